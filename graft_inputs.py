@@ -1,0 +1,217 @@
+"""Seeded synthetic inputs for the GRAFT draft-tree round.
+
+This module only *draws* inputs (random numbers, index sets, dtype rounding); it holds none of
+the method's arithmetic and is the one piece of code that both the CPU oracle's tests and the
+CUDA library's tests / benchmark use.  Every sequence is generated from its own counter-based
+stream (Philox keyed by (seed, tensor tag, sequence index)), so sequence b has the same bytes
+whatever the batch size or the rank that generates it.
+
+Workload shapes (block length 16; vocabularies 32,000 / 128,256 / 151,936; hidden widths
+256 / 2560 / 4096) stand in for a diffusion drafter's one-pass outputs:
+
+* logits[b, j, v] = 2 n + boost, n ~ N(0,1); at position j a seeded set of 64 distinct token ids
+  with ranks r = 1..64 gets boost H_{b,j} r^-1.1, H_{b,j} = H_b - 0.4 j;
+* hidden[b, j, :]: i.i.d. N(0,1), or an AR(1) chain h_j = rho_j h_{j-1} + sqrt(1-rho_j^2) g_j with
+  rho_j rising from 0.2 to 0.8 so that adjacent rows grow more similar at later positions;
+* TDES tables: either (emb, W_p, b_p, W_c, b_c, u) for the table-precompute step (small cases)
+  or the projected tables P, C ~ N(0,1) directly (large cases), u ~ N(0, 0.25), s = 1;
+* SABA: phi = (-160, +20, -5; bias 200), tau_min = 8, cost table t(n) = 18 + 0.02 max(0, n - 64) ms;
+* target ids: a continuation y_1..y_{L+1} per sequence, drawn before and independently of any tree.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, replace
+
+import numpy as np
+import torch
+
+N_BOOST = 64
+ZIPF_S = 1.1
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    batch: int
+    L: int
+    V: int
+    K: int
+    hidden_dim: int
+    logits_dtype: str  # "f32" | "bf16"
+    hidden_dtype: str
+    budget_min: int
+    budget_max: int
+    budget_step: int = 16
+    fixed_budget: int | None = None  # None -> SABA
+    boost_lo: float = 12.0  # H_b ~ U[boost_lo, boost_hi]; equal -> constant
+    boost_hi: float = 12.0
+    hidden_ar1: bool = True
+    m: int = 128
+    beta: float = 0.2
+    target_mode: str = "sampled"  # "sampled" (from the boosted distribution) | "decay" (match rate 0.9 -> 0.3)
+    seed: int = 20375
+
+    @property
+    def nmax(self) -> int:
+        return self.budget_max + 1
+
+    @property
+    def mask_words(self) -> int:
+        return (self.nmax + 31) // 32
+
+    def with_batch(self, batch: int) -> "Workload":
+        return replace(self, batch=batch)
+
+
+# The five stated configurations and the headline metric's configuration "M".
+C1 = Workload("C1", 1, 16, 32000, 8, 256, "f32", "f32", 64, 64, 16, fixed_budget=64, hidden_ar1=False, seed=20375)
+C2 = Workload("C2", 16, 16, 151936, 16, 2560, "bf16", "bf16", 16, 256, seed=20376)
+C3 = Workload("C3", 64, 16, 128256, 32, 4096, "bf16", "bf16", 16, 512, boost_lo=6.0, boost_hi=14.0, seed=20377)
+C4 = Workload("C4", 256, 16, 151936, 32, 4096, "bf16", "bf16", 16, 512, seed=20378)
+C5 = Workload("C5", 128, 16, 151936, 32, 4096, "bf16", "bf16", 16, 512, target_mode="decay", seed=20379)
+M = Workload("M", 64, 16, 151936, 32, 4096, "bf16", "bf16", 16, 512, target_mode="decay", seed=20380)
+WORKLOADS = {w.name: w for w in (C1, C2, C3, C4, C5, M)}
+
+_TAGS = {"logits": 1, "hidden": 2, "boost_ids": 3, "boost_h": 4, "tables": 5, "scalars": 6, "target": 7, "emb": 8}
+
+
+def _rng(seed: int, tag: str, b: int = 0) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=[(seed << 8) | _TAGS[tag], b]))
+
+
+def _to_dtype(x: np.ndarray, dtype: str) -> torch.Tensor:
+    t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32))
+    return t.to(torch.bfloat16) if dtype == "bf16" else t  # round-to-nearest-even
+
+
+def boost_ids(w: Workload, b: int) -> np.ndarray:
+    """[L, 64] distinct token ids per position; column r-1 holds the rank-r boosted token."""
+    g = _rng(w.seed, "boost_ids", b)
+    n = min(N_BOOST, w.V)
+    return np.stack([g.choice(w.V, size=n, replace=False) for _ in range(w.L)]).astype(np.int64)
+
+
+def boost_height(w: Workload, b: int) -> float:
+    if w.boost_hi == w.boost_lo:
+        return w.boost_lo
+    return float(_rng(w.seed, "boost_h", b).uniform(w.boost_lo, w.boost_hi))
+
+
+def logits_seq(w: Workload, b: int) -> torch.Tensor:
+    """[L, V] logits of sequence b in the workload's dtype."""
+    g = _rng(w.seed, "logits", b)
+    z = g.standard_normal((w.L, w.V), dtype=np.float32)
+    z *= 2.0
+    ids = boost_ids(w, b)
+    H = boost_height(w, b)
+    ranks = np.arange(1, ids.shape[1] + 1, dtype=np.float64) ** (-ZIPF_S)
+    for j in range(w.L):
+        z[j, ids[j]] += ((H - 0.4 * j) * ranks).astype(np.float32)
+    return _to_dtype(z, w.logits_dtype)
+
+
+def hidden_seq(w: Workload, b: int) -> torch.Tensor:
+    g = _rng(w.seed, "hidden", b)
+    x = g.standard_normal((w.L, w.hidden_dim), dtype=np.float32)
+    if w.hidden_ar1 and w.L > 1:
+        for j in range(1, w.L):
+            rho = 0.2 + 0.6 * j / (w.L - 1)
+            x[j] = rho * x[j - 1] + np.sqrt(1.0 - rho * rho) * x[j]
+    return _to_dtype(x, w.hidden_dtype)
+
+
+def batch_inputs(w: Workload, lo: int = 0, hi: int | None = None) -> dict:
+    """Inputs of sequences lo..hi-1 (default: the whole batch) as CPU torch tensors."""
+    hi = w.batch if hi is None else hi
+    n = hi - lo
+    logits = torch.empty((n, w.L, w.V), dtype=torch.bfloat16 if w.logits_dtype == "bf16" else torch.float32)
+    hidden = torch.empty((n, w.L, w.hidden_dim), dtype=torch.bfloat16 if w.hidden_dtype == "bf16" else torch.float32)
+    root = np.empty(n, np.int32)
+    hist = np.empty(n, np.float32)
+    prefix = np.empty(n, np.int32)
+    for i, b in enumerate(range(lo, hi)):
+        logits[i] = logits_seq(w, b)
+        hidden[i] = hidden_seq(w, b)
+        g = _rng(w.seed, "scalars", b)
+        root[i] = g.integers(0, w.V)
+        hist[i] = g.uniform(1.0, 9.0)
+        prefix[i] = g.integers(128, 4097)
+    out = dict(logits=logits, hidden=hidden, root_token=torch.from_numpy(root), hist=torch.from_numpy(hist),
+               prefix_len=torch.from_numpy(prefix))
+    out["fixed_budget"] = None if w.fixed_budget is None else torch.full((n,), w.fixed_budget, dtype=torch.int32)
+    return out
+
+
+def tdes_tables(w: Workload) -> dict:
+    """Projected tables P, C [V, m] ~ N(0,1) (what emb W^T + b looks like for W ~ N(0, 1/E)), u, s."""
+    g = _rng(w.seed, "tables")
+    P = g.standard_normal((w.V, w.m), dtype=np.float32)
+    Cc = g.standard_normal((w.V, w.m), dtype=np.float32)
+    u = (0.5 * g.standard_normal((w.L, w.m), dtype=np.float32)).astype(np.float32)
+    return dict(P=torch.from_numpy(P), C=torch.from_numpy(Cc), u=torch.from_numpy(u), s=1.0)
+
+
+def tdes_weights(V: int, E: int, m: int, L: int, seed: int, emb_dtype: str = "f32") -> dict:
+    """Raw scorer parameters for the table-precompute step: emb ~ N(0,1), W ~ N(0,1/E), b ~ N(0,0.01)."""
+    g = _rng(seed, "emb")
+    emb = _to_dtype(g.standard_normal((V, E), dtype=np.float32), emb_dtype)
+    sc = np.float32(1.0 / np.sqrt(E))
+    Wp = g.standard_normal((m, E), dtype=np.float32) * sc
+    Wc = g.standard_normal((m, E), dtype=np.float32) * sc
+    bp = (0.1 * g.standard_normal(m, dtype=np.float32)).astype(np.float32)
+    bc = (0.1 * g.standard_normal(m, dtype=np.float32)).astype(np.float32)
+    u = (0.5 * g.standard_normal((L, m), dtype=np.float32)).astype(np.float32)
+    return dict(emb=emb, Wp=torch.from_numpy(Wp), bp=torch.from_numpy(bp), Wc=torch.from_numpy(Wc),
+                bc=torch.from_numpy(bc), u=torch.from_numpy(u), s=1.0)
+
+
+def saba_defaults(w: Workload) -> dict:
+    """Synthetic SABA parameters (the fitted ones are not published) and the verification-cost table."""
+    return dict(phi_conf=-160.0, phi_degen=20.0, phi_hist=-5.0, phi_bias=200.0, tau_min=8.0, cost_mode=1,
+                c0=0.0, c1=0.0, c2=0.0, pts_n=[0.0, 64.0, float(w.budget_max)],
+                pts_t=[18.0, 18.0, 18.0 + 0.02 * max(0.0, w.budget_max - 64.0)])
+
+
+def target_tokens(w: Workload, b: int, logits_b: torch.Tensor | None = None) -> np.ndarray:
+    """y_1..y_{L+1} for sequence b (int32 [L+1]); y_{L+1} is a uniform random id.
+
+    "sampled": y_d is a draw from position d's distribution, taken as argmax(logits + Gumbel noise).
+    "decay":   with probability 0.9 - 0.6 (d-1)/(L-1), y_d is the boosted token of Zipf(1.1)-distributed
+               rank among that position's 64; otherwise a uniform random id.
+    """
+    g = _rng(w.seed, "target", b)
+    y = np.empty(w.L + 1, np.int32)
+    if w.target_mode == "sampled":
+        z = (logits_b if logits_b is not None else logits_seq(w, b)).to(torch.float32).numpy()
+        for j in range(w.L):
+            y[j] = int(np.argmax(z[j] + g.gumbel(size=w.V)))
+    else:
+        ids = boost_ids(w, b)
+        pr = np.arange(1, ids.shape[1] + 1, dtype=np.float64) ** (-ZIPF_S)
+        pr /= pr.sum()
+        for j in range(w.L):
+            p_match = 0.9 - 0.6 * j / max(1, w.L - 1)
+            if g.uniform() < p_match:
+                y[j] = ids[j, g.choice(ids.shape[1], p=pr)]
+            else:
+                y[j] = g.integers(0, w.V)
+    y[w.L] = g.integers(0, w.V)
+    return y
+
+
+def target_next_from_depth(y: np.ndarray, depth: np.ndarray) -> np.ndarray:
+    """target_next[i] = y_{depth(i)+1}: the target's next token after node i if the path to i was accepted.
+    Padding rows (depth -1) get -1."""
+    d = np.asarray(depth)
+    out = np.full(d.shape, -1, np.int32)
+    ok = d >= 0
+    out[ok] = y[d[ok]]
+    return out
+
+
+def small(name: str = "T", **kw) -> Workload:
+    """A small workload for tests; override any field."""
+    base = dict(name=name, batch=2, L=4, V=1000, K=4, hidden_dim=32, logits_dtype="f32", hidden_dtype="f32",
+                budget_min=8, budget_max=24, budget_step=8, fixed_budget=None, m=16, seed=7)
+    base.update(kw)
+    return Workload(**base)
