@@ -65,9 +65,10 @@ class Workload:
 
 # The five stated configurations and the headline metric's configuration "M".
 C1 = Workload("C1", 1, 16, 32000, 8, 256, "f32", "f32", 64, 64, 16, fixed_budget=64, hidden_ar1=False, seed=20375)
-C2 = Workload("C2", 16, 16, 151936, 16, 2560, "bf16", "bf16", 16, 256, seed=20376)
-C3 = Workload("C3", 64, 16, 128256, 32, 4096, "bf16", "bf16", 16, 512, boost_lo=6.0, boost_hi=14.0, seed=20377)
-C4 = Workload("C4", 256, 16, 151936, 32, 4096, "bf16", "bf16", 16, 512, seed=20378)
+C2 = Workload("C2", 16, 16, 151936, 16, 2560, "bf16", "bf16", 16, 256, target_mode="decay", seed=20376)
+C3 = Workload("C3", 64, 16, 128256, 32, 4096, "bf16", "bf16", 16, 512, boost_lo=6.0, boost_hi=14.0,
+              target_mode="decay", seed=20377)
+C4 = Workload("C4", 256, 16, 151936, 32, 4096, "bf16", "bf16", 16, 512, target_mode="decay", seed=20378)
 C5 = Workload("C5", 128, 16, 151936, 32, 4096, "bf16", "bf16", 16, 512, target_mode="decay", seed=20379)
 M = Workload("M", 64, 16, 151936, 32, 4096, "bf16", "bf16", 16, 512, target_mode="decay", seed=20380)
 WORKLOADS = {w.name: w for w in (C1, C2, C3, C4, C5, M)}

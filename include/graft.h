@@ -1,0 +1,186 @@
+/*
+ * graft.h -- C ABI of the B200 (sm_100a) GRAFT draft-tree builder.
+ *
+ * One decoding round of GRAFT (Sec. 3 "Method", overview in Sec. 3.1): given a diffusion
+ * drafter's one-pass block output -- logits q_{t,d}(.) over the vocabulary for d = 1..L and the
+ * hidden states h_{t,d} -- and the decoding state, build for every sequence of a batch the
+ * prefix-closed draft tree that the target model will verify, and afterwards walk the tree
+ * against the target's next tokens.
+ *
+ * Conventions
+ *   - Pointers named d_* are DEVICE pointers; all others are HOST pointers.  The caller owns
+ *     every buffer it passes in; the library never frees or reallocates them.  A context owns
+ *     only its own scratch (sized from max_batch at creation) and copies of the parameters.
+ *   - All tensors are dense, row-major, contiguous.  Logits rows may start at any address that
+ *     is a multiple of the element size (rows need not be 16-byte aligned).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls only
+ *     enqueue work on it and return; results are valid once the stream has reached that point.
+ *   - The return value reports host-side argument / launch errors, synchronously.  Data errors
+ *     are reported per sequence in d_status (bit flags below); nothing ever traps on the device.
+ *   - One context must not be used from two streams at the same time (the scratch is shared).
+ *   - There is no CPU fallback: without a CUDA device every entry point except
+ *     graft_status_str / graft_version returns GRAFT_ERR_CUDA.
+ *
+ * Limits (else GRAFT_ERR_UNSUPPORTED): 1 <= K <= 32, K <= V, 1 <= L <= 32, V < 2^31 - 64,
+ *   m a multiple of 4 with 4 <= m <= 512, budget_max <= 1023, budget_step >= 1,
+ *   L*K*K*4 bytes <= 128 KiB (edge scores live in shared memory), hidden_dim >= 1.
+ */
+#ifndef GRAFT_H_
+#define GRAFT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct graft_ctx graft_ctx; /* opaque */
+
+typedef enum {
+    GRAFT_OK = 0,
+    GRAFT_ERR_INVALID_ARG = 1, /* NULL where a pointer is required, batch out of range, ... */
+    GRAFT_ERR_UNSUPPORTED = 2, /* a size outside the limits above */
+    GRAFT_ERR_CUDA = 3,        /* a CUDA runtime call failed (no device, launch error, ...) */
+    GRAFT_ERR_WORKSPACE = 4,   /* scratch allocation failed */
+    GRAFT_ERR_STATE = 5        /* call order: TDES tables or SABA parameters not set */
+} graft_status;
+
+typedef enum { GRAFT_F32 = 0, GRAFT_BF16 = 1 } graft_dtype;
+
+/* per-sequence bits written to d_status */
+#define GRAFT_ST_BAD_LOGITS 1     /* a logits row holds NaN or +inf, or no finite entry: root-only tree */
+#define GRAFT_ST_TAU_CLAMPED 2    /* SABA: phi . s_t fell below tau_min and was clamped */
+#define GRAFT_ST_FRONTIER_EMPTY 4 /* fewer reachable prefixes than the budget */
+#define GRAFT_ST_INTERNAL 8       /* a bounded device-side wait ran out (should never happen) */
+
+typedef struct {
+    int32_t V;          /* vocabulary size */
+    int32_t L;          /* block length: future positions d = 1..L (the paper's D) */
+    int32_t K;          /* candidates kept per position */
+    int32_t m;          /* width of the TDES scoring space (Eq. 6) */
+    int32_t hidden_dim; /* width of h_{t,d} */
+    int32_t max_batch;
+    int32_t budget_min, budget_max, budget_step; /* SABA grid {min, min+step, .. <= max} (Sec. 3.3: 32..512 step 16) */
+    float beta;         /* residual strength of Eq. 4; 0 gives the DDTree score of Eq. 3 */
+    int32_t root_edge;  /* 1: depth-1 edges are scored against the root token; 0: f~ = 0 at depth 1 */
+    graft_dtype logits_dtype, hidden_dtype;
+} graft_config;
+
+/* SABA parameters (Sec. 3.3).  tau = phi . [conf, degen, hist] + phi_bias, clamped below by tau_min
+ * (Eq. 16's saturation scale).  Cost C_t(B): mode 0 = c0 + c1 B + c2 B prefix_t (Eq. 17); mode 1 = linear
+ * interpolation of the n_pts points (pts_n[i], pts_t[i]) (pts_n strictly increasing, n_pts <= 16), held
+ * constant outside them.  pts_* are host arrays and are copied. */
+typedef struct {
+    float phi_conf, phi_degen, phi_hist, phi_bias;
+    float tau_min;
+    int32_t cost_mode;
+    float c0, c1, c2;
+    int32_t n_pts;
+    const float* pts_n;
+    const float* pts_t;
+} graft_saba_params;
+
+/* Outputs of graft_build_trees.  Nmax = budget_max + 1 rows per sequence (node 0 is the root, i.e. the
+ * last committed token); W = ceil(Nmax / 32) mask words per row.  Nodes are in level order (depth
+ * ascending, then by the parent's index, then by candidate rank).  Rows n_nodes.. are padding: token,
+ * parent, depth, position = -1, path_score = 0, mask = 0. */
+typedef struct {
+    int32_t* d_n_nodes;    /* [batch] 1 + number of draft nodes */
+    int32_t* d_budget;     /* [batch] B_t */
+    int32_t* d_token;      /* [batch, Nmax] */
+    int32_t* d_parent;     /* [batch, Nmax] root: -1 */
+    int32_t* d_depth;      /* [batch, Nmax] root: 0 */
+    int32_t* d_position;   /* [batch, Nmax] prefix_len - 1 + depth */
+    float* d_path_score;   /* [batch, Nmax] S_TDES(u) of Eq. 13, accumulated root to leaf in fp32 */
+    uint32_t* d_mask;      /* [batch, Nmax, W] bit j of row i set iff j == i or j is an ancestor of i */
+    int32_t* d_status;     /* [batch] GRAFT_ST_* bits */
+    /* optional intermediate outputs, each may be NULL: */
+    int32_t* d_topk_id;    /* [batch, L, K] c^{(r)}_{t,d}, ranked by (logit descending, token id ascending) */
+    float* d_topk_lp;      /* [batch, L, K] log q_{t,d}(c^{(r)}) */
+    float* d_lse;          /* [batch, L] log sum_v exp(logit) */
+    float* d_edge;         /* [batch, L, K, K] S_TDES(v) indexed (depth, parent rank, child rank); depth 1 uses
+                              parent row 0 only, its other rows are 0 */
+    float* d_state;        /* [batch, 4] conf_t, degen_t, hist_t, tau (zeros when the budget is fixed) */
+} graft_tree_out;
+
+/* Create / destroy a context.  Allocates the scratch for max_batch sequences.  Sets *out = NULL on error. */
+graft_status graft_create(const graft_config* cfg, graft_ctx** out);
+graft_status graft_destroy(graft_ctx* ctx);
+size_t graft_nmax(const graft_ctx* ctx);       /* budget_max + 1 */
+size_t graft_mask_words(const graft_ctx* ctx); /* ceil(Nmax / 32) */
+
+/* SABA parameters (Sec. 3.3, Eq. 14-17).  Required before graft_build_trees is called without a
+ * fixed budget. */
+graft_status graft_set_saba(graft_ctx* ctx, const graft_saba_params* p);
+
+/* TDES tables (Sec. 3.2, text after Eq. 6: the projected embeddings depend only on the token id and are
+ * computed once).  d_P, d_C: [V, m] fp32, 16-byte aligned, P[v] = g_p(e_v), C[v] = g_c(e_v); d_u: [L, m]
+ * fp32 depth embeddings u_d; s: the scale of Eq. 6.  The tables are borrowed until the context is
+ * destroyed or the tables are set again.  u is copied on `stream`. */
+graft_status graft_set_tdes_tables(graft_ctx* ctx, const float* d_P, const float* d_C, const float* d_u, float s,
+                                   void* stream);
+
+/* Table precompute (same passage): d_out[v] = W e_v + b for one tower.  d_emb [V, E] (dtype as given),
+ * d_W [m, E] fp32, d_b [m] fp32 or NULL, d_out [V, m] fp32.  fp32 accumulation.  Call once per tower. */
+graft_status graft_tdes_precompute(graft_ctx* ctx, const void* d_emb, graft_dtype emb_dtype, int32_t E,
+                                   const float* d_W, const float* d_b, float* d_out, void* stream);
+
+/* The round (Sec. 3.1): candidates (Preliminaries, "DFlash one-pass marginals") -> SABA budget (Sec. 3.3)
+ * -> TDES edge scores (Eq. 4-6) -> best-first expansion by path score (Eq. 13) until B_t nodes -> emission.
+ *   d_logits       [batch, L, V]  drafter logits, dtype cfg.logits_dtype
+ *   d_hidden       [batch, L, hidden_dim], dtype cfg.hidden_dtype; may be NULL iff d_fixed_budget != NULL
+ *   d_root_token   [batch] last committed token (parent of the depth-1 edges)
+ *   d_hist         [batch] hist_t = mean of the last w accepted lengths (Eq. 15); may be NULL iff fixed budget
+ *   d_prefix_len   [batch] tokens in the prefix x^(t), the root included
+ *   d_fixed_budget [batch] or NULL.  NULL: B_t from SABA.  Else B_t = clamp(value, 0, budget_max).
+ * Requires graft_set_tdes_tables unless beta == 0 (then edge = log q and no table is read). */
+graft_status graft_build_trees(graft_ctx* ctx, int32_t batch, const void* d_logits, const void* d_hidden,
+                               const int32_t* d_root_token, const float* d_hist, const int32_t* d_prefix_len,
+                               const int32_t* d_fixed_budget, const graft_tree_out* out, void* stream);
+
+/* The steps of the round on their own (the same kernels graft_build_trees runs), for per-step timing
+ * and parity checks. */
+/* Vocab pass: per (sequence, position) log-sum-exp over V and the K top-ranked tokens with their log q.
+ * d_row_status [batch*L] (may be NULL) receives GRAFT_ST_BAD_LOGITS or 0 per row. */
+graft_status graft_vocab_pass(graft_ctx* ctx, int32_t batch, const void* d_logits, int32_t* d_topk_id,
+                              float* d_topk_lp, float* d_lse, int32_t* d_row_status, void* stream);
+/* TDES edge scores (Eq. 4-6) from candidates: d_edge [batch, L, K, K]. */
+graft_status graft_tdes_edges(graft_ctx* ctx, int32_t batch, const int32_t* d_topk_id, const float* d_topk_lp,
+                              const int32_t* d_root_token, float* d_edge, void* stream);
+
+/* Acceptance walk (Preliminaries, "Speculative decoding": a_t; "Tree-based speculative decoding": the longest
+ * accepted path is committed).  d_target_next[b, i] is the target model's next token after node i.
+ * Starting at the root, follow the child whose token equals target_next of the current node.
+ *   d_accept_len  [batch]     number of accepted draft tokens a_t (bonus token not counted)
+ *   d_accept_path [batch, L]  node indices of the accepted path, -1 padded
+ *   d_bonus_token [batch]     target_next of the last accepted node */
+graft_status graft_accept(graft_ctx* ctx, int32_t batch, const graft_tree_out* trees, const int32_t* d_target_next,
+                          int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus_token, void* stream);
+
+/* Host-buffer form of graft_build_trees for end-to-end use: every pointer here is a HOST pointer (pinned
+ * memory makes the copies asynchronous).  Copies the inputs host->device into context-owned staging buffers
+ * (allocated on first use, sized for max_batch), runs the same kernels as graft_build_trees, copies
+ * n_nodes, budget, status, token, parent, depth, position, path_score and mask device->host into h_out's
+ * arrays, and synchronises `stream` before returning.  h_out's optional fields must be NULL. */
+graft_status graft_build_trees_host(graft_ctx* ctx, int32_t batch, const void* h_logits, const void* h_hidden,
+                                    const int32_t* h_root_token, const float* h_hist, const int32_t* h_prefix_len,
+                                    const int32_t* h_fixed_budget, const graft_tree_out* h_out, void* stream);
+
+/* Number of kernels the library has launched through this context since creation. */
+uint64_t graft_launch_count(const graft_ctx* ctx);
+
+/* Per-kernel device timing of graft_build_trees.  graft_set_timing(ctx, 1) makes every later call record
+ * CUDA events on its stream around the vocab-pass kernel, the edge-score kernel and the tree kernel (a ring
+ * of the last 64 calls) and resets the call count.  graft_read_timing waits for the newest recorded call and
+ * returns the number of calls summed (at most 64) and the summed milliseconds of each kernel. */
+graft_status graft_set_timing(graft_ctx* ctx, int32_t enable);
+graft_status graft_read_timing(graft_ctx* ctx, int32_t* n_calls, float* vocab_ms, float* tdes_ms, float* tree_ms);
+
+const char* graft_status_str(graft_status s);
+const char* graft_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRAFT_H_ */

@@ -1,0 +1,7 @@
+"""B200-native GRAFT draft-tree builder: hand-written sm_100a kernels behind a C ABI (include/graft.h),
+with a thin ctypes binding.  PyTorch is used by callers only for device memory and streams."""
+from .binding import (  # noqa: F401
+    Graft, GraftError, TreeOut, BF16, F32, ST_BAD_LOGITS, ST_TAU_CLAMPED, ST_FRONTIER_EMPTY, ST_INTERNAL,
+    load_library, library_path,
+)
+from .shard import shard_range  # noqa: F401

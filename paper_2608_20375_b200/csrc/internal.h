@@ -1,0 +1,103 @@
+// Internal declarations shared by the translation units of libgraft (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/graft.h"
+
+namespace graft {
+
+constexpr int kMaxK = 32;
+constexpr int kMaxL = 32;
+constexpr int kMaxCostPts = 16;
+
+// ---- vocab pass -----------------------------------------------------------------------------
+constexpr int kVpConsumerWarps = 8;
+constexpr int kVpConsumers = kVpConsumerWarps * 32;  // 256
+constexpr int kVpThreads = kVpConsumers + 32;        // + one producer warp
+constexpr int kVpTileBytes = 16384;                  // one TMA bulk copy
+constexpr int kVpQuantum = 2048;                     // elements; granularity of the work partition
+constexpr int kVpCandCap = 1024;                     // candidate keys held in shared memory
+constexpr int kVpHitCap = 512;                       // chunk hits held in shared memory
+
+// What one CTA leaves behind for a row that it shares with other CTAs.
+struct VpRecord {
+    float c;      // reference exponent (log2 domain)
+    float s;      // sum_v 2^(z_v log2e - c) over the segment
+    float vmax;   // largest logit of the segment
+    uint32_t nkeys;
+    uint64_t keys[kMaxK];  // the segment's best keys, descending
+};
+
+struct VpPlan {
+    int grid;            // CTAs launched
+    int stages;          // ring depth
+    int max_seg_tiles;   // tiles in the longest segment a CTA can get
+    size_t smem_bytes;
+};
+
+struct SabaDev {
+    double phi_conf, phi_degen, phi_hist, phi_bias, tau_min;
+    int cost_mode;
+    double c0, c1, c2;
+    int n_pts;
+    double pts_n[kMaxCostPts], pts_t[kMaxCostPts];
+};
+
+}  // namespace graft
+
+struct graft_ctx {
+    graft_config cfg;
+    int device;
+    int num_sms;
+    int nmax, mask_words, grid_pts;
+    bool saba_set, tdes_set;
+    graft::SabaDev saba;
+    const float* d_P;
+    const float* d_C;
+    float* d_u;  // owned copy [L, m]
+    float tdes_s;
+    // scratch (one allocation)
+    void* ws;
+    size_t ws_bytes;
+    graft::VpRecord* vp_records;  // [grid, 2]
+    int* vp_row_counter;          // [max_batch * L], zero between launches
+    int32_t* w_topk_id;           // [max_batch, L, K]
+    float* w_topk_lp;             // [max_batch, L, K]
+    float* w_lse;                 // [max_batch, L]
+    int32_t* w_row_status;        // [max_batch, L]
+    float* w_edge;                // [max_batch, L, K, K]
+    double* w_cos;                // [max_batch, L]   adjacent-row cosines r_d
+    int32_t* w_errflag;           // [1] device-side internal error flag
+    graft::VpPlan vp_plan;
+    // host-buffer staging (allocated on first use of graft_build_trees_host)
+    void* stage;
+    size_t stage_bytes;
+    // bookkeeping
+    uint64_t launches;
+    int timing;
+    cudaEvent_t ev[6];
+};
+
+namespace graft {
+
+VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch);
+cudaError_t vp_configure(const graft_config& cfg, int num_sms, size_t* max_smem);
+cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* d_topk_id, float* d_topk_lp,
+                      float* d_lse, int32_t* d_row_status, cudaStream_t st);
+
+cudaError_t tdes_precompute_launch(graft_ctx* ctx, const void* d_emb, graft_dtype dt, int E, const float* d_W,
+                                   const float* d_b, float* d_out, cudaStream_t st);
+cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
+                              const int32_t* d_root_token, const int32_t* d_row_status, float* d_edge,
+                              cudaStream_t st);
+cudaError_t cosine_launch(graft_ctx* ctx, int batch, const void* d_hidden, double* d_cos, cudaStream_t st);
+cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
+                        const int32_t* d_row_status, const float* d_edge, const double* d_cos,
+                        const int32_t* d_root_token, const float* d_hist, const int32_t* d_prefix_len,
+                        const int32_t* d_fixed_budget, const graft_tree_out* out, cudaStream_t st);
+cudaError_t accept_launch(graft_ctx* ctx, int batch, const graft_tree_out* trees, const int32_t* d_target_next,
+                          int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus, cudaStream_t st);
+size_t tree_smem_bytes(const graft_config& cfg);
+
+}  // namespace graft

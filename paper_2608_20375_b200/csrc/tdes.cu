@@ -1,0 +1,212 @@
+// TDES (Sec. 3.2): the cached bi-tower projections and the per-round edge scores.
+//
+//   tdes_precompute_kernel   out[v] = W e_v + b            (text after Eq. 6: computed once per model)
+//   tdes_edges_kernel        edge[d][i][c] = log q_d(c) + beta * (f - mean_c f),
+//                            f = s (P[p_i] + u_d) . (C[c] + u_d) / sqrt(m)          (Eq. 4-6)
+//
+// The per-round scorer is a gather of token-indexed table rows followed by K x K dot products of length
+// m per depth -- not a dense contraction over hidden states -- so it runs as fp32 FMAs out of shared
+// memory (tensor-core tf32/bf16 products would also break the 1e-5 score tolerance).
+#include "common.cuh"
+#include "internal.h"
+
+namespace graft {
+namespace {
+
+// ---- table precompute: a plain shared-memory tiled fp32 GEMM (setup path, off the round) ---------------
+constexpr int PT_V = 64, PT_M = 64, PT_E = 16;
+
+template <bool BF16>
+__global__ void __launch_bounds__(256) tdes_precompute_kernel(const void* __restrict__ emb, const float* __restrict__ W,
+                                                              const float* __restrict__ bias, float* __restrict__ out,
+                                                              int V, int E, int m) {
+    __shared__ float sA[PT_E][PT_V + 1];  // emb tile, transposed
+    __shared__ float sB[PT_E][PT_M + 1];  // W tile, transposed
+    const int v0 = blockIdx.x * PT_V, k0 = blockIdx.y * PT_M;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;  // 16 x 16 threads, 4 x 4 outputs each
+    float acc[4][4] = {};
+    for (int e0 = 0; e0 < E; e0 += PT_E) {
+        for (int i = threadIdx.x; i < PT_V * PT_E; i += 256) {
+            int r = i / PT_E, c = i % PT_E;
+            int v = v0 + r, e = e0 + c;
+            float x = 0.f;
+            if (v < V && e < E) {
+                if (BF16)
+                    x = __uint_as_float(((uint32_t)((const uint16_t*)emb)[(size_t)v * E + e]) << 16);
+                else
+                    x = ((const float*)emb)[(size_t)v * E + e];
+            }
+            sA[c][r] = x;
+        }
+        for (int i = threadIdx.x; i < PT_M * PT_E; i += 256) {
+            int r = i / PT_E, c = i % PT_E;
+            int k = k0 + r, e = e0 + c;
+            sB[c][r] = (k < m && e < E) ? W[(size_t)k * E + e] : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < PT_E; ++e) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = sA[e][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = sB[e][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int v = v0 + ty * 4 + i;
+        if (v >= V) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int k = k0 + tx * 4 + j;
+            if (k < m) out[(size_t)v * m + k] = acc[i][j] + (bias ? bias[k] : 0.f);
+        }
+    }
+}
+
+// ---- edge scores: one CTA per (sequence, depth) --------------------------------------------------------
+struct EdgeParams {
+    const int32_t* topk_id;
+    const float* topk_lp;
+    const int32_t* root_token;
+    const int32_t* row_status;
+    const float* P;
+    const float* C;
+    const float* u;
+    float* edge;
+    int L, K, m, V;
+    float scale;  // s / sqrt(m)
+    float beta;
+    int root_edge;
+};
+
+__global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
+    extern __shared__ __align__(16) float smem[];
+    const int b = blockIdx.x / p.L, j = blockIdx.x % p.L;
+    const int K = p.K, m = p.m, ld = m + 4;  // padded row: 16-byte aligned, conflict-free float4 reads
+    float* sP = smem;                        // [K][ld]  parent rows + u_d
+    float* sC = smem + (size_t)kMaxK * ld;   // [K][ld]  child rows + u_d
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_par = (j == 0) ? 1 : K;
+    const size_t row = (size_t)b * p.L + j;
+    float* out = p.edge + row * K * K;
+    const int32_t* ids = p.topk_id + row * K;
+    const float* lps = p.topk_lp + row * K;
+
+    const bool bad = p.row_status != nullptr && (p.row_status[row] != 0 || (j > 0 && p.row_status[row - 1] != 0));
+    const bool neutral = (p.beta == 0.0f) || (j == 0 && !p.root_edge) || bad;
+    if (neutral) {
+        // edge = log q exactly (the DDTree score of Eq. 3); bad rows get zeros
+        for (int i = threadIdx.x; i < K * K; i += 256) {
+            int par = i / K, c = i % K;
+            out[i] = (bad || par >= n_par) ? 0.f : lps[c];
+        }
+        return;
+    }
+    // gather: one warp per table row, 16 bytes per lane
+    const float* urow = p.u + (size_t)j * m;
+    for (int r = warp; r < n_par + K; r += 8) {
+        const bool is_par = r < n_par;
+        const int idx = is_par ? r : r - n_par;
+        int32_t tok = is_par ? (j == 0 ? p.root_token[b] : p.topk_id[(row - 1) * K + idx]) : ids[idx];
+        tok = tok < 0 ? 0 : (tok >= p.V ? p.V - 1 : tok);
+        const float4* src = (const float4*)((is_par ? p.P : p.C) + (size_t)tok * m);
+        float* dst = (is_par ? sP : sC) + (size_t)idx * ld;
+        for (int k4 = lane; k4 < m / 4; k4 += 32) {
+            float4 t = __ldg(src + k4);
+            float4 uu = *(const float4*)(urow + k4 * 4);
+            t.x += uu.x;
+            t.y += uu.y;
+            t.z += uu.z;
+            t.w += uu.w;
+            *(float4*)(dst + k4 * 4) = t;
+        }
+    }
+    __syncthreads();
+    // lane = child c; each warp takes parents warp, warp+8, ...
+    const int c = lane;
+    float f[4] = {0.f, 0.f, 0.f, 0.f};
+    if (c < K) {
+        const float4* cc = (const float4*)(sC + (size_t)c * ld);
+        for (int k4 = 0; k4 < m / 4; ++k4) {
+            const float4 cv = cc[k4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int par = warp + 8 * t;
+                if (par < n_par) {
+                    const float4 pv = *(const float4*)(sP + (size_t)par * ld + k4 * 4);
+                    f[t] = fmaf(pv.x, cv.x, f[t]);
+                    f[t] = fmaf(pv.y, cv.y, f[t]);
+                    f[t] = fmaf(pv.z, cv.z, f[t]);
+                    f[t] = fmaf(pv.w, cv.w, f[t]);
+                }
+            }
+        }
+    }
+    const float lp = c < K ? lps[c] : 0.f;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        const int par = warp + 8 * t;
+        if (par >= K) continue;  // uniform per warp
+        float ft = (c < K) ? f[t] * p.scale : 0.f;
+        float sum = ft;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
+        const float mean = sum / (float)K;
+        if (c < K) out[(size_t)par * K + c] = (par < n_par) ? fmaf(p.beta, ft - mean, lp) : 0.f;
+    }
+}
+
+}  // namespace
+
+cudaError_t tdes_precompute_launch(graft_ctx* ctx, const void* d_emb, graft_dtype dt, int E, const float* d_W,
+                                   const float* d_b, float* d_out, cudaStream_t st) {
+    const int V = ctx->cfg.V, m = ctx->cfg.m;
+    dim3 grid((V + PT_V - 1) / PT_V, (m + PT_M - 1) / PT_M);
+    if (dt == GRAFT_BF16)
+        tdes_precompute_kernel<true><<<grid, 256, 0, st>>>(d_emb, d_W, d_b, d_out, V, E, m);
+    else
+        tdes_precompute_kernel<false><<<grid, 256, 0, st>>>(d_emb, d_W, d_b, d_out, V, E, m);
+    ctx->launches += 1;
+    return cudaGetLastError();
+}
+
+size_t tdes_edges_smem(const graft_config& cfg) { return (size_t)2 * kMaxK * (cfg.m + 4) * sizeof(float); }
+
+cudaError_t tdes_edges_configure(const graft_config& cfg) {
+    return cudaFuncSetAttribute(tdes_edges_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)tdes_edges_smem(cfg));
+}
+
+cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
+                              const int32_t* d_root_token, const int32_t* d_row_status, float* d_edge,
+                              cudaStream_t st) {
+    const graft_config& cfg = ctx->cfg;
+    EdgeParams p;
+    p.topk_id = d_topk_id;
+    p.topk_lp = d_topk_lp;
+    p.root_token = d_root_token;
+    p.row_status = d_row_status;
+    p.P = ctx->d_P;
+    p.C = ctx->d_C;
+    p.u = ctx->d_u;
+    p.edge = d_edge;
+    p.L = cfg.L;
+    p.K = cfg.K;
+    p.m = cfg.m;
+    p.V = cfg.V;
+    p.scale = ctx->tdes_s / sqrtf((float)cfg.m);
+    p.beta = ctx->tdes_set ? cfg.beta : 0.0f;
+    p.root_edge = cfg.root_edge;
+    tdes_edges_kernel<<<batch * cfg.L, 256, tdes_edges_smem(cfg), st>>>(p);
+    ctx->launches += 1;
+    return cudaGetLastError();
+}
+
+}  // namespace graft

@@ -1,0 +1,310 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import graft_inputs as gi
+import oracle
+from helpers import EPS, check_tree_invariants, compare_accept, compare_round, gpu_round, oracle_round
+
+pytestmark = pytest.mark.gpu
+
+DT = {"f32": 0, "bf16": 1}
+
+
+def _graft(w, max_batch=None, beta=None, root_edge=1):
+    from paper_2608_20375_b200 import Graft
+    g = Graft(w.V, w.L, w.K, w.m, w.hidden_dim, max_batch or w.batch, w.budget_min, w.budget_max, w.budget_step,
+              w.beta if beta is None else beta, root_edge, DT[w.logits_dtype], DT[w.hidden_dtype])
+    return g
+
+
+def _setup(w, g):
+    tb = gi.tdes_tables(w)
+    saba_kw = gi.saba_defaults(w)
+    keep = [tb["P"].cuda(), tb["C"].cuda(), tb["u"].cuda()]
+    g.set_tdes_tables(keep[0], keep[1], keep[2], tb["s"])
+    g.set_saba(**saba_kw)
+    return tb, saba_kw, keep
+
+
+# --------------------------------------------------------------------------- vocab pass
+def _vocab_case(z, K, dtype):
+    """z: [batch, L, V] CPU tensor in its dtype."""
+    from paper_2608_20375_b200 import Graft
+    Bt, L, V = z.shape
+    g = Graft(V, L, K, 16, 8, Bt, 8, 8, 8, 0.0, 1, DT[dtype], 0)
+    ids = torch.empty((Bt, L, K), dtype=torch.int32, device="cuda")
+    lp = torch.empty((Bt, L, K), dtype=torch.float32, device="cuda")
+    lse = torch.empty((Bt, L), dtype=torch.float32, device="cuda")
+    rs = torch.empty((Bt, L), dtype=torch.int32, device="cuda")
+    g.vocab_pass(z.cuda(), ids, lp, lse, rs)
+    torch.cuda.synchronize()
+    o_ids, o_lp, o_lse, o_st = oracle.vocab_pass(z.reshape(Bt * L, V), K)
+    ids, lp, lse, rs = (t.cpu().numpy().reshape(Bt * L, -1) for t in (ids, lp, lse, rs))
+    assert np.array_equal(rs[:, 0], o_st)
+    good = o_st == 0
+    assert np.array_equal(ids[good], o_ids[good])
+    a, b = lp[good].astype(np.float64), o_lp[good].astype(np.float64)
+    fin = np.isfinite(b)
+    assert np.array_equal(np.isneginf(a), np.isneginf(b))
+    assert np.abs(a[fin] - b[fin]).max(initial=0) <= EPS
+    assert np.abs(lse[good, 0] - o_lse[good]).max(initial=0) <= EPS
+    g.destroy()
+    return float(np.abs(lse[good, 0] - o_lse[good]).max(initial=0))
+
+
+@pytest.mark.parametrize("V,K,L,Bt,dtype", [
+    (32000, 8, 16, 1, "f32"),      # rows split over many CTAs
+    (4099, 32, 3, 5, "bf16"),      # odd V: rows start at 2-byte offsets
+    (4097, 16, 4, 3, "f32"),       # odd V in fp32
+    (33, 32, 2, 2, "bf16"),        # K almost V, everything through the ragged path
+    (8, 8, 1, 1, "f32"),           # K == V
+    (151936, 32, 2, 3, "bf16"),    # several tiles and a ragged tail per row
+    (20000, 16, 16, 40, "bf16"),   # many rows per CTA
+    (70001, 5, 1, 1, "bf16"),      # one row shared by every CTA
+])
+def test_vocab_pass_shapes(V, K, L, Bt, dtype):
+    g = torch.Generator().manual_seed(V + K)
+    z = 2.0 * torch.randn((Bt, L, V), generator=g)
+    z[:, :, : min(V, 7)] += 6.0
+    z = z.to(torch.bfloat16) if dtype == "bf16" else z
+    _vocab_case(z, K, dtype)
+
+
+def test_vocab_pass_ties_uniform_masked_and_bad_rows():
+    V, K = 9000, 32
+    g = torch.Generator().manual_seed(1)
+    z = torch.round(2.0 * torch.randn((1, 8, V), generator=g) * 2) / 2  # heavy ties
+    z[0, 1] = 1.25                        # all equal: ids 0..K-1
+    z[0, 2, 100:] = float("-inf")         # masked vocabulary
+    z[0, 3, 5] = float("nan")
+    z[0, 4, 77] = float("inf")
+    z[0, 5] = float("-inf")
+    z[0, 6] = torch.arange(V, dtype=torch.float32) * 1e-3   # ascending: every element a new maximum
+    z[0, 7] = -torch.arange(V, dtype=torch.float32) * 1e-3  # descending
+    _vocab_case(z, K, "f32")
+    _vocab_case(z.to(torch.bfloat16), K, "bf16")
+
+
+def test_vocab_pass_large_magnitudes_and_negative_zero():
+    V, K = 5000, 8
+    g = torch.Generator().manual_seed(2)
+    z = 30.0 * torch.randn((1, 4, V), generator=g)
+    z[0, 0] += 500.0
+    z[0, 1] -= 500.0
+    z[0, 2, ::2] = 0.0
+    z[0, 2, 1::2] = -0.0
+    z[0, 3] *= 1e-3
+    _vocab_case(z, K, "f32")
+    _vocab_case(z.to(torch.bfloat16), K, "bf16")
+
+
+def test_vocab_pass_is_reproducible_and_counters_reset():
+    w = gi.small(batch=3, L=4, V=50000, K=16, logits_dtype="bf16")
+    x = gi.batch_inputs(w)
+    g = _graft(w, beta=0.0)
+    z = x["logits"].cuda()
+    outs = []
+    for _ in range(3):
+        ids = torch.empty((3, 4, 16), dtype=torch.int32, device="cuda")
+        lp = torch.empty((3, 4, 16), dtype=torch.float32, device="cuda")
+        lse = torch.empty((3, 4), dtype=torch.float32, device="cuda")
+        g.vocab_pass(z, ids, lp, lse)
+        torch.cuda.synchronize()
+        outs.append((ids.cpu(), lp.cpu(), lse.cpu()))
+    for o in outs[1:]:
+        assert torch.equal(o[0], outs[0][0])
+        assert torch.equal(o[1], outs[0][1])
+
+
+# --------------------------------------------------------------------------- TDES
+def test_tdes_precompute_against_oracle():
+    V, E, m, L = 777, 200, 24, 4
+    wts = gi.tdes_weights(V, E, m, L, seed=5, emb_dtype="bf16")
+    w = gi.small(V=V, m=m, L=L)
+    g = _graft(w)
+    out = torch.empty((V, m), dtype=torch.float32, device="cuda")
+    for Wk, bk in (("Wp", "bp"), ("Wc", None)):
+        g.tdes_precompute(wts["emb"].cuda(), wts[Wk].cuda(), None if bk is None else wts[bk].cuda(), out)
+        torch.cuda.synchronize()
+        want = oracle.tdes_tables(wts["emb"], wts[Wk].numpy(), None if bk is None else wts[bk].numpy())
+        np.testing.assert_allclose(out.cpu().numpy(), want, rtol=1e-5, atol=1e-5)
+
+
+@pytest.mark.parametrize("K,L,m,beta,root_edge", [(4, 4, 16, 0.2, 1), (32, 16, 128, 0.2, 1), (7, 3, 36, 0.7, 0),
+                                                   (16, 5, 128, 0.0, 1)])
+def test_tdes_edges_against_oracle(K, L, m, beta, root_edge):
+    V, Bt = 3000, 3
+    w = gi.small(batch=Bt, V=V, K=K, L=L, m=m, beta=beta)
+    g = _graft(w, root_edge=root_edge)
+    tb, _, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    ids, lp, _, _ = oracle.vocab_pass(x["logits"].reshape(Bt * L, V), K)
+    ids, lp = ids.reshape(Bt, L, K), lp.reshape(Bt, L, K)
+    edge = torch.empty((Bt, L, K, K), dtype=torch.float32, device="cuda")
+    g.tdes_edges(torch.from_numpy(ids).cuda(), torch.from_numpy(lp).cuda(), x["root_token"].cuda(), edge)
+    torch.cuda.synchronize()
+    edge = edge.cpu().numpy()
+    for b in range(Bt):
+        want = oracle.tdes_edges(ids[b], lp[b], int(x["root_token"][b]), tb["P"].numpy(), tb["C"].numpy(),
+                                 tb["u"].numpy(), tb["s"], beta, root_edge)
+        assert np.abs(edge[b] - want).max() <= EPS
+        if beta == 0.0:
+            assert np.array_equal(edge[b], want)  # the DDTree score, bit for bit
+
+
+# --------------------------------------------------------------------------- whole round, small
+@pytest.mark.parametrize("kw", [
+    dict(batch=4, L=4, V=1000, K=4, budget_min=8, budget_max=24, budget_step=8),
+    dict(batch=3, L=6, V=5000, K=8, budget_min=16, budget_max=96, budget_step=16, logits_dtype="bf16",
+         hidden_dtype="bf16", hidden_dim=64, m=32),
+    dict(batch=2, L=16, V=20011, K=32, budget_min=32, budget_max=512, budget_step=16, logits_dtype="bf16", m=128,
+         hidden_dim=128, boost_lo=6.0, boost_hi=14.0),
+    dict(batch=2, L=3, V=50, K=4, budget_min=200, budget_max=200, fixed_budget=200),  # budget > all prefixes
+    dict(batch=2, L=5, V=300, K=1, budget_min=4, budget_max=12, budget_step=4),        # K = 1: a chain
+    dict(batch=2, L=1, V=300, K=8, budget_min=4, budget_max=4, fixed_budget=4),        # single position
+    dict(batch=3, L=8, V=3000, K=16, budget_min=0, budget_max=64, fixed_budget=0),     # empty budget
+    dict(batch=5, L=16, V=32000, K=8, budget_min=64, budget_max=64, fixed_budget=64, hidden_ar1=False),
+])
+@pytest.mark.parametrize("beta", [0.2, 0.0])
+def test_round_small(kw, beta):
+    w = gi.small(**kw, beta=beta)
+    g = _graft(w)
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    assert stats["excused_tree"] + stats["excused_budget"] <= max(1, w.batch // 4), stats
+    compare_accept(oracle, gi, g, w, out, gpu)
+
+
+def test_round_bad_rows_and_status_bits():
+    w = gi.small(batch=4, L=4, V=2000, K=4, budget_min=8, budget_max=24, budget_step=8)
+    g = _graft(w)
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    x["logits"][1, 2, 17] = float("nan")
+    x["logits"][3, 0, :] = float("-inf")
+    saba_kw = dict(saba_kw, phi_bias=-1e4)  # tau clamps on every sequence
+    g.set_saba(**saba_kw)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    assert gpu["status"].tolist() == [2, 1, 2, 1] == orc["status"].tolist()
+    compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+
+
+def test_round_affine_cost_and_paper_grid():
+    w = gi.small(batch=6, L=8, V=4000, K=8, budget_min=32, budget_max=512, budget_step=16, hidden_dim=96)
+    g = _graft(w)
+    tb, _, keep = _setup(w, g)
+    saba_kw = dict(phi_conf=-120.0, phi_degen=30.0, phi_hist=4.0, phi_bias=150.0, tau_min=8.0, cost_mode=0, c0=18.0,
+                   c1=0.02, c2=2e-6)
+    g.set_saba(**saba_kw)
+    x = gi.batch_inputs(w)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    assert len(set(gpu["budget"].tolist())) > 1  # budgets actually vary with the state
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    w = gi.small(batch=3, L=6, V=5000, K=8, budget_min=16, budget_max=96, budget_step=16, logits_dtype="bf16")
+    g = _graft(w)
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    out, gpu = gpu_round(g, w, x, debug=False)
+    pin = lambda t: None if t is None else t.pin_memory()  # noqa: E731
+    h = g.alloc_out(w.batch, device="cpu", pinned=True)
+    g.build_trees_host(pin(x["logits"]), pin(x["hidden"]), pin(x["root_token"]), pin(x["hist"]), pin(x["prefix_len"]),
+                       None, h)
+    for k in ("n_nodes", "budget", "token", "parent", "depth", "position", "path_score", "mask", "status"):
+        assert np.array_equal(getattr(h, k).numpy().view(gpu[k].dtype), gpu[k]), k
+
+
+def test_argument_validation():
+    from paper_2608_20375_b200 import Graft, GraftError
+    with pytest.raises(GraftError, match="supported"):
+        Graft(1000, 4, 64, 16, 8, 1, 8, 8)  # K > 32
+    with pytest.raises(GraftError, match="supported"):
+        Graft(1000, 4, 4, 18, 8, 1, 8, 8)   # m not a multiple of 4
+    with pytest.raises(GraftError, match="supported"):
+        Graft(1000, 4, 4, 16, 8, 1, 8, 2000)
+    w = gi.small()
+    g = _graft(w)
+    x = gi.batch_inputs(w)
+    out = g.alloc_out(w.batch)
+    cu = lambda t: t.cuda()  # noqa: E731
+    with pytest.raises(GraftError, match="not set"):  # TDES tables missing with beta != 0
+        g.build_trees(cu(x["logits"]), cu(x["hidden"]), cu(x["root_token"]), cu(x["hist"]), cu(x["prefix_len"]), None, out)
+    _setup(w, g)
+    with pytest.raises(GraftError, match="invalid"):  # SABA without hidden states
+        g.build_trees(cu(x["logits"]), None, cu(x["root_token"]), cu(x["hist"]), cu(x["prefix_len"]), None, out)
+    big = gi.batch_inputs(w.with_batch(w.batch + 1))
+    with pytest.raises(GraftError, match="invalid"):  # batch beyond max_batch
+        g.build_trees(cu(big["logits"]), cu(big["hidden"]), cu(big["root_token"]), cu(big["hist"]),
+                      cu(big["prefix_len"]), None, g.alloc_out(w.batch + 1))
+    assert g.launch_count() == 0
+
+
+# --------------------------------------------------------------------------- stated configurations
+def test_config_C1_full():
+    w = gi.C1
+    g = _graft(w)
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    a = compare_accept(oracle, gi, g, w, out, gpu)
+    assert 0 <= a[0] <= w.L
+    # beta = 0 reduces to DDTree: product-of-probabilities scores, and the tree is the top-B by path score
+    g0 = _graft(w, beta=0.0)
+    out0, gpu0 = gpu_round(g0, w, x)
+    w0 = gi.Workload(**{**w.__dict__, "beta": 0.0})
+    orc0 = oracle_round(oracle, w0, x, tb, saba_kw)
+    compare_round(oracle, w0, x, tb, saba_kw, gpu0, orc0)
+    n = gpu0["n_nodes"][0]
+    assert (gpu0["path_score"][0, 1:n] <= 0).all()
+
+
+@pytest.mark.parametrize("name,nseq", [("C2", 16), ("C3", 6), ("M", 6), ("C5", 4), ("C4", 3)])
+def test_config_full_size_sampled(name, nseq):
+    """Full-size launch configuration; the oracle checks a sample of sequences one by one, and the
+    invariants are checked on every sequence."""
+    w = gi.WORKLOADS[name]
+    g = _graft(w)
+    tb, saba_kw, keep = _setup(w, g)
+    # every sequence's inputs come from its own stream, so a sample can be generated without the rest
+    sample = sorted(set(np.linspace(0, w.batch - 1, nseq).astype(int).tolist()))
+    z = torch.empty((w.batch, w.L, w.V), dtype=torch.bfloat16, device="cuda")
+    h = torch.empty((w.batch, w.L, w.hidden_dim), dtype=torch.bfloat16, device="cuda")
+    root = torch.empty(w.batch, dtype=torch.int32)
+    hist = torch.empty(w.batch, dtype=torch.float32)
+    pref = torch.empty(w.batch, dtype=torch.int32)
+    xs = {}
+    for b in range(w.batch):
+        xb = gi.batch_inputs(w, b, b + 1)
+        z[b], h[b] = xb["logits"][0].cuda(), xb["hidden"][0].cuda()
+        root[b], hist[b], pref[b] = xb["root_token"][0], xb["hist"][0], xb["prefix_len"][0]
+        if b in sample:
+            xs[b] = xb
+    out = g.alloc_out(w.batch, debug=True)
+    g.build_trees(z, h, root.cuda(), hist.cuda(), pref.cuda(), None, out)
+    torch.cuda.synchronize()
+    gpu = out.cpu()
+    assert (gpu["status"] == 0).all()
+    for b in range(w.batch):
+        tree = {k: gpu[k][b] for k in ("n_nodes", "token", "parent", "depth", "position", "path_score", "mask")}
+        check_tree_invariants(tree, int(gpu["budget"][b]), w.L, None, int(root[b]), int(pref[b]))
+        assert gpu["n_nodes"][b] == gpu["budget"][b] + 1
+    excused = 0
+    for b in sample:
+        orc = oracle_round(oracle, w, xs[b], tb, saba_kw, threads=1)
+        one = {k: v[b:b + 1] for k, v in gpu.items()}
+        st = compare_round(oracle, w, xs[b], tb, saba_kw, one, orc)
+        excused += st["excused_tree"] + st["excused_budget"]
+    assert excused <= max(1, len(sample) // 3)
+    compare_accept(oracle, gi, g, w, out, gpu)
+    assert len(set(gpu["budget"].tolist())) > 1 or name in ("C2",)

@@ -9,6 +9,7 @@ import pytest
 import torch
 
 import oracle
+from helpers import check_tree_invariants
 
 RNG = np.random.default_rng(1234)
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
@@ -367,36 +368,6 @@ def test_select_special_cases():
 
 
 # ------------------------------------------------------------------ O5 emission
-def check_tree_invariants(o, budget, L, ids=None, root_token=None, prefix_len=None):
-    n = int(o["n_nodes"])
-    tok, par, dep, pos, msk = o["token"], o["parent"], o["depth"], o["position"], o["mask"]
-    Nmax, W = msk.shape
-    assert 1 <= n <= budget + 1 <= Nmax
-    assert par[0] == -1 and dep[0] == 0
-    kids = {}
-    for i in range(1, n):
-        p = int(par[i])
-        assert 0 <= p < i and dep[i] == dep[p] + 1 and 1 <= dep[i] <= L  # prefix-closed, level order
-        kids.setdefault(p, []).append(int(tok[i]))
-        row = 0
-        for w in range(W):
-            row |= int(msk[i, w]) << (32 * w)
-        prow = 0
-        for w in range(W):
-            prow |= int(msk[p, w]) << (32 * w)
-        assert row == prow | (1 << i) and bin(row).count("1") == dep[i] + 1 and row & 1
-    assert int(msk[0, 0]) == 1 and not msk[0, 1:].any()
-    for p, ts in kids.items():
-        assert len(set(ts)) == len(ts)  # sibling tokens distinct
-    assert list(dep[:n]) == sorted(dep[:n])
-    if prefix_len is not None:
-        assert np.array_equal(pos[:n], prefix_len - 1 + dep[:n])
-    if root_token is not None:
-        assert tok[0] == root_token
-    assert (tok[n:] == -1).all() and (par[n:] == -1).all() and (dep[n:] == -1).all() and (pos[n:] == -1).all()
-    assert (o["path_score"][n:] == 0).all() and not msk[n:].any()
-
-
 def test_emit_invariants_and_order():
     L, K, V = 4, 3, 50
     g = np.random.default_rng(11)
