@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the GRAFT draft-tree round on B200.
+
+One step = one whole round over one batch of synthetic drafter outputs: graft_build_trees (vocab pass ->
+SABA -> TDES edges -> best-first selection -> emission) followed by graft_accept.  Metric: trees/s (and
+microseconds per round) at batch 64, L = 16, V = 151,936 bf16 (workload "M").  Prints one JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload M] [--impl graft|reference]
+
+N > 1 (under torchrun): every rank runs the same per-GPU batch on its own sequences (weak scaling, no
+data-path collective); the time is the max over ranks.  --impl reference times the CPU oracle, as it stands,
+on the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import graft_inputs as gi  # noqa: E402
+
+METRIC = "draft trees built and verified-walked per second (batch 64, L=16, V=151,936 bf16)"
+UNIT = "trees/s"
+# DRAM bytes (read + write) of one vocab-pass launch on workload M, from the ncu capture summarised in
+# profiles/; None until a capture exists.
+NCU_VOCAB_TRAFFIC_BYTES_M = None
+L2_BYTES = 126 * 1024 * 1024
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Reads SM clock, power and clock-event reasons through NVML while the benchmark runs (read-only)."""
+
+    def __init__(self, index: int, period_s: float = 0.005):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples = []  # (t, sm_mhz, reasons_bitmask, power_w)
+        self.stop_flag = False
+        self.max_mhz = None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                pw = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                self.samples.append((time.perf_counter(), mhz, int(reasons), pw))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def summary(self, t0, t1):
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+                 0x80: "hw_power_brake", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting",
+                 0x10: "sync_boost"}
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "window": "none"}
+        win = [s for s in self.samples if t0 <= s[0] <= t1]
+        window = "timed"
+        if len(win) < 3:
+            win, window = self.samples, "whole run"
+        bits = 0
+        for s in win:
+            bits |= s[2]
+        return {"sm_mhz": float(np.median([s[1] for s in win])), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(n for b, n in names.items() if bits & b), "samples": len(win), "window": window,
+                "power_w_max": max(s[3] for s in win)}
+
+
+def _dist_setup(n_gpus):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    return rank, world, local
+
+
+def _host_inputs(w, lo, hi, n_buf):
+    """n_buf independent input sets for sequences lo..hi-1 (set k uses sequence index b + k * 1_000_003)."""
+    sets = []
+    for k in range(n_buf):
+        off = k * 1_000_003
+        parts = [gi.batch_inputs(w, b + off, b + off + 1) for b in range(lo, hi)]
+        s = {key: torch.cat([p[key] for p in parts]) for key in ("logits", "hidden", "root_token", "hist", "prefix_len")}
+        s["seq_ids"] = [b + off for b in range(lo, hi)]
+        sets.append(s)
+    return sets
+
+
+def run_graft(args):
+    from paper_2608_20375_b200 import Graft, BF16, F32, shard_range  # noqa: F401
+    import oracle  # CPU-baseline leg only
+
+    rank, world, local = _dist_setup(args.gpus)
+    w = gi.WORKLOADS[args.workload]
+    batch = w.batch  # per GPU (weak scaling)
+    lo = rank * batch
+    dev = torch.device("cuda", local)
+    dt = {"f32": 0, "bf16": 1}
+    g = Graft(w.V, w.L, w.K, w.m, w.hidden_dim, batch, w.budget_min, w.budget_max, w.budget_step, w.beta, 1,
+              dt[w.logits_dtype], dt[w.hidden_dtype])
+    tb = gi.tdes_tables(w)
+    P, Ct, u = tb["P"].to(dev), tb["C"].to(dev), tb["u"].to(dev)
+    g.set_tdes_tables(P, Ct, u, tb["s"])
+    saba_kw = gi.saba_defaults(w)
+    g.set_saba(**saba_kw)
+
+    logits_bytes = batch * w.L * w.V * (2 if w.logits_dtype == "bf16" else 4)
+    n_buf = max(2, int(np.ceil(2.5 * L2_BYTES / logits_bytes)))  # rotating sets: > 2.5x L2 in total
+    n_buf = min(n_buf, 8)
+    host_sets = _host_inputs(w, lo, lo + batch, n_buf)
+    dev_sets = [{k: (v.to(dev) if torch.is_tensor(v) else v) for k, v in s.items()} for s in host_sets]
+    fixed = None if w.fixed_budget is None else torch.full((batch,), w.fixed_budget, dtype=torch.int32, device=dev)
+    outs = [g.alloc_out(batch) for _ in range(n_buf)]
+    a_len = torch.empty(batch, dtype=torch.int32, device=dev)
+    a_path = torch.empty((batch, w.L), dtype=torch.int32, device=dev)
+    bonus = torch.empty(batch, dtype=torch.int32, device=dev)
+
+    def build(k):
+        s = dev_sets[k]
+        g.build_trees(s["logits"], s["hidden"], s["root_token"], s["hist"], s["prefix_len"], fixed, outs[k])
+
+    # target next-token ids per input set: drawn independently of the trees, indexed by each node's depth
+    tn_dev, tn_host = [], []
+    for k in range(n_buf):
+        build(k)
+        torch.cuda.synchronize()
+        depth = outs[k].depth.cpu().numpy()
+        tn = np.stack([gi.target_next_from_depth(gi.target_tokens(w, sid), depth[i])
+                       for i, sid in enumerate(host_sets[k]["seq_ids"])])
+        tn_host.append(torch.from_numpy(tn).pin_memory())
+        tn_dev.append(torch.from_numpy(tn).to(dev))
+
+    def step(i):
+        k = i % n_buf
+        build(k)
+        g.accept(outs[k], tn_dev[k], a_len, a_path, bonus)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    g.set_timing(True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    launches0 = g.launch_count()
+    t_wall0 = time.perf_counter()
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    torch.cuda.synchronize()
+    t_wall1 = time.perf_counter()
+    barrier()
+    launches = g.launch_count() - launches0
+    ms_total = ev0.elapsed_time(ev1)
+    n_t, vocab_ms, tdes_ms, tree_ms = g.read_timing()
+    g.set_timing(False)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * batch / (ms_step * 1e-3)
+    mean_accept = float(a_len.float().mean().item())
+    status_or = int(torch.stack([o.status for o in outs]).max().item())
+
+    # ---- end to end through the host-buffer entry point (host <-> device copies inside the timed region)
+    e2e_steps = max(3, min(args.steps, 10))
+    pinned = [{k: v.pin_memory() for k, v in s.items() if torch.is_tensor(v)} for s in host_sets[:2]]
+    h_out = g.alloc_out(batch, device="cpu", pinned=True)
+    h_alen = torch.empty(batch, dtype=torch.int32).pin_memory()
+    h_fixed = None if fixed is None else fixed.cpu().pin_memory()
+    d_out = outs[0]
+
+    def e2e_step(i):
+        s = pinned[i % len(pinned)]
+        g.build_trees_host(s["logits"], s["hidden"], s["root_token"], s["hist"], s["prefix_len"], h_fixed, h_out)
+        # the verifier's answer arrives on the host; the walk runs on the device copy of the tree it was built from
+        tnd = tn_host[i % len(pinned)].to(dev, non_blocking=True)
+        for name in ("n_nodes", "token", "parent"):
+            getattr(d_out, name).copy_(getattr(h_out, name), non_blocking=True)
+        g.accept(d_out, tnd, a_len, a_path, bonus)
+        h_alen.copy_(a_len, non_blocking=True)
+        torch.cuda.synchronize()
+
+    for i in range(2):
+        e2e_step(i)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    s0 = pinned[0]
+    h2d = sum(s0[k].numel() * s0[k].element_size() for k in ("logits", "hidden", "root_token", "hist", "prefix_len"))
+    h2d += tn_host[0].numel() * 4 + sum(getattr(h_out, n).numel() * 4 for n in ("n_nodes", "token", "parent"))
+    d2h = sum(getattr(h_out, n).numel() * getattr(h_out, n).element_size() for n in
+              ("n_nodes", "budget", "status", "token", "parent", "depth", "position", "path_score", "mask")) + batch * 4
+    sampler.stop_flag = True
+    sampler.join(timeout=2)
+
+    if rank != 0:
+        return
+    peak, peak_kind = _peaks()
+    vocab_s = vocab_ms * 1e-3 / max(1, n_t)
+    achieved = logits_bytes / vocab_s / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "us_per_round": ms_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32 (on bf16 logits; fp64 for the SABA scalars)", "data": "synthetic",
+        "config": {"workload": f"{w.name}: batch {batch} per GPU, L={w.L}, V={w.V} {w.logits_dtype} logits, "
+                               f"hidden d={w.hidden_dim} {w.hidden_dtype}, K={w.K}, m={w.m}, beta={w.beta}, SABA budgets "
+                               f"[{w.budget_min},{w.budget_max}] step {w.budget_step}, build_trees + accept",
+                   "parallelism": f"batch-sharded x{world}, no collective",
+                   "l2_policy": f"{n_buf} rotating input sets of {logits_bytes / 1e6:.0f} MB each (> L2 of 126 MB)"},
+        "gpu_launches": launches,
+        "kernel_ms": {"vocab_pass": vocab_ms / max(1, n_t), "tdes_edges": tdes_ms / max(1, n_t),
+                      "tree": tree_ms / max(1, n_t), "calls_averaged": n_t},
+        "roofline": {"bound": "hbm", "kernel": "vocab_pass_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "frac_of_nominal_8000": achieved / 8000.0, "algorithmic_bytes": logits_bytes,
+                     "traffic": NCU_VOCAB_TRAFFIC_BYTES_M if w.name == "M" else None},
+        "e2e": {"value": world * batch / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3, "steps": e2e_steps,
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+        "clocks": sampler.summary(t_wall0, t_wall1),
+        "mean_accepted_len": mean_accept, "status_or": status_or,
+    }
+    # ---- CPU baseline: the oracle as it stands, on this machine's host cores, on a bounded sample
+    if world == 1 and not args.no_cpu_baseline:
+        cores = os.cpu_count() or 1
+        threads = min(cores, 32)
+        n_seq = min(batch, max(threads, 2 * threads if w.V < 100000 else threads))
+        s = host_sets[0]
+        sub = {k: s[k][:n_seq] for k in ("logits", "hidden", "root_token", "hist", "prefix_len")}
+        sub["fixed_budget"] = None if w.fixed_budget is None else torch.full((n_seq,), w.fixed_budget, dtype=torch.int32)
+        sp = oracle.SabaParams(**saba_kw)
+        t0 = time.perf_counter()
+        orc = oracle.build_trees(sub["logits"], sub["hidden"], sub["root_token"].numpy(), sub["hist"].numpy(),
+                                 sub["prefix_len"].numpy(),
+                                 None if sub["fixed_budget"] is None else sub["fixed_budget"].numpy(), sp,
+                                 (w.budget_min, w.budget_max, w.budget_step), tb["P"].numpy(), tb["C"].numpy(),
+                                 tb["u"].numpy(), tb["s"], w.beta, w.K, threads=threads)
+        for i in range(n_seq):
+            tn = gi.target_next_from_depth(gi.target_tokens(w, s["seq_ids"][i]), orc["depth"][i])
+            oracle.accept(int(orc["n_nodes"][i]), orc["token"][i], orc["parent"][i], tn, w.L)
+        dt_s = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": n_seq / dt_s, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"{n_seq} of the {batch} sequences of input set 0, one round each, "
+                                          f"{threads} threads, {dt_s:.1f} s"}
+    print(json.dumps(line))
+
+
+def run_reference(args):
+    """The oracle (plain C, fp64), as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank != 0:
+        return
+    import oracle
+    w = gi.WORKLOADS[args.workload]
+    cores = os.cpu_count() or 1
+    threads = min(cores, 32, w.batch)
+    n_seq = threads  # one sequence per thread and step: a bounded sample of the batch
+    tb = gi.tdes_tables(w)
+    saba_kw = gi.saba_defaults(w)
+    sp = oracle.SabaParams(**saba_kw)
+    sets = _host_inputs(w, 0, n_seq, 2)
+    P, Ct, u = tb["P"].numpy(), tb["C"].numpy(), tb["u"].numpy()
+    ys = [[gi.target_tokens(w, sid) for sid in s["seq_ids"]] for s in sets]
+
+    def step(i):
+        s = sets[i % 2]
+        fb = None if w.fixed_budget is None else np.full(n_seq, w.fixed_budget, np.int32)
+        orc = oracle.build_trees(s["logits"], s["hidden"], s["root_token"].numpy(), s["hist"].numpy(),
+                                 s["prefix_len"].numpy(), fb, sp, (w.budget_min, w.budget_max, w.budget_step), P, Ct, u,
+                                 tb["s"], w.beta, w.K, threads=threads)
+        for j in range(n_seq):
+            tn = gi.target_next_from_depth(ys[i % 2][j], orc["depth"][j])
+            oracle.accept(int(orc["n_nodes"][j]), orc["token"][j], orc["parent"][j], tn, w.L)
+
+    for i in range(args.warmup):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step(i)
+    dt_s = (time.perf_counter() - t0) / args.steps
+    value = n_seq / dt_s
+    sample = f"{n_seq} of the {w.batch} sequences per step, one round each, {threads} threads"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt_s * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name}: batch {w.batch}, L={w.L}, V={w.V} {w.logits_dtype} logits, hidden "
+                               f"d={w.hidden_dim}, K={w.K}, SABA budgets [{w.budget_min},{w.budget_max}]; CPU oracle on "
+                               f"a sample of {n_seq} sequences per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="M", choices=sorted(gi.WORKLOADS))
+    ap.add_argument("--impl", default="graft", choices=["graft", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 10 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args)
+    else:
+        args.steps = 1000 if args.steps is None else args.steps
+        args.warmup = max(3, 20 if args.warmup is None else args.warmup)
+        run_graft(args)
+
+
+if __name__ == "__main__":
+    main()

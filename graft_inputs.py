@@ -169,8 +169,7 @@ def tdes_weights(V: int, E: int, m: int, L: int, seed: int, emb_dtype: str = "f3
 def saba_defaults(w: Workload) -> dict:
     """Synthetic SABA parameters (the fitted ones are not published) and the verification-cost table."""
     return dict(phi_conf=-160.0, phi_degen=20.0, phi_hist=-5.0, phi_bias=200.0, tau_min=8.0, cost_mode=1,
-                c0=0.0, c1=0.0, c2=0.0, pts_n=[0.0, 64.0, float(w.budget_max)],
-                pts_t=[18.0, 18.0, 18.0 + 0.02 * max(0.0, w.budget_max - 64.0)])
+                c0=0.0, c1=0.0, c2=0.0, pts_n=[0.0, 64.0, 1024.0], pts_t=[18.0, 18.0, 18.0 + 0.02 * (1024.0 - 64.0)])
 
 
 def target_tokens(w: Workload, b: int, logits_b: torch.Tensor | None = None) -> np.ndarray:

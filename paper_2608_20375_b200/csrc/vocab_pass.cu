@@ -562,15 +562,20 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
             }
             if (finish && warp == 0) {
                 // lse = (C + log2 S) ln 2, in double; every lane of warp 0 holds the same Cd, Sd, Vm
-                const double lse_d = (Cd + log2(Sd)) * kLn2;
-                const float lse_f = (float)lse_d;
+                // The stream accumulates 2^(z c - ref) with c = fp32(log2 e), so (C + log2 S) ln 2 is the
+                // log-sum-exp of the logits scaled by a = c ln 2 = 1 + 1.3e-8.  To first order that adds
+                // (a - 1) E_q[z]; the largest logit stands in for the mean under q (the difference is a few
+                // units times 1e-8).
                 const float vmax = __uint_as_float(bits_from_ord(Vm));
+                const double a_minus_1 = (double)kLog2e * kLn2 - 1.0;
+                const double lse_d = (Cd + log2(Sd)) * kLn2 - a_minus_1 * (double)vmax;
+                const float lse_f = (float)lse_d;
                 const bool bad = !(Sd > 0.0) || !(Sd < 1e300) || Vm == 0u || vmax == INFINITY || vmax == -INFINITY ||
                                  nk < p.K;
                 if (lane < p.K) {
                     const uint64_t key = lane < nk ? sh->outk[lane] : 0ull;
                     p.topk_id[(size_t)sg.row * p.K + lane] = lane < nk ? (int32_t)key_id(key) : -1;
-                    p.topk_lp[(size_t)sg.row * p.K + lane] = lane < nk ? key_value(key) - lse_f : 0.f;
+                    p.topk_lp[(size_t)sg.row * p.K + lane] = lane < nk ? (float)((double)key_value(key) - lse_d) : 0.f;
                 }
                 if (lane == 0) {
                     p.lse[sg.row] = lse_f;

@@ -49,7 +49,8 @@ def _vocab_case(z, K, dtype):
     fin = np.isfinite(b)
     assert np.array_equal(np.isneginf(a), np.isneginf(b))
     assert np.abs(a[fin] - b[fin]).max(initial=0) <= EPS
-    assert np.abs(lse[good, 0] - o_lse[good]).max(initial=0) <= EPS
+    # lse is returned as an fp32 number: allow its own rounding on top of EPS
+    assert np.all(np.abs(lse[good, 0] - o_lse[good]) <= EPS + np.spacing(np.abs(lse[good, 0])))
     g.destroy()
     return float(np.abs(lse[good, 0] - o_lse[good]).max(initial=0))
 
