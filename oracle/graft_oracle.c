@@ -255,18 +255,26 @@ int oracle_tdes_edges(const int32_t *topk_id /* [L,K] */, const float *topk_lp /
  * O4.  Best-first expansion (the "max-heap of candidate prefixes" of the DDTree paragraph,
  * ranked by the TDES path score of Eq. 13, stopped at B_t nodes, Sec. 3.1).  A prefix is a
  * tuple of candidate indices (c_1..c_l).  S(()) = 0; S(u) = fp32(S(parent) + edge).  The
- * frontier starts with the K depth-1 prefixes; each step removes the frontier maximum under
- * the total order (S descending, length ascending, tuple lexicographic ascending), adds it
+ * frontier starts with the K depth-1 prefixes; each step removes the frontier maximum, adds it
  * to the tree and inserts its K extensions.  The frontier is an explicit array scanned
  * linearly; no heap.
+ *
+ * The paper does not say how equal scores are ordered.  The total order used here is the one
+ * a heap of (score, insertion) pairs gives when every parent's children are pushed in the
+ * order of their edge scores:  path score descending; then length ascending; then the prefix
+ * whose parent was selected earlier (the root counts as selected first); then, under one
+ * parent, edge score descending and candidate rank ascending.
+ *
  * Output: sel_tuple [n_sel, L] (unused slots -1), sel_len, sel_S in pop order.
- * Pins: exhaustive enumeration for L,K <= 4 (top-B by path score when edges <= 0; top-B by
- * bottleneck key always); an independently written from-scratch frontier recomputation;
- * chain of top-1 tokens; complete tree when B >= number of prefixes.
+ * Pins: exhaustive enumeration for L,K <= 4 (a top-B set by path score when edges <= 0; a
+ * top-B set by bottleneck key always); an independently written from-scratch frontier
+ * recomputation; chain of top-1 tokens; complete tree when B >= number of prefixes.
  * ------------------------------------------------------------------------------------------ */
 typedef struct {
     float S;
+    float e;        /* the last edge's score */
     int32_t len;
+    int32_t ppop;   /* selection index of the parent: 0 = root, k = the k-th selected prefix */
     int8_t t[ORC_MAX_L];
 } orc_prefix;
 
@@ -274,9 +282,10 @@ static int orc_before(const orc_prefix *a, const orc_prefix *b) { /* does a pop 
     if (a->S > b->S) return 1;
     if (a->S < b->S) return 0;
     if (a->len != b->len) return a->len < b->len;
-    for (int i = 0; i < a->len; ++i)
-        if (a->t[i] != b->t[i]) return a->t[i] < b->t[i];
-    return 0;
+    if (a->ppop != b->ppop) return a->ppop < b->ppop;
+    if (a->e > b->e) return 1;
+    if (a->e < b->e) return 0;
+    return a->t[a->len - 1] < b->t[b->len - 1];
 }
 
 int oracle_select(const float *edge /* [L,K,K] */, int L, int K, int budget, int32_t *sel_tuple /* [budget,L] */,
@@ -289,8 +298,10 @@ int oracle_select(const float *edge /* [L,K,K] */, int L, int K, int budget, int
     for (int c = 0; c < K; ++c) {
         orc_prefix x;
         memset(&x, 0, sizeof x);
-        x.S = (float)(0.0f + edge[c]); /* depth 1, parent row 0 */
+        x.e = edge[c]; /* depth 1, parent row 0 */
+        x.S = (float)(0.0f + x.e);
         x.len = 1;
+        x.ppop = 0;
         x.t[0] = (int8_t)c;
         fr[nf++] = x;
     }
@@ -311,10 +322,12 @@ int oracle_select(const float *edge /* [L,K,K] */, int L, int K, int budget, int
             int par = x.t[x.len - 1];
             for (int c = 0; c < K; ++c) {
                 orc_prefix y = x;
-                volatile float sum = x.S + edge[((size_t)j * K + par) * K + c]; /* one fp32 rounding */
+                y.e = edge[((size_t)j * K + par) * K + c];
+                volatile float sum = x.S + y.e; /* one fp32 rounding */
                 y.S = sum;
                 y.t[y.len] = (int8_t)c;
                 y.len = x.len + 1;
+                y.ppop = n; /* x was the n-th selection */
                 fr[nf++] = y;
             }
         }

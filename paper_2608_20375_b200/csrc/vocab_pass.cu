@@ -286,13 +286,13 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
         if (lane == 0) {
             uint64_t policy = 0;
             if (p.use_hint) policy = l2_policy_evict_first();
-            uint32_t t = 0;
+            uint32_t t = 0, st = 0, ph = 1;  // ph: parity of the "empty" phase to wait for (first lap: none)
+            const uint32_t nst = (uint32_t)p.stages;
             for (long long qi = q0; qi < q1;) {
                 Seg sg = make_seg<BF16>(p, qi, q1);
                 qi += (sg.e1 - sg.e0 + kVpQuantum - 1) / kVpQuantum;
                 for (int tile = 0; tile < sg.ntiles; ++tile, ++t) {
-                    const uint32_t st = t % p.stages, use = t / p.stages;
-                    if (use > 0) mbar_wait_bounded(empty0 + 8 * st, (use - 1) & 1, &sh->abort_flag);
+                    if (t >= nst) mbar_wait_bounded(empty0 + 8 * st, ph, &sh->abort_flag);
                     uint32_t off = (uint32_t)tile * TILE;
                     uint32_t bytes = sg.body_bytes - off < (uint32_t)TILE ? sg.body_bytes - off : (uint32_t)TILE;
                     mbar_arrive_expect_tx(full0 + 8 * st, bytes);
@@ -300,6 +300,10 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
                         tma_load_1d_hint(smem_u32(ring + (size_t)st * TILE), sg.body + off, bytes, full0 + 8 * st, policy);
                     else
                         tma_load_1d(smem_u32(ring + (size_t)st * TILE), sg.body + off, bytes, full0 + 8 * st);
+                    if (++st == nst) {
+                        st = 0;
+                        ph ^= 1;
+                    }
                 }
             }
             if (sh->abort_flag) {
@@ -314,7 +318,8 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
         }
     } else {
         // ------------------------------ consumer warps -------------------------------------------
-        uint32_t t = 0;
+        uint32_t st = 0, ph = 0;  // ring position and parity of the "full" phase to wait for
+        const uint32_t nst = (uint32_t)p.stages;
         for (long long qi = q0; qi < q1;) {
             const Seg sg = make_seg<BF16>(p, qi, q1);
             qi += (sg.e1 - sg.e0 + kVpQuantum - 1) / kVpQuantum;
@@ -342,22 +347,26 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
                 }
             }
 
-            for (int tile = 0; tile < sg.ntiles; ++tile, ++t) {
-                const uint32_t st = t % p.stages, use = t / p.stages;
-                mbar_wait_bounded(full0 + 8 * st, use & 1, &sh->abort_flag);
-                const uint4* wb = (const uint4*)(ring + (size_t)st * TILE + (size_t)warp * WBLK);
-                const uint32_t off = (uint32_t)tile * TILE;
-                const uint32_t bytes = sg.body_bytes - off < (uint32_t)TILE ? sg.body_bytes - off : (uint32_t)TILE;
-                typename T::cm_t* slot = cmax + ((size_t)tile * NT + tid);
-                if (bytes == (uint32_t)TILE) {
-                    process_chunk<BF16, false>(wb, lane, 0, a, slot);
-                } else {
-                    int nv = ((int)bytes - warp * WBLK) / 16;
-                    nv = nv < 0 ? 0 : (nv > WBLK / 16 ? WBLK / 16 : nv);
-                    process_chunk<BF16, true>(wb, lane, nv, a, slot);
+            {
+                const int nfull = (int)(sg.body_bytes / TILE);
+                typename T::cm_t* slot = cmax + tid;
+                for (int tile = 0; tile < sg.ntiles; ++tile, slot += NT) {
+                    mbar_wait_bounded(full0 + 8 * st, ph, &sh->abort_flag);
+                    const uint4* wb = (const uint4*)(ring + (size_t)st * TILE + (size_t)warp * WBLK);
+                    if (tile < nfull) {
+                        process_chunk<BF16, false>(wb, lane, 0, a, slot);
+                    } else {
+                        int nv = ((int)(sg.body_bytes - (uint32_t)tile * TILE) - warp * WBLK) / 16;
+                        nv = nv < 0 ? 0 : (nv > WBLK / 16 ? WBLK / 16 : nv);
+                        process_chunk<BF16, true>(wb, lane, nv, a, slot);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty0 + 8 * st);
+                    if (++st == nst) {
+                        st = 0;
+                        ph ^= 1;
+                    }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * st);
             }
 
             // ---------------- segment epilogue -------------------------------------------------------

@@ -286,22 +286,24 @@ def _all_prefixes(edge):
     return out
 
 
-def _order_key(t, S):
-    return (-float(S), len(t), t)
+def _edge_of(edge, t):
+    return float(edge[len(t) - 1, t[-2] if len(t) > 1 else 0, t[-1]])
 
 
 def _best_first_rescan(edge, budget):
-    """Independent restatement: rebuild the frontier from the selected set at every step."""
+    """Independent restatement: rebuild the frontier from the selected set at every step.  Equal scores:
+    shorter prefix first, then the prefix whose parent was selected earlier, then under one parent the
+    larger edge score, then the lower candidate rank."""
     L, K, _ = edge.shape
     allp = _all_prefixes(edge)
     sel = []
-    chosen = {()}
-    for _ in range(budget):
-        frontier = [t for t in allp if t not in chosen and t[:-1] in chosen]
+    when = {(): 0}
+    for step in range(budget):
+        frontier = [t for t in allp if t not in when and t[:-1] in when]
         if not frontier:
             break
-        best = min(frontier, key=lambda t: _order_key(t, allp[t][0]))
-        chosen.add(best)
+        best = min(frontier, key=lambda t: (-float(allp[t][0]), len(t), when[t[:-1]], -_edge_of(edge, t), t[-1]))
+        when[best] = step + 1
         sel.append(best)
     return sel
 
@@ -333,8 +335,11 @@ def test_select_against_exhaustive_enumeration(L, K, budget, mono, seed):
     if mono:
         # all edges <= 0: the selection is the global top-B by path score (DDTree's rule),
         # and exp(S) is the product of the edge probabilities
-        ranked = sorted(allp, key=lambda t: _order_key(t, allp[t][0]))[: len(got)]
-        assert sorted(got) == sorted(ranked)
+        smin = min(float(allp[t][0]) for t in got)
+        smax_rest = max([float(v[0]) for t, v in allp.items() if t not in got], default=-np.inf)
+        assert smin >= smax_rest
+        assert sorted(float(allp[t][0]) for t in got) == sorted((float(v[0]) for v in allp.values()), reverse=True)[
+            : len(got)][::-1]
         for t in got[:5]:
             prod = math.prod(math.exp(float(edge[d, t[d - 1] if d else 0, t[d]])) for d in range(len(t)))
             assert abs(math.exp(float(allp[t][0])) - prod) < 1e-5
@@ -355,10 +360,25 @@ def test_select_special_cases():
     tup, ln, S = oracle.select(e2, 1)
     assert ln.tolist() == [1] and tup[0, 0] == int(np.argmax(e2[0, 0])) and S[0] == e2[0, 0].max()
     assert len(oracle.select(e2, 0)[1]) == 0
-    # all scores equal: order is (length, tuple) ascending
+    # all scores equal: shorter first, then earlier-selected parent, then candidate rank
     e3 = np.zeros((3, 2, 2), np.float32)
     tup, ln, S = oracle.select(e3, 6)
     assert [tuple(t[:n]) for t, n in zip(tup, ln)] == [(0,), (1,), (0, 0), (0, 1), (1, 0), (1, 1)]
+    # equal path scores, different parents: the prefix whose parent was selected earlier goes first, even
+    # when it is lexicographically later
+    e5 = np.full((2, 2, 2), -9.0, np.float32)
+    e5[0, 0] = [-1.0, 0.0]          # (1,) is selected first, then (0,)
+    e5[1, 1, 0] = -5.0              # (1,0): 0 - 5
+    e5[1, 0, 0] = -4.0              # (0,0): -1 - 4
+    tup, ln, S = oracle.select(e5, 3)
+    assert [tuple(t[:n]) for t, n in zip(tup, ln)] == [(1,), (0,), (1, 0)] and S[2] == -5.0
+    # equal path scores under one parent although the edges differ (4e7 + 1 and 4e7 + 2 both round to 4e7):
+    # the larger edge first, here the higher rank
+    e6 = np.full((2, 2, 2), -9.0, np.float32)
+    e6[0, 0] = [4.0e7, -1.0]
+    e6[1, 0] = [1.0, 2.0]
+    tup, ln, S = oracle.select(e6, 2)
+    assert [tuple(t[:n]) for t, n in zip(tup, ln)] == [(0,), (0, 1)] and S[1] == np.float32(4.0e7)
     # the parent row is the PARENT's candidate index: make child 1 great only under parent 1
     e4 = np.full((2, 2, 2), -5.0, np.float32)
     e4[0, 0] = [-1.0, -2.0]
@@ -454,7 +474,7 @@ def test_replay_check_accepts_own_tree_and_rejects_a_worse_one():
     # find a leaf to drop and a clearly worse frontier node to add
     allp = _all_prefixes(edge)
     frontier = [t for t in allp if t not in have and (t[:-1] == () or t[:-1] in have)]
-    worst_t = max(frontier, key=lambda t: _order_key(t, allp[t][0]))
+    worst_t = min(frontier, key=lambda t: float(allp[t][0]))
     last = tuple(int(x) for x in tup[-1][: ln[-1]])
     if worst_t[:-1] != last and allp[worst_t][0] < S[-1] - 1e-3:
         tup2[-1] = -1
