@@ -123,6 +123,7 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     const size_t o_cnt = take(B * L * sizeof(int));
     const size_t o_id = take(B * L * K * 4), o_lp = take(B * L * K * 4), o_lse = take(B * L * 4);
     const size_t o_rs = take(B * L * 4), o_edge = take(B * L * K * K * 4), o_cos = take(B * L * 8);
+    const size_t o_es = take(B * L * K * K * 4), o_ei = take(B * L * K * K);
     const size_t o_u = take(L * (size_t)cfg->m * 4), o_err = take(256);
     ctx->ws_bytes = off;
     if (cudaMalloc(&ctx->ws, ctx->ws_bytes) != cudaSuccess) {
@@ -147,6 +148,8 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     ctx->w_row_status = (int32_t*)(base + o_rs);
     ctx->w_edge = (float*)(base + o_edge);
     ctx->w_cos = (double*)(base + o_cos);
+    ctx->w_esort = (float*)(base + o_es);
+    ctx->w_eidx = (uint8_t*)(base + o_ei);
     ctx->d_u = (float*)(base + o_u);
     ctx->w_errflag = (int32_t*)(base + o_err);
     *out = ctx;
@@ -245,8 +248,8 @@ graft_status graft_tdes_edges(graft_ctx* ctx, int32_t batch, const int32_t* d_to
     if (!ctx || !d_topk_id || !d_topk_lp || !d_root_token || !d_edge) return GRAFT_ERR_INVALID_ARG;
     if (batch < 1 || batch > ctx->cfg.max_batch) return GRAFT_ERR_INVALID_ARG;
     if (ctx->cfg.beta != 0.0f && !ctx->tdes_set) return GRAFT_ERR_STATE;
-    if (tdes_edges_launch(ctx, batch, d_topk_id, d_topk_lp, d_root_token, nullptr, d_edge, (cudaStream_t)stream) !=
-        cudaSuccess)
+    if (tdes_edges_launch(ctx, batch, d_topk_id, d_topk_lp, d_root_token, nullptr, d_edge, ctx->w_esort, ctx->w_eidx,
+                          (cudaStream_t)stream) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     return GRAFT_OK;
 }
@@ -316,10 +319,11 @@ graft_status graft_build_trees(graft_ctx* ctx, int32_t batch, const void* d_logi
     if (ev) cudaEventRecord(ev[0], st);
     if (vp_launch(ctx, batch, d_logits, ids, lps, lse, ctx->w_row_status, st) != cudaSuccess) return GRAFT_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], st);
-    if (tdes_edges_launch(ctx, batch, ids, lps, d_root_token, ctx->w_row_status, edge, st) != cudaSuccess)
+    if (tdes_edges_launch(ctx, batch, ids, lps, d_root_token, ctx->w_row_status, edge, ctx->w_esort, ctx->w_eidx, st) !=
+        cudaSuccess)
         return GRAFT_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], st);
-    if (tree_launch(ctx, batch, ids, lps, ctx->w_row_status, edge, ctx->w_cos, d_root_token, d_hist, d_prefix_len,
+    if (tree_launch(ctx, batch, ids, lps, ctx->w_row_status, ctx->w_esort, ctx->w_eidx, ctx->w_cos, d_root_token, d_hist, d_prefix_len,
                     d_fixed_budget, out, st) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     if (ev) {

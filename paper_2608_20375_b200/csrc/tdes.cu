@@ -79,7 +79,9 @@ struct EdgeParams {
     const float* P;
     const float* C;
     const float* u;
-    float* edge;
+    float* edge;      // [batch, L, K, K] by (parent rank, child rank)
+    float* esort;     // same rows, each sorted by (edge descending, child rank ascending)
+    uint8_t* eidx;    // child rank of every sorted entry
     int L, K, m, V;
     float scale;  // s / sqrt(m)
     float beta;
@@ -96,6 +98,8 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
     const int n_par = (j == 0) ? 1 : K;
     const size_t row = (size_t)b * p.L + j;
     float* out = p.edge + row * K * K;
+    float* outs = p.esort + row * K * K;
+    uint8_t* outi = p.eidx + row * K * K;
     const int32_t* ids = p.topk_id + row * K;
     const float* lps = p.topk_lp + row * K;
 
@@ -103,9 +107,13 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
     const bool neutral = (p.beta == 0.0f) || (j == 0 && !p.root_edge) || bad;
     if (neutral) {
         // edge = log q exactly (the DDTree score of Eq. 3); bad rows get zeros
+        // (log q is already ordered by rank, so the sorted rows are the rows themselves)
         for (int i = threadIdx.x; i < K * K; i += 256) {
             int par = i / K, c = i % K;
-            out[i] = (bad || par >= n_par) ? 0.f : lps[c];
+            const float v = (bad || par >= n_par) ? 0.f : lps[c];
+            out[i] = v;
+            outs[i] = v;
+            outi[i] = (uint8_t)c;
         }
         return;
     }
@@ -159,7 +167,24 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
         const float mean = sum / (float)K;
-        if (c < K) out[(size_t)par * K + c] = (par < n_par) ? fmaf(p.beta, ft - mean, lp) : 0.f;
+        const float val = (par < n_par) ? fmaf(p.beta, ft - mean, lp) : 0.f;
+        if (c < K) out[(size_t)par * K + c] = val;
+        // the row again, sorted by (edge descending, child rank ascending): a 32-lane bitonic network on
+        // 64-bit keys; lanes beyond K hold the empty key 0 and sink to the end
+        uint64_t key = (c < K) ? (((uint64_t)ord_from_float(val) << 32) | (uint32_t)(31 - c)) : 0ull;
+#pragma unroll
+        for (int k = 2; k <= 32; k <<= 1) {
+#pragma unroll
+            for (int jj = k >> 1; jj > 0; jj >>= 1) {
+                const uint64_t other = __shfl_xor_sync(0xFFFFFFFFu, key, jj);
+                const bool keep_max = (((lane & k) == 0) == ((lane & jj) == 0));
+                key = keep_max ? (key > other ? key : other) : (key < other ? key : other);
+            }
+        }
+        if (lane < K) {
+            outs[(size_t)par * K + lane] = __uint_as_float(bits_from_ord((uint32_t)(key >> 32)));
+            outi[(size_t)par * K + lane] = (uint8_t)(31 - (uint32_t)(key & 0xFFu));
+        }
     }
 }
 
@@ -186,7 +211,7 @@ cudaError_t tdes_edges_configure(const graft_config& cfg) {
 
 cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                               const int32_t* d_root_token, const int32_t* d_row_status, float* d_edge,
-                              cudaStream_t st) {
+                              float* d_esort, uint8_t* d_eidx, cudaStream_t st) {
     const graft_config& cfg = ctx->cfg;
     EdgeParams p;
     p.topk_id = d_topk_id;
@@ -197,6 +222,8 @@ cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_i
     p.C = ctx->d_C;
     p.u = ctx->d_u;
     p.edge = d_edge;
+    p.esort = d_esort;
+    p.eidx = d_eidx;
     p.L = cfg.L;
     p.K = cfg.K;
     p.m = cfg.m;

@@ -53,7 +53,8 @@ struct TreeParams {
     const int32_t* topk_id;
     const float* topk_lp;
     const int32_t* row_status;
-    const float* edge;
+    const float* esort;   // [batch, L, K, K] edge rows sorted by (edge desc, child rank asc)
+    const uint8_t* eidx;  // child rank of each sorted entry
     const double* cosv;
     const int32_t* root_token;
     const float* hist;
@@ -68,18 +69,20 @@ struct TreeParams {
 constexpr int TREE_THREADS = 256;
 
 struct TreeSmem {
-    float* edge;         // [L*K*K]
-    float* S;            // [nmax]  path score, pop order
-    uint32_t* taken;     // [nmax]  children already selected (bit per candidate rank)
-    uint32_t* cur_key;   // [nmax]  ord(score) of the node's best unselected child, 0 = none
+    float* es;           // [L*K*K]  sorted edge rows
+    uint8_t* ei;         // [L*K*K]  child rank of each sorted entry
+    uint64_t* ent;       // [32*33]  frontier entry of node n at [(n & 31) * 33 + (n >> 5)], 0 = none
+    uint32_t* chmask;    // [nmax]   candidate ranks of the node's selected children, one bit each
+    int* cc;             // [nmax]   per-level scratch: child counts in level order, then their exclusive scan
+    uint32_t* stage;     // [8 warps * 32 rows * W] mask rows staged for coalesced stores
+    float* S;            // [nmax]   path score, selection order
     uint32_t* sortkey;   // [nmax]
-    int16_t* parent;     // [nmax]  pop-order index of the parent
-    int16_t* canon;      // [nmax]  level-order index of pop-order node n
-    int16_t* cparent;    // [nmax]  level-order parent, by level-order index
+    int16_t* parent;     // [nmax]   selection-order index of the parent
+    int16_t* canon;      // [nmax]   level-order index of selection-order node n
+    int16_t* cparent;    // [nmax]   level-order parent, by level-order index
     int16_t* lvl_list;   // [nmax]
     uint8_t* cand;       // [nmax]
     uint8_t* depth;      // [nmax]
-    uint8_t* cur_child;  // [nmax]
     int* lvl_count;      // [kMaxL + 2]
     int* lvl_start;      // [kMaxL + 2]
     int* lvl_fill;       // [kMaxL + 2]
@@ -93,16 +96,19 @@ __host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, TreeS
         off += (bytes + 15) & ~(size_t)15;
         return o;
     };
-    size_t o_edge = take((size_t)L * K * K * 4), o_S = take((size_t)nmax * 4), o_tk = take((size_t)nmax * 4),
-           o_ck = take((size_t)nmax * 4), o_sk = take((size_t)nmax * 4), o_par = take((size_t)nmax * 2),
+    size_t o_es = take((size_t)L * K * K * 4), o_ei = take((size_t)L * K * K), o_ent = take((size_t)32 * 33 * 8), o_chm = take((size_t)nmax * 4), o_cc = take((size_t)nmax * 4), o_stage = take((size_t)8 * 32 * ((nmax + 31) / 32) * 4),
+           o_S = take((size_t)nmax * 4), o_sk = take((size_t)nmax * 4), o_par = take((size_t)nmax * 2),
            o_can = take((size_t)nmax * 2), o_cp = take((size_t)nmax * 2), o_ll = take((size_t)nmax * 2),
-           o_cand = take(nmax), o_dep = take(nmax), o_cc = take(nmax), o_lc = take((kMaxL + 2) * 4),
-           o_ls = take((kMaxL + 2) * 4), o_lf = take((kMaxL + 2) * 4), o_sc = take(8 * 4);
+           o_cand = take(nmax), o_dep = take(nmax), o_lc = take((kMaxL + 2) * 4), o_ls = take((kMaxL + 2) * 4),
+           o_lf = take((kMaxL + 2) * 4), o_sc = take(8 * 4);
     if (s) {
-        s->edge = (float*)(base + o_edge);
+        s->es = (float*)(base + o_es);
+        s->ei = base + o_ei;
+        s->ent = (uint64_t*)(base + o_ent);
+        s->chmask = (uint32_t*)(base + o_chm);
+        s->cc = (int*)(base + o_cc);
+        s->stage = (uint32_t*)(base + o_stage);
         s->S = (float*)(base + o_S);
-        s->taken = (uint32_t*)(base + o_tk);
-        s->cur_key = (uint32_t*)(base + o_ck);
         s->sortkey = (uint32_t*)(base + o_sk);
         s->parent = (int16_t*)(base + o_par);
         s->canon = (int16_t*)(base + o_can);
@@ -110,7 +116,6 @@ __host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, TreeS
         s->lvl_list = (int16_t*)(base + o_ll);
         s->cand = base + o_cand;
         s->depth = base + o_dep;
-        s->cur_child = base + o_cc;
         s->lvl_count = (int*)(base + o_lc);
         s->lvl_start = (int*)(base + o_ls);
         s->lvl_fill = (int*)(base + o_lf);
@@ -130,32 +135,33 @@ __device__ __forceinline__ double saba_cost(const SabaDev& sp, double B, double 
     return sp.pts_t[sp.n_pts - 1];
 }
 
-// The best unselected child of node n under (score descending, rank ascending); executed by a full warp.
-__device__ __forceinline__ void compute_cursor(const TreeSmem& sm, int n, int L, int K, int lane) {
-    const int d = sm.depth[n];
-    uint32_t key = 0;
-    if (d < L && lane < K && !((sm.taken[n] >> lane) & 1u)) {
-        const float sc = sm.S[n] + sm.edge[((size_t)d * K + sm.cand[n]) * K + lane];
-        key = ord_from_float(sc);
-    }
-    const uint32_t kmax = __reduce_max_sync(0xFFFFFFFFu, key);
-    const uint32_t who = __ballot_sync(0xFFFFFFFFu, key == kmax && key != 0u);
-    if (lane == 0) {
-        sm.cur_key[n] = kmax;
-        sm.cur_child[n] = (uint8_t)(who ? __ffs(who) - 1 : 0);
-    }
+// Frontier entry: one per selected node, naming that node's best child not yet selected.  A plain 64-bit
+// maximum over the entries is the next node to select:
+//   bits 63..32  ord(path score of the child)                      -> score descending
+//   bits 30..25  32 - depth of the child                           -> then the shallower child
+//   bits 24..15  1023 - selection index of the parent              -> then the parent selected earlier
+//   bits 14..10  position of the child in the parent's sorted row  (under one parent the sorted row gives
+//   bits  9..5   candidate rank of the parent                       edge descending, rank ascending)
+//   bits  4..0   candidate rank of the child
+__device__ __forceinline__ uint64_t pack_entry(float score, int child_depth, int parent_sel, int pos, int parent_cand,
+                                               int child_cand) {
+    const uint32_t lo = ((uint32_t)(32 - child_depth) << 25) | ((uint32_t)(1023 - parent_sel) << 15) |
+                        ((uint32_t)pos << 10) | ((uint32_t)parent_cand << 5) | (uint32_t)child_cand;
+    return ((uint64_t)ord_from_float(score) << 32) | lo;
 }
 
-// Among frontier entries with equal score: the shallower child first, then the lexicographically smaller
-// prefix.  n1, n2 are the PARENTS of the competing children (distinct nodes).
-__device__ __forceinline__ bool pops_before(const TreeSmem& sm, int n1, int n2) {
-    const int d1 = sm.depth[n1], d2 = sm.depth[n2];
-    if (d1 != d2) return d1 < d2;
-    while (sm.parent[n1] != sm.parent[n2]) {
-        n1 = sm.parent[n1];
-        n2 = sm.parent[n2];
-    }
-    return sm.cand[n1] < sm.cand[n2];
+// Warp-wide maximum of a 64-bit key: one redux on the high word, then the low word of the (usually single)
+// lane that holds it.
+__device__ __forceinline__ uint64_t warp_max64(uint64_t x) {
+    const uint32_t hi = (uint32_t)(x >> 32), lo = (uint32_t)x;
+    const uint32_t hm = __reduce_max_sync(0xFFFFFFFFu, hi);
+    const uint32_t tie = __ballot_sync(0xFFFFFFFFu, hi == hm);
+    uint32_t lm;
+    if ((tie & (tie - 1)) == 0u)
+        lm = __shfl_sync(0xFFFFFFFFu, lo, __ffs(tie) - 1);
+    else
+        lm = __reduce_max_sync(0xFFFFFFFFu, hi == hm ? lo : 0u);
+    return ((uint64_t)hm << 32) | lm;
 }
 
 __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) {
@@ -167,7 +173,19 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     const graft_tree_out& o = p.out;
 
     // ---- status and budget ---------------------------------------------------------------------------
-    for (int i = tid; i < L * K * K; i += TREE_THREADS) sm.edge[i] = p.edge[(size_t)b * L * K * K + i];
+#ifdef GRAFT_TREE_PROF
+    long long t_prof0 = clock64(), t_prof1 = 0, t_prof2 = 0;
+#endif
+    {
+        const int ne = L * K * K;
+        if ((ne & 3) == 0) {
+            const float4* src = (const float4*)(p.esort + (size_t)b * ne);
+            for (int i = tid; i < ne / 4; i += TREE_THREADS) ((float4*)sm.es)[i] = src[i];
+        } else {
+            for (int i = tid; i < ne; i += TREE_THREADS) sm.es[i] = p.esort[(size_t)b * ne + i];
+        }
+        for (int i = tid; i < L * K * K; i += TREE_THREADS) sm.ei[i] = p.eidx[(size_t)b * L * K * K + i];
+    }
     if (warp == 0) {
         int st = 0;
         for (int j = lane; j < L; j += 32) st |= p.row_status[(size_t)b * L + j];
@@ -233,75 +251,78 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     }
     __syncthreads();
 
+#ifdef GRAFT_TREE_PROF
+    t_prof1 = clock64();
+#endif
     // ---- best-first expansion (warp 0) -----------------------------------------------------------------
     if (warp == 0) {
+        // Column `lane` of the entry table (nodes n with n & 31 == lane) belongs to this lane, which keeps the
+        // column's maximum in a register.  One step selects `cur`, the maximum entry: the parent's entry moves
+        // to its next sorted child and the new node gets an entry.  Only the parent's column changes, so the
+        // next maximum is the largest of (a) that column re-reduced by the 32 lanes together, (b) the new
+        // node's entry and (c) the maximum over all other columns, which does not depend on this step's
+        // updates and is reduced in the shadow of the loads.
+        constexpr int NSP = 33;
         const int budget = sm.scal[0];
         int st = sm.scal[2];
+        for (int i = lane; i < 32 * NSP; i += 32) sm.ent[i] = 0ull;
+        for (int i = lane; i < nmax; i += 32) sm.chmask[i] = 0u;
+        uint64_t best = 0ull;
         if (lane == 0) {
             sm.parent[0] = -1;
             sm.cand[0] = 0;
             sm.depth[0] = 0;
             sm.S[0] = 0.0f;
-            sm.taken[0] = 0u;
         }
         __syncwarp();
-        int n_sel = 0;
-        if (budget > 0) {
-            compute_cursor(sm, 0, L, K, lane);
-            __syncwarp();
+        if (lane == 0) {
+            best = pack_entry(0.0f + sm.es[0], 1, 0, 0, 0, sm.ei[0]);
+            sm.ent[0] = best;
         }
+        __syncwarp();
+        uint64_t cur = warp_max64(best);
+        int n_sel = 0;
         while (n_sel < budget) {
-            uint32_t best_key = 0;
-            int best_n = -1;
-            bool multi = false;
-            for (int n = lane; n <= n_sel; n += 32) {
-                const uint32_t k = sm.cur_key[n];
-                if (k > best_key) {
-                    best_key = k;
-                    best_n = n;
-                    multi = false;
-                } else if (k == best_key && k != 0u) {
-                    multi = true;
-                }
-            }
-            const uint32_t gmax = __reduce_max_sync(0xFFFFFFFFu, best_key);
-            if (gmax == 0u) {
+            const uint32_t hmax = (uint32_t)(cur >> 32), lmax = (uint32_t)cur;
+            if (hmax == 0u) {
                 st |= GRAFT_ST_FRONTIER_EMPTY;
                 break;
             }
-            const uint32_t tied = __ballot_sync(0xFFFFFFFFu, best_key == gmax);
-            const uint32_t anym = __ballot_sync(0xFFFFFFFFu, best_key == gmax && multi);
-            int win;
-            if (__popc(tied) == 1 && anym == 0u) {
-                win = __shfl_sync(0xFFFFFFFFu, best_n, __ffs(tied) - 1);
-            } else {
-                // equal scores: order by (depth ascending, prefix lexicographic ascending)
-                int mine = -1;
-                for (int n = lane; n <= n_sel; n += 32)
-                    if (sm.cur_key[n] == gmax && (mine < 0 || pops_before(sm, n, mine))) mine = n;
-#pragma unroll
-                for (int d = 16; d > 0; d >>= 1) {
-                    const int other = __shfl_xor_sync(0xFFFFFFFFu, mine, d);
-                    if (other >= 0 && (mine < 0 || pops_before(sm, other, mine))) mine = other;
-                }
-                win = mine;
-            }
-            const int c = sm.cur_child[win];
-            const int d = sm.depth[win] + 1;
-            const float s_new = sm.S[win] + sm.edge[((size_t)(d - 1) * K + sm.cand[win]) * K + c];
+            const int d = 32 - (int)((lmax >> 25) & 63u);  // depth of the selected child
+            const int n_par = 1023 - (int)((lmax >> 15) & 1023u);
+            const int pos = (int)((lmax >> 10) & 31u);
+            const int cpar = (int)((lmax >> 5) & 31u);
+            const int c = (int)(lmax & 31u);
+            const float s_new = __uint_as_float(bits_from_ord(hmax));
             const int n_new = ++n_sel;
-            __syncwarp();
+            const int colA = n_par & 31, slotA = n_par >> 5, colB = n_new & 31, slotB = n_new >> 5;
+            const uint64_t others = warp_max64(lane == colA ? 0ull : best);
+            // every lane reads the same few words (broadcasts) and its own entry of the parent's column
+            const bool adv = pos + 1 < K, deeper = d < L;
+            const int at1 = adv ? ((d - 1) * K + cpar) * K + pos + 1 : 0;
+            const int at2 = deeper ? (d * K + c) * K : 0;
+            const float sp = sm.S[n_par];
+            const float e1 = sm.es[at1], e2 = sm.es[at2];
+            const int i1 = sm.ei[at1], i2 = sm.ei[at2];
+            uint64_t col = sm.ent[colA * NSP + lane];
+            const uint64_t e_adv = adv ? pack_entry(sp + e1, d, n_par, pos + 1, cpar, i1) : 0ull;
+            const uint64_t e_new = deeper ? pack_entry(s_new + e2, d + 1, n_new, 0, c, i2) : 0ull;
             if (lane == 0) {
-                sm.parent[n_new] = (int16_t)win;
+                sm.ent[colA * NSP + slotA] = e_adv;
+                sm.ent[colB * NSP + slotB] = e_new;
+                sm.parent[n_new] = (int16_t)n_par;
                 sm.cand[n_new] = (uint8_t)c;
                 sm.depth[n_new] = (uint8_t)d;
                 sm.S[n_new] = s_new;
-                sm.taken[n_new] = 0u;
-                sm.taken[win] |= (1u << c);
+                sm.chmask[n_par] |= 1u << c;
             }
-            __syncwarp();
-            compute_cursor(sm, win, L, K, lane);
-            compute_cursor(sm, n_new, L, K, lane);
+            if (lane == slotA) col = e_adv;
+            if (colB == colA && lane == slotB) col = e_new;
+            const uint64_t colbest = warp_max64(col);
+            if (lane == colA) best = colbest;
+            if (lane == colB) best = e_new > best ? e_new : best;
+            cur = others > colbest ? others : colbest;
+            cur = e_new > cur ? e_new : cur;
             __syncwarp();
         }
         if (lane == 0) {
@@ -315,7 +336,13 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     }
     __syncthreads();
 
+#ifdef GRAFT_TREE_PROF
+    t_prof2 = clock64();
+#endif
     // ---- emission in level order -------------------------------------------------------------------------
+    // Level order = depth ascending, then the parent's level-order index, then candidate rank.  Level by level:
+    // the child counts of level d-1, laid out in level order, are scanned; a node of level d lands at
+    // (start of level d) + (children of earlier parents) + (selected siblings of lower rank).
     const int n_nodes = sm.scal[1];
     for (int n = tid; n < n_nodes; n += TREE_THREADS) atomicAdd(&sm.lvl_count[sm.depth[n]], 1);
     __syncthreads();
@@ -334,19 +361,38 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     }
     __syncthreads();
     for (int d = 1; d <= L; ++d) {
-        const int s0 = sm.lvl_start[d], cnt = sm.lvl_count[d];
-        if (cnt == 0) break;  // uniform: deeper levels are empty too
-        for (int i = tid; i < cnt; i += TREE_THREADS) {
-            const int n = sm.lvl_list[s0 + i];
-            sm.sortkey[n] = (uint32_t)sm.canon[sm.parent[n]] * 32u + sm.cand[n];
+        const int s_prev = sm.lvl_start[d - 1], n_prev = sm.lvl_count[d - 1];
+        const int s_cur = sm.lvl_start[d], n_cur = sm.lvl_count[d];
+        if (n_cur == 0) break;  // uniform: deeper levels are empty too
+        for (int i = tid; i < n_prev; i += TREE_THREADS) {
+            const int y = sm.lvl_list[s_prev + i];
+            sm.cc[sm.canon[y] - s_prev] = __popc(sm.chmask[y]);
         }
         __syncthreads();
-        for (int i = tid; i < cnt; i += TREE_THREADS) {
-            const int n = sm.lvl_list[s0 + i];
-            const uint32_t key = sm.sortkey[n];
-            int rank = 0;
-            for (int j = 0; j < cnt; ++j) rank += (sm.sortkey[sm.lvl_list[s0 + j]] < key) ? 1 : 0;
-            sm.canon[n] = (int16_t)(s0 + rank);
+        if (warp == 0) {  // exclusive scan of cc[0..n_prev): a contiguous chunk per lane, then a warp scan
+            const int ch = (n_prev + 31) / 32;
+            const int lo_i = lane * ch, hi_i = min(n_prev, lo_i + ch);
+            int sum = 0;
+            for (int i = lo_i; i < hi_i; ++i) sum += sm.cc[i];
+            int incl = sum;
+#pragma unroll
+            for (int o2 = 1; o2 < 32; o2 <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
+                if (lane >= o2) incl += t;
+            }
+            int run = incl - sum;
+            for (int i = lo_i; i < hi_i; ++i) {
+                const int v = sm.cc[i];
+                sm.cc[i] = run;
+                run += v;
+            }
+        }
+        __syncthreads();
+        for (int i = tid; i < n_cur; i += TREE_THREADS) {
+            const int x = sm.lvl_list[s_cur + i];
+            const int y = sm.parent[x];
+            sm.canon[x] = (int16_t)(s_cur + sm.cc[sm.canon[y] - s_prev] +
+                                    __popc(sm.chmask[y] & ((1u << sm.cand[x]) - 1u)));
         }
         __syncthreads();
     }
@@ -371,15 +417,46 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         o.d_path_score[ob + i] = 0.f;
     }
     __syncthreads();
-    for (int idx = tid; idx < nmax * W; idx += TREE_THREADS) {
-        const int i = idx / W, w = idx % W;
-        uint32_t bits = 0u;
-        if (i < n_nodes) {
-            for (int a = i; a >= 0 && (a >> 5) >= w; a = sm.cparent[a])
-                if ((a >> 5) == w) bits |= 1u << (a & 31);
+    // ancestor masks: each thread builds one row in its warp's staging tile (walking up, level-order indices
+    // only decrease, so the row is produced from its highest word down); the warp then stores its 32 rows,
+    // which are contiguous in the output, with coalesced writes
+    {
+        uint32_t* tile = sm.stage + (size_t)warp * 32 * W;
+        for (int i0 = warp * 32; i0 < nmax; i0 += TREE_THREADS) {
+            const int i = i0 + lane;
+            uint32_t* row = tile + lane * W;
+            if (i < n_nodes) {
+                int w = W - 1;
+                uint32_t bits = 0u;
+                for (int a = i; a >= 0; a = sm.cparent[a]) {
+                    const int wa = a >> 5;
+                    while (w > wa) {
+                        row[w] = bits;
+                        bits = 0u;
+                        --w;
+                    }
+                    bits |= 1u << (a & 31);
+                }
+                row[w] = bits;
+                for (--w; w >= 0; --w) row[w] = 0u;
+            } else {
+                for (int w = 0; w < W; ++w) row[w] = 0u;
+            }
+            __syncwarp();
+            const int rows = min(32, nmax - i0);
+            uint32_t* dst = o.d_mask + (ob + i0) * W;
+            for (int k = lane; k < rows * W; k += 32) dst[k] = tile[k];
+            __syncwarp();
         }
-        o.d_mask[ob * W + idx] = bits;
     }
+#ifdef GRAFT_TREE_PROF
+    __syncthreads();
+    if (tid == 0 && o.d_state) {
+        o.d_state[(size_t)b * 4 + 0] = (float)(t_prof1 - t_prof0);
+        o.d_state[(size_t)b * 4 + 1] = (float)(t_prof2 - t_prof1);
+        o.d_state[(size_t)b * 4 + 2] = (float)(clock64() - t_prof2);
+    }
+#endif
     if (tid == 0) {
         o.d_n_nodes[b] = n_nodes;
         o.d_budget[b] = sm.scal[0];
@@ -442,7 +519,7 @@ cudaError_t cosine_launch(graft_ctx* ctx, int batch, const void* d_hidden, doubl
 }
 
 cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
-                        const int32_t* d_row_status, const float* d_edge, const double* d_cos,
+                        const int32_t* d_row_status, const float* d_esort, const uint8_t* d_eidx, const double* d_cos,
                         const int32_t* d_root_token, const float* d_hist, const int32_t* d_prefix_len,
                         const int32_t* d_fixed_budget, const graft_tree_out* out, cudaStream_t st) {
     const graft_config& cfg = ctx->cfg;
@@ -450,7 +527,8 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     p.topk_id = d_topk_id;
     p.topk_lp = d_topk_lp;
     p.row_status = d_row_status;
-    p.edge = d_edge;
+    p.esort = d_esort;
+    p.eidx = d_eidx;
     p.cosv = d_cos;
     p.root_token = d_root_token;
     p.hist = d_hist;
