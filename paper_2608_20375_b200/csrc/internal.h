@@ -14,7 +14,8 @@ constexpr int kMaxCostPts = 16;
 // ---- vocab pass -----------------------------------------------------------------------------
 constexpr int kVpConsumerWarps = 8;
 constexpr int kVpConsumers = kVpConsumerWarps * 32;  // 256
-constexpr int kVpThreads = kVpConsumers + 32;        // + one producer warp
+constexpr int kVpEpiThreads = 128;                   // four epilogue warps
+constexpr int kVpThreads = kVpConsumers + kVpEpiThreads + 32;  // + one producer warp
 constexpr int kVpTileBytes = 16384;                  // one TMA bulk copy
 constexpr int kVpQuantum = 2048;                     // elements; granularity of the work partition
 constexpr int kVpCandCap = 1024;                     // candidate keys held in shared memory

@@ -72,6 +72,7 @@ struct TreeSmem {
     float* es;           // [L*K*K]  sorted edge rows
     uint8_t* ei;         // [L*K*K]  child rank of each sorted entry
     uint64_t* ent;       // [32*33]  frontier entry of node n at [(n & 31) * 33 + (n >> 5)], 0 = none
+    uint64_t* poplog;    // [nmax]   the entry that was selected as node n (node 0: the root's pseudo entry)
     uint32_t* chmask;    // [nmax]   candidate ranks of the node's selected children, one bit each
     int* cc;             // [nmax]   per-level scratch: child counts in level order, then their exclusive scan
     uint32_t* stage;     // [8 warps * 32 rows * W] mask rows staged for coalesced stores
@@ -96,7 +97,7 @@ __host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, TreeS
         off += (bytes + 15) & ~(size_t)15;
         return o;
     };
-    size_t o_es = take((size_t)L * K * K * 4), o_ei = take((size_t)L * K * K), o_ent = take((size_t)32 * 33 * 8), o_chm = take((size_t)nmax * 4), o_cc = take((size_t)nmax * 4), o_stage = take((size_t)8 * 32 * ((nmax + 31) / 32) * 4),
+    size_t o_es = take((size_t)L * K * K * 4), o_ei = take((size_t)L * K * K), o_ent = take((size_t)32 * 33 * 8), o_log = take((size_t)nmax * 8), o_chm = take((size_t)nmax * 4), o_cc = take((size_t)nmax * 4), o_stage = take((size_t)8 * 32 * ((nmax + 31) / 32) * 4),
            o_S = take((size_t)nmax * 4), o_sk = take((size_t)nmax * 4), o_par = take((size_t)nmax * 2),
            o_can = take((size_t)nmax * 2), o_cp = take((size_t)nmax * 2), o_ll = take((size_t)nmax * 2),
            o_cand = take(nmax), o_dep = take(nmax), o_lc = take((kMaxL + 2) * 4), o_ls = take((kMaxL + 2) * 4),
@@ -105,6 +106,7 @@ __host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, TreeS
         s->es = (float*)(base + o_es);
         s->ei = base + o_ei;
         s->ent = (uint64_t*)(base + o_ent);
+        s->poplog = (uint64_t*)(base + o_log);
         s->chmask = (uint32_t*)(base + o_chm);
         s->cc = (int*)(base + o_cc);
         s->stage = (uint32_t*)(base + o_stage);
@@ -266,55 +268,53 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         const int budget = sm.scal[0];
         int st = sm.scal[2];
         for (int i = lane; i < 32 * NSP; i += 32) sm.ent[i] = 0ull;
-        for (int i = lane; i < nmax; i += 32) sm.chmask[i] = 0u;
         uint64_t best = 0ull;
-        if (lane == 0) {
-            sm.parent[0] = -1;
-            sm.cand[0] = 0;
-            sm.depth[0] = 0;
-            sm.S[0] = 0.0f;
-        }
-        __syncwarp();
         if (lane == 0) {
             best = pack_entry(0.0f + sm.es[0], 1, 0, 0, 0, sm.ei[0]);
             sm.ent[0] = best;
+            sm.poplog[0] = (uint64_t)ord_from_float(0.0f) << 32;
         }
         __syncwarp();
         uint64_t cur = warp_max64(best);
         int n_sel = 0;
+        // Inside the loop a path score is never -0 (sums that start from +0), so the order-preserving map
+        // needs no zero canonicalisation here.
         while (n_sel < budget) {
             const uint32_t hmax = (uint32_t)(cur >> 32), lmax = (uint32_t)cur;
             if (hmax == 0u) {
                 st |= GRAFT_ST_FRONTIER_EMPTY;
                 break;
             }
-            const int d = 32 - (int)((lmax >> 25) & 63u);  // depth of the selected child
+            const int n_new = ++n_sel;
+            const uint32_t dm = (lmax >> 25) & 63u;  // 32 - depth of the selected child
+            const int d = 32 - (int)dm;
             const int n_par = 1023 - (int)((lmax >> 15) & 1023u);
             const int pos = (int)((lmax >> 10) & 31u);
             const int cpar = (int)((lmax >> 5) & 31u);
             const int c = (int)(lmax & 31u);
-            const float s_new = __uint_as_float(bits_from_ord(hmax));
-            const int n_new = ++n_sel;
             const int colA = n_par & 31, slotA = n_par >> 5, colB = n_new & 31, slotB = n_new >> 5;
             const uint64_t others = warp_max64(lane == colA ? 0ull : best);
             // every lane reads the same few words (broadcasts) and its own entry of the parent's column
             const bool adv = pos + 1 < K, deeper = d < L;
             const int at1 = adv ? ((d - 1) * K + cpar) * K + pos + 1 : 0;
             const int at2 = deeper ? (d * K + c) * K : 0;
-            const float sp = sm.S[n_par];
+            const uint32_t sp_o = ((const uint32_t*)sm.poplog)[2 * n_par + 1];  // ord(path score of the parent)
             const float e1 = sm.es[at1], e2 = sm.es[at2];
-            const int i1 = sm.ei[at1], i2 = sm.ei[at2];
+            const uint32_t i1 = sm.ei[at1], i2 = sm.ei[at2];
             uint64_t col = sm.ent[colA * NSP + lane];
-            const uint64_t e_adv = adv ? pack_entry(sp + e1, d, n_par, pos + 1, cpar, i1) : 0ull;
-            const uint64_t e_new = deeper ? pack_entry(s_new + e2, d + 1, n_new, 0, c, i2) : 0ull;
+            const float sp = __uint_as_float(sp_o ^ (~(uint32_t)((int32_t)sp_o >> 31) | 0x80000000u));
+            const float s_new = __uint_as_float(hmax ^ (~(uint32_t)((int32_t)hmax >> 31) | 0x80000000u));
+            const uint32_t u1 = __float_as_uint(sp + e1), u2 = __float_as_uint(s_new + e2);
+            const uint32_t h1 = u1 ^ ((uint32_t)((int32_t)u1 >> 31) | 0x80000000u);
+            const uint32_t h2 = u2 ^ ((uint32_t)((int32_t)u2 >> 31) | 0x80000000u);
+            const uint32_t l1 = ((lmax & ~31u) + (1u << 10)) | i1;
+            const uint32_t l2 = ((dm - 1u) << 25) | ((uint32_t)(1023 - n_new) << 15) | ((uint32_t)c << 5) | i2;
+            const uint64_t e_adv = adv ? (((uint64_t)h1 << 32) | l1) : 0ull;
+            const uint64_t e_new = deeper ? (((uint64_t)h2 << 32) | l2) : 0ull;
             if (lane == 0) {
                 sm.ent[colA * NSP + slotA] = e_adv;
                 sm.ent[colB * NSP + slotB] = e_new;
-                sm.parent[n_new] = (int16_t)n_par;
-                sm.cand[n_new] = (uint8_t)c;
-                sm.depth[n_new] = (uint8_t)d;
-                sm.S[n_new] = s_new;
-                sm.chmask[n_par] |= 1u << c;
+                sm.poplog[n_new] = cur;
             }
             if (lane == slotA) col = e_adv;
             if (colB == colA && lane == slotB) col = e_new;
@@ -344,7 +344,20 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     // the child counts of level d-1, laid out in level order, are scanned; a node of level d lands at
     // (start of level d) + (children of earlier parents) + (selected siblings of lower rank).
     const int n_nodes = sm.scal[1];
-    for (int n = tid; n < n_nodes; n += TREE_THREADS) atomicAdd(&sm.lvl_count[sm.depth[n]], 1);
+    for (int n = tid; n < nmax; n += TREE_THREADS) sm.chmask[n] = 0u;
+    __syncthreads();
+    for (int n = tid; n < n_nodes; n += TREE_THREADS) {  // unpack the selection log
+        const uint64_t e = sm.poplog[n];
+        const uint32_t lo = (uint32_t)e;
+        const int d = n == 0 ? 0 : 32 - (int)((lo >> 25) & 63u);
+        const int par = n == 0 ? -1 : 1023 - (int)((lo >> 15) & 1023u);
+        sm.parent[n] = (int16_t)par;
+        sm.cand[n] = (uint8_t)(lo & 31u);
+        sm.depth[n] = (uint8_t)d;
+        sm.S[n] = __uint_as_float(bits_from_ord((uint32_t)(e >> 32)));
+        if (n > 0) atomicOr(&sm.chmask[par], 1u << (lo & 31u));
+        atomicAdd(&sm.lvl_count[d], 1);
+    }
     __syncthreads();
     if (tid == 0) {
         int acc = 0;

@@ -4,31 +4,46 @@
 //
 // Shape of the kernel (sm_100a):
 //   * persistent grid, two CTAs per SM; the rows*V element stream is cut into equal contiguous shares,
-//     one per CTA, so a CTA sees at most two partial rows plus whole rows in between;
-//   * one producer warp feeds a shared-memory ring with 16 KiB TMA bulk copies (cp.async.bulk +
-//     mbarrier complete_tx); eight consumer warps read the ring with 16-byte shared loads;
-//   * per 32-element chunk a consumer lane takes a packed max (stored for the second stage, 2 bytes per
+//     one per CTA, so a CTA sees at most two partial rows plus whole rows in between ("segments");
+//   * warp roles: one producer warp feeds a shared-memory ring with 16 KiB TMA bulk copies (cp.async.bulk +
+//     mbarrier complete_tx); eight streaming warps read the ring with 16-byte shared loads; one epilogue
+//     warp finishes segment k while the streaming warps are already in segment k+1;
+//   * per 32-element chunk a streaming lane takes a packed max (stored for the second stage, 2 bytes per
 //     chunk), keeps a lazily rescaled reference exponent and adds 2^(z log2e - ref) with ex2.approx;
 //   * top-K needs no per-element work in the stream: after the segment, the K-th largest per-thread
 //     maximum is a lower bound T for the K-th largest element; only chunks whose stored max reaches T
 //     (about K of them) are re-read, their elements >= T become 64-bit keys (value desc, id asc) and the
 //     exact top-K is found by rank counting.  An overflow of the small key buffer (adversarial rows)
-//     falls back to an exact chunked selection;
+//     falls back to an exact sliced selection;
 //   * rows shared by several CTAs are merged by the last CTA to arrive (a counter, no waiting).
+// Every wait on an mbarrier is bounded; when one runs out the kernel raises an error flag and drains.
+#include <stdlib.h>
+
 #include "common.cuh"
 #include "internal.h"
+
+#ifndef GRAFT_VP_F32X2
+#define GRAFT_VP_F32X2 1  // packed fp32 pair arithmetic (fma.rn.f32x2 / add.rn.f32x2)
+#endif
 
 namespace graft {
 
 namespace {
 
-constexpr int NW = kVpConsumerWarps;
-constexpr int NT = kVpConsumers;
+#ifdef GRAFT_VP_PROF
+#define VP_T(i) do { long long _t = clock64(); if (blockIdx.x == 1 && lane == 0) atomicAdd(p.errflag + 2 + (i), (int)((_t - tprof) >> 4)); tprof = _t; } while (0)
+#else
+#define VP_T(i) do { } while (0)
+#endif
+
+constexpr int NW = kVpConsumerWarps;          // streaming warps
+constexpr int NT = kVpConsumers;              // streaming threads
+constexpr int PROD_WARP = NW + kVpEpiThreads / 32;  // warp index of the producer warp
 constexpr int TILE = kVpTileBytes;
-constexpr int WBLK = TILE / NW;  // bytes of a tile owned by one warp (2048)
+constexpr int WBLK = TILE / NW;               // bytes of a tile owned by one warp (2048)
 constexpr int VEC_PER_LANE = WBLK / 16 / 32;  // 4
-constexpr int CONS_BAR = 1;
 static_assert(VEC_PER_LANE == 4, "chunk layout assumes four 16-byte vectors per lane per tile");
+static_assert(kVpThreads == NT + kVpEpiThreads + 32, "thread count = streaming warps + epilogue warps + producer warp");
 
 template <bool BF16>
 struct VT;
@@ -51,7 +66,8 @@ struct VpParams {
     long long nq;  // quanta per row
     long long Q;   // quanta in total
     int stages;
-    int n_cmax;    // chunk-max slots in shared memory
+    int n_cmax;    // chunk-max slots per buffer (two buffers): 256 threads x max_tiles
+    int max_tiles; // slots per streaming thread
     VpRecord* records;
     int* row_counter;
     int32_t* topk_id;
@@ -60,6 +76,7 @@ struct VpParams {
     int32_t* row_status;
     int32_t* errflag;
     int use_hint;
+    int dbg;  // experiments only: 1 = stream without arithmetic, 2 = arithmetic without streaming, 3 = no epilogue
 };
 
 struct Seg {
@@ -84,8 +101,7 @@ __device__ __forceinline__ Seg make_seg(const VpParams& p, long long qi, long lo
     long long qr1 = qr0 + (qend - qi);
     if (qr1 > p.nq) qr1 = p.nq;
     s.e0 = (int)(qr0 * kVpQuantum);
-    long long e1 = qr1 * kVpQuantum;
-    s.e1 = e1 > p.V ? p.V : (int)e1;
+    s.e1 = qr1 == p.nq ? p.V : (int)(qr1 * kVpQuantum);  // the last quantum of a row also takes the remainder
     const char* a0 = p.logits + ((size_t)s.row * p.V + s.e0) * T::ESZ;
     const char* a1 = p.logits + ((size_t)s.row * p.V + s.e1) * T::ESZ;
     uintptr_t b0 = ((uintptr_t)a0 + 15) & ~(uintptr_t)15;
@@ -100,6 +116,45 @@ __device__ __forceinline__ Seg make_seg(const VpParams& p, long long qi, long lo
     s.e_tail0 = s.e_body0 + (int)(s.body_bytes / T::ESZ);
     s.ntiles = (int)((s.body_bytes + TILE - 1) / TILE);
     return s;
+}
+__device__ __forceinline__ int seg_quanta(const Seg& s) {
+    const int n = (s.e1 - s.e0) / kVpQuantum;  // a row's last quantum holds up to 2 * kVpQuantum - 1 elements
+    return n < 1 ? 1 : n;
+}
+
+
+// A CTA's share of the stream as a list of segments.  The share's last segment (usually a partial row that is
+// shared with the next CTA) is visited FIRST, so that the cross-CTA merge of shared rows happens early instead
+// of at the kernel's tail; the remaining segments follow in stream order.
+struct SegIter {
+    long long q0, q1, qi, q_last;  // q_last: first quantum of the share's last segment
+    int state;                     // 0: emit the last segment, 1: walk [q0, q_last)
+};
+template <bool BF16>
+__device__ __forceinline__ SegIter seg_iter_begin(const VpParams& p, long long q0, long long q1) {
+    SegIter it;
+    it.q0 = q0;
+    it.q1 = q1;
+    it.qi = q0;
+    // the last segment starts at the last row boundary inside the share (or at q0)
+    const long long r_last = (q1 - 1) / p.nq;
+    const long long b = r_last * p.nq;
+    it.q_last = b > q0 ? b : q0;
+    it.state = 0;
+    return it;
+}
+template <bool BF16>
+__device__ __forceinline__ bool seg_iter_next(const VpParams& p, SegIter& it, Seg& sg) {
+    if (it.q0 >= it.q1) return false;
+    if (it.state == 0) {
+        sg = make_seg<BF16>(p, it.q_last, it.q1);
+        it.state = 1;
+        return true;
+    }
+    if (it.qi >= it.q_last) return false;
+    sg = make_seg<BF16>(p, it.qi, it.q_last);
+    it.qi += seg_quanta(sg);
+    return true;
 }
 
 __device__ __forceinline__ float load_elem_f32(const char* p, bool bf16) {
@@ -124,6 +179,36 @@ __device__ __forceinline__ float acc_begin_chunk(Acc& a, float cm) {
     }
     return (a.ref == -INFINITY) ? 0.0f : -a.ref;
 }
+
+// (c, s) pairs stand for s * 2^c; merge two of them
+__device__ __forceinline__ void merge_cs(float& c, float& s, float c2, float s2) {
+    const float cn = fmaxf(c, c2);
+    const float f1 = (c == -INFINITY) ? 0.f : ex2_approx(c - cn);
+    const float f2 = (c2 == -INFINITY) ? 0.f : ex2_approx(c2 - cn);
+    s = s * f1 + s2 * f2;
+    c = cn;
+}
+
+#if GRAFT_VP_F32X2
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+#endif
 
 template <bool BF16, bool GUARD>
 __device__ __forceinline__ void process_chunk(const uint4* __restrict__ wb, int lane, int nvalid_vec, Acc& a,
@@ -159,6 +244,37 @@ __device__ __forceinline__ void process_chunk(const uint4* __restrict__ wb, int 
     uint32_t o = ord_from_float(cm);
     a.tmo = o > a.tmo ? o : a.tmo;
     const float nref = acc_begin_chunk(a, cm);
+#if GRAFT_VP_F32X2
+    const uint64_t c2 = pack2(kLog2e, kLog2e), r2 = pack2(nref, nref);
+    uint64_t acc0 = 0ull, acc1 = 0ull;  // two (+0, +0) pairs
+#pragma unroll
+    for (int i = 0; i < VEC_PER_LANE; ++i) {
+        const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+        if (BF16) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint64_t x2 = pack2(__uint_as_float(w[k] << 16), __uint_as_float(w[k] & 0xFFFF0000u));
+                float t0, t1;
+                unpack2(fma2(x2, c2, r2), t0, t1);
+                const uint64_t e2 = pack2(ex2_approx(t0), ex2_approx(t1));
+                if (k & 1)
+                    acc1 = add2(acc1, e2);
+                else
+                    acc0 = add2(acc0, e2);
+            }
+        } else {
+            float t0, t1, t2, t3;
+            unpack2(fma2(pack2(__uint_as_float(w[0]), __uint_as_float(w[1])), c2, r2), t0, t1);
+            unpack2(fma2(pack2(__uint_as_float(w[2]), __uint_as_float(w[3])), c2, r2), t2, t3);
+            acc0 = add2(acc0, pack2(ex2_approx(t0), ex2_approx(t1)));
+            acc1 = add2(acc1, pack2(ex2_approx(t2), ex2_approx(t3)));
+        }
+    }
+    float s0, s1, s2, s3;
+    unpack2(acc0, s0, s1);
+    unpack2(acc1, s2, s3);
+    a.s += (s0 + s1) + (s2 + s3);
+#else
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
     for (int i = 0; i < VEC_PER_LANE; ++i) {
@@ -184,114 +300,132 @@ __device__ __forceinline__ void process_chunk(const uint4* __restrict__ wb, int 
         }
     }
     a.s += (s0 + s1) + (s2 + s3);
+#endif
 }
 
 // ---- shared-memory control block ---------------------------------------------------------------
 struct __align__(16) VpShared {
-    uint64_t cand[kVpCandCap];
+    uint64_t cand[kVpCandCap];  // epilogue warp only
     uint64_t outk[kMaxK];
     uint32_t hits[kVpHitCap];
-    uint32_t tmax[NT];
-    float wc[NW], ws[NW];
-    uint32_t wv[NW];
-    int ncand, nhits, overflow;
-    uint32_t T;
-    float segC, segS;
-    uint32_t segV;
-    int is_last;
+    uint32_t tmax[2][NT];       // per-thread maxima of a finished segment, double-buffered by segment parity
+    float wc[2][NW], ws[2][NW];
+    uint16_t hthreads[NT];      // epilogue warp only: streaming threads whose maximum reaches T
+    int nhits, ncand, nht, ovf;  // epilogue group only
+    uint32_t Tv;
     volatile int abort_flag;
 };
 
-__device__ __forceinline__ void cons_bar() { named_bar_sync(CONS_BAR, NT); }
+__device__ __forceinline__ void epi_bar() { named_bar_sync(2, kVpEpiThreads); }
 
-// Exact top-K of cand[0..n) by rank counting; result sorted descending in outk[0..min(n,K)).
-// Keys are distinct (ids are), so ranks are a permutation.  Ends with a consumer barrier.
-__device__ void select_topk(VpShared* sh, int n, int K, int tid) {
-    for (int i = tid; i < n; i += NT) {
+// ---- epilogue-warp helpers (32 threads, warp-synchronous) ----------------------------------------------
+// Append `key` for the lanes with pred set; returns the new count.  Entries beyond the capacity are dropped
+// and *overflow is raised.
+__device__ __forceinline__ int warp_append(uint64_t* buf, int n, int cap, bool pred, uint64_t key, int lane,
+                                           int* overflow) {
+    const uint32_t m = __ballot_sync(0xFFFFFFFFu, pred);
+    if (pred) {
+        const int pos = n + __popc(m & ((1u << lane) - 1u));
+        if (pos < cap)
+            buf[pos] = key;
+        else
+            *overflow = 1;
+    }
+    n += __popc(m);
+    if (n > cap) {
+        *overflow = 1;
+        n = cap;
+    }
+    return n;
+}
+
+// Exact top-K of cand[0..n) by rank counting; result sorted descending in outk[0..min(n,K)).  Keys are
+// distinct (ids are), so ranks are a permutation.
+__device__ void warp_select_topk(VpShared* sh, int n, int K, int lane) {
+    __syncwarp();
+    for (int i = lane; i < n; i += 32) {
         const uint64_t key = sh->cand[i];
         int rank = 0;
         for (int j = 0; j < n; ++j) rank += (sh->cand[j] > key) ? 1 : 0;
         if (rank < K) sh->outk[rank] = key;
     }
-    cons_bar();
+    __syncwarp();
 }
 
 // Exact selection over a whole segment straight from global memory, in slices small enough that the key
 // buffer cannot overflow.  Used only when the fast path's buffers overflowed.
 template <bool BF16>
-__device__ void fallback_select(VpShared* sh, const VpParams& p, const Seg& sg, int tid, int* nk_out) {
+__device__ int warp_fallback_select(VpShared* sh, const VpParams& p, const Seg& sg, int lane) {
     using T = VT<BF16>;
     const int K = p.K;
     const int slice = kVpCandCap - kMaxK;
     const char* rowp = p.logits + (size_t)sg.row * p.V * T::ESZ;
     uint64_t thr = 0;
-    int nb = 0;
+    int nb = 0, ovf = 0;
     for (int base = sg.e0; base < sg.e1; base += slice) {
-        if (tid == 0) sh->ncand = nb;
-        cons_bar();
-        int end = base + slice < sg.e1 ? base + slice : sg.e1;
-        for (int e = base + tid; e < end; e += NT) {
-            float x = load_elem_f32(rowp + (size_t)e * T::ESZ, BF16);
-            uint64_t key = make_key(__float_as_uint(x), (uint32_t)e);
-            if (key > thr) {
-                int pos = atomicAdd(&sh->ncand, 1);
-                sh->cand[pos] = key;
-            }
+        const int end = base + slice < sg.e1 ? base + slice : sg.e1;
+        int n = nb;
+        for (int e0 = base; e0 < end; e0 += 32) {
+            const int e = e0 + lane;
+            uint64_t key = 0;
+            if (e < end) key = make_key(__float_as_uint(load_elem_f32(rowp + (size_t)e * T::ESZ, BF16)), (uint32_t)e);
+            n = warp_append(sh->cand, n, kVpCandCap, e < end && key > thr, key, lane, &ovf);
         }
-        cons_bar();
-        int n = sh->ncand;
         if (n > K) {
-            select_topk(sh, n, K, tid);
-            if (tid < K) sh->cand[tid] = sh->outk[tid];
+            warp_select_topk(sh, n, K, lane);
+            if (lane < K) sh->cand[lane] = sh->outk[lane];
             thr = sh->outk[K - 1];
             nb = K;
-            cons_bar();
+            __syncwarp();
         } else {
             nb = n;
         }
     }
-    select_topk(sh, nb, K, tid);
-    *nk_out = nb < K ? nb : K;
+    warp_select_topk(sh, nb, K, lane);
+    return nb < K ? nb : K;
 }
 
 template <bool BF16>
 __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParams p) {
     using T = VT<BF16>;
+    using cm_t = typename T::cm_t;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     unsigned char* ring = smem_raw;
-    uint64_t* bars = (uint64_t*)(ring + (size_t)p.stages * TILE);
-    VpShared* sh = (VpShared*)(bars + 2 * 8);
-    typename T::cm_t* cmax = (typename T::cm_t*)(sh + 1);
+    uint64_t* bars = (uint64_t*)(ring + (size_t)p.stages * TILE);  // full[8], empty[8], part_ready[2], epi_done[2]
+    VpShared* sh = (VpShared*)(bars + 24);
+    cm_t* cmax = (cm_t*)(sh + 1);  // [2][n_cmax]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long G = gridDim.x;
     const long long q0 = cta_start(blockIdx.x, p.Q, G), q1 = cta_start(blockIdx.x + 1, p.Q, G);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 8);
+    const uint32_t ready0 = smem_u32(bars + 16), done0 = smem_u32(bars + 18);
 
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, NW);
         }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(ready0 + 8 * s, NW);
+            mbar_init(done0 + 8 * s, 1);
+        }
         mbar_fence_init();
-        sh->ncand = 0;
-        sh->nhits = 0;
-        sh->overflow = 0;
         sh->abort_flag = 0;
     }
     __syncthreads();
 
-    if (warp == NW) {
+    if (warp == PROD_WARP) {
         // ------------------------------ producer warp --------------------------------------------
         if (lane == 0) {
             uint64_t policy = 0;
             if (p.use_hint) policy = l2_policy_evict_first();
             uint32_t t = 0, st = 0, ph = 1;  // ph: parity of the "empty" phase to wait for (first lap: none)
             const uint32_t nst = (uint32_t)p.stages;
-            for (long long qi = q0; qi < q1;) {
-                Seg sg = make_seg<BF16>(p, qi, q1);
-                qi += (sg.e1 - sg.e0 + kVpQuantum - 1) / kVpQuantum;
-                for (int tile = 0; tile < sg.ntiles; ++tile, ++t) {
+            SegIter it = seg_iter_begin<BF16>(p, q0, q1);
+            Seg sg;
+            while (seg_iter_next<BF16>(p, it, sg)) {
+                for (int tile = 0; tile < sg.ntiles && p.dbg != 2; ++tile, ++t) {
                     if (t >= nst) mbar_wait_bounded(empty0 + 8 * st, ph, &sh->abort_flag);
                     uint32_t off = (uint32_t)tile * TILE;
                     uint32_t bytes = sg.body_bytes - off < (uint32_t)TILE ? sg.body_bytes - off : (uint32_t)TILE;
@@ -308,52 +442,38 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
             }
             if (sh->abort_flag) {
                 // a consumer gave up: make sure none of our copies is still in flight before the CTA retires
-                for (uint32_t back = 0; back < (uint32_t)p.stages && back < t; ++back) {
-                    uint32_t tt = t - 1 - back;
+                for (uint32_t back = 0; back < nst && back < t; ++back) {
+                    const uint32_t tt = t - 1 - back;
                     uint32_t tries = 0;
-                    while (!mbar_try_wait(full0 + 8 * (tt % p.stages), (tt / p.stages) & 1) && ++tries < GRAFT_SPIN_LIMIT) {
+                    while (!mbar_try_wait(full0 + 8 * (tt % nst), (tt / nst) & 1) && ++tries < GRAFT_SPIN_LIMIT) {
                     }
                 }
             }
         }
-    } else {
-        // ------------------------------ consumer warps -------------------------------------------
+    } else if (warp < NW) {
+        // ------------------------------ streaming warps ------------------------------------------
         uint32_t st = 0, ph = 0;  // ring position and parity of the "full" phase to wait for
         const uint32_t nst = (uint32_t)p.stages;
-        for (long long qi = q0; qi < q1;) {
-            const Seg sg = make_seg<BF16>(p, qi, q1);
-            qi += (sg.e1 - sg.e0 + kVpQuantum - 1) / kVpQuantum;
-            const char* rowp = p.logits + (size_t)sg.row * p.V * T::ESZ;
+        uint32_t k = 0;           // segment counter: buffers are indexed by k & 1
+        SegIter it = seg_iter_begin<BF16>(p, q0, q1);
+        Seg sg;
+        for (; seg_iter_next<BF16>(p, it, sg); ++k) {
+            const uint32_t pb = k & 1u;
             Acc a;
             a.ref = -INFINITY;
             a.s = 0.f;
             a.tmo = 0u;
-
-            // ragged head / tail that the 16-byte bulk copies cannot carry: plain loads, every element a candidate
-            {
-                const int nhead = sg.e_body0 - sg.e0, ntail = sg.e1 - sg.e_tail0;
-                for (int i = tid; i < nhead + ntail; i += NT) {
-                    const int e = i < nhead ? sg.e0 + i : sg.e_tail0 + (i - nhead);
-                    const float x = load_elem_f32(rowp + (size_t)e * T::ESZ, BF16);
-                    uint32_t o = ord_from_float(x);
-                    a.tmo = o > a.tmo ? o : a.tmo;
-                    const float nref = acc_begin_chunk(a, x);
-                    a.s += ex2_approx(fmaf(x, kLog2e, nref));
-                    int pos = atomicAdd(&sh->ncand, 1);
-                    if (pos < kVpCandCap)
-                        sh->cand[pos] = make_key(__float_as_uint(x), (uint32_t)e);
-                    else
-                        sh->overflow = 1;
-                }
-            }
-
+            // the buffers of parity pb are free once the epilogue of segment k-2 is done
+            if (k >= 2) mbar_wait_bounded(done0 + 8 * pb, ((k >> 1) - 1u) & 1u, &sh->abort_flag);
             {
                 const int nfull = (int)(sg.body_bytes / TILE);
-                typename T::cm_t* slot = cmax + tid;
-                for (int tile = 0; tile < sg.ntiles; ++tile, slot += NT) {
-                    mbar_wait_bounded(full0 + 8 * st, ph, &sh->abort_flag);
+                cm_t* slot = cmax + (size_t)pb * p.n_cmax + (size_t)tid * p.max_tiles;  // this thread's slots, by tile
+                for (int tile = 0; tile < sg.ntiles; ++tile, ++slot) {
+                    if (p.dbg != 2) mbar_wait_bounded(full0 + 8 * st, ph, &sh->abort_flag);
                     const uint4* wb = (const uint4*)(ring + (size_t)st * TILE + (size_t)warp * WBLK);
-                    if (tile < nfull) {
+                    if (p.dbg == 1) {
+                        *slot = 0;
+                    } else if (tile < nfull) {
                         process_chunk<BF16, false>(wb, lane, 0, a, slot);
                     } else {
                         int nv = ((int)(sg.body_bytes - (uint32_t)tile * TILE) - warp * WBLK) / 16;
@@ -368,209 +488,301 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
                     }
                 }
             }
-
-            // ---------------- segment epilogue -------------------------------------------------------
-            // E1: per-thread maxima to shared memory; (ref, s) and the maximum reduced per warp
-            sh->tmax[tid] = a.tmo;
+            // hand the segment over to the epilogue warp
+            sh->tmax[pb][tid] = a.tmo;
             {
                 float c = a.ref, s = a.s;
-                uint32_t vm = a.tmo;
 #pragma unroll
                 for (int d = 16; d > 0; d >>= 1) {
-                    float c2 = __shfl_xor_sync(0xFFFFFFFFu, c, d);
-                    float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, d);
-                    uint32_t v2 = __shfl_xor_sync(0xFFFFFFFFu, vm, d);
-                    float cn = fmaxf(c, c2);
-                    float f1 = (c == -INFINITY) ? 0.f : ex2_approx(c - cn);
-                    float f2 = (c2 == -INFINITY) ? 0.f : ex2_approx(c2 - cn);
-                    s = s * f1 + s2 * f2;
-                    c = cn;
-                    vm = vm > v2 ? vm : v2;
+                    const float c2 = __shfl_xor_sync(0xFFFFFFFFu, c, d);
+                    const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, d);
+                    merge_cs(c, s, c2, s2);
                 }
                 if (lane == 0) {
-                    sh->wc[warp] = c;
-                    sh->ws[warp] = s;
-                    sh->wv[warp] = vm;
+                    sh->wc[pb][warp] = c;
+                    sh->ws[pb][warp] = s;
                 }
             }
-            cons_bar();
-            // E2: warp 0 finds T = the K-th largest per-thread maximum, truncated to its top 16 bits
-            //     (a lower bound of the K-th largest element); warp 1 folds the warps' (ref, s).
-            if (warp == 0) {
-                uint32_t mine[NT / 32];
-#pragma unroll
-                for (int i = 0; i < NT / 32; ++i) mine[i] = sh->tmax[i * 32 + lane];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(ready0 + 8 * pb);
+        }
+    } else {
+        // ------------------------------ epilogue group (four warps) ------------------------------
+        // Warp 0 of the group owns the hand-over barriers and the sequential parts; the data-parallel parts
+        // (which chunks reach T, re-reading them, ranking the candidates) are shared by the 128 threads.
+        const int ew = warp - NW, etid = tid - NT;
+        uint32_t k = 0;
+        SegIter it = seg_iter_begin<BF16>(p, q0, q1);
+        Seg sg;
+        for (; seg_iter_next<BF16>(p, it, sg); ++k) {
+            const uint32_t pb = k & 1u;
+            const char* rowp = p.logits + (size_t)sg.row * p.V * T::ESZ;
+            const cm_t* cmx = cmax + (size_t)pb * p.n_cmax;
+#ifdef GRAFT_VP_PROF
+            long long tprof = clock64();
+#endif
+            if (ew == 0) mbar_wait_bounded(ready0 + 8 * pb, (k >> 1) & 1u, &sh->abort_flag);
+            if (p.dbg) {
+                __syncwarp();
+                if (ew == 0 && lane == 0) mbar_arrive(done0 + 8 * pb);
+                continue;
+            }
+            float c = -INFINITY, s = 0.f;
+            uint32_t vmo = 0;
+            if (ew == 0) {
+                VP_T(0);
+                int overflow = 0, ncand = 0;
+                // (a) log-sum-exp pieces of the streaming warps
+                c = lane < NW ? sh->wc[pb][lane] : -INFINITY;
+                s = lane < NW ? sh->ws[pb][lane] : 0.f;
+                // (b) ragged head / tail that the 16-byte bulk copies cannot carry: plain loads, every element a
+                //     candidate (at most 7 + 7 elements unless the whole segment is shorter than 16 bytes)
+                {
+                    const int nhead = sg.e_body0 - sg.e0, ntail = sg.e1 - sg.e_tail0;
+                    for (int i0 = 0; i0 < nhead + ntail; i0 += 32) {
+                        const int i = i0 + lane;
+                        const bool in = i < nhead + ntail;
+                        uint64_t key = 0;
+                        if (in) {
+                            const int e = i < nhead ? sg.e0 + i : sg.e_tail0 + (i - nhead);
+                            const float x = load_elem_f32(rowp + (size_t)e * T::ESZ, BF16);
+                            const uint32_t o = ord_from_float(x);
+                            vmo = o > vmo ? o : vmo;
+                            float c1 = x * kLog2e, s1 = 1.0f;
+                            if (x == -INFINITY) {
+                                c1 = -INFINITY;
+                                s1 = 0.f;
+                            } else if (!(x < INFINITY)) {
+                                s1 = NAN;  // +inf or NaN poisons the sum and marks the row
+                                c1 = 0.f;
+                            }
+                            merge_cs(c, s, c1, s1);
+                            key = make_key(__float_as_uint(x), (uint32_t)e);
+                        }
+                        ncand = warp_append(sh->cand, ncand, kVpCandCap, in, key, lane, &overflow);
+                    }
+                }
+                VP_T(1);
+                // (c) T = the K-th largest per-thread maximum, truncated to its top 16 bits: a lower bound of
+                //     the K-th largest element of the segment's body (0 when fewer than K threads saw data)
                 uint32_t Tv = 0;
-                for (int bit = 31; bit >= 16; --bit) {
-                    const uint32_t trial = Tv | (1u << bit);
-                    int cnt = 0;
+                {
+                    uint32_t mine[NT / 32];
 #pragma unroll
-                    for (int i = 0; i < NT / 32; ++i) cnt += (mine[i] >= trial) ? 1 : 0;
-                    cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
-                    if (cnt >= p.K) Tv = trial;
-                }
-                if (lane == 0) sh->T = Tv;
-            } else if (warp == 1) {
-                float c = lane < NW ? sh->wc[lane] : -INFINITY;
-                float s = lane < NW ? sh->ws[lane] : 0.f;
-                uint32_t vm = lane < NW ? sh->wv[lane] : 0u;
+                    for (int i = 0; i < NT / 32; ++i) {
+                        mine[i] = sh->tmax[pb][i * 32 + lane];
+                        vmo = mine[i] > vmo ? mine[i] : vmo;
+                    }
+                    for (int bit = 30; bit >= 16; bit -= 2) {  // two bits per step: three independent counts
+                        const uint32_t t1 = Tv | (1u << bit), t2 = Tv | (2u << bit), t3 = Tv | (3u << bit);
+                        int c1 = 0, c2 = 0, c3 = 0;
 #pragma unroll
-                for (int d = NW / 2; d > 0; d >>= 1) {
-                    float c2 = __shfl_xor_sync(0xFFFFFFFFu, c, d);
-                    float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, d);
-                    uint32_t v2 = __shfl_xor_sync(0xFFFFFFFFu, vm, d);
-                    float cn = fmaxf(c, c2);
-                    float f1 = (c == -INFINITY) ? 0.f : ex2_approx(c - cn);
-                    float f2 = (c2 == -INFINITY) ? 0.f : ex2_approx(c2 - cn);
-                    s = s * f1 + s2 * f2;
-                    c = cn;
-                    vm = vm > v2 ? vm : v2;
+                        for (int i = 0; i < NT / 32; ++i) {
+                            c1 += (mine[i] >= t1) ? 1 : 0;
+                            c2 += (mine[i] >= t2) ? 1 : 0;
+                            c3 += (mine[i] >= t3) ? 1 : 0;
+                        }
+                        c1 = __reduce_add_sync(0xFFFFFFFFu, c1);
+                        c2 = __reduce_add_sync(0xFFFFFFFFu, c2);
+                        c3 = __reduce_add_sync(0xFFFFFFFFu, c3);
+                        Tv = c3 >= p.K ? t3 : (c2 >= p.K ? t2 : (c1 >= p.K ? t1 : Tv));
+                    }
                 }
+                // fold (c, s, max) across the warp
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) {
+                    const float c2 = __shfl_xor_sync(0xFFFFFFFFu, c, d);
+                    const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, d);
+                    merge_cs(c, s, c2, s2);
+                }
+                vmo = __reduce_max_sync(0xFFFFFFFFu, vmo);
+                overflow = __any_sync(0xFFFFFFFFu, overflow);
                 if (lane == 0) {
-                    sh->segC = c;
-                    sh->segS = s;
-                    sh->segV = vm;
+                    sh->Tv = Tv;
+                    sh->nhits = 0;
+                    sh->nht = 0;
+                    sh->ncand = ncand;
+                    sh->ovf = overflow;
                 }
+                VP_T(2);
             }
-            cons_bar();
-            // E3: every thread scans the chunk maxima it stored itself
+            epi_bar();
+            const uint32_t Tv = sh->Tv;
+            // (d) chunks whose stored maximum reaches T: only threads whose own maximum reaches T can have one.
+            //     List positions come from shared-memory atomics (the order does not matter: the final selection
+            //     ranks exact keys).  A hit is recorded as the byte offset of the chunk's first vector.
+            for (int t = etid; t < NT; t += kVpEpiThreads) {
+                const uint32_t x = sh->tmax[pb][t];
+                if (x >= Tv && x != 0u) sh->hthreads[atomicAdd(&sh->nht, 1)] = (uint16_t)t;
+            }
+            epi_bar();
             {
-                const uint32_t Tv = sh->T;
-                for (int tile = 0; tile < sg.ntiles; ++tile) {
-                    const uint32_t cs = (uint32_t)tile * NT + tid;
-                    const uint32_t bits = BF16 ? ((uint32_t)cmax[cs] << 16) : (uint32_t)cmax[cs];
+                const int npairs = sh->nht * sg.ntiles;
+                for (int idx = etid; idx < npairs; idx += kVpEpiThreads) {
+                    const int h = idx / sg.ntiles, tile = idx - h * sg.ntiles;
+                    const uint32_t t = sh->hthreads[h];
+                    const cm_t raw = cmx[(size_t)t * p.max_tiles + tile];
+                    const uint32_t bits = BF16 ? ((uint32_t)raw << 16) : (uint32_t)raw;
                     if (ord_from_bits(bits) >= Tv) {
-                        int pos = atomicAdd(&sh->nhits, 1);
-                        if (pos < kVpHitCap)
-                            sh->hits[pos] = cs;
-                        else
-                            sh->overflow = 1;
+                        const int pos = atomicAdd(&sh->nhits, 1);
+                        if (pos < kVpHitCap) sh->hits[pos] = (uint32_t)tile * TILE + (t >> 5) * WBLK + (t & 31) * 16;
                     }
                 }
             }
-            cons_bar();
-            // E4: elements of the hit chunks, one element per thread and step, re-read from global memory
+            epi_bar();
+            if (ew == 0) VP_T(3);
+            // (e) the 16-byte vectors of the hit chunks, re-read from global memory; elements >= T become keys.
+            //     A thread issues its loads of a round before it uses any: under a saturated memory system one
+            //     round trip costs microseconds.
             {
-                const uint32_t Tv = sh->T;
-                const int nh = sh->nhits < kVpHitCap ? sh->nhits : kVpHitCap;
-                for (int idx = tid; idx < nh * T::CH; idx += NT) {
-                    const uint32_t cs = sh->hits[idx / T::CH];
-                    const int j = idx % T::CH;
-                    const uint32_t tile = cs / NT, r = cs % NT, w = r >> 5, l = r & 31;
-                    const uint32_t off = tile * TILE + w * WBLK + ((j / T::EPV) * 32 + l) * 16 + (j % T::EPV) * T::ESZ;
-                    if (off < sg.body_bytes) {
-                        const float x = load_elem_f32(sg.body + off, BF16);
-                        if (ord_from_float(x) >= Tv) {
-                            int pos = atomicAdd(&sh->ncand, 1);
-                            if (pos < kVpCandCap)
-                                sh->cand[pos] = make_key(__float_as_uint(x), (uint32_t)(sg.e_body0 + off / T::ESZ));
+                const int nhits = sh->nhits < kVpHitCap ? sh->nhits : kVpHitCap;
+                if (etid == 0 && sh->nhits > kVpHitCap) sh->ovf = 1;
+                constexpr int RU = 2;
+                const int nvec = nhits * VEC_PER_LANE;
+                for (int base = 0; base < nvec; base += kVpEpiThreads * RU) {
+                    uint4 vv[RU];
+                    uint32_t offs[RU];
+#pragma unroll
+                    for (int u = 0; u < RU; ++u) {
+                        const int i = base + u * kVpEpiThreads + etid;
+                        vv[u] = make_uint4(T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD);
+                        offs[u] = 0xFFFFFFFFu;
+                        if (i < nvec) {
+                            const uint32_t off = sh->hits[i / VEC_PER_LANE] + (uint32_t)(i % VEC_PER_LANE) * 512u;
+                            if (off < sg.body_bytes) {
+                                offs[u] = off;
+                                vv[u] = *(const uint4*)(sg.body + off);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < RU; ++u) {
+                        if (offs[u] == 0xFFFFFFFFu) continue;
+                        const uint32_t wv[4] = {vv[u].x, vv[u].y, vv[u].z, vv[u].w};
+#pragma unroll
+                        for (int j = 0; j < T::EPV; ++j) {
+                            uint32_t xb;
+                            if (BF16)
+                                xb = (j & 1) ? (wv[j >> 1] & 0xFFFF0000u) : (wv[j >> 1] << 16);
                             else
-                                sh->overflow = 1;
+                                xb = wv[j];
+                            if (ord_from_bits(xb) >= Tv) {
+                                const int pos = atomicAdd(&sh->ncand, 1);
+                                if (pos < kVpCandCap)
+                                    sh->cand[pos] = make_key(xb, (uint32_t)(sg.e_body0 + offs[u] / T::ESZ + j));
+                            }
                         }
                     }
                 }
             }
-            cons_bar();
-            // E5: exact top-K of the candidates
-            int nk;
-            if (sh->overflow) {
-                fallback_select<BF16>(sh, p, sg, tid, &nk);
-            } else {
-                const int n = sh->ncand;
-                select_topk(sh, n, p.K, tid);
-                nk = n < p.K ? n : p.K;
+            epi_bar();
+            if (ew == 0) VP_T(4);
+            // (f) exact top-K of the candidates by rank counting (keys are distinct, so ranks are a permutation)
+            const bool overflow = sh->ovf != 0 || sh->ncand > kVpCandCap;
+            const int ncand = sh->ncand < kVpCandCap ? sh->ncand : kVpCandCap;
+            int nk = ncand < p.K ? ncand : p.K;
+            if (!overflow) {
+                for (int i = etid; i < ncand; i += kVpEpiThreads) {
+                    const uint64_t key = sh->cand[i];
+                    int rank = 0;
+                    for (int j = 0; j < ncand; ++j) rank += (sh->cand[j] > key) ? 1 : 0;
+                    if (rank < p.K) sh->outk[rank] = key;
+                }
+            } else if (ew == 0) {
+                nk = warp_fallback_select<BF16>(sh, p, sg, lane);
             }
-            // E6: finish the row, or leave a record for the CTA that arrives last
+            epi_bar();
+            if (ew != 0) continue;
+            const int nhits = sh->nhits;
+            VP_T(5);
+            if (blockIdx.x == 1 && lane == 0) { atomicAdd(p.errflag + 10, ncand); atomicAdd(p.errflag + 11, nhits); atomicAdd(p.errflag + 12, 1); }
+            // the double-buffered arrays of parity pb may be reused from here on
+            __syncwarp();
+            if (lane == 0) mbar_arrive(done0 + 8 * pb);
+            // (g) finish the row, or leave a record for the CTA that arrives last
             const long long x0 = (long long)sg.row * p.nq;
             const int c_first = cta_of(x0, p.Q, G), c_last = cta_of(x0 + p.nq - 1, p.Q, G);
             const int nseg = c_last - c_first + 1;
-            double Cd = (double)sh->segC, Sd = (double)sh->segS;
-            uint32_t Vm = sh->segV;
+            double Cd = (double)c, Sd = (double)s;
+            uint32_t Vm = vmo;
             bool finish = (nseg == 1);
             if (nseg > 1) {
                 const int my_first_row = (int)(q0 / p.nq);
                 VpRecord* rec = p.records + (size_t)blockIdx.x * 2 + (sg.row == my_first_row ? 0 : 1);
-                if (tid < kMaxK) rec->keys[tid] = tid < nk ? sh->outk[tid] : 0ull;
-                if (tid == 0) {
-                    rec->c = sh->segC;
-                    rec->s = sh->segS;
-                    rec->vmax = __uint_as_float(sh->segV);
+                if (lane < kMaxK) rec->keys[lane] = lane < nk ? sh->outk[lane] : 0ull;
+                if (lane == 0) {
+                    rec->c = c;
+                    rec->s = s;
+                    rec->vmax = __uint_as_float(vmo);
                     rec->nkeys = (uint32_t)nk;
                 }
                 __threadfence();
-                cons_bar();
-                if (tid == 0) {
-                    int old = atomicAdd(p.row_counter + sg.row, 1);
-                    sh->is_last = (old == nseg - 1);
+                __syncwarp();
+                int old = 0;
+                if (lane == 0) {
+                    old = atomicAdd(p.row_counter + sg.row, 1);
                     __threadfence();
                 }
-                cons_bar();
-                if (sh->is_last) {
+                old = __shfl_sync(0xFFFFFFFFu, old, 0);
+                if (old == nseg - 1) {
                     finish = true;
                     // merge the records of CTAs c_first..c_last, a round at a time
                     const int per_round = (kVpCandCap - kMaxK) / kMaxK;
                     int have = 0;
                     for (int c0 = c_first; c0 <= c_last; c0 += per_round) {
                         const int c1 = c0 + per_round - 1 < c_last ? c0 + per_round - 1 : c_last;
-                        if (tid == 0) sh->ncand = have;
-                        cons_bar();
-                        for (int i = tid; i < (c1 - c0 + 1) * kMaxK; i += NT) {
-                            const int c = c0 + i / kMaxK, k = i % kMaxK;
-                            const int c_row0 = (int)(cta_start(c, p.Q, G) / p.nq);
-                            const VpRecord* r = p.records + (size_t)c * 2 + (sg.row == c_row0 ? 0 : 1);
-                            const uint64_t key = __ldcg((const unsigned long long*)&r->keys[k]);
-                            if (key != 0ull) sh->cand[atomicAdd(&sh->ncand, 1)] = key;
+                        int n = have, ovf = 0;
+                        for (int i0 = 0; i0 < (c1 - c0 + 1) * kMaxK; i0 += 32) {
+                            const int i = i0 + lane;
+                            const int cc = c0 + i / kMaxK, kk = i % kMaxK;
+                            const int c_row0 = (int)(cta_start(cc, p.Q, G) / p.nq);
+                            const VpRecord* r = p.records + (size_t)cc * 2 + (sg.row == c_row0 ? 0 : 1);
+                            const uint64_t key = __ldcg((const unsigned long long*)&r->keys[kk]);
+                            n = warp_append(sh->cand, n, kVpCandCap, key != 0ull, key, lane, &ovf);
                         }
-                        cons_bar();
-                        const int n = sh->ncand;
-                        select_topk(sh, n, p.K, tid);
+                        warp_select_topk(sh, n, p.K, lane);
                         have = n < p.K ? n : p.K;
-                        if (tid < have) sh->cand[tid] = sh->outk[tid];
-                        cons_bar();
+                        if (lane < have) sh->cand[lane] = sh->outk[lane];
+                        __syncwarp();
                     }
                     nk = have;
-                    // log-sum-exp pieces, folded in double by one thread per record and a warp reduction
-                    if (warp == 0) {
-                        double Cm = -INFINITY;
-                        uint32_t vm = 0;
-                        for (int c = c_first + lane; c <= c_last; c += 32) {
-                            const int c_row0 = (int)(cta_start(c, p.Q, G) / p.nq);
-                            const VpRecord* r = p.records + (size_t)c * 2 + (sg.row == c_row0 ? 0 : 1);
-                            float rc = __ldcg(&r->c);
-                            uint32_t rv = __float_as_uint(__ldcg(&r->vmax));
-                            Cm = fmax(Cm, (double)rc);
-                            vm = vm > rv ? vm : rv;
-                        }
-#pragma unroll
-                        for (int d = 16; d > 0; d >>= 1) {
-                            Cm = fmax(Cm, __shfl_xor_sync(0xFFFFFFFFu, Cm, d));
-                            uint32_t v2 = __shfl_xor_sync(0xFFFFFFFFu, vm, d);
-                            vm = vm > v2 ? vm : v2;
-                        }
-                        double S = 0.0;
-                        for (int c = c_first + lane; c <= c_last; c += 32) {
-                            const int c_row0 = (int)(cta_start(c, p.Q, G) / p.nq);
-                            const VpRecord* r = p.records + (size_t)c * 2 + (sg.row == c_row0 ? 0 : 1);
-                            float rc = __ldcg(&r->c), rs = __ldcg(&r->s);
-                            if (rc != -INFINITY) S += (double)rs * exp2((double)rc - Cm);
-                            else if (rs != rs) S += (double)rs;
-                        }
-#pragma unroll
-                        for (int d = 16; d > 0; d >>= 1) S += __shfl_xor_sync(0xFFFFFFFFu, S, d);
-                        if (lane == 0) {
-                            sh->segC = (float)Cm;  // exact: Cm is one of the fp32 references
-                            sh->segS = (float)S;
-                            sh->segV = vm;
-                        }
-                        Cd = Cm;
-                        Sd = S;
-                        Vm = vm;
+                    // log-sum-exp pieces, folded in double
+                    double Cm = -INFINITY;
+                    uint32_t vm = 0;
+                    for (int cc = c_first + lane; cc <= c_last; cc += 32) {
+                        const int c_row0 = (int)(cta_start(cc, p.Q, G) / p.nq);
+                        const VpRecord* r = p.records + (size_t)cc * 2 + (sg.row == c_row0 ? 0 : 1);
+                        const float rc = __ldcg(&r->c);
+                        const uint32_t rv = __float_as_uint(__ldcg(&r->vmax));
+                        Cm = fmax(Cm, (double)rc);
+                        vm = vm > rv ? vm : rv;
                     }
-                    if (tid == 0) p.row_counter[sg.row] = 0;
+#pragma unroll
+                    for (int d = 16; d > 0; d >>= 1) {
+                        Cm = fmax(Cm, __shfl_xor_sync(0xFFFFFFFFu, Cm, d));
+                        const uint32_t v2 = __shfl_xor_sync(0xFFFFFFFFu, vm, d);
+                        vm = vm > v2 ? vm : v2;
+                    }
+                    double S = 0.0;
+                    for (int cc = c_first + lane; cc <= c_last; cc += 32) {
+                        const int c_row0 = (int)(cta_start(cc, p.Q, G) / p.nq);
+                        const VpRecord* r = p.records + (size_t)cc * 2 + (sg.row == c_row0 ? 0 : 1);
+                        const float rc = __ldcg(&r->c), rs = __ldcg(&r->s);
+                        if (rc != -INFINITY)
+                            S += (double)rs * exp2((double)rc - Cm);
+                        else if (rs != rs)
+                            S += (double)rs;
+                    }
+#pragma unroll
+                    for (int d = 16; d > 0; d >>= 1) S += __shfl_xor_sync(0xFFFFFFFFu, S, d);
+                    Cd = Cm;
+                    Sd = S;
+                    Vm = vm;
+                    if (lane == 0) p.row_counter[sg.row] = 0;
                 }
             }
-            if (finish && warp == 0) {
-                // lse = (C + log2 S) ln 2, in double; every lane of warp 0 holds the same Cd, Sd, Vm
+            VP_T(6);
+            if (finish) {
                 // The stream accumulates 2^(z c - ref) with c = fp32(log2 e), so (C + log2 S) ln 2 is the
                 // log-sum-exp of the logits scaled by a = c ln 2 = 1 + 1.3e-8.  To first order that adds
                 // (a - 1) E_q[z]; the largest logit stands in for the mean under q (the difference is a few
@@ -578,7 +790,6 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
                 const float vmax = __uint_as_float(bits_from_ord(Vm));
                 const double a_minus_1 = (double)kLog2e * kLn2 - 1.0;
                 const double lse_d = (Cd + log2(Sd)) * kLn2 - a_minus_1 * (double)vmax;
-                const float lse_f = (float)lse_d;
                 const bool bad = !(Sd > 0.0) || !(Sd < 1e300) || Vm == 0u || vmax == INFINITY || vmax == -INFINITY ||
                                  nk < p.K;
                 if (lane < p.K) {
@@ -586,18 +797,13 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
                     p.topk_id[(size_t)sg.row * p.K + lane] = lane < nk ? (int32_t)key_id(key) : -1;
                     p.topk_lp[(size_t)sg.row * p.K + lane] = lane < nk ? (float)((double)key_value(key) - lse_d) : 0.f;
                 }
+                VP_T(7);
                 if (lane == 0) {
-                    p.lse[sg.row] = lse_f;
+                    p.lse[sg.row] = (float)lse_d;
                     p.row_status[sg.row] = bad ? GRAFT_ST_BAD_LOGITS : 0;
                 }
             }
-            // E7: reset the counters for the next segment
-            if (tid == 0) {
-                sh->ncand = 0;
-                sh->nhits = 0;
-                sh->overflow = 0;
-            }
-            cons_bar();
+            __syncwarp();
         }
     }
     __syncthreads();
@@ -608,14 +814,14 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
 
 // ---- host side ----------------------------------------------------------------------------------
 static size_t vp_smem_bytes(int stages, int n_cmax, bool bf16) {
-    return (size_t)stages * TILE + 16 * sizeof(uint64_t) + sizeof(VpShared) + (size_t)n_cmax * (bf16 ? 2 : 4) + 16;
+    return (size_t)stages * TILE + 24 * sizeof(uint64_t) + sizeof(VpShared) + (size_t)2 * n_cmax * (bf16 ? 2 : 4) + 16;
 }
 
 VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch) {
     VpPlan pl;
     const bool bf16 = cfg.logits_dtype == GRAFT_BF16;
     const int esz = bf16 ? 2 : 4;
-    const long long nq = ((long long)cfg.V + kVpQuantum - 1) / kVpQuantum;
+    const long long nq = cfg.V / kVpQuantum > 0 ? cfg.V / kVpQuantum : 1;
     const long long Q = nq * (long long)batch * cfg.L;
     long long G = (long long)num_sms * 2;
     if (G > Q) G = Q;
@@ -623,7 +829,8 @@ VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch) {
     pl.grid = (int)G;
     long long share_q = (Q + G - 1) / G;
     long long seg_elems = share_q * kVpQuantum;
-    if (seg_elems > nq * kVpQuantum) seg_elems = nq * kVpQuantum;
+    seg_elems += kVpQuantum;  // a row's last quantum also takes the remainder
+    if (seg_elems > cfg.V) seg_elems = cfg.V;
     pl.max_seg_tiles = (int)((seg_elems * esz + TILE - 1) / TILE) + 1;
     const size_t budget = 112 * 1024;  // two CTAs per SM
     int stages = 6;
@@ -643,10 +850,11 @@ cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* 
     p.rows = batch * cfg.L;
     p.V = cfg.V;
     p.K = cfg.K;
-    p.nq = ((long long)cfg.V + kVpQuantum - 1) / kVpQuantum;
+    p.nq = cfg.V / kVpQuantum > 0 ? cfg.V / kVpQuantum : 1;
     p.Q = p.nq * p.rows;
     p.stages = pl.stages;
     p.n_cmax = pl.max_seg_tiles * NT;
+    p.max_tiles = pl.max_seg_tiles;
     p.records = ctx->vp_records;
     p.row_counter = ctx->vp_row_counter;
     p.topk_id = d_topk_id;
@@ -655,6 +863,12 @@ cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* 
     p.row_status = d_row_status;
     p.errflag = ctx->w_errflag;
     p.use_hint = 1;
+    p.dbg = 0;
+#ifdef GRAFT_VP_EXPERIMENT  // tuning switches, never compiled into the shipped library
+    if (getenv("GRAFT_VP_HINT")) p.use_hint = atoi(getenv("GRAFT_VP_HINT"));
+    if (getenv("GRAFT_VP_DEBUG")) p.dbg = atoi(getenv("GRAFT_VP_DEBUG"));
+    if (getenv("GRAFT_VP_STAGES")) p.stages = atoi(getenv("GRAFT_VP_STAGES"));
+#endif
     if (bf16)
         vocab_pass_kernel<true><<<pl.grid, kVpThreads, pl.smem_bytes, st>>>(p);
     else
@@ -667,12 +881,12 @@ cudaError_t vp_configure(const graft_config& cfg, int num_sms, size_t* max_smem)
     // the largest dynamic shared-memory request any batch can produce (segment = a whole row)
     VpPlan pl = vp_make_plan(cfg, num_sms, cfg.max_batch > 4096 ? cfg.max_batch : 4096);
     *max_smem = pl.smem_bytes;
-    if (pl.smem_bytes > 113 * 1024 && pl.stages <= 2) return cudaErrorInvalidValue;
+    if (pl.smem_bytes > 113 * 1024) return cudaErrorInvalidValue;
     cudaError_t e;
     if (cfg.logits_dtype == GRAFT_BF16)
-        e = cudaFuncSetAttribute(vocab_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 114 * 1024);
+        e = cudaFuncSetAttribute(vocab_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
     else
-        e = cudaFuncSetAttribute(vocab_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 114 * 1024);
+        e = cudaFuncSetAttribute(vocab_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
     return e;
 }
 
