@@ -149,6 +149,23 @@ graft_status graft_vocab_pass(graft_ctx* ctx, int32_t batch, const void* d_logit
 graft_status graft_tdes_edges(graft_ctx* ctx, int32_t batch, const int32_t* d_topk_id, const float* d_topk_lp,
                               const int32_t* d_root_token, float* d_edge, void* stream);
 
+/* Allocation-free vocab pass (the paper has no counterpart: this entry point exists for the host side only).
+ * Same computation and outputs as graft_vocab_pass, but it needs no context and calls no cudaMalloc, cudaFree
+ * or other allocating routine: the kernel's scratch (records of rows shared between CTAs, per-row arrival
+ * counters) lives in a static device array inside the library (about 0.4 MB, held by every GPU that loads the
+ * library until the process exits).  It is meant for callers that cannot let a library allocate -- a serving
+ * process that gave all device memory to its own pool at start-up, or code that has to stay off the driver's
+ * allocation lock on its latency path.
+ *   Limits: batch * L <= 16384 rows and at most 512 CTAs (two per SM); beyond them GRAFT_ERR_UNSUPPORTED.
+ *   d_row_status [batch * L] is required here.
+ *   The first call on each device looks up the array's device address and sets the kernel's shared-memory
+ *   attribute; make that first call before any stream capture begins.
+ *   All calls on a device share the one array: two calls whose kernels overlap on the GPU (different streams
+ *   without ordering) race on it.  Calls ordered on one stream are fine; each clears what must start at zero. */
+graft_status graft_vocab_pass_static(int32_t batch, int32_t L, int32_t V, int32_t K, graft_dtype logits_dtype,
+                                     const void* d_logits, int32_t* d_topk_id, float* d_topk_lp, float* d_lse,
+                                     int32_t* d_row_status, void* stream);
+
 /* Acceptance walk (Preliminaries, "Speculative decoding": a_t; "Tree-based speculative decoding": the longest
  * accepted path is committed).  d_target_next[b, i] is the target model's next token after node i.
  * Starting at the root, follow the child whose token equals target_next of the current node.

@@ -20,7 +20,8 @@ ST_BAD_LOGITS, ST_TAU_CLAMPED, ST_FRONTIER_EMPTY, ST_INTERNAL = 1, 2, 4, 8
 
 ENTRY_POINTS = [
     "graft_create", "graft_destroy", "graft_nmax", "graft_mask_words", "graft_set_saba", "graft_set_tdes_tables",
-    "graft_tdes_precompute", "graft_build_trees", "graft_vocab_pass", "graft_tdes_edges", "graft_accept",
+    "graft_tdes_precompute", "graft_build_trees", "graft_vocab_pass", "graft_vocab_pass_static", "graft_tdes_edges",
+    "graft_accept",
     "graft_build_trees_host", "graft_launch_count", "graft_set_timing", "graft_read_timing", "graft_status_str",
     "graft_version",
 ]
@@ -83,6 +84,7 @@ def load_library():
     lib.graft_build_trees_host.argtypes = lib.graft_build_trees.argtypes
     lib.graft_vocab_pass.argtypes = [vp, C.c_int32, vp, vp, vp, vp, vp, vp]
     lib.graft_tdes_edges.argtypes = [vp, C.c_int32, vp, vp, vp, vp, vp]
+    lib.graft_vocab_pass_static.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int, vp, vp, vp, vp, vp, vp]
     lib.graft_accept.argtypes = [vp, C.c_int32, C.POINTER(_TreeOut), vp, vp, vp, vp, vp]
     lib.graft_launch_count.argtypes = [vp]
     lib.graft_launch_count.restype = C.c_uint64
@@ -117,6 +119,17 @@ def _ptr(t, dtype=None, cuda=True):
 
 def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def vocab_pass_static(logits, K, topk_id, topk_lp, lse, row_status):
+    """graft_vocab_pass_static: the vocab pass for callers that cannot let the library allocate (no context;
+    the scratch is a static device array inside the library).  logits [batch, L, V] on the GPU."""
+    lib = load_library()
+    batch, L, V = logits.shape
+    dt = BF16 if logits.dtype == torch.bfloat16 else F32
+    _check(lib, lib.graft_vocab_pass_static(batch, L, V, K, dt, _ptr(logits), _ptr(topk_id, torch.int32),
+                                            _ptr(topk_lp, torch.float32), _ptr(lse, torch.float32),
+                                            _ptr(row_status, torch.int32), _stream()), "graft_vocab_pass_static")
 
 
 @dataclass

@@ -18,6 +18,9 @@
 //   * rows shared by several CTAs are merged by the last CTA to arrive (a counter, no waiting).
 // Every wait on an mbarrier is bounded; when one runs out the kernel raises an error flag and drains.
 #include <stdlib.h>
+#include <string.h>
+
+#include <mutex>
 
 #include "common.cuh"
 #include "internal.h"
@@ -891,3 +894,120 @@ cudaError_t vp_configure(const graft_config& cfg, int num_sms, size_t* max_smem)
 }
 
 }  // namespace graft
+
+// ---- allocation-free variant of the vocab pass ------------------------------------------------------------
+// Some callers cannot let this library allocate: a serving process that handed all device memory to its own
+// pool at start-up (a cudaMalloc there fails, or stalls every stream while the driver synchronises), or code
+// that must stay off the driver's allocation lock on its latency path.  For them the scratch of the vocab
+// pass -- the per-CTA records of rows shared between CTAs, the per-row arrival counters and the error word --
+// lives in the file-scope device array below instead of a context's cudaMalloc'ed workspace.  Every GPU that
+// loads this library holds the array (about 0.4 MB) until the process exits.
+namespace graft {
+namespace {
+
+constexpr int kStaticMaxGrid = 512;     // CTAs: two per SM on up to 256 SMs
+constexpr int kStaticMaxRows = 16384;   // batch * L
+
+struct VpStaticScratch {
+    VpRecord records[kStaticMaxGrid * 2];
+    int row_counter[kStaticMaxRows];
+    int errflag[64];
+};
+
+static __device__ __align__(256) unsigned char g_vp_static_scratch[sizeof(VpStaticScratch)];
+
+struct VpStaticDevice {
+    bool ready = false;
+    VpStaticScratch* scratch = nullptr;  // device address of g_vp_static_scratch on this device
+    int num_sms = 0;
+};
+VpStaticDevice g_vp_static_dev[64];
+std::mutex g_vp_static_mutex;
+
+}  // namespace
+}  // namespace graft
+
+extern "C" graft_status graft_vocab_pass_static(int32_t batch, int32_t L, int32_t V, int32_t K,
+                                                graft_dtype logits_dtype, const void* d_logits, int32_t* d_topk_id,
+                                                float* d_topk_lp, float* d_lse, int32_t* d_row_status, void* stream) {
+    using namespace graft;
+    if (!d_logits || !d_topk_id || !d_topk_lp || !d_lse || !d_row_status) return GRAFT_ERR_INVALID_ARG;
+    if (logits_dtype != GRAFT_F32 && logits_dtype != GRAFT_BF16) return GRAFT_ERR_INVALID_ARG;
+    if (batch < 1 || L < 1 || V < 1 || K < 1) return GRAFT_ERR_INVALID_ARG;
+    if ((uintptr_t)d_logits % (logits_dtype == GRAFT_BF16 ? 2 : 4)) return GRAFT_ERR_INVALID_ARG;
+    if (K > kMaxK || K > V || L > kMaxL || (long long)V > 2147483647LL - 64) return GRAFT_ERR_UNSUPPORTED;
+    if ((long long)batch * L > kStaticMaxRows) return GRAFT_ERR_UNSUPPORTED;  // beyond the static scratch
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return GRAFT_ERR_CUDA;
+    }
+    graft_config cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.V = V;
+    cfg.L = L;
+    cfg.K = K;
+    cfg.max_batch = batch;
+    cfg.logits_dtype = logits_dtype;
+    VpStaticDevice* sd = &g_vp_static_dev[dev];
+    {
+        // set-up, once per device, with that device current: the array's name is only a host-side stand-in
+        // here, so its device address has to be asked for
+        std::lock_guard<std::mutex> lock(g_vp_static_mutex);
+        if (!sd->ready) {
+            void* ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_vp_static_scratch) != cudaSuccess || !ptr) {
+                cudaGetLastError();
+                return GRAFT_ERR_CUDA;
+            }
+            int sms = 0;
+            if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+                cudaGetLastError();
+                return GRAFT_ERR_CUDA;
+            }
+            if (cudaFuncSetAttribute(vocab_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024) !=
+                    cudaSuccess ||
+                cudaFuncSetAttribute(vocab_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024) !=
+                    cudaSuccess) {
+                cudaGetLastError();
+                return GRAFT_ERR_CUDA;
+            }
+            sd->scratch = (VpStaticScratch*)ptr;
+            sd->num_sms = sms;
+            sd->ready = true;
+        }
+    }
+    const VpPlan pl = vp_make_plan(cfg, sd->num_sms, batch);
+    if (pl.grid > kStaticMaxGrid || pl.smem_bytes > 113 * 1024) return GRAFT_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps whatever the previous call left: the arrival counters and the error word must start at 0
+    if (cudaMemsetAsync(sd->scratch->row_counter, 0, sizeof(int) * (size_t)batch * L, st) != cudaSuccess ||
+        cudaMemsetAsync(sd->scratch->errflag, 0, sizeof(sd->scratch->errflag), st) != cudaSuccess) {
+        cudaGetLastError();
+        return GRAFT_ERR_CUDA;
+    }
+    VpParams p;
+    p.logits = (const char*)d_logits;
+    p.rows = batch * L;
+    p.V = V;
+    p.K = K;
+    p.nq = V / kVpQuantum > 0 ? V / kVpQuantum : 1;
+    p.Q = p.nq * p.rows;
+    p.stages = pl.stages;
+    p.n_cmax = pl.max_seg_tiles * NT;
+    p.max_tiles = pl.max_seg_tiles;
+    p.records = sd->scratch->records;
+    p.row_counter = sd->scratch->row_counter;
+    p.topk_id = d_topk_id;
+    p.topk_lp = d_topk_lp;
+    p.lse = d_lse;
+    p.row_status = d_row_status;
+    p.errflag = sd->scratch->errflag;
+    p.use_hint = 1;
+    p.dbg = 0;
+    if (logits_dtype == GRAFT_BF16)
+        vocab_pass_kernel<true><<<pl.grid, kVpThreads, pl.smem_bytes, st>>>(p);
+    else
+        vocab_pass_kernel<false><<<pl.grid, kVpThreads, pl.smem_bytes, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? GRAFT_OK : GRAFT_ERR_CUDA;
+}
