@@ -117,23 +117,37 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
         }
         return;
     }
-    // gather: one warp per table row, 16 bytes per lane
+    // gather: token ids first (one round trip), then every warp issues the loads of all its rows before it uses
+    // any of them (a second round trip); one warp per table row, 16 bytes per lane
+    __shared__ int toks[2 * kMaxK];
+    if (threadIdx.x < n_par + K) {
+        const int r = threadIdx.x;
+        int32_t tok = r < n_par ? (j == 0 ? p.root_token[b] : p.topk_id[(row - 1) * K + r]) : ids[r - n_par];
+        toks[r] = tok < 0 ? 0 : (tok >= p.V ? p.V - 1 : tok);
+    }
+    __syncthreads();
     const float* urow = p.u + (size_t)j * m;
-    for (int r = warp; r < n_par + K; r += 8) {
-        const bool is_par = r < n_par;
-        const int idx = is_par ? r : r - n_par;
-        int32_t tok = is_par ? (j == 0 ? p.root_token[b] : p.topk_id[(row - 1) * K + idx]) : ids[idx];
-        tok = tok < 0 ? 0 : (tok >= p.V ? p.V - 1 : tok);
-        const float4* src = (const float4*)((is_par ? p.P : p.C) + (size_t)tok * m);
-        float* dst = (is_par ? sP : sC) + (size_t)idx * ld;
-        for (int k4 = lane; k4 < m / 4; k4 += 32) {
-            float4 t = __ldg(src + k4);
-            float4 uu = *(const float4*)(urow + k4 * 4);
-            t.x += uu.x;
-            t.y += uu.y;
-            t.z += uu.z;
-            t.w += uu.w;
-            *(float4*)(dst + k4 * 4) = t;
+    constexpr int RPW = 2 * kMaxK / 8;  // rows per warp at most
+    for (int k40 = 0; k40 < m / 4; k40 += 32) {
+        const int k4 = k40 + lane;
+        float4 t[RPW];
+#pragma unroll
+        for (int q = 0; q < RPW; ++q) {
+            const int r = warp + 8 * q;
+            t[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (r < n_par + K && k4 < m / 4)
+                t[q] = __ldg((const float4*)((r < n_par ? p.P : p.C) + (size_t)toks[r] * m) + k4);
+        }
+        if (k4 < m / 4) {
+            const float4 uu = *(const float4*)(urow + k4 * 4);
+#pragma unroll
+            for (int q = 0; q < RPW; ++q) {
+                const int r = warp + 8 * q;
+                if (r < n_par + K) {
+                    float* dst = (r < n_par ? sP + (size_t)r * ld : sC + (size_t)(r - n_par) * ld) + k4 * 4;
+                    *(float4*)dst = make_float4(t[q].x + uu.x, t[q].y + uu.y, t[q].z + uu.z, t[q].w + uu.w);
+                }
+            }
         }
     }
     __syncthreads();
