@@ -259,11 +259,11 @@ int oracle_tdes_edges(const int32_t *topk_id /* [L,K] */, const float *topk_lp /
  * to the tree and inserts its K extensions.  The frontier is an explicit array scanned
  * linearly; no heap.
  *
- * The paper does not say how equal scores are ordered.  The total order used here is the one
- * a heap of (score, insertion) pairs gives when every parent's children are pushed in the
- * order of their edge scores:  path score descending; then length ascending; then the prefix
- * whose parent was selected earlier (the root counts as selected first); then, under one
- * parent, edge score descending and candidate rank ascending.
+ * The paper does not say how equal scores are ordered.  The total order used here depends only
+ * on the prefixes themselves (not on the history of the expansion):  path score descending;
+ * then length ascending; then the parent prefix in lexicographic order of its candidate ranks;
+ * then, under one parent, edge score descending and candidate rank ascending (a parent's
+ * children are taken in the order of their edge scores).
  *
  * Output: sel_tuple [n_sel, L] (unused slots -1), sel_len, sel_S in pop order.
  * Pins: exhaustive enumeration for L,K <= 4 (a top-B set by path score when edges <= 0; a
@@ -274,7 +274,6 @@ typedef struct {
     float S;
     float e;        /* the last edge's score */
     int32_t len;
-    int32_t ppop;   /* selection index of the parent: 0 = root, k = the k-th selected prefix */
     int8_t t[ORC_MAX_L];
 } orc_prefix;
 
@@ -282,7 +281,8 @@ static int orc_before(const orc_prefix *a, const orc_prefix *b) { /* does a pop 
     if (a->S > b->S) return 1;
     if (a->S < b->S) return 0;
     if (a->len != b->len) return a->len < b->len;
-    if (a->ppop != b->ppop) return a->ppop < b->ppop;
+    for (int i = 0; i + 1 < a->len; ++i) /* the parents, lexicographically */
+        if (a->t[i] != b->t[i]) return a->t[i] < b->t[i];
     if (a->e > b->e) return 1;
     if (a->e < b->e) return 0;
     return a->t[a->len - 1] < b->t[b->len - 1];
@@ -301,7 +301,6 @@ int oracle_select(const float *edge /* [L,K,K] */, int L, int K, int budget, int
         x.e = edge[c]; /* depth 1, parent row 0 */
         x.S = (float)(0.0f + x.e);
         x.len = 1;
-        x.ppop = 0;
         x.t[0] = (int8_t)c;
         fr[nf++] = x;
     }
@@ -327,7 +326,6 @@ int oracle_select(const float *edge /* [L,K,K] */, int L, int K, int budget, int
                 y.S = sum;
                 y.t[y.len] = (int8_t)c;
                 y.len = x.len + 1;
-                y.ppop = n; /* x was the n-th selection */
                 fr[nf++] = y;
             }
         }

@@ -62,68 +62,95 @@ struct TreeParams {
     const int32_t* fixed_budget;
     graft_tree_out out;
     int L, K, nmax, W, bmin, bmax, bstep;
+    int ncap;  // capacity of the node table of the parallel phase
     int use_saba;
     SabaDev saba;
 };
 
-constexpr int TREE_THREADS = 256;
+constexpr int TREE_THREADS = 1024;  // one CTA per SM (shared memory bound): all warps serve the parallel phases
+constexpr int TREE_MASK_WARPS = 8;  // warps that build mask rows (each needs a 32-row staging tile)
 
 struct TreeSmem {
     float* es;           // [L*K*K]  sorted edge rows
     uint8_t* ei;         // [L*K*K]  child rank of each sorted entry
-    uint64_t* ent;       // [32*33]  frontier entry of node n at [(n & 31) * 33 + (n >> 5)], 0 = none
-    uint64_t* poplog;    // [nmax]   the entry that was selected as node n (node 0: the root's pseudo entry)
+    // node table of the parallel phase (append-only; node 0 = root)
+    uint32_t* nkey;      // [ncap]   bottleneck key = min over the path of ord(path score); later: compact index
+    float* nS;           // [ncap]   path score
+    uint32_t* ninfo;     // [ncap]   parent's table index | candidate rank << 13 | depth << 18
+    // compact arrays by selection index n (0 = root; a parent's index is smaller than its children's)
+    uint64_t* ent;       // [nmax]   frontier entry of node n: its best unselected child, 0 = none
+    float* S;            // [nmax]   path score
     uint32_t* chmask;    // [nmax]   candidate ranks of the node's selected children, one bit each
-    int* cc;             // [nmax]   per-level scratch: child counts in level order, then their exclusive scan
-    uint32_t* stage;     // [8 warps * 32 rows * W] mask rows staged for coalesced stores
-    float* S;            // [nmax]   path score, selection order
-    uint32_t* sortkey;   // [nmax]
-    int16_t* parent;     // [nmax]   selection-order index of the parent
-    int16_t* canon;      // [nmax]   level-order index of selection-order node n
+    int16_t* parent;     // [nmax]
+    int16_t* canon;      // [nmax]   level-order index of node n
     int16_t* cparent;    // [nmax]   level-order parent, by level-order index
-    int16_t* lvl_list;   // [nmax]
     uint8_t* cand;       // [nmax]
     uint8_t* depth;      // [nmax]
+    // emission scratch, laid over the node table (dead by then)
+    int16_t* lvl_list;   // [nmax]
+    int* cc;             // [nmax]   per-level child counts in level order, then their exclusive scan
+    uint32_t* stage;     // [8 warps * 32 rows * W] mask rows staged for coalesced stores
+    uint32_t* hist;      // [4 * 256]
     int* lvl_count;      // [kMaxL + 2]
     int* lvl_start;      // [kMaxL + 2]
     int* lvl_fill;       // [kMaxL + 2]
-    int* scal;           // [8]  0: budget, 1: n_nodes, 2: status
+    int* scal;           // [16] 0 budget, 1 n_nodes, 2 status, 3 table size, 4 overflow, 6/7 radix-select hand-over
 };
 
-__host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, TreeSmem* s, unsigned char* base) {
+__host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, int ncap, TreeSmem* s, unsigned char* base) {
     size_t off = 0;
     auto take = [&](size_t bytes) {
         size_t o = off;
         off += (bytes + 15) & ~(size_t)15;
         return o;
     };
-    size_t o_es = take((size_t)L * K * K * 4), o_ei = take((size_t)L * K * K), o_ent = take((size_t)32 * 33 * 8), o_log = take((size_t)nmax * 8), o_chm = take((size_t)nmax * 4), o_cc = take((size_t)nmax * 4), o_stage = take((size_t)8 * 32 * ((nmax + 31) / 32) * 4),
-           o_S = take((size_t)nmax * 4), o_sk = take((size_t)nmax * 4), o_par = take((size_t)nmax * 2),
-           o_can = take((size_t)nmax * 2), o_cp = take((size_t)nmax * 2), o_ll = take((size_t)nmax * 2),
-           o_cand = take(nmax), o_dep = take(nmax), o_lc = take((kMaxL + 2) * 4), o_ls = take((kMaxL + 2) * 4),
-           o_lf = take((kMaxL + 2) * 4), o_sc = take(8 * 4);
+    const int W = (nmax + 31) / 32;
+    size_t o_es = take((size_t)L * K * K * 4), o_ei = take((size_t)L * K * K);
+    size_t emis = (((size_t)nmax * 2 + 15) & ~(size_t)15) + (((size_t)nmax * 4 + 15) & ~(size_t)15) + (size_t)8 * 32 * W * 4;
+    size_t table = (size_t)ncap * 12;
+    size_t o_tab = take(table > emis ? table : emis);
+    size_t o_ent = take((size_t)nmax * 8), o_S = take((size_t)nmax * 4), o_chm = take((size_t)nmax * 4),
+           o_par = take((size_t)nmax * 2), o_can = take((size_t)nmax * 2), o_cp = take((size_t)nmax * 2),
+           o_cand = take(nmax), o_dep = take(nmax), o_hist = take(1024 * 4), o_lc = take((kMaxL + 2) * 4),
+           o_ls = take((kMaxL + 2) * 4), o_lf = take((kMaxL + 2) * 4), o_sc = take(16 * 4);
     if (s) {
         s->es = (float*)(base + o_es);
         s->ei = base + o_ei;
+        s->nkey = (uint32_t*)(base + o_tab);
+        s->nS = (float*)(base + o_tab + (size_t)ncap * 4);
+        s->ninfo = (uint32_t*)(base + o_tab + (size_t)ncap * 8);
+        s->lvl_list = (int16_t*)(base + o_tab);
+        s->cc = (int*)(base + o_tab + (((size_t)nmax * 2 + 15) & ~(size_t)15));
+        s->stage = (uint32_t*)(base + o_tab + (((size_t)nmax * 2 + 15) & ~(size_t)15) + (((size_t)nmax * 4 + 15) & ~(size_t)15));
         s->ent = (uint64_t*)(base + o_ent);
-        s->poplog = (uint64_t*)(base + o_log);
-        s->chmask = (uint32_t*)(base + o_chm);
-        s->cc = (int*)(base + o_cc);
-        s->stage = (uint32_t*)(base + o_stage);
         s->S = (float*)(base + o_S);
-        s->sortkey = (uint32_t*)(base + o_sk);
+        s->chmask = (uint32_t*)(base + o_chm);
         s->parent = (int16_t*)(base + o_par);
         s->canon = (int16_t*)(base + o_can);
         s->cparent = (int16_t*)(base + o_cp);
-        s->lvl_list = (int16_t*)(base + o_ll);
         s->cand = base + o_cand;
         s->depth = base + o_dep;
+        s->hist = (uint32_t*)(base + o_hist);
         s->lvl_count = (int*)(base + o_lc);
         s->lvl_start = (int*)(base + o_ls);
         s->lvl_fill = (int*)(base + o_lf);
         s->scal = (int*)(base + o_sc);
     }
     return off;
+}
+
+// capacity of the node table: what fits beside the edge rows in ~200 KB of shared memory, at most 6144 nodes
+// (parent indices are 13 bits) and at least enough for a full budget's worth of nodes
+__host__ __device__ inline int tree_node_cap(int L, int K, int nmax) {
+    const int W = (nmax + 31) / 32;
+    const size_t emis = (((size_t)nmax * 2 + 15) & ~(size_t)15) + (((size_t)nmax * 4 + 15) & ~(size_t)15) +
+                        (size_t)8 * 32 * W * 4;
+    const size_t fixed = tree_smem_layout(L, K, nmax, 0, nullptr, nullptr);  // counts `emis` for the table
+    const size_t room = fixed < (size_t)200 * 1024 ? (size_t)200 * 1024 - fixed : 0;
+    long long cap = (long long)((emis + room) / 12);
+    if (cap > 6144) cap = 6144;
+    if (cap < 2 * nmax) cap = 2 * nmax;
+    return (int)cap;
 }
 
 __device__ __forceinline__ double saba_cost(const SabaDev& sp, double B, double prefix) {
@@ -137,46 +164,101 @@ __device__ __forceinline__ double saba_cost(const SabaDev& sp, double B, double 
     return sp.pts_t[sp.n_pts - 1];
 }
 
-// Frontier entry: one per selected node, naming that node's best child not yet selected.  A plain 64-bit
-// maximum over the entries is the next node to select:
-//   bits 63..32  ord(path score of the child)                      -> score descending
-//   bits 30..25  32 - depth of the child                           -> then the shallower child
-//   bits 24..15  1023 - selection index of the parent              -> then the parent selected earlier
-//   bits 14..10  position of the child in the parent's sorted row  (under one parent the sorted row gives
-//   bits  9..5   candidate rank of the parent                       edge descending, rank ascending)
+// Frontier entry of a selected node: its best child that is not selected yet.
+//   bits 63..32  ord(path score of the child)
+//   bits 30..25  32 - depth of the child (larger = shallower)
+//   bits 14..10  position of the child in the parent's sorted row
+//   bits  9..5   candidate rank of the parent
 //   bits  4..0   candidate rank of the child
-__device__ __forceinline__ uint64_t pack_entry(float score, int child_depth, int parent_sel, int pos, int parent_cand,
-                                               int child_cand) {
-    const uint32_t lo = ((uint32_t)(32 - child_depth) << 25) | ((uint32_t)(1023 - parent_sel) << 15) |
-                        ((uint32_t)pos << 10) | ((uint32_t)parent_cand << 5) | (uint32_t)child_cand;
+__device__ __forceinline__ uint64_t pack_entry(float score, int child_depth, int pos, int parent_cand, int child_cand) {
+    const uint32_t lo = ((uint32_t)(32 - child_depth) << 25) | ((uint32_t)pos << 10) | ((uint32_t)parent_cand << 5) |
+                        (uint32_t)child_cand;
     return ((uint64_t)ord_from_float(score) << 32) | lo;
 }
 
-// Warp-wide maximum of a 64-bit key: one redux on the high word, then the low word of the (usually single)
-// lane that holds it.
-__device__ __forceinline__ uint64_t warp_max64(uint64_t x) {
-    const uint32_t hi = (uint32_t)(x >> 32), lo = (uint32_t)x;
-    const uint32_t hm = __reduce_max_sync(0xFFFFFFFFu, hi);
-    const uint32_t tie = __ballot_sync(0xFFFFFFFFu, hi == hm);
-    uint32_t lm;
-    if ((tie & (tie - 1)) == 0u)
-        lm = __shfl_sync(0xFFFFFFFFu, lo, __ffs(tie) - 1);
-    else
-        lm = __reduce_max_sync(0xFFFFFFFFu, hi == hm ? lo : 0u);
-    return ((uint64_t)hm << 32) | lm;
+// Does the prefix of node n1 come before the prefix of node n2 in lexicographic order of candidate ranks?
+// Both at the same depth, n1 != n2.
+__device__ __forceinline__ bool path_less(const TreeSmem& sm, int n1, int n2) {
+    while (sm.parent[n1] != sm.parent[n2]) {
+        n1 = sm.parent[n1];
+        n2 = sm.parent[n2];
+    }
+    return sm.cand[n1] < sm.cand[n2];
+}
+
+// Order of two frontier entries (owned by nodes n1, n2): path score descending, then the shallower child,
+// then the parent whose prefix is lexicographically smaller.  n < 0 = no entry.
+__device__ __forceinline__ bool entry_before(const TreeSmem& sm, uint64_t e1, int n1, uint64_t e2, int n2) {
+    if (n2 < 0) return n1 >= 0;
+    if (n1 < 0) return false;
+    const uint32_t h1 = (uint32_t)(e1 >> 32), h2 = (uint32_t)(e2 >> 32);
+    if (h1 != h2) return h1 > h2;
+    const uint32_t d1 = ((uint32_t)e1 >> 25) & 63u, d2 = ((uint32_t)e2 >> 25) & 63u;
+    if (d1 != d2) return d1 > d2;
+    return path_less(sm, n1, n2);
+}
+
+// B-th largest of keys[lo..hi) (hi - lo >= kth >= 1) by an 8-bit radix select; every thread of the CTA calls it.
+__device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, int lo, int hi, int kth, int tid) {
+    const int warp = tid >> 5, lane = tid & 31;
+    uint32_t prefix = 0, mask = 0;
+    int remaining = kth;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        sm.hist[tid] = 0u;  // four copies of the 256 bins (TREE_THREADS == 1024): neighbouring warps do not collide
+        __syncthreads();
+        for (int i = lo + tid; i < hi; i += TREE_THREADS) {
+            const uint32_t k = keys[i];
+            if ((k & mask) == prefix) atomicAdd(&sm.hist[(warp & 3) * 256 + ((k >> shift) & 255u)], 1u);
+        }
+        __syncthreads();
+        if (warp == 0) {  // lane l owns bins 255-8l .. 248-8l, from the top down
+            int c[8], sum = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int bin = 255 - 8 * lane - j;
+                c[j] = (int)(sm.hist[bin] + sm.hist[256 + bin] + sm.hist[512 + bin] + sm.hist[768 + bin]);
+                sum += c[j];
+            }
+            int incl = sum;
+#pragma unroll
+            for (int o2 = 1; o2 < 32; o2 <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
+                if (lane >= o2) incl += t;
+            }
+            const int excl = incl - sum;
+            if (excl < remaining && remaining <= incl) {
+                int acc = excl, digit = 255 - 8 * lane, rem = remaining - excl;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (acc < remaining && remaining <= acc + c[j]) {
+                        digit = 255 - 8 * lane - j;
+                        rem = remaining - acc;
+                    }
+                    acc += c[j];
+                }
+                sm.scal[6] = digit;
+                sm.scal[7] = rem;
+            }
+        }
+        __syncthreads();
+        prefix |= (uint32_t)sm.scal[6] << shift;
+        mask |= 255u << shift;
+        remaining = sm.scal[7];
+    }
+    return prefix;
 }
 
 __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TreeSmem sm;
-    tree_smem_layout(p.L, p.K, p.nmax, &sm, smem_raw);
+    tree_smem_layout(p.L, p.K, p.nmax, p.ncap, &sm, smem_raw);
     const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int L = p.L, K = p.K, nmax = p.nmax, W = p.W;
     const graft_tree_out& o = p.out;
 
     // ---- status and budget ---------------------------------------------------------------------------
 #ifdef GRAFT_TREE_PROF
-    long long t_prof0 = clock64(), t_prof1 = 0, t_prof2 = 0;
+    long long t_prof0 = clock64(), t_prof1 = 0, t_prof2 = 0, t_prof15 = 0;
 #endif
     {
         const int ne = L * K * K;
@@ -256,73 +338,235 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
 #ifdef GRAFT_TREE_PROF
     t_prof1 = clock64();
 #endif
-    // ---- best-first expansion (warp 0) -----------------------------------------------------------------
-    if (warp == 0) {
-        // Column `lane` of the entry table (nodes n with n & 31 == lane) belongs to this lane, which keeps the
-        // column's maximum in a register.  One step selects `cur`, the maximum entry: the parent's entry moves
-        // to its next sorted child and the new node gets an entry.  Only the parent's column changes, so the
-        // next maximum is the largest of (a) that column re-reduced by the 32 lanes together, (b) the new
-        // node's entry and (c) the maximum over all other columns, which does not depend on this step's
-        // updates and is reduced in the shadow of the loads.
-        constexpr int NSP = 33;
-        const int budget = sm.scal[0];
-        int st = sm.scal[2];
-        for (int i = lane; i < 32 * NSP; i += 32) sm.ent[i] = 0ull;
-        uint64_t best = 0ull;
-        if (lane == 0) {
-            best = pack_entry(0.0f + sm.es[0], 1, 0, 0, 0, sm.ei[0]);
-            sm.ent[0] = best;
-            sm.poplog[0] = (uint64_t)ord_from_float(0.0f) << 32;
+    // ---- best-first expansion ------------------------------------------------------------------------------
+    // Best-first expansion selects prefixes in non-increasing order of their bottleneck key (the minimum path
+    // score along the prefix), so after B selections the tree is the set of prefixes with key above the B-th
+    // largest key theta, plus some of those with key == theta.  Phase 1 (whole CTA) finds theta and the set
+    // {key > theta} level by level: the alive nodes of depth d append their children that can still matter
+    // (key >= current theta; a prefix of the parent's sorted row), then theta becomes the B-th largest key seen
+    // so far (radix select).  Phase 2 (one warp) continues the exact sequential expansion from that state for
+    // the few remaining selections among equal keys.  If the node table overflows, phase 2 does everything.
+    const int budget = sm.scal[0];
+    int n_gt = 0;  // selected so far (root excluded)
+    if (tid == 0) {
+        sm.nkey[0] = 0xFFFFFFFFu;
+        sm.nS[0] = 0.0f;
+        sm.ninfo[0] = 0u;
+        sm.scal[3] = 1;
+        sm.scal[4] = 0;
+        sm.lvl_start[0] = 0;
+        sm.lvl_start[1] = 1;
+        sm.parent[0] = -1;
+        sm.cand[0] = 0;
+        sm.depth[0] = 0;
+        sm.S[0] = 0.0f;
+    }
+    __syncthreads();
+    bool table_ok = budget > 0;
+    uint32_t theta = 0u;
+    if (budget > 0) {
+        int ntot = 1, n_at_select = 1;
+        for (int d = 0; d < L; ++d) {
+#ifdef GRAFT_TREE_PROF
+            long long tl0 = clock64();
+#endif
+            const int b0 = sm.lvl_start[d], b1 = sm.lvl_start[d + 1];
+            if (b1 == b0) break;
+            if (theta == 0u) {
+                // no threshold yet (fewer than B nodes so far): every child of every node of the level is appended,
+                // one thread per (node, child), at a position that needs no atomic
+                const int total = (b1 - b0) * K;
+                if (ntot + total > p.ncap) {
+                    if (tid == 0) sm.scal[4] = 1;
+                } else {
+                    for (int j = tid; j < total; j += TREE_THREADS) {
+                        const int xi = j / K, r = j - xi * K, x = b0 + xi;
+                        const uint32_t kx = sm.nkey[x];
+                        const int row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
+                        const float sc = sm.nS[x] + sm.es[row + r];
+                        const uint32_t oc = ord_from_float(sc);
+                        sm.nkey[ntot + j] = oc < kx ? oc : kx;
+                        sm.nS[ntot + j] = sc;
+                        sm.ninfo[ntot + j] = (uint32_t)x | ((uint32_t)sm.ei[row + r] << 13) | ((uint32_t)(d + 1) << 18);
+                    }
+                    if (tid == 0) sm.scal[3] = ntot + total;
+                }
+            } else {
+                // one thread per node: the children that can still matter are a prefix of the node's sorted row
+                // (scores only fall along the row); its length comes from a binary search, one atomic reserves the
+                // slots, and the writes are independent of each other
+                for (int x = b0 + tid; x < b1; x += TREE_THREADS) {
+                    const uint32_t kx = sm.nkey[x];
+                    if (kx < theta) continue;  // dead: none of its descendants can be selected
+                    const int row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
+                    const float sx = sm.nS[x];
+                    int lo_r = 0, hi_r = K;  // first r in [0, K] whose key falls below theta
+                    while (lo_r < hi_r) {
+                        const int mid = (lo_r + hi_r) >> 1;
+                        const uint32_t oc = ord_from_float(sx + sm.es[row + mid]);
+                        if ((oc < kx ? oc : kx) >= theta)
+                            lo_r = mid + 1;
+                        else
+                            hi_r = mid;
+                    }
+                    const int cnt = lo_r;
+                    if (cnt == 0) continue;
+                    const int base = atomicAdd(&sm.scal[3], cnt);
+                    if (base + cnt > p.ncap) {
+                        sm.scal[4] = 1;
+                        continue;
+                    }
+                    for (int r = 0; r < cnt; ++r) {
+                        const float sc = sx + sm.es[row + r];
+                        const uint32_t oc = ord_from_float(sc);
+                        sm.nkey[base + r] = oc < kx ? oc : kx;
+                        sm.nS[base + r] = sc;
+                        sm.ninfo[base + r] = (uint32_t)x | ((uint32_t)sm.ei[row + r] << 13) | ((uint32_t)(d + 1) << 18);
+                    }
+                }
+            }
+            __syncthreads();
+#ifdef GRAFT_TREE_PROF
+            long long tl1 = clock64();
+#endif
+            const int nt = sm.scal[3];
+            if (sm.scal[4]) {
+                table_ok = false;
+                break;
+            }
+            if (tid == 0) sm.lvl_start[d + 2] = nt;
+            if (nt == ntot) break;  // nothing appended: no deeper level
+            ntot = nt;
+            // theta only has to be a lower bound of its final value while the levels are built (it prunes), so
+            // the exact B-th largest key is recomputed only when the table has grown noticeably
+            if (ntot - 1 >= budget && (theta == 0u || ntot - n_at_select >= ntot / 2)) {
+                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, tid);
+                n_at_select = ntot;
+            }
+            __syncthreads();
+#ifdef GRAFT_TREE_PROF
+            if (tid == 0 && o.d_edge) {
+                float* dbg = o.d_edge + (size_t)b * L * K * K;
+                dbg[4 * d] = (float)(tl1 - tl0);
+                dbg[4 * d + 1] = (float)(clock64() - tl1);
+                dbg[4 * d + 2] = (float)ntot;
+                dbg[4 * d + 3] = (float)(b1 - b0);
+            }
+#endif
         }
-        __syncwarp();
-        uint64_t cur = warp_max64(best);
-        int n_sel = 0;
-        // Inside the loop a path score is never -0 (sums that start from +0), so the order-preserving map
-        // needs no zero canonicalisation here.
+        __syncthreads();
+        if (table_ok && ntot - 1 >= budget && n_at_select != ntot) {
+            theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, tid);  // the exact final value
+        }
+        __syncthreads();
+        if (table_ok) {
+            // compact {key > theta} in table order (parents stay before their children)
+            const int per = (ntot + TREE_THREADS - 1) / TREE_THREADS;
+            const int i0 = tid * per < ntot ? tid * per : ntot, i1 = i0 + per < ntot ? i0 + per : ntot;
+            int cnt = 0;
+            for (int i = i0; i < i1; ++i) cnt += (i == 0 || sm.nkey[i] > theta) ? 1 : 0;
+            int incl = cnt;
+#pragma unroll
+            for (int o2 = 1; o2 < 32; o2 <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
+                if (lane >= o2) incl += t;
+            }
+            if (lane == 31) sm.hist[warp] = (uint32_t)incl;
+            __syncthreads();
+            int woff = 0;
+            for (int w = 0; w < warp; ++w) woff += (int)sm.hist[w];
+            int total = 0;
+            for (int w = 0; w < TREE_THREADS / 32; ++w) total += (int)sm.hist[w];
+            int run = woff + incl - cnt;
+            __syncthreads();
+            for (int i = i0; i < i1; ++i) {
+                const bool sel = (i == 0 || sm.nkey[i] > theta);
+                sm.nkey[i] = sel ? (uint32_t)run : 0xFFFFFFFFu;  // the key is no longer needed: keep the compact index
+                run += sel ? 1 : 0;
+            }
+            __syncthreads();
+            for (int i = i0; i < i1; ++i) {
+                const uint32_t n = sm.nkey[i];
+                if (n == 0xFFFFFFFFu || i == 0) continue;
+                const uint32_t info = sm.ninfo[i];
+                sm.parent[n] = (int16_t)sm.nkey[info & 8191u];
+                sm.cand[n] = (uint8_t)((info >> 13) & 31u);
+                sm.depth[n] = (uint8_t)(info >> 18);
+                sm.S[n] = sm.nS[i];
+            }
+            n_gt = total - 1;
+            __syncthreads();
+            // frontier entries of the selected nodes: the first child of the sorted row that is not selected,
+            // i.e. the first with ord(score) <= theta
+            for (int n = tid; n <= n_gt; n += TREE_THREADS) {
+                const int d = sm.depth[n];
+                uint64_t e = 0ull;
+                if (d < L) {
+                    const int row = (d * K + sm.cand[n]) * K;
+                    const float sn = sm.S[n];
+                    int pos = 0;
+                    while (pos < K && ord_from_float(sn + sm.es[row + pos]) > theta) ++pos;
+                    if (pos < K) e = pack_entry(sn + sm.es[row + pos], d + 1, pos, sm.cand[n], sm.ei[row + pos]);
+                }
+                sm.ent[n] = e;
+            }
+        }
+    }
+#ifdef GRAFT_TREE_PROF
+    t_prof15 = clock64();
+#endif
+    if (!table_ok && tid == 0) sm.ent[0] = budget > 0 ? pack_entry(0.0f + sm.es[0], 1, 0, 0, sm.ei[0]) : 0ull;
+    __syncthreads();
+    if (warp == 0) {
+        // Phase 2: exact sequential expansion.  Every step scans all frontier entries (one per selected node)
+        // for the best under the full order, including the lexicographic rule for equal scores.
+        int st = sm.scal[2];
+        int n_sel = table_ok ? n_gt : 0;
         while (n_sel < budget) {
-            const uint32_t hmax = (uint32_t)(cur >> 32), lmax = (uint32_t)cur;
-            if (hmax == 0u) {
+            uint64_t be = 0ull;
+            int bn = -1;
+            for (int n = lane; n <= n_sel; n += 32) {
+                const uint64_t e = sm.ent[n];
+                if (e != 0ull && entry_before(sm, e, n, be, bn)) {
+                    be = e;
+                    bn = n;
+                }
+            }
+#pragma unroll
+            for (int o2 = 16; o2 > 0; o2 >>= 1) {
+                const uint64_t oe = __shfl_xor_sync(0xFFFFFFFFu, be, o2);
+                const int on = __shfl_xor_sync(0xFFFFFFFFu, bn, o2);
+                if (entry_before(sm, oe, on, be, bn)) {
+                    be = oe;
+                    bn = on;
+                }
+            }
+            if (bn < 0) {
                 st |= GRAFT_ST_FRONTIER_EMPTY;
                 break;
             }
+            const uint32_t lo = (uint32_t)be;
+            const int d = 32 - (int)((lo >> 25) & 63u), pos = (int)((lo >> 10) & 31u);
+            const int cpar = (int)((lo >> 5) & 31u), c = (int)(lo & 31u);
+            const float s_new = __uint_as_float(bits_from_ord((uint32_t)(be >> 32)));
             const int n_new = ++n_sel;
-            const uint32_t dm = (lmax >> 25) & 63u;  // 32 - depth of the selected child
-            const int d = 32 - (int)dm;
-            const int n_par = 1023 - (int)((lmax >> 15) & 1023u);
-            const int pos = (int)((lmax >> 10) & 31u);
-            const int cpar = (int)((lmax >> 5) & 31u);
-            const int c = (int)(lmax & 31u);
-            const int colA = n_par & 31, slotA = n_par >> 5, colB = n_new & 31, slotB = n_new >> 5;
-            const uint64_t others = warp_max64(lane == colA ? 0ull : best);
-            // every lane reads the same few words (broadcasts) and its own entry of the parent's column
-            const bool adv = pos + 1 < K, deeper = d < L;
-            const int at1 = adv ? ((d - 1) * K + cpar) * K + pos + 1 : 0;
-            const int at2 = deeper ? (d * K + c) * K : 0;
-            const uint32_t sp_o = ((const uint32_t*)sm.poplog)[2 * n_par + 1];  // ord(path score of the parent)
-            const float e1 = sm.es[at1], e2 = sm.es[at2];
-            const uint32_t i1 = sm.ei[at1], i2 = sm.ei[at2];
-            uint64_t col = sm.ent[colA * NSP + lane];
-            const float sp = __uint_as_float(sp_o ^ (~(uint32_t)((int32_t)sp_o >> 31) | 0x80000000u));
-            const float s_new = __uint_as_float(hmax ^ (~(uint32_t)((int32_t)hmax >> 31) | 0x80000000u));
-            const uint32_t u1 = __float_as_uint(sp + e1), u2 = __float_as_uint(s_new + e2);
-            const uint32_t h1 = u1 ^ ((uint32_t)((int32_t)u1 >> 31) | 0x80000000u);
-            const uint32_t h2 = u2 ^ ((uint32_t)((int32_t)u2 >> 31) | 0x80000000u);
-            const uint32_t l1 = ((lmax & ~31u) + (1u << 10)) | i1;
-            const uint32_t l2 = ((dm - 1u) << 25) | ((uint32_t)(1023 - n_new) << 15) | ((uint32_t)c << 5) | i2;
-            const uint64_t e_adv = adv ? (((uint64_t)h1 << 32) | l1) : 0ull;
-            const uint64_t e_new = deeper ? (((uint64_t)h2 << 32) | l2) : 0ull;
             if (lane == 0) {
-                sm.ent[colA * NSP + slotA] = e_adv;
-                sm.ent[colB * NSP + slotB] = e_new;
-                sm.poplog[n_new] = cur;
+                sm.parent[n_new] = (int16_t)bn;
+                sm.cand[n_new] = (uint8_t)c;
+                sm.depth[n_new] = (uint8_t)d;
+                sm.S[n_new] = s_new;
+                uint64_t e_adv = 0ull, e_new = 0ull;
+                if (pos + 1 < K) {
+                    const int at = ((d - 1) * K + cpar) * K + pos + 1;
+                    e_adv = pack_entry(sm.S[bn] + sm.es[at], d, pos + 1, cpar, sm.ei[at]);
+                }
+                if (d < L) {
+                    const int at = (d * K + c) * K;
+                    e_new = pack_entry(s_new + sm.es[at], d + 1, 0, c, sm.ei[at]);
+                }
+                sm.ent[bn] = e_adv;
+                sm.ent[n_new] = e_new;
             }
-            if (lane == slotA) col = e_adv;
-            if (colB == colA && lane == slotB) col = e_new;
-            const uint64_t colbest = warp_max64(col);
-            if (lane == colA) best = colbest;
-            if (lane == colB) best = e_new > best ? e_new : best;
-            cur = others > colbest ? others : colbest;
-            cur = e_new > cur ? e_new : cur;
             __syncwarp();
         }
         if (lane == 0) {
@@ -346,17 +590,9 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     const int n_nodes = sm.scal[1];
     for (int n = tid; n < nmax; n += TREE_THREADS) sm.chmask[n] = 0u;
     __syncthreads();
-    for (int n = tid; n < n_nodes; n += TREE_THREADS) {  // unpack the selection log
-        const uint64_t e = sm.poplog[n];
-        const uint32_t lo = (uint32_t)e;
-        const int d = n == 0 ? 0 : 32 - (int)((lo >> 25) & 63u);
-        const int par = n == 0 ? -1 : 1023 - (int)((lo >> 15) & 1023u);
-        sm.parent[n] = (int16_t)par;
-        sm.cand[n] = (uint8_t)(lo & 31u);
-        sm.depth[n] = (uint8_t)d;
-        sm.S[n] = __uint_as_float(bits_from_ord((uint32_t)(e >> 32)));
-        if (n > 0) atomicOr(&sm.chmask[par], 1u << (lo & 31u));
-        atomicAdd(&sm.lvl_count[d], 1);
+    for (int n = tid; n < n_nodes; n += TREE_THREADS) {
+        if (n > 0) atomicOr(&sm.chmask[sm.parent[n]], 1u << sm.cand[n]);
+        atomicAdd(&sm.lvl_count[sm.depth[n]], 1);
     }
     __syncthreads();
     if (tid == 0) {
@@ -435,7 +671,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     // which are contiguous in the output, with coalesced writes
     {
         uint32_t* tile = sm.stage + (size_t)warp * 32 * W;
-        for (int i0 = warp * 32; i0 < nmax; i0 += TREE_THREADS) {
+        for (int i0 = warp * 32; i0 < nmax && warp < TREE_MASK_WARPS; i0 += TREE_MASK_WARPS * 32) {
             const int i = i0 + lane;
             uint32_t* row = tile + lane * W;
             if (i < n_nodes) {
@@ -466,8 +702,9 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     __syncthreads();
     if (tid == 0 && o.d_state) {
         o.d_state[(size_t)b * 4 + 0] = (float)(t_prof1 - t_prof0);
-        o.d_state[(size_t)b * 4 + 1] = (float)(t_prof2 - t_prof1);
-        o.d_state[(size_t)b * 4 + 2] = (float)(clock64() - t_prof2);
+        o.d_state[(size_t)b * 4 + 1] = (float)(t_prof15 - t_prof1);
+        o.d_state[(size_t)b * 4 + 2] = (float)(t_prof2 - t_prof15);
+        o.d_state[(size_t)b * 4 + 3] = (float)(clock64() - t_prof2);
     }
 #endif
     if (tid == 0) {
@@ -513,7 +750,8 @@ __global__ void __launch_bounds__(128) accept_kernel(const int32_t* __restrict__
 }  // namespace
 
 size_t tree_smem_bytes(const graft_config& cfg) {
-    return tree_smem_layout(cfg.L, cfg.K, cfg.budget_max + 1, nullptr, nullptr);
+    const int nmax = cfg.budget_max + 1;
+    return tree_smem_layout(cfg.L, cfg.K, nmax, tree_node_cap(cfg.L, cfg.K, nmax), nullptr, nullptr);
 }
 
 cudaError_t tree_configure(const graft_config& cfg) {
@@ -552,6 +790,7 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     p.K = cfg.K;
     p.nmax = ctx->nmax;
     p.W = ctx->mask_words;
+    p.ncap = tree_node_cap(cfg.L, cfg.K, ctx->nmax);
     p.bmin = cfg.budget_min;
     p.bmax = cfg.budget_max;
     p.bstep = cfg.budget_step;

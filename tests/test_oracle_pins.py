@@ -292,8 +292,8 @@ def _edge_of(edge, t):
 
 def _best_first_rescan(edge, budget):
     """Independent restatement: rebuild the frontier from the selected set at every step.  Equal scores:
-    shorter prefix first, then the prefix whose parent was selected earlier, then under one parent the
-    larger edge score, then the lower candidate rank."""
+    shorter prefix first, then the lexicographically smaller parent, then under one parent the larger edge
+    score, then the lower candidate rank."""
     L, K, _ = edge.shape
     allp = _all_prefixes(edge)
     sel = []
@@ -302,7 +302,7 @@ def _best_first_rescan(edge, budget):
         frontier = [t for t in allp if t not in when and t[:-1] in when]
         if not frontier:
             break
-        best = min(frontier, key=lambda t: (-float(allp[t][0]), len(t), when[t[:-1]], -_edge_of(edge, t), t[-1]))
+        best = min(frontier, key=lambda t: (-float(allp[t][0]), len(t), t[:-1], -_edge_of(edge, t), t[-1]))
         when[best] = step + 1
         sel.append(best)
     return sel
@@ -360,18 +360,18 @@ def test_select_special_cases():
     tup, ln, S = oracle.select(e2, 1)
     assert ln.tolist() == [1] and tup[0, 0] == int(np.argmax(e2[0, 0])) and S[0] == e2[0, 0].max()
     assert len(oracle.select(e2, 0)[1]) == 0
-    # all scores equal: shorter first, then earlier-selected parent, then candidate rank
+    # all scores equal: shorter first, then the parent's ranks lexicographically, then candidate rank
     e3 = np.zeros((3, 2, 2), np.float32)
     tup, ln, S = oracle.select(e3, 6)
     assert [tuple(t[:n]) for t, n in zip(tup, ln)] == [(0,), (1,), (0, 0), (0, 1), (1, 0), (1, 1)]
-    # equal path scores, different parents: the prefix whose parent was selected earlier goes first, even
-    # when it is lexicographically later
+    # equal path scores, different parents: the lexicographically smaller parent goes first, even when it was
+    # selected later
     e5 = np.full((2, 2, 2), -9.0, np.float32)
     e5[0, 0] = [-1.0, 0.0]          # (1,) is selected first, then (0,)
     e5[1, 1, 0] = -5.0              # (1,0): 0 - 5
     e5[1, 0, 0] = -4.0              # (0,0): -1 - 4
     tup, ln, S = oracle.select(e5, 3)
-    assert [tuple(t[:n]) for t, n in zip(tup, ln)] == [(1,), (0,), (1, 0)] and S[2] == -5.0
+    assert [tuple(t[:n]) for t, n in zip(tup, ln)] == [(1,), (0,), (0, 0)] and S[2] == -5.0
     # equal path scores under one parent although the edges differ (4e7 + 1 and 4e7 + 2 both round to 4e7):
     # the larger edge first, here the higher rank
     e6 = np.full((2, 2, 2), -9.0, np.float32)
