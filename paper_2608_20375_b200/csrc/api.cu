@@ -124,7 +124,7 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     const size_t o_rec = take((size_t)ctx->num_sms * 2 * 2 * sizeof(VpRecord));
     const size_t o_cnt = take(B * L * sizeof(int));
     const size_t o_id = take(B * L * K * 4), o_lp = take(B * L * K * 4), o_lse = take(B * L * 4);
-    const size_t o_rs = take(B * L * 4), o_edge = take(B * L * K * K * 4), o_cos = take(B * L * 8);
+    const size_t o_rs = take(B * L * 4), o_edge = take(B * L * K * K * 4);
     const size_t o_es = take(B * L * K * K * 4), o_ei = take(B * L * K * K);
     const size_t o_u = take(L * (size_t)cfg->m * 4), o_err = take(256);
     ctx->ws_bytes = off;
@@ -149,7 +149,6 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     ctx->w_lse = (float*)(base + o_lse);
     ctx->w_row_status = (int32_t*)(base + o_rs);
     ctx->w_edge = (float*)(base + o_edge);
-    ctx->w_cos = (double*)(base + o_cos);
     ctx->w_esort = (float*)(base + o_es);
     ctx->w_eidx = (uint8_t*)(base + o_ei);
     ctx->d_u = (float*)(base + o_u);
@@ -317,7 +316,6 @@ graft_status graft_build_trees(graft_ctx* ctx, int32_t batch, const void* d_logi
     float* lse = out->d_lse ? out->d_lse : ctx->w_lse;
     float* edge = out->d_edge ? out->d_edge : ctx->w_edge;
 
-    if (use_saba && cosine_launch(ctx, batch, d_hidden, ctx->w_cos, st) != cudaSuccess) return GRAFT_ERR_CUDA;
     if (ev) cudaEventRecord(ev[0], st);
     if (vp_launch(ctx, batch, d_logits, ids, lps, lse, ctx->w_row_status, st) != cudaSuccess) return GRAFT_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], st);
@@ -325,7 +323,7 @@ graft_status graft_build_trees(graft_ctx* ctx, int32_t batch, const void* d_logi
         cudaSuccess)
         return GRAFT_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], st);
-    if (tree_launch(ctx, batch, ids, lps, ctx->w_row_status, ctx->w_esort, ctx->w_eidx, ctx->w_cos, d_root_token, d_hist, d_prefix_len,
+    if (tree_launch(ctx, batch, ids, lps, ctx->w_row_status, ctx->w_esort, ctx->w_eidx, d_hidden, d_root_token, d_hist, d_prefix_len,
                     d_fixed_budget, out, st) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     if (ev) {

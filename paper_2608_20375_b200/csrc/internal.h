@@ -70,7 +70,6 @@ struct graft_ctx {
     float* w_edge;                // [max_batch, L, K, K]
     float* w_esort;               // [max_batch, L, K, K] rows sorted by edge score
     uint8_t* w_eidx;              // [max_batch, L, K, K] child rank of each sorted entry
-    double* w_cos;                // [max_batch, L]   adjacent-row cosines r_d
     int32_t* w_errflag;           // [1] device-side internal error flag
     graft::VpPlan vp_plan;
     // host-buffer staging (allocated on first use of graft_build_trees_host)
@@ -94,9 +93,8 @@ cudaError_t tdes_precompute_launch(graft_ctx* ctx, const void* d_emb, graft_dtyp
 cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                               const int32_t* d_root_token, const int32_t* d_row_status, float* d_edge,
                               float* d_esort, uint8_t* d_eidx, cudaStream_t st);
-cudaError_t cosine_launch(graft_ctx* ctx, int batch, const void* d_hidden, double* d_cos, cudaStream_t st);
 cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
-                        const int32_t* d_row_status, const float* d_esort, const uint8_t* d_eidx, const double* d_cos,
+                        const int32_t* d_row_status, const float* d_esort, const uint8_t* d_eidx, const void* d_hidden,
                         const int32_t* d_root_token, const float* d_hist, const int32_t* d_prefix_len,
                         const int32_t* d_fixed_budget, const graft_tree_out* out, cudaStream_t st);
 cudaError_t accept_launch(graft_ctx* ctx, int batch, const graft_tree_out* trees, const int32_t* d_target_next,

@@ -7,47 +7,6 @@
 namespace graft {
 namespace {
 
-// ---- adjacent-position cosines r_d = cos(h_d, h_{d+1}) (Eq. 15), one CTA per (sequence, d) ------------
-template <bool BF16>
-__global__ void __launch_bounds__(128) cosine_kernel(const void* __restrict__ hidden, double* __restrict__ cosv, int L,
-                                                     int dh) {
-    const int b = blockIdx.x / (L - 1), d = blockIdx.x % (L - 1);
-    const size_t ra = ((size_t)b * L + d) * dh, rb = ra + dh;
-    double ab = 0.0, aa = 0.0, bb = 0.0;
-    for (int k = threadIdx.x; k < dh; k += 128) {
-        float x, y;
-        if (BF16) {
-            x = __uint_as_float(((uint32_t)((const uint16_t*)hidden)[ra + k]) << 16);
-            y = __uint_as_float(((uint32_t)((const uint16_t*)hidden)[rb + k]) << 16);
-        } else {
-            x = ((const float*)hidden)[ra + k];
-            y = ((const float*)hidden)[rb + k];
-        }
-        ab += (double)x * (double)y;
-        aa += (double)x * (double)x;
-        bb += (double)y * (double)y;
-    }
-    __shared__ double red[3][4];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        ab += __shfl_xor_sync(0xFFFFFFFFu, ab, o);
-        aa += __shfl_xor_sync(0xFFFFFFFFu, aa, o);
-        bb += __shfl_xor_sync(0xFFFFFFFFu, bb, o);
-    }
-    if ((threadIdx.x & 31) == 0) {
-        red[0][threadIdx.x >> 5] = ab;
-        red[1][threadIdx.x >> 5] = aa;
-        red[2][threadIdx.x >> 5] = bb;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        ab = red[0][0] + red[0][1] + red[0][2] + red[0][3];
-        aa = red[1][0] + red[1][1] + red[1][2] + red[1][3];
-        bb = red[2][0] + red[2][1] + red[2][2] + red[2][3];
-        cosv[(size_t)b * L + d] = (aa > 0.0 && bb > 0.0) ? ab / (sqrt(aa) * sqrt(bb)) : 0.0;
-    }
-}
-
 // ---- tree kernel -------------------------------------------------------------------------------------------
 struct TreeParams {
     const int32_t* topk_id;
@@ -55,7 +14,8 @@ struct TreeParams {
     const int32_t* row_status;
     const float* esort;   // [batch, L, K, K] edge rows sorted by (edge desc, child rank asc)
     const uint8_t* eidx;  // child rank of each sorted entry
-    const double* cosv;
+    const void* hidden;   // [batch, L, hidden_dim] (SABA only)
+    int hidden_dim, hidden_bf16;
     const int32_t* root_token;
     const float* hist;
     const int32_t* prefix_len;
@@ -68,7 +28,6 @@ struct TreeParams {
 };
 
 constexpr int TREE_THREADS = 1024;  // one CTA per SM (shared memory bound): all warps serve the parallel phases
-constexpr int TREE_MASK_WARPS = 8;  // warps that build mask rows (each needs a 32-row staging tile)
 
 struct TreeSmem {
     float* es;           // [L*K*K]  sorted edge rows
@@ -90,10 +49,11 @@ struct TreeSmem {
     int16_t* lvl_list;   // [nmax]
     int* cc;             // [nmax]   per-level child counts in level order, then their exclusive scan
     uint32_t* stage;     // [8 warps * 32 rows * W] mask rows staged for coalesced stores
-    uint32_t* hist;      // [4 * 256]
+    uint32_t* hist;      // [2 * 4 * 256]
     int* lvl_count;      // [kMaxL + 2]
     int* lvl_start;      // [kMaxL + 2]
     int* lvl_fill;       // [kMaxL + 2]
+    double* cosv;        // [kMaxL]  adjacent-position cosines r_d (Eq. 15)
     int* scal;           // [16] 0 budget, 1 n_nodes, 2 status, 3 table size, 4 overflow, 6/7 radix-select hand-over
 };
 
@@ -111,8 +71,8 @@ __host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, int n
     size_t o_tab = take(table > emis ? table : emis);
     size_t o_ent = take((size_t)nmax * 8), o_S = take((size_t)nmax * 4), o_chm = take((size_t)nmax * 4),
            o_par = take((size_t)nmax * 2), o_can = take((size_t)nmax * 2), o_cp = take((size_t)nmax * 2),
-           o_cand = take(nmax), o_dep = take(nmax), o_hist = take(1024 * 4), o_lc = take((kMaxL + 2) * 4),
-           o_ls = take((kMaxL + 2) * 4), o_lf = take((kMaxL + 2) * 4), o_sc = take(16 * 4);
+           o_cand = take(nmax), o_dep = take(nmax), o_hist = take(2048 * 4), o_lc = take((kMaxL + 2) * 4),
+           o_ls = take((kMaxL + 2) * 4), o_lf = take((kMaxL + 2) * 4), o_sc = take(16 * 4), o_cos = take(kMaxL * 8);
     if (s) {
         s->es = (float*)(base + o_es);
         s->ei = base + o_ei;
@@ -135,6 +95,7 @@ __host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, int n
         s->lvl_start = (int*)(base + o_ls);
         s->lvl_fill = (int*)(base + o_lf);
         s->scal = (int*)(base + o_sc);
+        s->cosv = (double*)(base + o_cos);
     }
     return off;
 }
@@ -199,24 +160,31 @@ __device__ __forceinline__ bool entry_before(const TreeSmem& sm, uint64_t e1, in
 }
 
 // B-th largest of keys[lo..hi) (hi - lo >= kth >= 1) by an 8-bit radix select; every thread of the CTA calls it.
-__device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, int lo, int hi, int kth, int tid) {
+// With passes < 4 only the top 8 * passes bits are resolved and the rest is returned as zero: a lower bound
+// of the B-th largest key.  The 256 bins exist in four copies (neighbouring warps use different ones) and in two
+// generations, so that the next pass's bins are cleared while this pass's are scanned.
+__device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, int lo, int hi, int kth, int passes,
+                                    int tid) {
     const int warp = tid >> 5, lane = tid & 31;
     uint32_t prefix = 0, mask = 0;
     int remaining = kth;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        sm.hist[tid] = 0u;  // four copies of the 256 bins (TREE_THREADS == 1024): neighbouring warps do not collide
-        __syncthreads();
+    sm.hist[tid] = 0u;
+    __syncthreads();
+    for (int pass = 0; pass < passes; ++pass) {
+        const int shift = 24 - 8 * pass;
+        uint32_t* h = sm.hist + (pass & 1) * 1024;
         for (int i = lo + tid; i < hi; i += TREE_THREADS) {
             const uint32_t k = keys[i];
-            if ((k & mask) == prefix) atomicAdd(&sm.hist[(warp & 3) * 256 + ((k >> shift) & 255u)], 1u);
+            if ((k & mask) == prefix) atomicAdd(&h[(warp & 3) * 256 + ((k >> shift) & 255u)], 1u);
         }
+        sm.hist[((pass + 1) & 1) * 1024 + tid] = 0u;  // the other generation, for the next pass
         __syncthreads();
         if (warp == 0) {  // lane l owns bins 255-8l .. 248-8l, from the top down
             int c[8], sum = 0;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const int bin = 255 - 8 * lane - j;
-                c[j] = (int)(sm.hist[bin] + sm.hist[256 + bin] + sm.hist[512 + bin] + sm.hist[768 + bin]);
+                c[j] = (int)(h[bin] + h[256 + bin] + h[512 + bin] + h[768 + bin]);
                 sum += c[j];
             }
             int incl = sum;
@@ -260,15 +228,93 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
 #ifdef GRAFT_TREE_PROF
     long long t_prof0 = clock64(), t_prof1 = 0, t_prof2 = 0, t_prof15 = 0;
 #endif
-    {
-        const int ne = L * K * K;
-        if ((ne & 3) == 0) {
-            const float4* src = (const float4*)(p.esort + (size_t)b * ne);
-            for (int i = tid; i < ne / 4; i += TREE_THREADS) ((float4*)sm.es)[i] = src[i];
-        } else {
-            for (int i = tid; i < ne; i += TREE_THREADS) sm.es[i] = p.esort[(size_t)b * ne + i];
+    // the sorted edge rows of this sequence: bulk copies through the TMA unit when the 16-byte rules allow it
+    // (they land while warp 0 works out the budget), plain loads otherwise
+    __shared__ __align__(8) uint64_t rows_bar;
+    const int ne = L * K * K;
+    const bool bulk = (ne % 16) == 0;
+    if (bulk) {
+        if (tid == 0) {
+            mbar_init(smem_u32(&rows_bar), 1);
+            mbar_fence_init();
+            mbar_arrive_expect_tx(smem_u32(&rows_bar), (uint32_t)ne * 5u);
+            const char* g_es = (const char*)(p.esort + (size_t)b * ne);
+            const char* g_ei = (const char*)(p.eidx + (size_t)b * ne);
+            for (uint32_t off = 0; off < (uint32_t)ne * 4u; off += 16384u) {
+                const uint32_t bytes = (uint32_t)ne * 4u - off < 16384u ? (uint32_t)ne * 4u - off : 16384u;
+                tma_load_1d(smem_u32((char*)sm.es + off), g_es + off, bytes, smem_u32(&rows_bar));
+            }
+            for (uint32_t off = 0; off < (uint32_t)ne; off += 16384u) {
+                const uint32_t bytes = (uint32_t)ne - off < 16384u ? (uint32_t)ne - off : 16384u;
+                tma_load_1d(smem_u32((char*)sm.ei + off), g_ei + off, bytes, smem_u32(&rows_bar));
+            }
         }
-        for (int i = tid; i < L * K * K; i += TREE_THREADS) sm.ei[i] = p.eidx[(size_t)b * L * K * K + i];
+    } else {
+        for (int i = tid; i < ne; i += TREE_THREADS) {
+            sm.es[i] = p.esort[(size_t)b * ne + i];
+            sm.ei[i] = p.eidx[(size_t)b * ne + i];
+        }
+    }
+    // adjacent-position cosines r_d = cos(h_d, h_{d+1}) (Eq. 15): one warp per pair, fp64 accumulation
+    if (p.use_saba) {
+        for (int d = warp; d < L - 1; d += TREE_THREADS / 32) {
+            const int dh = p.hidden_dim;
+            const size_t ra = ((size_t)b * L + d) * dh, rb = ra + dh;
+            double ab = 0.0, aa = 0.0, bb = 0.0;
+            if (p.hidden_bf16 && (dh & 7) == 0 && ((uintptr_t)p.hidden & 15) == 0) {
+                const uint4* pa = (const uint4*)((const uint16_t*)p.hidden + ra);
+                const uint4* pb = (const uint4*)((const uint16_t*)p.hidden + rb);
+                constexpr int CU = 4;  // vectors in flight per row and lane: the loads of a step are issued together
+                for (int k0 = lane; k0 < dh / 8; k0 += 32 * CU) {
+                    uint4 va[CU], vb[CU];
+#pragma unroll
+                    for (int u = 0; u < CU; ++u) {
+                        const int k = k0 + 32 * u;
+                        va[u] = k < dh / 8 ? pa[k] : make_uint4(0u, 0u, 0u, 0u);
+                        vb[u] = k < dh / 8 ? pb[k] : make_uint4(0u, 0u, 0u, 0u);
+                    }
+#pragma unroll
+                    for (int u = 0; u < CU; ++u) {
+                        const uint32_t wa[4] = {va[u].x, va[u].y, va[u].z, va[u].w};
+                        const uint32_t wb[4] = {vb[u].x, vb[u].y, vb[u].z, vb[u].w};
+                        float fab = 0.f, faa = 0.f, fbb = 0.f;  // eight exact bf16 products per sum: fp32 is enough
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float x0 = __uint_as_float(wa[q] << 16), x1 = __uint_as_float(wa[q] & 0xFFFF0000u);
+                            const float y0 = __uint_as_float(wb[q] << 16), y1 = __uint_as_float(wb[q] & 0xFFFF0000u);
+                            fab = fmaf(x0, y0, fmaf(x1, y1, fab));
+                            faa = fmaf(x0, x0, fmaf(x1, x1, faa));
+                            fbb = fmaf(y0, y0, fmaf(y1, y1, fbb));
+                        }
+                        ab += (double)fab;
+                        aa += (double)faa;
+                        bb += (double)fbb;
+                    }
+                }
+            } else {
+                for (int k = lane; k < dh; k += 32) {
+                    float x, y;
+                    if (p.hidden_bf16) {
+                        x = __uint_as_float(((uint32_t)((const uint16_t*)p.hidden)[ra + k]) << 16);
+                        y = __uint_as_float(((uint32_t)((const uint16_t*)p.hidden)[rb + k]) << 16);
+                    } else {
+                        x = ((const float*)p.hidden)[ra + k];
+                        y = ((const float*)p.hidden)[rb + k];
+                    }
+                    ab += (double)x * (double)y;
+                    aa += (double)x * (double)x;
+                    bb += (double)y * (double)y;
+                }
+            }
+#pragma unroll
+            for (int o2 = 16; o2 > 0; o2 >>= 1) {
+                ab += __shfl_xor_sync(0xFFFFFFFFu, ab, o2);
+                aa += __shfl_xor_sync(0xFFFFFFFFu, aa, o2);
+                bb += __shfl_xor_sync(0xFFFFFFFFu, bb, o2);
+            }
+            if (lane == 0) sm.cosv[d] = (aa > 0.0 && bb > 0.0) ? ab / (sqrt(aa) * sqrt(bb)) : 0.0;
+        }
+        __syncthreads();
     }
     if (warp == 0) {
         int st = 0;
@@ -283,7 +329,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             } else {
                 double conf = 0.0, rs = 0.0;
                 for (int j = lane; j < L; j += 32) conf += exp((double)p.topk_lp[((size_t)b * L + j) * K]);
-                for (int j = lane; j < L - 1; j += 32) rs += p.cosv[(size_t)b * L + j];
+                for (int j = lane; j < L - 1; j += 32) rs += sm.cosv[j];
 #pragma unroll
                 for (int d = 16; d > 0; d >>= 1) {
                     conf += __shfl_xor_sync(0xFFFFFFFFu, conf, d);
@@ -291,7 +337,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 }
                 conf /= (double)L;
                 double degen = 0.0;
-                if (L >= 2) degen = rs / (double)(L - 1) + (p.cosv[(size_t)b * L + L - 2] - p.cosv[(size_t)b * L]);
+                if (L >= 2) degen = rs / (double)(L - 1) + (sm.cosv[L - 2] - sm.cosv[0]);
                 const double hist = (double)p.hist[b];
                 double tau = p.saba.phi_conf * conf + p.saba.phi_degen * degen + p.saba.phi_hist * hist + p.saba.phi_bias;
                 if (!(tau >= p.saba.tau_min)) {
@@ -334,6 +380,14 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         }
     }
     __syncthreads();
+    if (bulk) {
+        // bounded wait for the bulk copies; on a timeout the sequence is reported through its status word
+        __shared__ int rows_abort;
+        if (tid == 0) rows_abort = 0;
+        __syncthreads();
+        if (!mbar_wait_bounded(smem_u32(&rows_bar), 0, &rows_abort) && tid == 0) sm.scal[2] |= GRAFT_ST_INTERNAL;
+        __syncthreads();
+    }
 
 #ifdef GRAFT_TREE_PROF
     t_prof1 = clock64();
@@ -440,7 +494,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             // theta only has to be a lower bound of its final value while the levels are built (it prunes), so
             // the exact B-th largest key is recomputed only when the table has grown noticeably
             if (ntot - 1 >= budget && (theta == 0u || ntot - n_at_select >= ntot / 2)) {
-                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, tid);
+                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 2, tid);  // a 16-bit lower bound is enough here
                 n_at_select = ntot;
             }
             __syncthreads();
@@ -455,9 +509,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
 #endif
         }
         __syncthreads();
-        if (table_ok && ntot - 1 >= budget && n_at_select != ntot) {
-            theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, tid);  // the exact final value
-        }
+        if (table_ok && ntot - 1 >= budget) theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 4, tid);  // exact
         __syncthreads();
         if (table_ok) {
             // compact {key > theta} in table order (parents stay before their children)
@@ -668,10 +720,15 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     __syncthreads();
     // ancestor masks: each thread builds one row in its warp's staging tile (walking up, level-order indices
     // only decrease, so the row is produced from its highest word down); the warp then stores its 32 rows,
-    // which are contiguous in the output, with coalesced writes
+    // which are contiguous in the output, with coalesced writes.  Padding rows are zero-filled directly.
     {
+        const size_t stage_off = (((size_t)nmax * 2 + 15) & ~(size_t)15) + (((size_t)nmax * 4 + 15) & ~(size_t)15);
+        const size_t region = (size_t)p.ncap * 12 > stage_off + (size_t)8 * 32 * W * 4 ? (size_t)p.ncap * 12
+                                                                                         : stage_off + (size_t)8 * 32 * W * 4;
+        int mw = (int)((region - stage_off) / ((size_t)32 * W * 4));
+        mw = mw > TREE_THREADS / 32 ? TREE_THREADS / 32 : mw;
         uint32_t* tile = sm.stage + (size_t)warp * 32 * W;
-        for (int i0 = warp * 32; i0 < nmax && warp < TREE_MASK_WARPS; i0 += TREE_MASK_WARPS * 32) {
+        for (int i0 = warp * 32; i0 < n_nodes && warp < mw; i0 += mw * 32) {
             const int i = i0 + lane;
             uint32_t* row = tile + lane * W;
             if (i < n_nodes) {
@@ -697,6 +754,9 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             for (int k = lane; k < rows * W; k += 32) dst[k] = tile[k];
             __syncwarp();
         }
+        // rows from the first multiple of 32 at or above n_nodes on are all padding
+        const int z0 = ((n_nodes + 31) / 32) * 32;
+        for (size_t k = (size_t)z0 * W + tid; k < (size_t)nmax * W; k += TREE_THREADS) o.d_mask[ob * W + k] = 0u;
     }
 #ifdef GRAFT_TREE_PROF
     __syncthreads();
@@ -714,26 +774,50 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     }
 }
 
-// ---- acceptance walk: one warp per sequence --------------------------------------------------------------
+// ---- acceptance walk: one warp per sequence ------------------------------------------------------------------
+// The tree (parents, tokens) and the target's next tokens are staged in shared memory with one coalesced read;
+// the walk itself then runs out of shared memory.  In level order the parent indices never decrease, so the
+// children of the current node are found by a binary search for the first node whose parent is >= it.
 __global__ void __launch_bounds__(128) accept_kernel(const int32_t* __restrict__ n_nodes, const int32_t* __restrict__ token,
                                                      const int32_t* __restrict__ parent,
                                                      const int32_t* __restrict__ target_next, int batch, int nmax, int L,
                                                      int32_t* __restrict__ accept_len, int32_t* __restrict__ accept_path,
                                                      int32_t* __restrict__ bonus) {
-    const int b = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    extern __shared__ __align__(16) int32_t acc_smem[];
+    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x * 4 + wib;
     if (b >= batch) return;
+    int32_t* par = acc_smem + (size_t)wib * 3 * nmax;
+    int32_t* tok = par + nmax;
+    int32_t* tn = tok + nmax;
     const size_t ob = (size_t)b * nmax;
     int nn = n_nodes[b];
     nn = nn < 1 ? 1 : (nn > nmax ? nmax : nn);
+    for (int i = lane; i < nn; i += 32) {
+        par[i] = parent[ob + i];
+        tok[i] = token[ob + i];
+        tn[i] = target_next[ob + i];
+    }
+    __syncwarp();
     int cur = 0, a = 0;
     while (a < L) {
-        const int want = target_next[ob + cur];
+        const int want = tn[cur];
+        int lo = cur + 1, hi = nn;  // first index in (cur, nn) whose parent is >= cur
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (par[mid] >= cur)
+                hi = mid;
+            else
+                lo = mid + 1;
+        }
         int found = -1;
-        for (int i0 = cur + 1; i0 < nn && found < 0; i0 += 32) {  // children come after their parent
+        for (int i0 = lo; i0 < nn && found < 0; i0 += 32) {  // the children of cur are contiguous from lo on
             const int i = i0 + lane;
-            const bool hit = i < nn && parent[ob + i] == cur && token[ob + i] == want;
-            const uint32_t m = __ballot_sync(0xFFFFFFFFu, hit);
-            if (m) found = i0 + __ffs(m) - 1;
+            const bool child = i < nn && par[i] == cur;
+            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, child && tok[i] == want);
+            const uint32_t more = __ballot_sync(0xFFFFFFFFu, child);
+            if (hit) found = i0 + __ffs(hit) - 1;
+            if (more != 0xFFFFFFFFu) break;  // ran past the last child
         }
         if (found < 0) break;
         if (lane == 0) accept_path[(size_t)b * L + a] = found;
@@ -743,7 +827,7 @@ __global__ void __launch_bounds__(128) accept_kernel(const int32_t* __restrict__
     for (int i = a + lane; i < L; i += 32) accept_path[(size_t)b * L + i] = -1;
     if (lane == 0) {
         accept_len[b] = a;
-        bonus[b] = target_next[ob + cur];
+        bonus[b] = tn[cur];
     }
 }
 
@@ -758,19 +842,8 @@ cudaError_t tree_configure(const graft_config& cfg) {
     return cudaFuncSetAttribute(tree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tree_smem_bytes(cfg));
 }
 
-cudaError_t cosine_launch(graft_ctx* ctx, int batch, const void* d_hidden, double* d_cos, cudaStream_t st) {
-    const graft_config& cfg = ctx->cfg;
-    if (cfg.L < 2) return cudaSuccess;
-    if (cfg.hidden_dtype == GRAFT_BF16)
-        cosine_kernel<true><<<batch * (cfg.L - 1), 128, 0, st>>>(d_hidden, d_cos, cfg.L, cfg.hidden_dim);
-    else
-        cosine_kernel<false><<<batch * (cfg.L - 1), 128, 0, st>>>(d_hidden, d_cos, cfg.L, cfg.hidden_dim);
-    ctx->launches += 1;
-    return cudaGetLastError();
-}
-
 cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
-                        const int32_t* d_row_status, const float* d_esort, const uint8_t* d_eidx, const double* d_cos,
+                        const int32_t* d_row_status, const float* d_esort, const uint8_t* d_eidx, const void* d_hidden,
                         const int32_t* d_root_token, const float* d_hist, const int32_t* d_prefix_len,
                         const int32_t* d_fixed_budget, const graft_tree_out* out, cudaStream_t st) {
     const graft_config& cfg = ctx->cfg;
@@ -780,7 +853,9 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     p.row_status = d_row_status;
     p.esort = d_esort;
     p.eidx = d_eidx;
-    p.cosv = d_cos;
+    p.hidden = d_hidden;
+    p.hidden_dim = cfg.hidden_dim;
+    p.hidden_bf16 = cfg.hidden_dtype == GRAFT_BF16 ? 1 : 0;
     p.root_token = d_root_token;
     p.hist = d_hist;
     p.prefix_len = d_prefix_len;
@@ -803,7 +878,7 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
 
 cudaError_t accept_launch(graft_ctx* ctx, int batch, const graft_tree_out* trees, const int32_t* d_target_next,
                           int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus, cudaStream_t st) {
-    accept_kernel<<<(batch + 3) / 4, 128, 0, st>>>(trees->d_n_nodes, trees->d_token, trees->d_parent, d_target_next,
+    accept_kernel<<<(batch + 3) / 4, 128, (size_t)4 * 3 * ctx->nmax * sizeof(int32_t), st>>>(trees->d_n_nodes, trees->d_token, trees->d_parent, d_target_next,
                                                    batch, ctx->nmax, ctx->cfg.L, d_accept_len, d_accept_path, d_bonus);
     ctx->launches += 1;
     return cudaGetLastError();

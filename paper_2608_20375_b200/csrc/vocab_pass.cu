@@ -399,6 +399,9 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
     cm_t* cmax = (cm_t*)(sh + 1);  // [2][n_cmax]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef GRAFT_VP_PROF
+    const long long t_kernel0 = clock64();
+#endif
     const long long G = gridDim.x;
     const long long q0 = cta_start(blockIdx.x, p.Q, G), q1 = cta_start(blockIdx.x + 1, p.Q, G);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 8);
@@ -509,6 +512,9 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
             __syncwarp();
             if (lane == 0) mbar_arrive(ready0 + 8 * pb);
         }
+#ifdef GRAFT_VP_PROF
+        if (warp == 0 && lane == 0 && blockIdx.x < 8) p.errflag[16 + blockIdx.x * 2] = (int)((clock64() - t_kernel0) >> 4);
+#endif
     } else {
         // ------------------------------ epilogue group (four warps) ------------------------------
         // Warp 0 of the group owns the hand-over barriers and the sequential parts; the data-parallel parts
@@ -810,6 +816,9 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
         }
     }
     __syncthreads();
+#ifdef GRAFT_VP_PROF
+    if (tid == 0 && blockIdx.x < 8) p.errflag[17 + blockIdx.x * 2] = (int)((clock64() - t_kernel0) >> 4);
+#endif
     if (tid == 0 && sh->abort_flag) atomicOr(p.errflag, 1);
 }
 
