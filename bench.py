@@ -259,7 +259,7 @@ def run_graft(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "us_per_round": ms_step * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32 (on bf16 logits; fp64 for the SABA scalars)", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{w.name}: batch {batch} per GPU, L={w.L}, V={w.V} {w.logits_dtype} logits, "
                                f"hidden d={w.hidden_dim} {w.hidden_dtype}, K={w.K}, m={w.m}, beta={w.beta}, SABA budgets "
                                f"[{w.budget_min},{w.budget_max}] step {w.budget_step}, build_trees + accept",
@@ -281,7 +281,7 @@ def run_graft(args):
     if world == 1 and not args.no_cpu_baseline:
         cores = os.cpu_count() or 1
         threads = min(cores, 32)
-        n_seq = min(batch, max(threads, 2 * threads if w.V < 100000 else threads))
+        n_seq = batch  # the whole batch of input set 0: about 20 s of CPU work at workload M
         s = host_sets[0]
         sub = {k: s[k][:n_seq] for k in ("logits", "hidden", "root_token", "hist", "prefix_len")}
         sub["fixed_budget"] = None if w.fixed_budget is None else torch.full((n_seq,), w.fixed_budget, dtype=torch.int32)
