@@ -12,11 +12,13 @@ constexpr int kMaxL = 32;
 constexpr int kMaxCostPts = 16;
 
 // ---- vocab pass -----------------------------------------------------------------------------
-constexpr int kVpConsumerWarps = 8;
-constexpr int kVpConsumers = kVpConsumerWarps * 32;  // 256
-constexpr int kVpEpiThreads = 128;                   // four epilogue warps
-constexpr int kVpThreads = kVpConsumers + kVpEpiThreads + 32;  // + one producer warp
-constexpr int kVpTileBytes = 16384;                  // one TMA bulk copy
+constexpr int kVpConsumerWarps = 16;                 // streaming warps (one CTA per SM)
+constexpr int kVpConsumers = kVpConsumerWarps * 32;  // 512
+constexpr int kVpEpiThreads = 128;                   // four warps per epilogue group
+constexpr int kVpEpiGroups = 2;                      // the groups take alternate segments
+constexpr int kVpBufs = 4;                           // hand-over buffers between streaming and epilogue warps
+constexpr int kVpThreads = kVpConsumers + kVpEpiGroups * kVpEpiThreads + 32;  // + one producer warp
+constexpr int kVpTileBytes = 32768;                  // one ring stage (2 KiB per streaming warp)
 constexpr int kVpQuantum = 2048;                     // elements; granularity of the work partition
 constexpr int kVpCandCap = 1024;                     // candidate keys held in shared memory
 constexpr int kVpHitCap = 512;                       // chunk hits held in shared memory

@@ -41,12 +41,13 @@ namespace {
 
 constexpr int NW = kVpConsumerWarps;          // streaming warps
 constexpr int NT = kVpConsumers;              // streaming threads
-constexpr int PROD_WARP = NW + kVpEpiThreads / 32;  // warp index of the producer warp
+constexpr int PROD_WARP = NW + kVpEpiGroups * kVpEpiThreads / 32;  // warp index of the producer warp
 constexpr int TILE = kVpTileBytes;
 constexpr int WBLK = TILE / NW;               // bytes of a tile owned by one warp (2048)
+static_assert(WBLK == 2048, "one warp owns 2 KiB of every tile");
 constexpr int VEC_PER_LANE = WBLK / 16 / 32;  // 4
 static_assert(VEC_PER_LANE == 4, "chunk layout assumes four 16-byte vectors per lane per tile");
-static_assert(kVpThreads == NT + kVpEpiThreads + 32, "thread count = streaming warps + epilogue warps + producer warp");
+static_assert(kVpThreads == NT + kVpEpiGroups * kVpEpiThreads + 32, "thread count = streaming warps + epilogue warps + producer warp");
 
 template <bool BF16>
 struct VT;
@@ -58,7 +59,7 @@ struct VT<true> {
 };
 template <>
 struct VT<false> {
-    using cm_t = uint32_t;
+    using cm_t = uint16_t;  // the chunk maximum rounded UP to bf16 precision: an upper bound is all the scan needs
     static constexpr int ESZ = 4, EPV = 4, CH = 16;
     static constexpr uint32_t NEG_INF_WORD = 0xFF800000u;
 };
@@ -79,6 +80,7 @@ struct VpParams {
     int32_t* row_status;
     int32_t* errflag;
     int use_hint;
+    float* dbg_out;  // profiling builds only
     int dbg;  // experiments only: 1 = stream without arithmetic, 2 = arithmetic without streaming, 3 = no epilogue
 };
 
@@ -242,7 +244,11 @@ __device__ __forceinline__ void process_chunk(const uint4* __restrict__ wb, int 
                                fmaxf(__uint_as_float(v[i].z), __uint_as_float(v[i].w))));
         }
         cm = m;
-        *cmax_slot = (typename T::cm_t)__float_as_uint(cm);
+        {
+            // round toward +inf onto the bf16 grid: positive values round their magnitude up, negative ones truncate
+            const uint32_t mb = __float_as_uint(cm);
+            *cmax_slot = (typename T::cm_t)((mb >> 31) ? (mb >> 16) : ((mb + 0xFFFFu) >> 16));
+        }
     }
     uint32_t o = ord_from_float(cm);
     a.tmo = o > a.tmo ? o : a.tmo;
@@ -307,19 +313,23 @@ __device__ __forceinline__ void process_chunk(const uint4* __restrict__ wb, int 
 }
 
 // ---- shared-memory control block ---------------------------------------------------------------
-struct __align__(16) VpShared {
-    uint64_t cand[kVpCandCap];  // epilogue warp only
+struct __align__(16) EpiShared {  // private to one epilogue group
+    uint64_t cand[kVpCandCap];
     uint64_t outk[kMaxK];
     uint32_t hits[kVpHitCap];
-    uint32_t tmax[2][NT];       // per-thread maxima of a finished segment, double-buffered by segment parity
-    float wc[2][NW], ws[2][NW];
-    uint16_t hthreads[NT];      // epilogue warp only: streaming threads whose maximum reaches T
-    int nhits, ncand, nht, ovf;  // epilogue group only
+    uint16_t hthreads[NT];  // streaming threads whose maximum reaches T
+    int nhits, ncand, nht, ovf;
     uint32_t Tv;
+};
+struct __align__(16) VpShared {
+    EpiShared epi[kVpEpiGroups];
+    uint32_t tmax[kVpBufs][NT];  // per-thread maxima of a finished segment, one buffer per segment in flight
+    float wc[kVpBufs][NW], ws[kVpBufs][NW];
+    long long t_stream_end;      // profiling builds only
     volatile int abort_flag;
 };
 
-__device__ __forceinline__ void epi_bar() { named_bar_sync(2, kVpEpiThreads); }
+__device__ __forceinline__ void epi_bar(int group) { named_bar_sync(2 + group, kVpEpiThreads); }
 
 // ---- epilogue-warp helpers (32 threads, warp-synchronous) ----------------------------------------------
 // Append `key` for the lanes with pred set; returns the new count.  Entries beyond the capacity are dropped
@@ -344,7 +354,7 @@ __device__ __forceinline__ int warp_append(uint64_t* buf, int n, int cap, bool p
 
 // Exact top-K of cand[0..n) by rank counting; result sorted descending in outk[0..min(n,K)).  Keys are
 // distinct (ids are), so ranks are a permutation.
-__device__ void warp_select_topk(VpShared* sh, int n, int K, int lane) {
+__device__ void warp_select_topk(EpiShared* sh, int n, int K, int lane) {
     __syncwarp();
     for (int i = lane; i < n; i += 32) {
         const uint64_t key = sh->cand[i];
@@ -358,7 +368,7 @@ __device__ void warp_select_topk(VpShared* sh, int n, int K, int lane) {
 // Exact selection over a whole segment straight from global memory, in slices small enough that the key
 // buffer cannot overflow.  Used only when the fast path's buffers overflowed.
 template <bool BF16>
-__device__ int warp_fallback_select(VpShared* sh, const VpParams& p, const Seg& sg, int lane) {
+__device__ int warp_fallback_select(EpiShared* sh, const VpParams& p, const Seg& sg, int lane) {
     using T = VT<BF16>;
     const int K = p.K;
     const int slice = kVpCandCap - kMaxK;
@@ -389,14 +399,14 @@ __device__ int warp_fallback_select(VpShared* sh, const VpParams& p, const Seg& 
 }
 
 template <bool BF16>
-__global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParams p) {
+__global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParams p) {
     using T = VT<BF16>;
     using cm_t = typename T::cm_t;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     unsigned char* ring = smem_raw;
-    uint64_t* bars = (uint64_t*)(ring + (size_t)p.stages * TILE);  // full[8], empty[8], part_ready[2], epi_done[2]
+    uint64_t* bars = (uint64_t*)(ring + (size_t)p.stages * TILE);  // full[8], empty[8], ready[4], done[4]
     VpShared* sh = (VpShared*)(bars + 24);
-    cm_t* cmax = (cm_t*)(sh + 1);  // [2][n_cmax]
+    cm_t* cmax = (cm_t*)(sh + 1);  // [kVpBufs][n_cmax]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef GRAFT_VP_PROF
@@ -405,14 +415,14 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
     const long long G = gridDim.x;
     const long long q0 = cta_start(blockIdx.x, p.Q, G), q1 = cta_start(blockIdx.x + 1, p.Q, G);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 8);
-    const uint32_t ready0 = smem_u32(bars + 16), done0 = smem_u32(bars + 18);
+    const uint32_t ready0 = smem_u32(bars + 16), done0 = smem_u32(bars + 20);
 
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, NW);
         }
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < kVpBufs; ++s) {
             mbar_init(ready0 + 8 * s, NW);
             mbar_init(done0 + 8 * s, 1);
         }
@@ -460,17 +470,17 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
         // ------------------------------ streaming warps ------------------------------------------
         uint32_t st = 0, ph = 0;  // ring position and parity of the "full" phase to wait for
         const uint32_t nst = (uint32_t)p.stages;
-        uint32_t k = 0;           // segment counter: buffers are indexed by k & 1
+        uint32_t k = 0;           // segment counter: hand-over buffers are indexed by k % kVpBufs
         SegIter it = seg_iter_begin<BF16>(p, q0, q1);
         Seg sg;
         for (; seg_iter_next<BF16>(p, it, sg); ++k) {
-            const uint32_t pb = k & 1u;
+            const uint32_t pb = k % kVpBufs;
             Acc a;
             a.ref = -INFINITY;
             a.s = 0.f;
             a.tmo = 0u;
-            // the buffers of parity pb are free once the epilogue of segment k-2 is done
-            if (k >= 2) mbar_wait_bounded(done0 + 8 * pb, ((k >> 1) - 1u) & 1u, &sh->abort_flag);
+            // buffer pb is free once the epilogue of segment k - kVpBufs is done
+            if (k >= kVpBufs) mbar_wait_bounded(done0 + 8 * pb, ((k / kVpBufs) - 1u) & 1u, &sh->abort_flag);
             {
                 const int nfull = (int)(sg.body_bytes / TILE);
                 cm_t* slot = cmax + (size_t)pb * p.n_cmax + (size_t)tid * p.max_tiles;  // this thread's slots, by tile
@@ -513,24 +523,28 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
             if (lane == 0) mbar_arrive(ready0 + 8 * pb);
         }
 #ifdef GRAFT_VP_PROF
-        if (warp == 0 && lane == 0 && blockIdx.x < 8) p.errflag[16 + blockIdx.x * 2] = (int)((clock64() - t_kernel0) >> 4);
+        if (warp == 0 && lane == 0) sh->t_stream_end = clock64() - t_kernel0;
 #endif
     } else {
-        // ------------------------------ epilogue group (four warps) ------------------------------
-        // Warp 0 of the group owns the hand-over barriers and the sequential parts; the data-parallel parts
-        // (which chunks reach T, re-reading them, ranking the candidates) are shared by the 128 threads.
-        const int ew = warp - NW, etid = tid - NT;
+        // ------------------------------ epilogue groups (four warps each) ------------------------
+        // Group g finishes the segments with k % 2 == g, so a group has two segment times for one epilogue.
+        // Warp 0 of a group owns the hand-over barriers and the sequential parts; the data-parallel parts (which
+        // chunks reach T, re-reading them, ranking the candidates) are shared by the group's 128 threads.
+        const int grp = (warp - NW) / (kVpEpiThreads / 32), ew = (warp - NW) % (kVpEpiThreads / 32);
+        const int etid = (tid - NT) % kVpEpiThreads;
+        EpiShared* const es = &sh->epi[grp];
         uint32_t k = 0;
         SegIter it = seg_iter_begin<BF16>(p, q0, q1);
         Seg sg;
         for (; seg_iter_next<BF16>(p, it, sg); ++k) {
-            const uint32_t pb = k & 1u;
+            if ((int)(k % kVpEpiGroups) != grp) continue;
+            const uint32_t pb = k % kVpBufs;
             const char* rowp = p.logits + (size_t)sg.row * p.V * T::ESZ;
             const cm_t* cmx = cmax + (size_t)pb * p.n_cmax;
 #ifdef GRAFT_VP_PROF
             long long tprof = clock64();
 #endif
-            if (ew == 0) mbar_wait_bounded(ready0 + 8 * pb, (k >> 1) & 1u, &sh->abort_flag);
+            if (ew == 0) mbar_wait_bounded(ready0 + 8 * pb, (k / kVpBufs) & 1u, &sh->abort_flag);
             if (p.dbg) {
                 __syncwarp();
                 if (ew == 0 && lane == 0) mbar_arrive(done0 + 8 * pb);
@@ -568,7 +582,7 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
                             merge_cs(c, s, c1, s1);
                             key = make_key(__float_as_uint(x), (uint32_t)e);
                         }
-                        ncand = warp_append(sh->cand, ncand, kVpCandCap, in, key, lane, &overflow);
+                        ncand = warp_append(es->cand, ncand, kVpCandCap, in, key, lane, &overflow);
                     }
                 }
                 VP_T(1);
@@ -607,45 +621,45 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
                 vmo = __reduce_max_sync(0xFFFFFFFFu, vmo);
                 overflow = __any_sync(0xFFFFFFFFu, overflow);
                 if (lane == 0) {
-                    sh->Tv = Tv;
-                    sh->nhits = 0;
-                    sh->nht = 0;
-                    sh->ncand = ncand;
-                    sh->ovf = overflow;
+                    es->Tv = Tv;
+                    es->nhits = 0;
+                    es->nht = 0;
+                    es->ncand = ncand;
+                    es->ovf = overflow;
                 }
                 VP_T(2);
             }
-            epi_bar();
-            const uint32_t Tv = sh->Tv;
+            epi_bar(grp);
+            const uint32_t Tv = es->Tv;
             // (d) chunks whose stored maximum reaches T: only threads whose own maximum reaches T can have one.
             //     List positions come from shared-memory atomics (the order does not matter: the final selection
             //     ranks exact keys).  A hit is recorded as the byte offset of the chunk's first vector.
             for (int t = etid; t < NT; t += kVpEpiThreads) {
                 const uint32_t x = sh->tmax[pb][t];
-                if (x >= Tv && x != 0u) sh->hthreads[atomicAdd(&sh->nht, 1)] = (uint16_t)t;
+                if (x >= Tv && x != 0u) es->hthreads[atomicAdd(&es->nht, 1)] = (uint16_t)t;
             }
-            epi_bar();
+            epi_bar(grp);
             {
-                const int npairs = sh->nht * sg.ntiles;
+                const int npairs = es->nht * sg.ntiles;
                 for (int idx = etid; idx < npairs; idx += kVpEpiThreads) {
                     const int h = idx / sg.ntiles, tile = idx - h * sg.ntiles;
-                    const uint32_t t = sh->hthreads[h];
+                    const uint32_t t = es->hthreads[h];
                     const cm_t raw = cmx[(size_t)t * p.max_tiles + tile];
-                    const uint32_t bits = BF16 ? ((uint32_t)raw << 16) : (uint32_t)raw;
+                    const uint32_t bits = (uint32_t)raw << 16;
                     if (ord_from_bits(bits) >= Tv) {
-                        const int pos = atomicAdd(&sh->nhits, 1);
-                        if (pos < kVpHitCap) sh->hits[pos] = (uint32_t)tile * TILE + (t >> 5) * WBLK + (t & 31) * 16;
+                        const int pos = atomicAdd(&es->nhits, 1);
+                        if (pos < kVpHitCap) es->hits[pos] = (uint32_t)tile * TILE + (t >> 5) * WBLK + (t & 31) * 16;
                     }
                 }
             }
-            epi_bar();
+            epi_bar(grp);
             if (ew == 0) VP_T(3);
             // (e) the 16-byte vectors of the hit chunks, re-read from global memory; elements >= T become keys.
             //     A thread issues its loads of a round before it uses any: under a saturated memory system one
             //     round trip costs microseconds.
             {
-                const int nhits = sh->nhits < kVpHitCap ? sh->nhits : kVpHitCap;
-                if (etid == 0 && sh->nhits > kVpHitCap) sh->ovf = 1;
+                const int nhits = es->nhits < kVpHitCap ? es->nhits : kVpHitCap;
+                if (etid == 0 && es->nhits > kVpHitCap) es->ovf = 1;
                 constexpr int RU = 2;
                 const int nvec = nhits * VEC_PER_LANE;
                 for (int base = 0; base < nvec; base += kVpEpiThreads * RU) {
@@ -657,7 +671,7 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
                         vv[u] = make_uint4(T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD);
                         offs[u] = 0xFFFFFFFFu;
                         if (i < nvec) {
-                            const uint32_t off = sh->hits[i / VEC_PER_LANE] + (uint32_t)(i % VEC_PER_LANE) * 512u;
+                            const uint32_t off = es->hits[i / VEC_PER_LANE] + (uint32_t)(i % VEC_PER_LANE) * 512u;
                             if (off < sg.body_bytes) {
                                 offs[u] = off;
                                 vv[u] = *(const uint4*)(sg.body + off);
@@ -676,33 +690,33 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
                             else
                                 xb = wv[j];
                             if (ord_from_bits(xb) >= Tv) {
-                                const int pos = atomicAdd(&sh->ncand, 1);
+                                const int pos = atomicAdd(&es->ncand, 1);
                                 if (pos < kVpCandCap)
-                                    sh->cand[pos] = make_key(xb, (uint32_t)(sg.e_body0 + offs[u] / T::ESZ + j));
+                                    es->cand[pos] = make_key(xb, (uint32_t)(sg.e_body0 + offs[u] / T::ESZ + j));
                             }
                         }
                     }
                 }
             }
-            epi_bar();
+            epi_bar(grp);
             if (ew == 0) VP_T(4);
             // (f) exact top-K of the candidates by rank counting (keys are distinct, so ranks are a permutation)
-            const bool overflow = sh->ovf != 0 || sh->ncand > kVpCandCap;
-            const int ncand = sh->ncand < kVpCandCap ? sh->ncand : kVpCandCap;
+            const bool overflow = es->ovf != 0 || es->ncand > kVpCandCap;
+            const int ncand = es->ncand < kVpCandCap ? es->ncand : kVpCandCap;
             int nk = ncand < p.K ? ncand : p.K;
             if (!overflow) {
                 for (int i = etid; i < ncand; i += kVpEpiThreads) {
-                    const uint64_t key = sh->cand[i];
+                    const uint64_t key = es->cand[i];
                     int rank = 0;
-                    for (int j = 0; j < ncand; ++j) rank += (sh->cand[j] > key) ? 1 : 0;
-                    if (rank < p.K) sh->outk[rank] = key;
+                    for (int j = 0; j < ncand; ++j) rank += (es->cand[j] > key) ? 1 : 0;
+                    if (rank < p.K) es->outk[rank] = key;
                 }
             } else if (ew == 0) {
-                nk = warp_fallback_select<BF16>(sh, p, sg, lane);
+                nk = warp_fallback_select<BF16>(es, p, sg, lane);
             }
-            epi_bar();
+            epi_bar(grp);
             if (ew != 0) continue;
-            const int nhits = sh->nhits;
+            const int nhits = es->nhits;
             VP_T(5);
             if (blockIdx.x == 1 && lane == 0) { atomicAdd(p.errflag + 10, ncand); atomicAdd(p.errflag + 11, nhits); atomicAdd(p.errflag + 12, 1); }
             // the double-buffered arrays of parity pb may be reused from here on
@@ -718,7 +732,7 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
             if (nseg > 1) {
                 const int my_first_row = (int)(q0 / p.nq);
                 VpRecord* rec = p.records + (size_t)blockIdx.x * 2 + (sg.row == my_first_row ? 0 : 1);
-                if (lane < kMaxK) rec->keys[lane] = lane < nk ? sh->outk[lane] : 0ull;
+                if (lane < kMaxK) rec->keys[lane] = lane < nk ? es->outk[lane] : 0ull;
                 if (lane == 0) {
                     rec->c = c;
                     rec->s = s;
@@ -747,11 +761,11 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
                             const int c_row0 = (int)(cta_start(cc, p.Q, G) / p.nq);
                             const VpRecord* r = p.records + (size_t)cc * 2 + (sg.row == c_row0 ? 0 : 1);
                             const uint64_t key = __ldcg((const unsigned long long*)&r->keys[kk]);
-                            n = warp_append(sh->cand, n, kVpCandCap, key != 0ull, key, lane, &ovf);
+                            n = warp_append(es->cand, n, kVpCandCap, key != 0ull, key, lane, &ovf);
                         }
-                        warp_select_topk(sh, n, p.K, lane);
+                        warp_select_topk(es, n, p.K, lane);
                         have = n < p.K ? n : p.K;
-                        if (lane < have) sh->cand[lane] = sh->outk[lane];
+                        if (lane < have) es->cand[lane] = es->outk[lane];
                         __syncwarp();
                     }
                     nk = have;
@@ -802,7 +816,7 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
                 const bool bad = !(Sd > 0.0) || !(Sd < 1e300) || Vm == 0u || vmax == INFINITY || vmax == -INFINITY ||
                                  nk < p.K;
                 if (lane < p.K) {
-                    const uint64_t key = lane < nk ? sh->outk[lane] : 0ull;
+                    const uint64_t key = lane < nk ? es->outk[lane] : 0ull;
                     p.topk_id[(size_t)sg.row * p.K + lane] = lane < nk ? (int32_t)key_id(key) : -1;
                     p.topk_lp[(size_t)sg.row * p.K + lane] = lane < nk ? (float)((double)key_value(key) - lse_d) : 0.f;
                 }
@@ -817,7 +831,17 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
     }
     __syncthreads();
 #ifdef GRAFT_VP_PROF
-    if (tid == 0 && blockIdx.x < 8) p.errflag[17 + blockIdx.x * 2] = (int)((clock64() - t_kernel0) >> 4);
+    if (tid == 0) {
+        unsigned smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        long long gt;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
+        float* dbg = p.dbg_out + (size_t)blockIdx.x * 4;
+        dbg[0] = (float)sh->t_stream_end;
+        dbg[1] = (float)(clock64() - t_kernel0);
+        dbg[2] = (float)smid;
+        dbg[3] = (float)(gt & 0xFFFFFF);
+    }
 #endif
     if (tid == 0 && sh->abort_flag) atomicOr(p.errflag, 1);
 }
@@ -826,7 +850,7 @@ __global__ void __launch_bounds__(kVpThreads, 2) vocab_pass_kernel(const VpParam
 
 // ---- host side ----------------------------------------------------------------------------------
 static size_t vp_smem_bytes(int stages, int n_cmax, bool bf16) {
-    return (size_t)stages * TILE + 24 * sizeof(uint64_t) + sizeof(VpShared) + (size_t)2 * n_cmax * (bf16 ? 2 : 4) + 16;
+    return (size_t)stages * TILE + 24 * sizeof(uint64_t) + sizeof(VpShared) + (size_t)kVpBufs * n_cmax * 2 + 16;
 }
 
 VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch) {
@@ -835,7 +859,7 @@ VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch) {
     const int esz = bf16 ? 2 : 4;
     const long long nq = cfg.V / kVpQuantum > 0 ? cfg.V / kVpQuantum : 1;
     const long long Q = nq * (long long)batch * cfg.L;
-    long long G = (long long)num_sms * 2;
+    long long G = (long long)num_sms;  // one CTA per SM
     if (G > Q) G = Q;
     if (G < 1) G = 1;
     pl.grid = (int)G;
@@ -844,7 +868,7 @@ VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch) {
     seg_elems += kVpQuantum;  // a row's last quantum also takes the remainder
     if (seg_elems > cfg.V) seg_elems = cfg.V;
     pl.max_seg_tiles = (int)((seg_elems * esz + TILE - 1) / TILE) + 1;
-    const size_t budget = 112 * 1024;  // two CTAs per SM
+    const size_t budget = 224 * 1024;  // one CTA per SM
     int stages = 6;
     while (stages > 2 && vp_smem_bytes(stages, pl.max_seg_tiles * NT, bf16) > budget) --stages;
     pl.stages = stages;
@@ -876,6 +900,7 @@ cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* 
     p.errflag = ctx->w_errflag;
     p.use_hint = 1;
     p.dbg = 0;
+    p.dbg_out = ctx->w_edge;
 #ifdef GRAFT_VP_EXPERIMENT  // tuning switches, never compiled into the shipped library
     if (getenv("GRAFT_VP_HINT")) p.use_hint = atoi(getenv("GRAFT_VP_HINT"));
     if (getenv("GRAFT_VP_DEBUG")) p.dbg = atoi(getenv("GRAFT_VP_DEBUG"));
@@ -893,12 +918,12 @@ cudaError_t vp_configure(const graft_config& cfg, int num_sms, size_t* max_smem)
     // the largest dynamic shared-memory request any batch can produce (segment = a whole row)
     VpPlan pl = vp_make_plan(cfg, num_sms, cfg.max_batch > 4096 ? cfg.max_batch : 4096);
     *max_smem = pl.smem_bytes;
-    if (pl.smem_bytes > 113 * 1024) return cudaErrorInvalidValue;
+    if (pl.smem_bytes > 225 * 1024) return cudaErrorInvalidValue;
     cudaError_t e;
     if (cfg.logits_dtype == GRAFT_BF16)
-        e = cudaFuncSetAttribute(vocab_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+        e = cudaFuncSetAttribute(vocab_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
     else
-        e = cudaFuncSetAttribute(vocab_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+        e = cudaFuncSetAttribute(vocab_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
     return e;
 }
 
@@ -974,9 +999,9 @@ extern "C" graft_status graft_vocab_pass_static(int32_t batch, int32_t L, int32_
                 cudaGetLastError();
                 return GRAFT_ERR_CUDA;
             }
-            if (cudaFuncSetAttribute(vocab_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024) !=
+            if (cudaFuncSetAttribute(vocab_pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) !=
                     cudaSuccess ||
-                cudaFuncSetAttribute(vocab_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024) !=
+                cudaFuncSetAttribute(vocab_pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024) !=
                     cudaSuccess) {
                 cudaGetLastError();
                 return GRAFT_ERR_CUDA;
@@ -987,7 +1012,7 @@ extern "C" graft_status graft_vocab_pass_static(int32_t batch, int32_t L, int32_
         }
     }
     const VpPlan pl = vp_make_plan(cfg, sd->num_sms, batch);
-    if (pl.grid > kStaticMaxGrid || pl.smem_bytes > 113 * 1024) return GRAFT_ERR_UNSUPPORTED;
+    if (pl.grid > kStaticMaxGrid || pl.smem_bytes > 225 * 1024) return GRAFT_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     // the array keeps whatever the previous call left: the arrival counters and the error word must start at 0
     if (cudaMemsetAsync(sd->scratch->row_counter, 0, sizeof(int) * (size_t)batch * L, st) != cudaSuccess ||
@@ -1014,6 +1039,7 @@ extern "C" graft_status graft_vocab_pass_static(int32_t batch, int32_t L, int32_
     p.errflag = sd->scratch->errflag;
     p.use_hint = 1;
     p.dbg = 0;
+    p.dbg_out = nullptr;
     if (logits_dtype == GRAFT_BF16)
         vocab_pass_kernel<true><<<pl.grid, kVpThreads, pl.smem_bytes, st>>>(p);
     else
