@@ -135,8 +135,10 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
         for (int q = 0; q < RPW; ++q) {
             const int r = warp + 8 * q;
             t[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+#ifndef TDES_NO_GATHER
             if (r < n_par + K && k4 < m / 4)
                 t[q] = __ldg((const float4*)((r < n_par ? p.P : p.C) + (size_t)toks[r] * m) + k4);
+#endif
         }
         if (k4 < m / 4) {
             const float4 uu = *(const float4*)(urow + k4 * 4);
@@ -151,24 +153,34 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
         }
     }
     __syncthreads();
-    // lane = child c; each warp takes parents warp, warp+8, ...
+    // lane = child c; each warp takes parents warp, warp+8, ...  The dot products run on packed fp32 pairs
+    // (fma.rn.f32x2): a 16-byte shared load is two ready-made pairs.
     const int c = lane;
     float f[4] = {0.f, 0.f, 0.f, 0.f};
     if (c < K) {
-        const float4* cc = (const float4*)(sC + (size_t)c * ld);
+        const ulonglong2* cc = (const ulonglong2*)(sC + (size_t)c * ld);
+        unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};  // (+0, +0) pairs
+        int npw = 0;                                           // parents of this warp: warp, warp+8, ...
+#pragma unroll
+        for (int t = 0; t < 4; ++t) npw += (warp + 8 * t < n_par) ? 1 : 0;
+#ifndef TDES_NO_FMA
         for (int k4 = 0; k4 < m / 4; ++k4) {
-            const float4 cv = cc[k4];
+            const ulonglong2 cv = cc[k4];
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
-                const int par = warp + 8 * t;
-                if (par < n_par) {
-                    const float4 pv = *(const float4*)(sP + (size_t)par * ld + k4 * 4);
-                    f[t] = fmaf(pv.x, cv.x, f[t]);
-                    f[t] = fmaf(pv.y, cv.y, f[t]);
-                    f[t] = fmaf(pv.z, cv.z, f[t]);
-                    f[t] = fmaf(pv.w, cv.w, f[t]);
+                if (t < npw) {  // uniform per warp
+                    const ulonglong2 pv = *(const ulonglong2*)(sP + (size_t)(warp + 8 * t) * ld + k4 * 4);
+                    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc[t]) : "l"(pv.x), "l"(cv.x));
+                    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc[t]) : "l"(pv.y), "l"(cv.y));
                 }
             }
+        }
+#endif
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            float lo2, hi2;
+            asm("mov.b64 {%0, %1}, %2;" : "=f"(lo2), "=f"(hi2) : "l"(acc[t]));
+            f[t] = lo2 + hi2;
         }
     }
     const float lp = c < K ? lps[c] : 0.f;
@@ -186,6 +198,7 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
         // the row again, sorted by (edge descending, child rank ascending): a 32-lane bitonic network on
         // 64-bit keys; lanes beyond K hold the empty key 0 and sink to the end
         uint64_t key = (c < K) ? (((uint64_t)ord_from_float(val) << 32) | (uint32_t)(31 - c)) : 0ull;
+#ifndef TDES_NO_SORT
 #pragma unroll
         for (int k = 2; k <= 32; k <<= 1) {
 #pragma unroll
@@ -195,6 +208,7 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
                 key = keep_max ? (key > other ? key : other) : (key < other ? key : other);
             }
         }
+#endif
         if (lane < K) {
             outs[(size_t)par * K + lane] = __uint_as_float(bits_from_ord((uint32_t)(key >> 32)));
             outi[(size_t)par * K + lane] = (uint8_t)(31 - (uint32_t)(key & 0xFFu));

@@ -774,31 +774,46 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     }
 }
 
-// ---- acceptance walk: one warp per sequence ------------------------------------------------------------------
-// The tree (parents, tokens) and the target's next tokens are staged in shared memory with one coalesced read;
-// the walk itself then runs out of shared memory.  In level order the parent indices never decrease, so the
-// children of the current node are found by a binary search for the first node whose parent is >= it.
+// ---- acceptance walk: one CTA per sequence ---------------------------------------------------------------------
+// The tree (parents, tokens) and the target's next tokens are staged in shared memory by 128 threads with all
+// loads in flight together; warp 0 then walks out of shared memory.  In level order the parent indices never
+// decrease, so the children of the current node are found by a binary search for the first node whose parent
+// is >= it.
 __global__ void __launch_bounds__(128) accept_kernel(const int32_t* __restrict__ n_nodes, const int32_t* __restrict__ token,
                                                      const int32_t* __restrict__ parent,
                                                      const int32_t* __restrict__ target_next, int batch, int nmax, int L,
                                                      int32_t* __restrict__ accept_len, int32_t* __restrict__ accept_path,
                                                      int32_t* __restrict__ bonus) {
     extern __shared__ __align__(16) int32_t acc_smem[];
-    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = blockIdx.x * 4 + wib;
-    if (b >= batch) return;
-    int32_t* par = acc_smem + (size_t)wib * 3 * nmax;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+    int32_t* par = acc_smem;
     int32_t* tok = par + nmax;
     int32_t* tn = tok + nmax;
     const size_t ob = (size_t)b * nmax;
     int nn = n_nodes[b];
     nn = nn < 1 ? 1 : (nn > nmax ? nmax : nn);
-    for (int i = lane; i < nn; i += 32) {
-        par[i] = parent[ob + i];
-        tok[i] = token[ob + i];
-        tn[i] = target_next[ob + i];
+    {
+        constexpr int U = 8;  // 128 threads x 8 covers the largest tree (1024 nodes) in one round
+        int32_t vp[U], vt[U], vn[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i = tid + 128 * u;
+            vp[u] = i < nn ? parent[ob + i] : 0;
+            vt[u] = i < nn ? token[ob + i] : 0;
+            vn[u] = i < nn ? target_next[ob + i] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i = tid + 128 * u;
+            if (i < nn) {
+                par[i] = vp[u];
+                tok[i] = vt[u];
+                tn[i] = vn[u];
+            }
+        }
     }
-    __syncwarp();
+    __syncthreads();
+    if (tid >= 32) return;
     int cur = 0, a = 0;
     while (a < L) {
         const int want = tn[cur];
@@ -878,7 +893,7 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
 
 cudaError_t accept_launch(graft_ctx* ctx, int batch, const graft_tree_out* trees, const int32_t* d_target_next,
                           int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus, cudaStream_t st) {
-    accept_kernel<<<(batch + 3) / 4, 128, (size_t)4 * 3 * ctx->nmax * sizeof(int32_t), st>>>(trees->d_n_nodes, trees->d_token, trees->d_parent, d_target_next,
+    accept_kernel<<<batch, 128, (size_t)3 * ctx->nmax * sizeof(int32_t), st>>>(trees->d_n_nodes, trees->d_token, trees->d_parent, d_target_next,
                                                    batch, ctx->nmax, ctx->cfg.L, d_accept_len, d_accept_path, d_bonus);
     ctx->launches += 1;
     return cudaGetLastError();
