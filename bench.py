@@ -142,6 +142,8 @@ def run_graft(args):
     g.set_tdes_tables(P, Ct, u, tb["s"])
     saba_kw = gi.saba_defaults(w)
     g.set_saba(**saba_kw)
+    if args.edge_rows is not None:
+        g.set_edge_rows(args.edge_rows)
 
     logits_bytes = batch * w.L * w.V * (2 if w.logits_dtype == "bf16" else 4)
     n_buf = max(2, int(np.ceil(2.5 * L2_BYTES / logits_bytes)))  # rotating sets: > 2.5x L2 in total
@@ -263,6 +265,7 @@ def run_graft(args):
         "config": {"workload": f"{w.name}: batch {batch} per GPU, L={w.L}, V={w.V} {w.logits_dtype} logits, "
                                f"hidden d={w.hidden_dim} {w.hidden_dtype}, K={w.K}, m={w.m}, beta={w.beta}, SABA budgets "
                                f"[{w.budget_min},{w.budget_max}] step {w.budget_step}, build_trees + accept",
+                   "edge_rows": g.edge_rows(),
                    "parallelism": f"batch-sharded x{world}, no collective",
                    "l2_policy": f"{n_buf} rotating input sets of {logits_bytes / 1e6:.0f} MB each (> L2 of 126 MB)"},
         "gpu_launches": launches,
@@ -358,6 +361,8 @@ def main():
     ap.add_argument("--workload", default="M", choices=sorted(gi.WORKLOADS))
     ap.add_argument("--impl", default="graft", choices=["graft", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--edge-rows", type=int, default=None,
+                    help="depths scored ahead of the expansion (default: the library's)")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 10 if args.steps is None else args.steps

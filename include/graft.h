@@ -121,6 +121,16 @@ graft_status graft_set_saba(graft_ctx* ctx, const graft_saba_params* p);
 graft_status graft_set_tdes_tables(graft_ctx* ctx, const float* d_P, const float* d_C, const float* d_u, float s,
                                    void* stream);
 
+/* How many depths the edge-score kernel covers ahead of the expansion.  The scores of Eq. 4-6 are needed only for
+ * depths that the best-first expansion reaches, which is not known in advance: depths [0, rows) are scored for every
+ * sequence by a kernel of their own, deeper ones inside the tree kernel when an expansion gets there.  The trees do
+ * not depend on the split beyond fp32 rounding of the scores (the two scorers add in different orders).
+ * rows in [0, L]; the default is min(L, 8), or L when the on-demand scorer's buffers do not fit in shared memory
+ * (then any other value is GRAFT_ERR_INVALID_ARG).  Host-only call; takes effect from the next round.
+ * (A tuning knob of this implementation; the paper scores all edges.) */
+graft_status graft_set_edge_rows(graft_ctx* ctx, int32_t rows);
+int32_t graft_edge_rows(const graft_ctx* ctx);
+
 /* Table precompute (same passage): d_out[v] = W e_v + b for one tower.  d_emb [V, E] (dtype as given),
  * d_W [m, E] fp32, d_b [m] fp32 or NULL, d_out [V, m] fp32.  fp32 accumulation.  Call once per tower. */
 graft_status graft_tdes_precompute(graft_ctx* ctx, const void* d_emb, graft_dtype emb_dtype, int32_t E,

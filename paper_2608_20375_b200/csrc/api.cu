@@ -154,6 +154,7 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     ctx->w_esort = (float*)(base + o_es);
     ctx->w_eidx = (uint8_t*)(base + o_ei);
     ctx->d_u = (float*)(base + o_u);
+    ctx->edge_rows = tree_lazy_fits(*cfg) ? (cfg->L < 8 ? cfg->L : 8) : cfg->L;
     ctx->w_errflag = (int32_t*)(base + o_err);
     *out = ctx;
     return GRAFT_OK;
@@ -225,6 +226,15 @@ graft_status graft_set_tdes_tables(graft_ctx* ctx, const float* d_P, const float
     return GRAFT_OK;
 }
 
+graft_status graft_set_edge_rows(graft_ctx* ctx, int32_t rows) {
+    if (!ctx || rows < 0 || rows > ctx->cfg.L) return GRAFT_ERR_INVALID_ARG;
+    if (rows < ctx->cfg.L && !tree_lazy_fits(ctx->cfg)) return GRAFT_ERR_INVALID_ARG;
+    ctx->edge_rows = rows;
+    return GRAFT_OK;
+}
+
+int32_t graft_edge_rows(const graft_ctx* ctx) { return ctx ? ctx->edge_rows : -1; }
+
 graft_status graft_tdes_precompute(graft_ctx* ctx, const void* d_emb, graft_dtype emb_dtype, int32_t E,
                                    const float* d_W, const float* d_b, float* d_out, void* stream) {
     if (!ctx || !d_emb || !d_W || !d_out || E < 1) return GRAFT_ERR_INVALID_ARG;
@@ -252,6 +262,7 @@ graft_status graft_tdes_edges(graft_ctx* ctx, int32_t batch, const int32_t* d_to
     if (batch < 1 || batch > ctx->cfg.max_batch) return GRAFT_ERR_INVALID_ARG;
     if (ctx->cfg.beta != 0.0f && !ctx->tdes_set) return GRAFT_ERR_STATE;
     if (tdes_edges_launch(ctx, batch, d_topk_id, d_topk_lp, d_root_token, nullptr, d_edge, ctx->w_esort, ctx->w_eidx,
+                          ctx->cfg.L,
                           (cudaStream_t)stream) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     return GRAFT_OK;
@@ -321,9 +332,14 @@ graft_status graft_build_trees(graft_ctx* ctx, int32_t batch, const void* d_logi
     if (ev) cudaEventRecord(ev[0], st);
     if (vp_launch(ctx, batch, d_logits, ids, lps, lse, ctx->w_row_status, st) != cudaSuccess) return GRAFT_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], st);
-    if (tdes_edges_launch(ctx, batch, ids, lps, d_root_token, ctx->w_row_status, edge, ctx->w_esort, ctx->w_eidx, st) !=
-        cudaSuccess)
-        return GRAFT_ERR_CUDA;
+    // Edge scores of Eq. 4-6: the kernel scores the depths [0, edge_rows) for every sequence (all depths when the
+    // caller asks for the score array); the tree kernel scores deeper rows itself if an expansion gets that far.
+    {
+        const int rows = out->d_edge ? ctx->cfg.L : ctx->edge_rows;
+        if (rows > 0 && tdes_edges_launch(ctx, batch, ids, lps, d_root_token, ctx->w_row_status, edge, ctx->w_esort,
+                                          ctx->w_eidx, rows, st) != cudaSuccess)
+            return GRAFT_ERR_CUDA;
+    }
     if (ev) cudaEventRecord(ev[2], st);
     if (tree_launch(ctx, batch, ids, lps, ctx->w_row_status, ctx->w_esort, ctx->w_eidx, d_hidden, d_root_token, d_hist, d_prefix_len,
                     d_fixed_budget, out, st) != cudaSuccess)

@@ -1,0 +1,112 @@
+// TDES edge scores of one depth out of shared memory (Eq. 4-6), shared by the edge-score kernel (which scores the
+// first depths for every sequence) and the tree kernel (which scores deeper depths when an expansion gets there),
+// so that a row has the same bits whichever kernel produced it.
+//
+//   f[p][c]    = s/sqrt(m) * (P[p] + u_d) . (C[c] + u_d)                                   (Eq. 4-6)
+//   edge[p][c] = log q_d(c) + beta * (f[p][c] - mean_c f[p][c])                            (TDES score)
+//   and every parent's row ordered by (edge descending, child rank ascending).
+#pragma once
+#include "common.cuh"
+
+namespace graft {
+
+// K x K dot products by 8 warps.  Warp ty takes parents ty, ty+8, ty+16, ty+24; lane = (ks, tx): children tx,
+// tx+8, tx+16, tx+24 and every fourth float4 of the m axis starting at ks.  A lane keeps a 4 x 4 tile of running
+// sums (16 FMAs per pair of 16-byte loads); the four ks of a tile are then added by two butterfly steps, in a fixed
+// order.  rP / rC: [.][ld] rows in shared memory, ld = m + 4 floats (16-byte aligned, conflict-free float4 reads).
+// ADD_U: the rows hold P and C and u is added on the way into the registers; otherwise they already hold P + u and
+// C + u (the same fp32 sums either way).  part: [K][K] floats of shared memory; rows >= n_par are not written.
+template <bool ADD_U>
+__device__ __forceinline__ void edge_dots(const float* rP, const float* rC, const float* rU, int m, int K, int n_par,
+                                          float* part, int ty, int lane) {
+    if (ty >= n_par) return;
+    const int tx = lane & 7, ks = lane >> 3, q4 = m / 4, ld = m + 4;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int i2 = 0; i2 < 4; ++i2) acc[i][i2] = 0.f;
+    for (int k4 = ks; k4 < q4; k4 += 4) {
+        float4 uu = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ADD_U) uu = *(const float4*)(rU + 4 * k4);
+        float4 cv[4];
+#pragma unroll
+        for (int i2 = 0; i2 < 4; ++i2) {
+            cv[i2] = *(const float4*)(rC + (size_t)min(tx + 8 * i2, K - 1) * ld + 4 * k4);  // (rows past K: unused)
+            if (ADD_U) {
+                cv[i2].x += uu.x;
+                cv[i2].y += uu.y;
+                cv[i2].z += uu.z;
+                cv[i2].w += uu.w;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float4 pv = *(const float4*)(rP + (size_t)min(ty + 8 * i, n_par - 1) * ld + 4 * k4);
+            if (ADD_U) {
+                pv.x += uu.x;
+                pv.y += uu.y;
+                pv.z += uu.z;
+                pv.w += uu.w;
+            }
+#pragma unroll
+            for (int i2 = 0; i2 < 4; ++i2) {
+                float a = acc[i][i2];
+                a = fmaf(pv.x, cv[i2].x, a);
+                a = fmaf(pv.y, cv[i2].y, a);
+                a = fmaf(pv.z, cv[i2].z, a);
+                a = fmaf(pv.w, cv[i2].w, a);
+                acc[i][i2] = a;
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int i2 = 0; i2 < 4; ++i2) {
+            float a = acc[i][i2];
+            a += __shfl_xor_sync(0xFFFFFFFFu, a, 8);
+            a += __shfl_xor_sync(0xFFFFFFFFu, a, 16);
+            acc[i][i2] = a;
+        }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (ks == i && ty + 8 * i < n_par) {
+#pragma unroll
+            for (int i2 = 0; i2 < 4; ++i2)
+                if (tx + 8 * i2 < K) part[(size_t)(ty + 8 * i) * K + tx + 8 * i2] = acc[i][i2];
+        }
+    }
+}
+
+// One warp finishes one parent's row: scale, centre over the K children, add log q (lane = child c), and find the
+// place of every child in the order (edge descending, child rank ascending) by counting the children that come
+// before it.  dots: the parent's K dot products, or nullptr for a parent that does not exist (a row of zeros).
+// wsc: 32 words of shared memory of this warp.  Returns the score in `val` and the place in `rank` (lanes < K).
+__device__ __forceinline__ void edge_row_finish(const float* dots, const float* lps, float scale, float beta, int K,
+                                                uint32_t* wsc, int lane, float& val, int& rank) {
+    const int c = lane;
+    val = 0.f;
+    if (dots != nullptr) {
+        const float ft = c < K ? dots[c] * scale : 0.f;
+        float sum = ft;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
+        const float mean = sum / (float)K;
+        val = fmaf(beta, ft - mean, c < K ? lps[c] : 0.f);
+    }
+    const uint32_t mine = c < K ? ord_from_float(val) : 0u;  // 0 is below the image of every float
+    __syncwarp();
+    wsc[c] = mine;
+    __syncwarp();
+    rank = 0;
+#pragma unroll
+    for (int i4 = 0; i4 < 8; ++i4) {
+        const uint4 o4 = *(const uint4*)(wsc + 4 * i4);
+        rank += (o4.x > mine ? 1 : 0) + (o4.y > mine ? 1 : 0) + (o4.z > mine ? 1 : 0) + (o4.w > mine ? 1 : 0);
+    }
+    const uint32_t same = __match_any_sync(0xFFFFFFFFu, mine);
+    rank += __popc(same & ((1u << lane) - 1u));
+}
+
+}  // namespace graft

@@ -60,6 +60,7 @@ struct graft_ctx {
     const float* d_C;
     float* d_u;  // owned copy [L, m]
     float tdes_s;
+    int edge_rows;  // depths [0, edge_rows) are scored by the edge-score kernel, deeper ones on demand in the tree kernel
     // scratch (one allocation)
     void* ws;
     size_t ws_bytes;
@@ -94,7 +95,7 @@ cudaError_t tdes_precompute_launch(graft_ctx* ctx, const void* d_emb, graft_dtyp
                                    const float* d_b, float* d_out, cudaStream_t st);
 cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                               const int32_t* d_root_token, const int32_t* d_row_status, float* d_edge,
-                              float* d_esort, uint8_t* d_eidx, cudaStream_t st);
+                              float* d_esort, uint8_t* d_eidx, int rows, cudaStream_t st);  // depths [0, rows)
 cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                         const int32_t* d_row_status, const float* d_esort, const uint8_t* d_eidx, const void* d_hidden,
                         const int32_t* d_root_token, const float* d_hist, const int32_t* d_prefix_len,
@@ -102,5 +103,6 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
 cudaError_t accept_launch(graft_ctx* ctx, int batch, const graft_tree_out* trees, const int32_t* d_target_next,
                           int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus, cudaStream_t st);
 size_t tree_smem_bytes(const graft_config& cfg);
+bool tree_lazy_fits(const graft_config& cfg);  // edge scores are computed inside the tree kernel
 
 }  // namespace graft

@@ -9,6 +9,7 @@
 // memory (tensor-core tf32/bf16 products would also break the 1e-5 score tolerance).
 #include "common.cuh"
 #include "internal.h"
+#include "edge_score.cuh"
 
 namespace graft {
 namespace {
@@ -83,6 +84,7 @@ struct EdgeParams {
     float* esort;     // same rows, each sorted by (edge descending, child rank ascending)
     uint8_t* eidx;    // child rank of every sorted entry
     int L, K, m, V;
+    int rows;     // depths [0, rows) are scored: one CTA each
     float scale;  // s / sqrt(m)
     float beta;
     int root_edge;
@@ -90,7 +92,7 @@ struct EdgeParams {
 
 __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
     extern __shared__ __align__(16) float smem[];
-    const int b = blockIdx.x / p.L, j = blockIdx.x % p.L;
+    const int b = blockIdx.x / p.rows, j = blockIdx.x % p.rows;
     const int K = p.K, m = p.m, ld = m + 4;  // padded row: 16-byte aligned, conflict-free float4 reads
     float* sP = smem;                        // [K][ld]  parent rows + u_d
     float* sC = smem + (size_t)kMaxK * ld;   // [K][ld]  child rows + u_d
@@ -135,10 +137,8 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
         for (int q = 0; q < RPW; ++q) {
             const int r = warp + 8 * q;
             t[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-#ifndef TDES_NO_GATHER
             if (r < n_par + K && k4 < m / 4)
                 t[q] = __ldg((const float4*)((r < n_par ? p.P : p.C) + (size_t)toks[r] * m) + k4);
-#endif
         }
         if (k4 < m / 4) {
             const float4 uu = *(const float4*)(urow + k4 * 4);
@@ -153,65 +153,20 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
         }
     }
     __syncthreads();
-    // lane = child c; each warp takes parents warp, warp+8, ...  The dot products run on packed fp32 pairs
-    // (fma.rn.f32x2): a 16-byte shared load is two ready-made pairs.
-    const int c = lane;
-    float f[4] = {0.f, 0.f, 0.f, 0.f};
-    if (c < K) {
-        const ulonglong2* cc = (const ulonglong2*)(sC + (size_t)c * ld);
-        unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};  // (+0, +0) pairs
-        int npw = 0;                                           // parents of this warp: warp, warp+8, ...
-#pragma unroll
-        for (int t = 0; t < 4; ++t) npw += (warp + 8 * t < n_par) ? 1 : 0;
-#ifndef TDES_NO_FMA
-        for (int k4 = 0; k4 < m / 4; ++k4) {
-            const ulonglong2 cv = cc[k4];
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                if (t < npw) {  // uniform per warp
-                    const ulonglong2 pv = *(const ulonglong2*)(sP + (size_t)(warp + 8 * t) * ld + k4 * 4);
-                    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc[t]) : "l"(pv.x), "l"(cv.x));
-                    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc[t]) : "l"(pv.y), "l"(cv.y));
-                }
-            }
-        }
-#endif
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            float lo2, hi2;
-            asm("mov.b64 {%0, %1}, %2;" : "=f"(lo2), "=f"(hi2) : "l"(acc[t]));
-            f[t] = lo2 + hi2;
-        }
-    }
-    const float lp = c < K ? lps[c] : 0.f;
-#pragma unroll
-    for (int t = 0; t < 4; ++t) {
-        const int par = warp + 8 * t;
-        if (par >= K) continue;  // uniform per warp
-        float ft = (c < K) ? f[t] * p.scale : 0.f;
-        float sum = ft;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
-        const float mean = sum / (float)K;
-        const float val = (par < n_par) ? fmaf(p.beta, ft - mean, lp) : 0.f;
-        if (c < K) out[(size_t)par * K + c] = val;
-        // the row again, sorted by (edge descending, child rank ascending): a 32-lane bitonic network on
-        // 64-bit keys; lanes beyond K hold the empty key 0 and sink to the end
-        uint64_t key = (c < K) ? (((uint64_t)ord_from_float(val) << 32) | (uint32_t)(31 - c)) : 0ull;
-#ifndef TDES_NO_SORT
-#pragma unroll
-        for (int k = 2; k <= 32; k <<= 1) {
-#pragma unroll
-            for (int jj = k >> 1; jj > 0; jj >>= 1) {
-                const uint64_t other = __shfl_xor_sync(0xFFFFFFFFu, key, jj);
-                const bool keep_max = (((lane & k) == 0) == ((lane & jj) == 0));
-                key = keep_max ? (key > other ? key : other) : (key < other ? key : other);
-            }
-        }
-#endif
+    // dot products into shared memory, then every warp finishes the rows of parents warp, warp+8, ...
+    float* part = sC + (size_t)kMaxK * ld;  // [K][K]
+    __shared__ uint32_t wsc[8][32];
+    edge_dots<false>(sP, sC, nullptr, m, K, n_par, part, warp, lane);
+    __syncthreads();
+    for (int par = warp; par < K; par += 8) {
+        float val;
+        int rank;
+        edge_row_finish(par < n_par ? part + (size_t)par * K : nullptr, lps, p.scale, p.beta, K, wsc[warp], lane, val,
+                        rank);
         if (lane < K) {
-            outs[(size_t)par * K + lane] = __uint_as_float(bits_from_ord((uint32_t)(key >> 32)));
-            outi[(size_t)par * K + lane] = (uint8_t)(31 - (uint32_t)(key & 0xFFu));
+            out[(size_t)par * K + lane] = val;
+            outs[(size_t)par * K + rank] = val;
+            outi[(size_t)par * K + rank] = (uint8_t)lane;
         }
     }
 }
@@ -230,7 +185,9 @@ cudaError_t tdes_precompute_launch(graft_ctx* ctx, const void* d_emb, graft_dtyp
     return cudaGetLastError();
 }
 
-size_t tdes_edges_smem(const graft_config& cfg) { return (size_t)2 * kMaxK * (cfg.m + 4) * sizeof(float); }
+size_t tdes_edges_smem(const graft_config& cfg) {
+    return ((size_t)2 * kMaxK * (cfg.m + 4) + (size_t)kMaxK * kMaxK) * sizeof(float);  // P rows, C rows, dot products
+}
 
 cudaError_t tdes_edges_configure(const graft_config& cfg) {
     return cudaFuncSetAttribute(tdes_edges_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -239,7 +196,7 @@ cudaError_t tdes_edges_configure(const graft_config& cfg) {
 
 cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                               const int32_t* d_root_token, const int32_t* d_row_status, float* d_edge,
-                              float* d_esort, uint8_t* d_eidx, cudaStream_t st) {
+                              float* d_esort, uint8_t* d_eidx, int rows, cudaStream_t st) {
     const graft_config& cfg = ctx->cfg;
     EdgeParams p;
     p.topk_id = d_topk_id;
@@ -259,7 +216,8 @@ cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_i
     p.scale = ctx->tdes_s / sqrtf((float)cfg.m);
     p.beta = ctx->tdes_set ? cfg.beta : 0.0f;
     p.root_edge = cfg.root_edge;
-    tdes_edges_kernel<<<batch * cfg.L, 256, tdes_edges_smem(cfg), st>>>(p);
+    p.rows = rows;
+    tdes_edges_kernel<<<batch * rows, 256, tdes_edges_smem(cfg), st>>>(p);
     ctx->launches += 1;
     return cudaGetLastError();
 }

@@ -3,6 +3,7 @@
 // with the packed ancestor mask, and the acceptance walk.
 #include "common.cuh"
 #include "internal.h"
+#include "edge_score.cuh"
 
 namespace graft {
 namespace {
@@ -23,6 +24,16 @@ struct TreeParams {
     graft_tree_out out;
     int L, K, nmax, W, bmin, bmax, bstep;
     int ncap;  // capacity of the node table of the parallel phase
+    // Edge scores (Eq. 4-6): the rows of depths [0, rows_pre) come from the edge-score kernel through esort / eidx;
+    // deeper rows are scored inside this kernel (lazy = 1), level by level, only if the expansion gets there.
+    int rows_pre;
+    int lazy;
+    int lazy_m;  // m when the shared-memory layout holds the buffers of the on-demand scorer, else 0
+    const float* P;
+    const float* C;
+    const float* u;
+    float scale, beta;
+    int root_edge, m, V;
     int use_saba;
     SabaDev saba;
 };
@@ -54,10 +65,17 @@ struct TreeSmem {
     int* lvl_start;      // [kMaxL + 2]
     int* lvl_fill;       // [kMaxL + 2]
     double* cosv;        // [kMaxL]  adjacent-position cosines r_d (Eq. 15)
+    // on-demand edge scoring only:
+    float* gP;           // [K][m+4]  gathered parent rows P[token]
+    float* gC;           // [K][m+4]  gathered child rows C[token]
+    float* gU;           // [m]       u_d
+    int32_t* tokid;      // [L*K]     candidate tokens
+    float* lpv;          // [L*K]     their log q
     int* scal;           // [16] 0 budget, 1 n_nodes, 2 status, 3 table size, 4 overflow, 6/7 radix-select hand-over
 };
 
-__host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, int ncap, TreeSmem* s, unsigned char* base) {
+__host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, int ncap, int lazy_m, TreeSmem* s,
+                                                   unsigned char* base) {
     size_t off = 0;
     auto take = [&](size_t bytes) {
         size_t o = off;
@@ -73,6 +91,14 @@ __host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, int n
            o_par = take((size_t)nmax * 2), o_can = take((size_t)nmax * 2), o_cp = take((size_t)nmax * 2),
            o_cand = take(nmax), o_dep = take(nmax), o_hist = take(2048 * 4), o_lc = take((kMaxL + 2) * 4),
            o_ls = take((kMaxL + 2) * 4), o_lf = take((kMaxL + 2) * 4), o_sc = take(16 * 4), o_cos = take(kMaxL * 8);
+    size_t o_gp = 0, o_gc = 0, o_gu = 0, o_tk = 0, o_lp = 0;
+    if (lazy_m > 0) {
+        o_gp = take((size_t)K * (lazy_m + 4) * 4);
+        o_gc = take((size_t)K * (lazy_m + 4) * 4);
+        o_gu = take((size_t)lazy_m * 4);
+        o_tk = take((size_t)L * K * 4);
+        o_lp = take((size_t)L * K * 4);
+    }
     if (s) {
         s->es = (float*)(base + o_es);
         s->ei = base + o_ei;
@@ -96,18 +122,23 @@ __host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, int n
         s->lvl_fill = (int*)(base + o_lf);
         s->scal = (int*)(base + o_sc);
         s->cosv = (double*)(base + o_cos);
+        s->gP = (float*)(base + o_gp);
+        s->gC = (float*)(base + o_gc);
+        s->gU = (float*)(base + o_gu);
+        s->tokid = (int32_t*)(base + o_tk);
+        s->lpv = (float*)(base + o_lp);
     }
     return off;
 }
 
 // capacity of the node table: what fits beside the edge rows in ~200 KB of shared memory, at most 6144 nodes
 // (parent indices are 13 bits) and at least enough for a full budget's worth of nodes
-__host__ __device__ inline int tree_node_cap(int L, int K, int nmax) {
+__host__ __device__ inline int tree_node_cap(int L, int K, int nmax, int lazy_m) {
     const int W = (nmax + 31) / 32;
     const size_t emis = (((size_t)nmax * 2 + 15) & ~(size_t)15) + (((size_t)nmax * 4 + 15) & ~(size_t)15) +
                         (size_t)8 * 32 * W * 4;
-    const size_t fixed = tree_smem_layout(L, K, nmax, 0, nullptr, nullptr);  // counts `emis` for the table
-    const size_t room = fixed < (size_t)200 * 1024 ? (size_t)200 * 1024 - fixed : 0;
+    const size_t fixed = tree_smem_layout(L, K, nmax, 0, lazy_m, nullptr, nullptr);  // counts `emis` for the table
+    const size_t room = fixed < (size_t)222 * 1024 ? (size_t)222 * 1024 - fixed : 0;
     long long cap = (long long)((emis + room) / 12);
     if (cap > 6144) cap = 6144;
     if (cap < 2 * nmax) cap = 2 * nmax;
@@ -216,10 +247,111 @@ __device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, in
     return prefix;
 }
 
+
+// ---- edge scores on demand --------------------------------------------------------------------------------------
+// Row j of the edge scores (children at depth j+1), Eq. 4-6: the table rows P[parent token], C[child token] and
+// u_j are copied into shared memory asynchronously (16-byte cp.async chunks spread over the CTA, issued while the
+// level above is expanded); K x K dot products of (P + u_j) and (C + u_j) in fp32, centred over the children, plus
+// log q; each parent's row is then ordered by (edge descending, child rank ascending).
+__device__ __forceinline__ bool lazy_neutral(const TreeParams& p, int j) {
+    return p.beta == 0.0f || (j == 0 && !p.root_edge);
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// Every thread calls this; the copies of one row form one group per thread.
+__device__ __forceinline__ void lazy_issue_gather(const TreeParams& p, const TreeSmem& sm, int j, int root_token, int tid) {
+    if (j >= p.L || lazy_neutral(p, j)) return;
+    const int K = p.K, m = p.m, ld = m + 4, q4 = m / 4, n_par = j == 0 ? 1 : K;
+    const int total = (n_par + K + 1) * q4;
+    for (int i = tid; i < total; i += TREE_THREADS) {
+        const int r = i / q4, k4 = i - r * q4;
+        const float* src;
+        float* dst;
+        if (r == n_par + K) {
+            src = p.u + (size_t)j * m;
+            dst = sm.gU;
+        } else {
+            int tok = r < n_par ? (j == 0 ? root_token : sm.tokid[(j - 1) * K + r]) : sm.tokid[j * K + r - n_par];
+            tok = tok < 0 ? 0 : (tok >= p.V ? p.V - 1 : tok);
+            src = (r < n_par ? p.P : p.C) + (size_t)tok * m;
+            dst = r < n_par ? sm.gP + (size_t)r * ld : sm.gC + (size_t)(r - n_par) * ld;
+        }
+        cp_async16(smem_u32(dst + 4 * k4), src + 4 * k4);
+    }
+    cp_async_commit();
+}
+// Every thread of the CTA calls this.
+// `inflight` is the depth whose table rows are on their way (or -1).
+__device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSmem& sm, int j, int root_token, int tid,
+                                               int& inflight) {
+    const int K = p.K, m = p.m, n_par = j == 0 ? 1 : K;
+    const int warp = tid >> 5, lane = tid & 31;
+    float* es = sm.es + (size_t)j * K * K;
+    uint8_t* ei = sm.ei + (size_t)j * K * K;
+    const float* lps = sm.lpv + j * K;
+    if (lazy_neutral(p, j)) {
+        // edge = log q exactly (the DDTree score of Eq. 3); log q is already ordered by rank
+        for (int i = tid; i < K * K; i += TREE_THREADS) {
+            es[i] = (i / K) < n_par ? lps[i % K] : 0.f;
+            ei[i] = (uint8_t)(i % K);
+        }
+        __syncthreads();
+        return;
+    }
+#ifdef GRAFT_TREE_PROF
+    long long lt0 = clock64();
+#endif
+    if (inflight != j) lazy_issue_gather(p, sm, j, root_token, tid);
+    cp_async_wait_all();
+    __syncthreads();
+#ifdef GRAFT_TREE_PROF
+    long long lt1 = clock64();
+#endif
+    float* part = (float*)sm.hist;                // [K][K] dot products (the histogram space is idle here)
+    uint32_t* wsc = sm.hist + 1024 + warp * 32;   // [32] per warp
+    if (warp < 8) edge_dots<true>(sm.gP, sm.gC, sm.gU, m, K, n_par, part, warp, lane);
+    __syncthreads();
+#ifdef GRAFT_TREE_PROF
+    long long lt2 = clock64();
+#endif
+    lazy_issue_gather(p, sm, j + 1, root_token, tid);  // the table rows of this depth are no longer read
+    inflight = j + 1;
+#ifdef GRAFT_TREE_PROF
+    long long lt3 = clock64();
+#endif
+    for (int par = warp; par < K; par += TREE_THREADS / 32) {  // one warp per parent
+        float val;
+        int rank;
+        edge_row_finish(par < n_par ? part + (size_t)par * K : nullptr, lps, p.scale, p.beta, K, wsc, lane, val, rank);
+        if (lane < K) {
+            es[(size_t)par * K + rank] = val;
+            ei[(size_t)par * K + rank] = (uint8_t)lane;
+        }
+    }
+#ifdef GRAFT_TREE_PROF
+    long long lt4 = clock64();
+#endif
+    __syncthreads();
+#ifdef GRAFT_TREE_PROF
+    if (tid == 0 && p.out.d_edge) {
+        float* dbg = p.out.d_edge + (size_t)blockIdx.x * p.L * K * K + 64 + 5 * j;
+        dbg[0] = (float)(lt1 - lt0);
+        dbg[1] = (float)(lt2 - lt1);
+        dbg[2] = (float)(lt3 - lt2);
+        dbg[3] = (float)(lt4 - lt3);
+        dbg[4] = (float)(clock64() - lt4);
+    }
+#endif
+}
+
 __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TreeSmem sm;
-    tree_smem_layout(p.L, p.K, p.nmax, p.ncap, &sm, smem_raw);
+    tree_smem_layout(p.L, p.K, p.nmax, p.ncap, p.lazy_m, &sm, smem_raw);
     const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int L = p.L, K = p.K, nmax = p.nmax, W = p.W;
     const graft_tree_out& o = p.out;
@@ -231,15 +363,34 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     // the sorted edge rows of this sequence: bulk copies through the TMA unit when the 16-byte rules allow it
     // (they land while warp 0 works out the budget), plain loads otherwise
     __shared__ __align__(8) uint64_t rows_bar;
-    const int ne = L * K * K;
-    const bool bulk = (ne % 16) == 0;
+    __shared__ int rows_abort;
+    const int ne = p.rows_pre * K * K;  // entries that come from the edge-score kernel
+    const bool bulk = ne > 0 && (ne % 16) == 0;
+    const int root = p.root_token[b];
+    int rows_done = p.rows_pre;  // rows [0, rows_done) are in shared memory
+    int inflight = -1;           // on-demand scoring: depth whose table rows are being fetched
+    if (tid == 0) {
+        rows_abort = 0;
+        mbar_init(smem_u32(&rows_bar), 1);
+        mbar_fence_init();
+    }
+    if (p.lazy) {  // the candidates of every depth, for the rows that may have to be scored here
+        for (int i = tid; i < L * K; i += TREE_THREADS) {
+            sm.tokid[i] = p.topk_id[(size_t)b * L * K + i];
+            sm.lpv[i] = p.topk_lp[(size_t)b * L * K + i];
+        }
+        if (p.rows_pre == 0) {  // the table rows of depth 0 arrive while the budget is worked out
+            __syncthreads();
+            lazy_issue_gather(p, sm, 0, root, tid);
+            inflight = 0;
+        }
+    }
+    const size_t seq_e = (size_t)b * L * K * K;  // this sequence's rows in esort / eidx
     if (bulk) {
         if (tid == 0) {
-            mbar_init(smem_u32(&rows_bar), 1);
-            mbar_fence_init();
             mbar_arrive_expect_tx(smem_u32(&rows_bar), (uint32_t)ne * 5u);
-            const char* g_es = (const char*)(p.esort + (size_t)b * ne);
-            const char* g_ei = (const char*)(p.eidx + (size_t)b * ne);
+            const char* g_es = (const char*)(p.esort + seq_e);
+            const char* g_ei = (const char*)(p.eidx + seq_e);
             for (uint32_t off = 0; off < (uint32_t)ne * 4u; off += 16384u) {
                 const uint32_t bytes = (uint32_t)ne * 4u - off < 16384u ? (uint32_t)ne * 4u - off : 16384u;
                 tma_load_1d(smem_u32((char*)sm.es + off), g_es + off, bytes, smem_u32(&rows_bar));
@@ -251,8 +402,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         }
     } else {
         for (int i = tid; i < ne; i += TREE_THREADS) {
-            sm.es[i] = p.esort[(size_t)b * ne + i];
-            sm.ei[i] = p.eidx[(size_t)b * ne + i];
+            sm.es[i] = p.esort[seq_e + i];
+            sm.ei[i] = p.eidx[seq_e + i];
         }
     }
     // adjacent-position cosines r_d = cos(h_d, h_{d+1}) (Eq. 15): one warp per pair, fp64 accumulation
@@ -382,9 +533,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     __syncthreads();
     if (bulk) {
         // bounded wait for the bulk copies; on a timeout the sequence is reported through its status word
-        __shared__ int rows_abort;
-        if (tid == 0) rows_abort = 0;
-        __syncthreads();
         if (!mbar_wait_bounded(smem_u32(&rows_bar), 0, &rows_abort) && tid == 0) sm.scal[2] |= GRAFT_ST_INTERNAL;
         __syncthreads();
     }
@@ -426,6 +574,10 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
 #endif
             const int b0 = sm.lvl_start[d], b1 = sm.lvl_start[d + 1];
             if (b1 == b0) break;
+            if (d >= rows_done) {  // the edge rows of this depth: scored now, never if the expansion stops above it
+                lazy_score_row(p, sm, d, root, tid, inflight);
+                rows_done = d + 1;
+            }
             if (theta == 0u) {
                 // no threshold yet (fewer than B nodes so far): every child of every node of the level is appended,
                 // one thread per (node, child), at a position that needs no atomic
@@ -567,6 +719,9 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
 #ifdef GRAFT_TREE_PROF
     t_prof15 = clock64();
 #endif
+    if (p.lazy && !table_ok && budget > 0) {  // the sequential fall-back may reach any depth
+        for (; rows_done < L; ++rows_done) lazy_score_row(p, sm, rows_done, root, tid, inflight);
+    }
     if (!table_ok && tid == 0) sm.ent[0] = budget > 0 ? pack_entry(0.0f + sm.es[0], 1, 0, 0, sm.ei[0]) : 0ull;
     __syncthreads();
     if (warp == 0) {
@@ -612,9 +767,15 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     const int at = ((d - 1) * K + cpar) * K + pos + 1;
                     e_adv = pack_entry(sm.S[bn] + sm.es[at], d, pos + 1, cpar, sm.ei[at]);
                 }
-                if (d < L) {
-                    const int at = (d * K + c) * K;
-                    e_new = pack_entry(s_new + sm.es[at], d + 1, 0, c, sm.ei[at]);
+                if (d < L && n_sel < budget) {  // (after the last selection the entry is never read)
+                    // a node selected here has a key >= theta, so it sits in the table and the row of its depth
+                    // was scored when its level was expanded
+                    if (d >= rows_done) {
+                        st |= GRAFT_ST_INTERNAL;
+                    } else {
+                        const int at = (d * K + c) * K;
+                        e_new = pack_entry(s_new + sm.es[at], d + 1, 0, c, sm.ei[at]);
+                    }
                 }
                 sm.ent[bn] = e_adv;
                 sm.ent[n_new] = e_new;
@@ -698,7 +859,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         __syncthreads();
     }
     const int prefix = p.prefix_len[b];
-    const int root = p.root_token[b];
     const size_t ob = (size_t)b * nmax;
     for (int n = tid; n < n_nodes; n += TREE_THREADS) {
         const int i = sm.canon[n], d = sm.depth[n];
@@ -767,10 +927,11 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         o.d_state[(size_t)b * 4 + 3] = (float)(clock64() - t_prof2);
     }
 #endif
+    if (p.lazy) cp_async_wait_all();  // table rows fetched ahead for a depth that was never scored
     if (tid == 0) {
         o.d_n_nodes[b] = n_nodes;
         o.d_budget[b] = sm.scal[0];
-        o.d_status[b] = sm.scal[2];
+        o.d_status[b] = sm.scal[2] | (rows_abort ? GRAFT_ST_INTERNAL : 0);
     }
 }
 
@@ -848,9 +1009,16 @@ __global__ void __launch_bounds__(128) accept_kernel(const int32_t* __restrict__
 
 }  // namespace
 
+// Edge scores are computed inside the tree kernel when its gather buffers fit in shared memory beside the rest.
+bool tree_lazy_fits(const graft_config& cfg) {
+    const int nmax = cfg.budget_max + 1;
+    return tree_smem_layout(cfg.L, cfg.K, nmax, 2 * nmax, cfg.m, nullptr, nullptr) <= (size_t)222 * 1024;
+}
+
 size_t tree_smem_bytes(const graft_config& cfg) {
     const int nmax = cfg.budget_max + 1;
-    return tree_smem_layout(cfg.L, cfg.K, nmax, tree_node_cap(cfg.L, cfg.K, nmax), nullptr, nullptr);
+    const int lazy_m = tree_lazy_fits(cfg) ? cfg.m : 0;
+    return tree_smem_layout(cfg.L, cfg.K, nmax, tree_node_cap(cfg.L, cfg.K, nmax, lazy_m), lazy_m, nullptr, nullptr);
 }
 
 cudaError_t tree_configure(const graft_config& cfg) {
@@ -880,7 +1048,18 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     p.K = cfg.K;
     p.nmax = ctx->nmax;
     p.W = ctx->mask_words;
-    p.ncap = tree_node_cap(cfg.L, cfg.K, ctx->nmax);
+    p.rows_pre = ctx->edge_rows;
+    p.lazy = p.rows_pre < cfg.L ? 1 : 0;  // (only possible when tree_lazy_fits)
+    p.lazy_m = tree_lazy_fits(cfg) ? cfg.m : 0;
+    p.ncap = tree_node_cap(cfg.L, cfg.K, ctx->nmax, p.lazy_m);
+    p.P = ctx->d_P;
+    p.C = ctx->d_C;
+    p.u = ctx->d_u;
+    p.scale = ctx->tdes_s / sqrtf((float)cfg.m);
+    p.beta = ctx->tdes_set ? cfg.beta : 0.0f;
+    p.root_edge = cfg.root_edge;
+    p.m = cfg.m;
+    p.V = cfg.V;
     p.bmin = cfg.budget_min;
     p.bmax = cfg.budget_max;
     p.bstep = cfg.budget_step;

@@ -181,6 +181,89 @@ def test_round_small(kw, beta):
     compare_accept(oracle, gi, g, w, out, gpu)
 
 
+def test_round_edge_rows_need_the_separate_kernel_when_the_tables_are_wide():
+    """m = 512 with K = 32, L = 16: the table rows do not fit in the tree kernel's shared memory, so every depth
+    is scored by the separate kernel and the split cannot be changed."""
+    from paper_2608_20375_b200 import GraftError
+    w = gi.small(batch=3, L=16, V=6000, K=32, budget_min=32, budget_max=512, budget_step=16, m=512, hidden_dim=64,
+                 boost_lo=6.0, boost_hi=14.0)
+    g = _graft(w)
+    assert g.edge_rows() == w.L
+    with pytest.raises(GraftError):
+        g.set_edge_rows(4)
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    assert stats["excused_tree"] + stats["excused_budget"] <= 1, stats
+
+
+_SPLIT_CASES = [
+    dict(batch=4, L=16, V=20011, K=32, budget_min=32, budget_max=512, budget_step=16, logits_dtype="bf16", m=128,
+         hidden_dim=128, boost_lo=6.0, boost_hi=14.0),
+    dict(batch=3, L=6, V=5000, K=8, budget_min=16, budget_max=96, budget_step=16, m=32),
+    dict(batch=2, L=5, V=300, K=1, budget_min=4, budget_max=12, budget_step=4),  # a chain: every depth is reached
+    dict(batch=3, L=16, V=32000, K=8, budget_min=64, budget_max=64, fixed_budget=64, hidden_ar1=False, m=36),
+    dict(batch=2, L=12, V=900, K=5, budget_min=40, budget_max=40, fixed_budget=40, m=20, boost_lo=14.0,
+         boost_hi=14.0),                                                          # peaked: deep and narrow
+]
+
+
+@pytest.mark.parametrize("kw", _SPLIT_CASES)
+@pytest.mark.parametrize("rows", [0, 1, 3, None])
+def test_round_edge_rows_split(kw, rows):
+    """The depths up to `rows` are scored by the separate kernel, the rest on demand inside the tree kernel
+    (None: all by the separate kernel).  Every split must give oracle-valid trees."""
+    w = gi.small(**kw)
+    g = _graft(w)
+    g.set_edge_rows(min(w.L, w.L if rows is None else rows))
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    assert stats["excused_tree"] + stats["excused_budget"] <= max(1, w.batch // 4), stats
+    assert int(gpu["depth"].max()) >= min(w.L, 3)  # the case does reach the depths scored on demand
+    g.destroy()
+
+
+@pytest.mark.parametrize("kw", _SPLIT_CASES)
+def test_round_does_not_depend_on_the_edge_rows_split(kw):
+    """Both scorers run the same arithmetic in the same order, so the trees are the same bit for bit."""
+    w = gi.small(**kw)
+    g = _graft(w)
+    _setup(w, g)
+    x = gi.batch_inputs(w)
+    outs = []
+    for rows in (0, 2, w.L):
+        g.set_edge_rows(min(rows, w.L))
+        outs.append(gpu_round(g, w, x, debug=False)[1])
+    for other in outs[1:]:
+        for k in ("n_nodes", "budget", "status", "token", "parent", "depth", "position", "path_score", "mask"):
+            assert np.array_equal(outs[0][k], other[k]), k
+    g.destroy()
+
+
+@pytest.mark.parametrize("kw", _SPLIT_CASES[:3] + [
+    dict(batch=3, L=16, V=6000, K=32, budget_min=32, budget_max=512, budget_step=16, m=512, hidden_dim=64)])
+@pytest.mark.parametrize("rows", [0, None])
+def test_round_without_debug_outputs_gives_the_same_trees(kw, rows):
+    """The production call (no candidate / edge / state outputs requested) must give the trees of the call
+    that also writes the debug arrays, bit for bit."""
+    w = gi.small(**kw)
+    g = _graft(w)
+    if rows is not None and w.m < 512:  # (m = 512: the split is fixed, every depth by the separate kernel)
+        g.set_edge_rows(rows)
+    _setup(w, g)
+    x = gi.batch_inputs(w)
+    _, a = gpu_round(g, w, x, debug=True)
+    _, b = gpu_round(g, w, x, debug=False)
+    for k in ("n_nodes", "budget", "status", "token", "parent", "depth", "position", "path_score", "mask"):
+        assert np.array_equal(a[k], b[k]), k
+    g.destroy()
+
+
 def test_round_bad_rows_and_status_bits():
     w = gi.small(batch=4, L=4, V=2000, K=4, budget_min=8, budget_max=24, budget_step=8)
     g = _graft(w)
