@@ -30,9 +30,9 @@ import graft_inputs as gi  # noqa: E402
 
 METRIC = "draft trees built and verified-walked per second (batch 64, L=16, V=151,936 bf16)"
 UNIT = "trees/s"
-# DRAM bytes (read + write) of one vocab-pass launch on workload M, from the ncu capture summarised in
-# profiles/; None until a capture exists.
-NCU_VOCAB_TRAFFIC_BYTES_M = None
+# DRAM bytes (read + write) of one vocab-pass launch on workload M: the mean of the two launches of the ncu
+# capture summarised in profiles/vocab_pass_kernel_M.md.
+NCU_VOCAB_TRAFFIC_BYTES_M = 321_486_208
 L2_BYTES = 126 * 1024 * 1024
 
 

@@ -70,9 +70,7 @@ const char* graft_status_str(graft_status s) {
     return "unknown status";
 }
 
-int graft_debug_read(graft_ctx* ctx, int32_t* out64) { return (int)cudaMemcpy(out64, ctx->w_errflag, 256, cudaMemcpyDeviceToHost); }
 
-int graft_debug_read2(graft_ctx* ctx, float* out, int n) { return (int)cudaMemcpy(out, ctx->w_edge, (size_t)n * 4, cudaMemcpyDeviceToHost); }
 
 const char* graft_version(void) { return "graft-b200 0.1 (sm_100a)"; }
 

@@ -302,27 +302,15 @@ __device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSm
         __syncthreads();
         return;
     }
-#ifdef GRAFT_TREE_PROF
-    long long lt0 = clock64();
-#endif
     if (inflight != j) lazy_issue_gather(p, sm, j, root_token, tid);
     cp_async_wait_all();
     __syncthreads();
-#ifdef GRAFT_TREE_PROF
-    long long lt1 = clock64();
-#endif
     float* part = (float*)sm.hist;                // [K][K] dot products (the histogram space is idle here)
     uint32_t* wsc = sm.hist + 1024 + warp * 32;   // [32] per warp
     if (warp < 8) edge_dots<true>(sm.gP, sm.gC, sm.gU, m, K, n_par, part, warp, lane);
     __syncthreads();
-#ifdef GRAFT_TREE_PROF
-    long long lt2 = clock64();
-#endif
     lazy_issue_gather(p, sm, j + 1, root_token, tid);  // the table rows of this depth are no longer read
     inflight = j + 1;
-#ifdef GRAFT_TREE_PROF
-    long long lt3 = clock64();
-#endif
     for (int par = warp; par < K; par += TREE_THREADS / 32) {  // one warp per parent
         float val;
         int rank;
@@ -332,20 +320,7 @@ __device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSm
             ei[(size_t)par * K + rank] = (uint8_t)lane;
         }
     }
-#ifdef GRAFT_TREE_PROF
-    long long lt4 = clock64();
-#endif
     __syncthreads();
-#ifdef GRAFT_TREE_PROF
-    if (tid == 0 && p.out.d_edge) {
-        float* dbg = p.out.d_edge + (size_t)blockIdx.x * p.L * K * K + 64 + 5 * j;
-        dbg[0] = (float)(lt1 - lt0);
-        dbg[1] = (float)(lt2 - lt1);
-        dbg[2] = (float)(lt3 - lt2);
-        dbg[3] = (float)(lt4 - lt3);
-        dbg[4] = (float)(clock64() - lt4);
-    }
-#endif
 }
 
 __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) {
