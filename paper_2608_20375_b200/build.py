@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgraft.so")
 SOURCES = ["api.cu", "vocab_pass.cu", "tdes.cu", "tree.cu"]
-HEADERS = ["common.cuh", "internal.h", "edge_score.cuh", os.path.join("..", "..", "include", "graft.h")]
+HEADERS = ["common.cuh", "internal.h", "edge_score.cuh", "cosine.cuh", os.path.join("..", "..", "include", "graft.h")]
 # no --use_fast_math: the fp64 pieces (log-sum-exp fold, SABA) and the fp32 divisions must stay IEEE
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]

@@ -126,7 +126,7 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     const size_t o_id = take(B * L * K * 4), o_lp = take(B * L * K * 4), o_lse = take(B * L * 4);
     const size_t o_rs = take(B * L * 4), o_edge = take(B * L * K * K * 4);
     const size_t o_es = take(B * L * K * K * 4), o_ei = take(B * L * K * K);
-    const size_t o_u = take(L * (size_t)cfg->m * 4), o_err = take(256);
+    const size_t o_u = take(L * (size_t)cfg->m * 4), o_err = take(256), o_cos = take(B * L * 8);
     ctx->ws_bytes = off;
     if (cudaMalloc(&ctx->ws, ctx->ws_bytes) != cudaSuccess) {
         cudaGetLastError();
@@ -154,6 +154,7 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     ctx->d_u = (float*)(base + o_u);
     ctx->edge_rows = tree_lazy_fits(*cfg) ? (cfg->L < 8 ? cfg->L : 8) : cfg->L;
     ctx->w_errflag = (int32_t*)(base + o_err);
+    ctx->w_cos = (double*)(base + o_cos);
     *out = ctx;
     return GRAFT_OK;
 }
@@ -249,7 +250,7 @@ graft_status graft_vocab_pass(graft_ctx* ctx, int32_t batch, const void* d_logit
     const int esz = ctx->cfg.logits_dtype == GRAFT_BF16 ? 2 : 4;
     if ((uintptr_t)d_logits % esz) return GRAFT_ERR_INVALID_ARG;
     if (vp_launch(ctx, batch, d_logits, d_topk_id, d_topk_lp, d_lse, d_row_status ? d_row_status : ctx->w_row_status,
-                  (cudaStream_t)stream) != cudaSuccess)
+                  nullptr, nullptr, (cudaStream_t)stream) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     return GRAFT_OK;
 }
@@ -260,8 +261,7 @@ graft_status graft_tdes_edges(graft_ctx* ctx, int32_t batch, const int32_t* d_to
     if (batch < 1 || batch > ctx->cfg.max_batch) return GRAFT_ERR_INVALID_ARG;
     if (ctx->cfg.beta != 0.0f && !ctx->tdes_set) return GRAFT_ERR_STATE;
     if (tdes_edges_launch(ctx, batch, d_topk_id, d_topk_lp, d_root_token, nullptr, d_edge, ctx->w_esort, ctx->w_eidx,
-                          ctx->cfg.L,
-                          (cudaStream_t)stream) != cudaSuccess)
+                          ctx->cfg.L, (cudaStream_t)stream) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     return GRAFT_OK;
 }
@@ -328,7 +328,9 @@ graft_status graft_build_trees(graft_ctx* ctx, int32_t batch, const void* d_logi
     float* edge = out->d_edge ? out->d_edge : ctx->w_edge;
 
     if (ev) cudaEventRecord(ev[0], st);
-    if (vp_launch(ctx, batch, d_logits, ids, lps, lse, ctx->w_row_status, st) != cudaSuccess) return GRAFT_ERR_CUDA;
+    if (vp_launch(ctx, batch, d_logits, ids, lps, lse, ctx->w_row_status, use_saba ? d_hidden : nullptr, ctx->w_cos,
+                  st) != cudaSuccess)
+        return GRAFT_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], st);
     // Edge scores of Eq. 4-6: the kernel scores the depths [0, edge_rows) for every sequence (all depths when the
     // caller asks for the score array); the tree kernel scores deeper rows itself if an expansion gets that far.
@@ -340,7 +342,7 @@ graft_status graft_build_trees(graft_ctx* ctx, int32_t batch, const void* d_logi
     }
     if (ev) cudaEventRecord(ev[2], st);
     if (tree_launch(ctx, batch, ids, lps, ctx->w_row_status, ctx->w_esort, ctx->w_eidx, d_hidden, d_root_token, d_hist, d_prefix_len,
-                    d_fixed_budget, out, st) != cudaSuccess)
+                    d_fixed_budget, ctx->w_cos, out, st) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     if (ev) {
         cudaEventRecord(ev[3], st);

@@ -17,7 +17,7 @@ constexpr int kVpConsumers = kVpConsumerWarps * 32;  // 512
 constexpr int kVpEpiThreads = 128;                   // four warps per epilogue group
 constexpr int kVpEpiGroups = 2;                      // the groups take alternate segments
 constexpr int kVpBufs = 4;                           // hand-over buffers between streaming and epilogue warps
-constexpr int kVpThreads = kVpConsumers + kVpEpiGroups * kVpEpiThreads + 32;  // + one producer warp
+constexpr int kVpThreads = kVpConsumers + kVpEpiGroups * kVpEpiThreads + 64;  // + one producer warp + one cosine warp
 constexpr int kVpTileBytes = 32768;                  // one ring stage (2 KiB per streaming warp)
 constexpr int kVpQuantum = 2048;                     // elements; granularity of the work partition
 constexpr int kVpCandCap = 1024;                     // candidate keys held in shared memory
@@ -73,6 +73,7 @@ struct graft_ctx {
     float* w_edge;                // [max_batch, L, K, K]
     float* w_esort;               // [max_batch, L, K, K] rows sorted by edge score
     uint8_t* w_eidx;              // [max_batch, L, K, K] child rank of each sorted entry
+    double* w_cos;                // [max_batch, L] adjacent-position cosines (Eq. 15)
     int32_t* w_errflag;           // [1] device-side internal error flag
     graft::VpPlan vp_plan;
     // host-buffer staging (allocated on first use of graft_build_trees_host)
@@ -89,7 +90,9 @@ namespace graft {
 VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch);
 cudaError_t vp_configure(const graft_config& cfg, int num_sms, size_t* max_smem);
 cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* d_topk_id, float* d_topk_lp,
-                      float* d_lse, int32_t* d_row_status, cudaStream_t st);
+                      float* d_lse, int32_t* d_row_status, const void* d_hidden, double* d_cos, cudaStream_t st);
+// d_hidden != NULL: one more warp per CTA also writes the adjacent-position cosines of the SABA state (Eq. 15)
+// to d_cos [batch, L]
 
 cudaError_t tdes_precompute_launch(graft_ctx* ctx, const void* d_emb, graft_dtype dt, int E, const float* d_W,
                                    const float* d_b, float* d_out, cudaStream_t st);
@@ -99,7 +102,7 @@ cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_i
 cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                         const int32_t* d_row_status, const float* d_esort, const uint8_t* d_eidx, const void* d_hidden,
                         const int32_t* d_root_token, const float* d_hist, const int32_t* d_prefix_len,
-                        const int32_t* d_fixed_budget, const graft_tree_out* out, cudaStream_t st);
+                        const int32_t* d_fixed_budget, const double* d_cos, const graft_tree_out* out, cudaStream_t st);
 cudaError_t accept_launch(graft_ctx* ctx, int batch, const graft_tree_out* trees, const int32_t* d_target_next,
                           int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus, cudaStream_t st);
 size_t tree_smem_bytes(const graft_config& cfg);

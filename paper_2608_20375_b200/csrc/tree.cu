@@ -13,10 +13,10 @@ struct TreeParams {
     const int32_t* topk_id;
     const float* topk_lp;
     const int32_t* row_status;
+    const double* cos_pre;  // [batch, L] adjacent-position cosines (Eq. 15), written by the vocab pass
+    const int32_t* vp_err;  // word 0: a bounded wait of the vocab pass ran out (sticky)
     const float* esort;   // [batch, L, K, K] edge rows sorted by (edge desc, child rank asc)
     const uint8_t* eidx;  // child rank of each sorted entry
-    const void* hidden;   // [batch, L, hidden_dim] (SABA only)
-    int hidden_dim, hidden_bf16;
     const int32_t* root_token;
     const float* hist;
     const int32_t* prefix_len;
@@ -381,71 +381,16 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             sm.ei[i] = p.eidx[seq_e + i];
         }
     }
-    // adjacent-position cosines r_d = cos(h_d, h_{d+1}) (Eq. 15): one warp per pair, fp64 accumulation
+    // adjacent-position cosines r_d = cos(h_d, h_{d+1}) (Eq. 15): written by the vocab pass
     if (p.use_saba) {
-        for (int d = warp; d < L - 1; d += TREE_THREADS / 32) {
-            const int dh = p.hidden_dim;
-            const size_t ra = ((size_t)b * L + d) * dh, rb = ra + dh;
-            double ab = 0.0, aa = 0.0, bb = 0.0;
-            if (p.hidden_bf16 && (dh & 7) == 0 && ((uintptr_t)p.hidden & 15) == 0) {
-                const uint4* pa = (const uint4*)((const uint16_t*)p.hidden + ra);
-                const uint4* pb = (const uint4*)((const uint16_t*)p.hidden + rb);
-                constexpr int CU = 4;  // vectors in flight per row and lane: the loads of a step are issued together
-                for (int k0 = lane; k0 < dh / 8; k0 += 32 * CU) {
-                    uint4 va[CU], vb[CU];
-#pragma unroll
-                    for (int u = 0; u < CU; ++u) {
-                        const int k = k0 + 32 * u;
-                        va[u] = k < dh / 8 ? pa[k] : make_uint4(0u, 0u, 0u, 0u);
-                        vb[u] = k < dh / 8 ? pb[k] : make_uint4(0u, 0u, 0u, 0u);
-                    }
-#pragma unroll
-                    for (int u = 0; u < CU; ++u) {
-                        const uint32_t wa[4] = {va[u].x, va[u].y, va[u].z, va[u].w};
-                        const uint32_t wb[4] = {vb[u].x, vb[u].y, vb[u].z, vb[u].w};
-                        float fab = 0.f, faa = 0.f, fbb = 0.f;  // eight exact bf16 products per sum: fp32 is enough
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float x0 = __uint_as_float(wa[q] << 16), x1 = __uint_as_float(wa[q] & 0xFFFF0000u);
-                            const float y0 = __uint_as_float(wb[q] << 16), y1 = __uint_as_float(wb[q] & 0xFFFF0000u);
-                            fab = fmaf(x0, y0, fmaf(x1, y1, fab));
-                            faa = fmaf(x0, x0, fmaf(x1, x1, faa));
-                            fbb = fmaf(y0, y0, fmaf(y1, y1, fbb));
-                        }
-                        ab += (double)fab;
-                        aa += (double)faa;
-                        bb += (double)fbb;
-                    }
-                }
-            } else {
-                for (int k = lane; k < dh; k += 32) {
-                    float x, y;
-                    if (p.hidden_bf16) {
-                        x = __uint_as_float(((uint32_t)((const uint16_t*)p.hidden)[ra + k]) << 16);
-                        y = __uint_as_float(((uint32_t)((const uint16_t*)p.hidden)[rb + k]) << 16);
-                    } else {
-                        x = ((const float*)p.hidden)[ra + k];
-                        y = ((const float*)p.hidden)[rb + k];
-                    }
-                    ab += (double)x * (double)y;
-                    aa += (double)x * (double)x;
-                    bb += (double)y * (double)y;
-                }
-            }
-#pragma unroll
-            for (int o2 = 16; o2 > 0; o2 >>= 1) {
-                ab += __shfl_xor_sync(0xFFFFFFFFu, ab, o2);
-                aa += __shfl_xor_sync(0xFFFFFFFFu, aa, o2);
-                bb += __shfl_xor_sync(0xFFFFFFFFu, bb, o2);
-            }
-            if (lane == 0) sm.cosv[d] = (aa > 0.0 && bb > 0.0) ? ab / (sqrt(aa) * sqrt(bb)) : 0.0;
-        }
+        if (tid < L - 1) sm.cosv[tid] = p.cos_pre[(size_t)b * L + tid];
         __syncthreads();
     }
     if (warp == 0) {
         int st = 0;
         for (int j = lane; j < L; j += 32) st |= p.row_status[(size_t)b * L + j];
         st = __reduce_or_sync(0xFFFFFFFFu, st);
+        if (p.vp_err[0] & 1) st |= GRAFT_ST_INTERNAL;
         int budget = 0;
         float state[4] = {0.f, 0.f, 0.f, 0.f};
         if (!(st & GRAFT_ST_BAD_LOGITS)) {
@@ -1003,17 +948,17 @@ cudaError_t tree_configure(const graft_config& cfg) {
 cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                         const int32_t* d_row_status, const float* d_esort, const uint8_t* d_eidx, const void* d_hidden,
                         const int32_t* d_root_token, const float* d_hist, const int32_t* d_prefix_len,
-                        const int32_t* d_fixed_budget, const graft_tree_out* out, cudaStream_t st) {
+                        const int32_t* d_fixed_budget, const double* d_cos, const graft_tree_out* out, cudaStream_t st) {
     const graft_config& cfg = ctx->cfg;
     TreeParams p;
     p.topk_id = d_topk_id;
     p.topk_lp = d_topk_lp;
     p.row_status = d_row_status;
+    p.vp_err = ctx->w_errflag;
+    p.cos_pre = d_cos;
     p.esort = d_esort;
     p.eidx = d_eidx;
-    p.hidden = d_hidden;
-    p.hidden_dim = cfg.hidden_dim;
-    p.hidden_bf16 = cfg.hidden_dtype == GRAFT_BF16 ? 1 : 0;
+    (void)d_hidden;  // read by the vocab pass, which leaves the cosines in d_cos
     p.root_token = d_root_token;
     p.hist = d_hist;
     p.prefix_len = d_prefix_len;

@@ -24,6 +24,7 @@
 
 #include "common.cuh"
 #include "internal.h"
+#include "cosine.cuh"
 
 #ifndef GRAFT_VP_F32X2
 #define GRAFT_VP_F32X2 1  // packed fp32 pair arithmetic (fma.rn.f32x2 / add.rn.f32x2)
@@ -47,7 +48,9 @@ constexpr int WBLK = TILE / NW;               // bytes of a tile owned by one wa
 static_assert(WBLK == 2048, "one warp owns 2 KiB of every tile");
 constexpr int VEC_PER_LANE = WBLK / 16 / 32;  // 4
 static_assert(VEC_PER_LANE == 4, "chunk layout assumes four 16-byte vectors per lane per tile");
-static_assert(kVpThreads == NT + kVpEpiGroups * kVpEpiThreads + 32, "thread count = streaming warps + epilogue warps + producer warp");
+constexpr int COS_WARP = PROD_WARP + 1;  // warp that computes the SABA cosines beside the stream
+static_assert(kVpThreads == NT + kVpEpiGroups * kVpEpiThreads + 64,
+              "thread count = streaming warps + epilogue warps + producer warp + cosine warp");
 
 template <bool BF16>
 struct VT;
@@ -79,6 +82,11 @@ struct VpParams {
     float* lse;
     int32_t* row_status;
     int32_t* errflag;
+    // adjacent-position cosines of the SABA state (Eq. 15), computed by a warp of their own beside the stream;
+    // cos_out == nullptr: not asked for
+    const void* hidden;
+    int hidden_bf16, hidden_dim, L;
+    double* cos_out;  // [rows / L, L]
     int use_hint;
     float* dbg_out;  // profiling builds only
     int dbg;  // experiments only: 1 = stream without arithmetic, 2 = arithmetic without streaming, 3 = no epilogue
@@ -525,6 +533,19 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
 #ifdef GRAFT_VP_PROF
         if (warp == 0 && lane == 0) sh->t_stream_end = clock64() - t_kernel0;
 #endif
+    } else if (warp == COS_WARP) {
+        // ------------------------------ cosine warp ----------------------------------------------
+        // Adjacent-position cosines of the SABA state (Eq. 15): a few pairs of hidden-state rows per CTA, read
+        // beside the logits stream (under 3 % of its bytes) so that nothing downstream waits for them.
+        if (p.cos_out != nullptr && !p.dbg) {
+            const int npairs = (p.rows / p.L) * (p.L - 1);
+            for (int q = (int)blockIdx.x; q < npairs; q += (int)gridDim.x) {
+                const int sb = q / (p.L - 1), d = q - sb * (p.L - 1);
+                const double r = warp_adjacent_cosine(p.hidden, p.hidden_bf16, p.hidden_dim,
+                                                      ((size_t)sb * p.L + d) * p.hidden_dim, lane);
+                if (lane == 0) p.cos_out[(size_t)sb * p.L + d] = r;
+            }
+        }
     } else {
         // ------------------------------ epilogue groups (four warps each) ------------------------
         // Group g finishes the segments with k % 2 == g, so a group has two segment times for one epilogue.
@@ -716,9 +737,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             }
             epi_bar(grp);
             if (ew != 0) continue;
-            const int nhits = es->nhits;
             VP_T(5);
-            if (blockIdx.x == 1 && lane == 0) { atomicAdd(p.errflag + 10, ncand); atomicAdd(p.errflag + 11, nhits); atomicAdd(p.errflag + 12, 1); }
             // the double-buffered arrays of parity pb may be reused from here on
             __syncwarp();
             if (lane == 0) mbar_arrive(done0 + 8 * pb);
@@ -877,7 +896,7 @@ VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch) {
 }
 
 cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* d_topk_id, float* d_topk_lp,
-                      float* d_lse, int32_t* d_row_status, cudaStream_t st) {
+                      float* d_lse, int32_t* d_row_status, const void* d_hidden, double* d_cos, cudaStream_t st) {
     const graft_config& cfg = ctx->cfg;
     const bool bf16 = cfg.logits_dtype == GRAFT_BF16;
     VpPlan pl = vp_make_plan(cfg, ctx->num_sms, batch);
@@ -898,6 +917,11 @@ cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* 
     p.lse = d_lse;
     p.row_status = d_row_status;
     p.errflag = ctx->w_errflag;
+    p.hidden = d_hidden;
+    p.hidden_bf16 = cfg.hidden_dtype == GRAFT_BF16 ? 1 : 0;
+    p.hidden_dim = cfg.hidden_dim;
+    p.L = cfg.L;
+    p.cos_out = (d_hidden != nullptr && cfg.L > 1) ? d_cos : nullptr;
     p.use_hint = 1;
     p.dbg = 0;
     p.dbg_out = ctx->w_edge;
@@ -1037,6 +1061,11 @@ extern "C" graft_status graft_vocab_pass_static(int32_t batch, int32_t L, int32_
     p.lse = d_lse;
     p.row_status = d_row_status;
     p.errflag = sd->scratch->errflag;
+    p.hidden = nullptr;
+    p.hidden_bf16 = 0;
+    p.hidden_dim = 0;
+    p.L = L;
+    p.cos_out = nullptr;
     p.use_hint = 1;
     p.dbg = 0;
     p.dbg_out = nullptr;
