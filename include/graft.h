@@ -200,8 +200,9 @@ uint64_t graft_launch_count(const graft_ctx* ctx);
 
 /* Per-kernel device timing of graft_build_trees.  graft_set_timing(ctx, 1) makes every later call record
  * CUDA events on its stream around the vocab-pass kernel, the edge-score kernel and the tree kernel (a ring
- * of the last 64 calls) and resets the call count.  graft_read_timing waits for the newest recorded call and
- * returns the number of calls summed (at most 64) and the summed milliseconds of each kernel. */
+ * of the last 64 calls) and resets the call count; graft_set_timing(ctx, 2) does the same without the reset
+ * (to sample some calls of a longer run), 0 stops recording.  graft_read_timing waits for the newest recorded
+ * call and returns the number of calls summed (at most 64) and the summed milliseconds of each kernel. */
 graft_status graft_set_timing(graft_ctx* ctx, int32_t enable);
 graft_status graft_read_timing(graft_ctx* ctx, int32_t* n_calls, float* vocab_ms, float* tdes_ms, float* tree_ms);
 

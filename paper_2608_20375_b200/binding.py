@@ -298,8 +298,9 @@ class Graft:
     def launch_count(self) -> int:
         return int(self.lib.graft_launch_count(self._ctx))
 
-    def set_timing(self, enable: bool):
-        _check(self.lib, self.lib.graft_set_timing(self._ctx, 1 if enable else 0), "graft_set_timing")
+    def set_timing(self, enable):
+        """0 / False: stop; 1 / True: record and reset the call count; 2: record, keep counting."""
+        _check(self.lib, self.lib.graft_set_timing(self._ctx, int(enable)), "graft_set_timing")
 
     def read_timing(self):
         n = C.c_int32()

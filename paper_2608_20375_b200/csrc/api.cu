@@ -275,7 +275,7 @@ graft_status graft_set_timing(graft_ctx* ctx, int32_t enable) {
                 if (cudaEventCreate(&ex->timing.ev[i][j]) != cudaSuccess) return GRAFT_ERR_CUDA;
         ex->timing.created = true;
     }
-    ex->timing.calls = 0;
+    if (enable == 1) ex->timing.calls = 0;
     ctx->timing = enable ? 1 : 0;
     return GRAFT_OK;
 }
