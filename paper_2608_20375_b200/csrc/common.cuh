@@ -44,6 +44,14 @@ __device__ __forceinline__ uint32_t hmax2_bf16(uint32_t a, uint32_t b) {
     return r;
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// A kernel launched with launch_pdl() may start before the kernel ahead of it in the stream has finished (once
+// every CTA of that kernel has called pdl_launch_dependents() or exited); it must call pdl_wait() before it touches
+// anything the earlier kernel writes.  pdl_wait() returns when the earlier grid has completed and its writes are
+// visible; in a kernel launched the ordinary way both calls do nothing.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- mbarrier + TMA bulk copy -------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");

@@ -87,6 +87,23 @@ struct graft_ctx {
 
 namespace graft {
 
+// Launch `kernel` so that it may overlap the tail of the kernel ahead of it in the stream (programmatic dependent
+// launch).  The kernel must call pdl_wait() before it reads what that kernel wrote.
+template <typename P>
+inline cudaError_t launch_pdl(void (*kernel)(P), dim3 grid, dim3 block, size_t smem, cudaStream_t st, const P& params) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute at;
+    at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at.val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = &at;
+    lc.numAttrs = 1;
+    return cudaLaunchKernelEx(&lc, kernel, params);
+}
+
 VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch);
 cudaError_t vp_configure(const graft_config& cfg, int num_sms, size_t* max_smem);
 cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* d_topk_id, float* d_topk_lp,

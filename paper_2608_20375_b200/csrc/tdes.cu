@@ -92,6 +92,8 @@ struct EdgeParams {
 
 __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
     extern __shared__ __align__(16) float smem[];
+    pdl_launch_dependents();  // the tree kernel may move in as SMs free up; it waits for this grid before it reads
+    pdl_wait();               // the candidates come from the vocab pass
     const int b = blockIdx.x / p.rows, j = blockIdx.x % p.rows;
     const int K = p.K, m = p.m, ld = m + 4;  // padded row: 16-byte aligned, conflict-free float4 reads
     float* sP = smem;                        // [K][ld]  parent rows + u_d
@@ -217,9 +219,9 @@ cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_i
     p.beta = ctx->tdes_set ? cfg.beta : 0.0f;
     p.root_edge = cfg.root_edge;
     p.rows = rows;
-    tdes_edges_kernel<<<batch * rows, 256, tdes_edges_smem(cfg), st>>>(p);
+    const cudaError_t e = launch_pdl(tdes_edges_kernel, dim3(batch * rows), dim3(256), tdes_edges_smem(cfg), st, p);
     ctx->launches += 1;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace graft

@@ -330,6 +330,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int L = p.L, K = p.K, nmax = p.nmax, W = p.W;
     const graft_tree_out& o = p.out;
+    pdl_launch_dependents();  // an acceptance walk queued behind this kernel may move in; it waits for this grid
+    pdl_wait();  // candidates, cosines and edge rows come from the kernels ahead in the stream
 
     // ---- status and budget ---------------------------------------------------------------------------
 #ifdef GRAFT_TREE_PROF
@@ -860,11 +862,27 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
 // loads in flight together; warp 0 then walks out of shared memory.  In level order the parent indices never
 // decrease, so the children of the current node are found by a binary search for the first node whose parent
 // is >= it.
-__global__ void __launch_bounds__(128) accept_kernel(const int32_t* __restrict__ n_nodes, const int32_t* __restrict__ token,
-                                                     const int32_t* __restrict__ parent,
-                                                     const int32_t* __restrict__ target_next, int batch, int nmax, int L,
-                                                     int32_t* __restrict__ accept_len, int32_t* __restrict__ accept_path,
-                                                     int32_t* __restrict__ bonus) {
+struct AcceptParams {
+    const int32_t* n_nodes;
+    const int32_t* token;
+    const int32_t* parent;
+    const int32_t* target_next;
+    int batch, nmax, L;
+    int32_t* accept_len;
+    int32_t* accept_path;
+    int32_t* bonus;
+};
+
+__global__ void __launch_bounds__(128) accept_kernel(const AcceptParams ap) {
+    const int32_t* __restrict__ n_nodes = ap.n_nodes;
+    const int32_t* __restrict__ token = ap.token;
+    const int32_t* __restrict__ parent = ap.parent;
+    const int32_t* __restrict__ target_next = ap.target_next;
+    const int nmax = ap.nmax, L = ap.L;
+    int32_t* __restrict__ accept_len = ap.accept_len;
+    int32_t* __restrict__ accept_path = ap.accept_path;
+    int32_t* __restrict__ bonus = ap.bonus;
+    pdl_wait();  // the tree may come from a tree kernel that is still running ahead in the stream
     extern __shared__ __align__(16) int32_t acc_smem[];
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     int32_t* par = acc_smem;
@@ -985,17 +1003,27 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     p.bstep = cfg.budget_step;
     p.use_saba = d_fixed_budget == nullptr;
     p.saba = ctx->saba;
-    tree_kernel<<<batch, TREE_THREADS, tree_smem_bytes(cfg), st>>>(p);
+    const cudaError_t e = launch_pdl(tree_kernel, dim3(batch), dim3(TREE_THREADS), tree_smem_bytes(cfg), st, p);
     ctx->launches += 1;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t accept_launch(graft_ctx* ctx, int batch, const graft_tree_out* trees, const int32_t* d_target_next,
                           int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus, cudaStream_t st) {
-    accept_kernel<<<batch, 128, (size_t)3 * ctx->nmax * sizeof(int32_t), st>>>(trees->d_n_nodes, trees->d_token, trees->d_parent, d_target_next,
-                                                   batch, ctx->nmax, ctx->cfg.L, d_accept_len, d_accept_path, d_bonus);
+    AcceptParams ap;
+    ap.n_nodes = trees->d_n_nodes;
+    ap.token = trees->d_token;
+    ap.parent = trees->d_parent;
+    ap.target_next = d_target_next;
+    ap.batch = batch;
+    ap.nmax = ctx->nmax;
+    ap.L = ctx->cfg.L;
+    ap.accept_len = d_accept_len;
+    ap.accept_path = d_accept_path;
+    ap.bonus = d_bonus;
+    const cudaError_t e = launch_pdl(accept_kernel, dim3(batch), dim3(128), (size_t)3 * ctx->nmax * sizeof(int32_t), st, ap);
     ctx->launches += 1;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace graft

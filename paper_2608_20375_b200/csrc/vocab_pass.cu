@@ -411,6 +411,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
     using T = VT<BF16>;
     using cm_t = typename T::cm_t;
     extern __shared__ __align__(128) unsigned char smem_raw[];
+    pdl_launch_dependents();  // the edge-score kernel's CTAs may move in as this grid's CTAs leave; they wait for it
     unsigned char* ring = smem_raw;
     uint64_t* bars = (uint64_t*)(ring + (size_t)p.stages * TILE);  // full[8], empty[8], ready[4], done[4]
     VpShared* sh = (VpShared*)(bars + 24);
