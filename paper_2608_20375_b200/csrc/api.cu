@@ -266,6 +266,12 @@ graft_status graft_tdes_edges(graft_ctx* ctx, int32_t batch, const int32_t* d_to
     return GRAFT_OK;
 }
 
+#if defined(GRAFT_VP_PROF) || defined(GRAFT_TREE_PROF)
+// profiling builds only (never in the shipped library): raw reads of the counters the instrumented kernels leave
+extern "C" int graft_debug_read(graft_ctx* ctx, int32_t* out64) { return (int)cudaMemcpy(out64, ctx->w_errflag, 256, cudaMemcpyDeviceToHost); }
+extern "C" int graft_debug_read2(graft_ctx* ctx, float* out, int n) { return (int)cudaMemcpy(out, ctx->w_edge, (size_t)n * 4, cudaMemcpyDeviceToHost); }
+#endif
+
 graft_status graft_set_timing(graft_ctx* ctx, int32_t enable) {
     if (!ctx) return GRAFT_ERR_INVALID_ARG;
     CtxExtra* ex = extra_of(ctx);

@@ -17,6 +17,7 @@ constexpr int kVpConsumers = kVpConsumerWarps * 32;  // 512
 constexpr int kVpEpiThreads = 128;                   // four warps per epilogue group
 constexpr int kVpEpiGroups = 2;                      // the groups take alternate segments
 constexpr int kVpBufs = 4;                           // hand-over buffers between streaming and epilogue warps
+constexpr int kVpGroups = 64;   // groups of streaming threads whose maxima bound the K-th largest element (>= kMaxK)
 constexpr int kVpThreads = kVpConsumers + kVpEpiGroups * kVpEpiThreads + 64;  // + one producer warp + one cosine warp
 constexpr int kVpTileBytes = 32768;                  // one ring stage (2 KiB per streaming warp)
 constexpr int kVpQuantum = 2048;                     // elements; granularity of the work partition

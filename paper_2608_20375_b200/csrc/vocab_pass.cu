@@ -332,6 +332,7 @@ struct __align__(16) EpiShared {  // private to one epilogue group
 struct __align__(16) VpShared {
     EpiShared epi[kVpEpiGroups];
     uint32_t tmax[kVpBufs][NT];  // per-thread maxima of a finished segment, one buffer per segment in flight
+    uint32_t gmax[kVpBufs][kVpGroups];  // the same maxima folded into 64 groups (lane, warp parity); zero when idle
     float wc[kVpBufs][NW], ws[kVpBufs][NW];
     long long t_stream_end;      // profiling builds only
     volatile int abort_flag;
@@ -438,6 +439,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
         mbar_fence_init();
         sh->abort_flag = 0;
     }
+    if (tid < kVpBufs * kVpGroups) (&sh->gmax[0][0])[tid] = 0u;
     __syncthreads();
 
     if (warp == PROD_WARP) {
@@ -515,6 +517,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             }
             // hand the segment over to the epilogue warp
             sh->tmax[pb][tid] = a.tmo;
+            atomicMax(&sh->gmax[pb][(warp & 1) * 32 + lane], a.tmo);
             {
                 float c = a.ref, s = a.s;
 #pragma unroll
@@ -608,21 +611,26 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     }
                 }
                 VP_T(1);
-                // (c) T = the K-th largest per-thread maximum, truncated to its top 16 bits: a lower bound of
+                // (c) T = the K-th largest group maximum, truncated to its top 16 bits: a lower bound of
                 //     the K-th largest element of the segment's body (0 when fewer than K threads saw data)
                 uint32_t Tv = 0;
                 {
-                    uint32_t mine[NT / 32];
+                    // over 64 group maxima rather than the 512 thread maxima: any partition of the elements into
+                    // at least K groups gives a lower bound, and this one costs an eighth of the compares for about
+                    // a third more candidates (groups = (lane, warp parity), so that a segment that only reaches
+                    // two streaming warps still fills all of them)
+                    uint32_t mine[kVpGroups / 32];
 #pragma unroll
-                    for (int i = 0; i < NT / 32; ++i) {
-                        mine[i] = sh->tmax[pb][i * 32 + lane];
+                    for (int i = 0; i < kVpGroups / 32; ++i) {
+                        mine[i] = sh->gmax[pb][i * 32 + lane];
+                        sh->gmax[pb][i * 32 + lane] = 0u;  // idle again (published by the `done` arrival below)
                         vmo = mine[i] > vmo ? mine[i] : vmo;
                     }
                     for (int bit = 30; bit >= 16; bit -= 2) {  // two bits per step: three independent counts
                         const uint32_t t1 = Tv | (1u << bit), t2 = Tv | (2u << bit), t3 = Tv | (3u << bit);
                         int c1 = 0, c2 = 0, c3 = 0;
 #pragma unroll
-                        for (int i = 0; i < NT / 32; ++i) {
+                        for (int i = 0; i < kVpGroups / 32; ++i) {
                             c1 += (mine[i] >= t1) ? 1 : 0;
                             c2 += (mine[i] >= t2) ? 1 : 0;
                             c3 += (mine[i] >= t3) ? 1 : 0;
@@ -739,6 +747,14 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             epi_bar(grp);
             if (ew != 0) continue;
             VP_T(5);
+#ifdef GRAFT_VP_PROF
+            if (blockIdx.x == 1 && lane == 0) {
+                atomicAdd(p.errflag + 10, ncand);
+                atomicAdd(p.errflag + 11, es->nhits);
+                atomicAdd(p.errflag + 12, 1);
+                atomicAdd(p.errflag + 13, es->nht);
+            }
+#endif
             // the double-buffered arrays of parity pb may be reused from here on
             __syncwarp();
             if (lane == 0) mbar_arrive(done0 + 8 * pb);
