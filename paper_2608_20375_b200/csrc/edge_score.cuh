@@ -10,30 +10,34 @@
 
 namespace graft {
 
-// K x K dot products by 8 warps.  Warp ty takes parents ty, ty+8, ty+16, ty+24; lane = (ks, tx): children tx,
-// tx+8, tx+16, tx+24 and every fourth float4 of the m axis starting at ks.  A lane keeps a 4 x 4 tile of running
-// sums (16 FMAs per pair of 16-byte loads); the four ks of a tile are then added by two butterfly steps, in a fixed
-// order.  rP / rC: [.][ld] rows in shared memory, ld = m + 4 floats (16-byte aligned, conflict-free float4 reads).
+// K x K dot products by 8 warps.  Warp ty takes parents ty, ty+8, ty+16, ty+24; lane = (ks, tx): children tx and
+// tx+16, and every second float4 of the m axis starting at ks.  A lane keeps a 4 x 2 tile of running sums, each as
+// a packed fp32 pair (even and odd elements of the m axis; `fma.rn.f32x2`, so 16 packed FMAs per six 16-byte
+// loads); the pair is added at the end and the two ks of a tile by one butterfly step, in a fixed order.
+// rP / rC: [.][ld] rows in shared memory, ld = m + 4 floats (16-byte aligned, conflict-free float4 reads).
 // ADD_U: the rows hold P and C and u is added on the way into the registers; otherwise they already hold P + u and
 // C + u (the same fp32 sums either way).  part: [K][K] floats of shared memory; rows >= n_par are not written.
 template <bool ADD_U>
 __device__ __forceinline__ void edge_dots(const float* rP, const float* rC, const float* rU, int m, int K, int n_par,
                                           float* part, int ty, int lane) {
     if (ty >= n_par) return;
-    const int tx = lane & 7, ks = lane >> 3, q4 = m / 4, ld = m + 4;
-    float acc[4][4];
+    const int tx = lane & 15, ks = lane >> 4, q4 = m / 4, ld = m + 4;
+    float2 acc[4][2];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int i2 = 0; i2 < 4; ++i2) acc[i][i2] = 0.f;
-    for (int k4 = ks; k4 < q4; k4 += 4) {
+        for (int i2 = 0; i2 < 2; ++i2) acc[i][i2] = make_float2(0.f, 0.f);
+    const float* c0 = rC + (size_t)min(tx, K - 1) * ld;  // (rows past K: read, never used)
+    const float* c1 = rC + (size_t)min(tx + 16, K - 1) * ld;
+    for (int k4 = ks; k4 < q4; k4 += 2) {
         float4 uu = make_float4(0.f, 0.f, 0.f, 0.f);
         if (ADD_U) uu = *(const float4*)(rU + 4 * k4);
-        float4 cv[4];
+        float4 cv[2];
+        cv[0] = *(const float4*)(c0 + 4 * k4);
+        cv[1] = *(const float4*)(c1 + 4 * k4);
+        if (ADD_U) {
 #pragma unroll
-        for (int i2 = 0; i2 < 4; ++i2) {
-            cv[i2] = *(const float4*)(rC + (size_t)min(tx + 8 * i2, K - 1) * ld + 4 * k4);  // (rows past K: unused)
-            if (ADD_U) {
+            for (int i2 = 0; i2 < 2; ++i2) {
                 cv[i2].x += uu.x;
                 cv[i2].y += uu.y;
                 cv[i2].z += uu.z;
@@ -50,31 +54,26 @@ __device__ __forceinline__ void edge_dots(const float* rP, const float* rC, cons
                 pv.w += uu.w;
             }
 #pragma unroll
-            for (int i2 = 0; i2 < 4; ++i2) {
-                float a = acc[i][i2];
-                a = fmaf(pv.x, cv[i2].x, a);
-                a = fmaf(pv.y, cv[i2].y, a);
-                a = fmaf(pv.z, cv[i2].z, a);
-                a = fmaf(pv.w, cv[i2].w, a);
+            for (int i2 = 0; i2 < 2; ++i2) {
+                float2 a = acc[i][i2];
+                a = __ffma2_rn(make_float2(pv.x, pv.y), make_float2(cv[i2].x, cv[i2].y), a);
+                a = __ffma2_rn(make_float2(pv.z, pv.w), make_float2(cv[i2].z, cv[i2].w), a);
                 acc[i][i2] = a;
             }
         }
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int i2 = 0; i2 < 4; ++i2) {
-            float a = acc[i][i2];
-            a += __shfl_xor_sync(0xFFFFFFFFu, a, 8);
-            a += __shfl_xor_sync(0xFFFFFFFFu, a, 16);
-            acc[i][i2] = a;
-        }
-#pragma unroll
     for (int i = 0; i < 4; ++i) {
-        if (ks == i && ty + 8 * i < n_par) {
+        float v[2];
 #pragma unroll
-            for (int i2 = 0; i2 < 4; ++i2)
-                if (tx + 8 * i2 < K) part[(size_t)(ty + 8 * i) * K + tx + 8 * i2] = acc[i][i2];
+        for (int i2 = 0; i2 < 2; ++i2) {
+            float a = acc[i][i2].x + acc[i][i2].y;
+            a += __shfl_xor_sync(0xFFFFFFFFu, a, 16);
+            v[i2] = a;
+        }
+        if (ks == (i & 1) && ty + 8 * i < n_par) {
+            if (tx < K) part[(size_t)(ty + 8 * i) * K + tx] = v[0];
+            if (tx + 16 < K) part[(size_t)(ty + 8 * i) * K + tx + 16] = v[1];
         }
     }
 }
