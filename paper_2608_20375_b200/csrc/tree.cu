@@ -191,31 +191,37 @@ __device__ __forceinline__ bool entry_before(const TreeSmem& sm, uint64_t e1, in
 }
 
 // B-th largest of keys[lo..hi) (hi - lo >= kth >= 1) by an 8-bit radix select; every thread of the CTA calls it.
-// With passes < 4 only the top 8 * passes bits are resolved and the rest is returned as zero: a lower bound
-// of the B-th largest key.  The 256 bins exist in four copies (neighbouring warps use different ones) and in two
-// generations, so that the next pass's bins are cleared while this pass's are scanned.
-__device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, int lo, int hi, int kth, int passes,
-                                    int tid) {
+// Passes [pass0, pass1) of four are run: with pass1 < 4 only the top 8 * pass1 bits are resolved and the rest is
+// returned as zero, a lower bound of the B-th largest key; a later call on the same keys can take up the search
+// where this one stopped (pass0 = the earlier pass1, prefix and remaining as returned).  The 256 bins exist in four
+// copies (neighbouring warps use different ones) and in two generations, so that the next pass's bins are cleared
+// while this pass's are scanned.
+__device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, int lo, int hi, int kth, int pass0,
+                                    int pass1, uint32_t prefix, int& remaining, int tid) {
     const int warp = tid >> 5, lane = tid & 31;
-    uint32_t prefix = 0, mask = 0;
-    int remaining = kth;
-    sm.hist[tid] = 0u;
+    uint32_t mask = pass0 == 0 ? 0u : 0xFFFFFFFFu << (32 - 8 * pass0);
+    if (pass0 == 0) {
+        prefix = 0u;
+        remaining = kth;
+    }
+    sm.hist[(pass0 & 1) * 1024 + tid] = 0u;
     __syncthreads();
-    for (int pass = 0; pass < passes; ++pass) {
+    for (int pass = pass0; pass < pass1; ++pass) {
         const int shift = 24 - 8 * pass;
-        uint32_t* h = sm.hist + (pass & 1) * 1024;
+        uint32_t* h = sm.hist + (pass & 1) * 1024 + (warp & 3) * 256;
         for (int i = lo + tid; i < hi; i += TREE_THREADS) {
             const uint32_t k = keys[i];
-            if ((k & mask) == prefix) atomicAdd(&h[(warp & 3) * 256 + ((k >> shift) & 255u)], 1u);
+            if ((k & mask) == prefix) atomicAdd(&h[(k >> shift) & 255u], 1u);
         }
         sm.hist[((pass + 1) & 1) * 1024 + tid] = 0u;  // the other generation, for the next pass
         __syncthreads();
         if (warp == 0) {  // lane l owns bins 255-8l .. 248-8l, from the top down
+            const uint32_t* hh = sm.hist + (pass & 1) * 1024;
             int c[8], sum = 0;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const int bin = 255 - 8 * lane - j;
-                c[j] = (int)(h[bin] + h[256 + bin] + h[512 + bin] + h[768 + bin]);
+                c[j] = (int)(hh[bin] + hh[256 + bin] + hh[512 + bin] + hh[768 + bin]);
                 sum += c[j];
             }
             int incl = sum;
@@ -246,7 +252,6 @@ __device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, in
     }
     return prefix;
 }
-
 
 // ---- edge scores on demand --------------------------------------------------------------------------------------
 // Row j of the edge scores (children at depth j+1), Eq. 4-6: the table rows P[parent token], C[child token] and
@@ -489,7 +494,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     bool table_ok = budget > 0;
     uint32_t theta = 0u;
     if (budget > 0) {
-        int ntot = 1, n_at_select = 1;
+        int ntot = 1, n_at_select = 1, sel_rem = 0;
         for (int d = 0; d < L; ++d) {
 #ifdef GRAFT_TREE_PROF
             long long tl0 = clock64();
@@ -520,36 +525,112 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     if (tid == 0) sm.scal[3] = ntot + total;
                 }
             } else {
-                // one thread per node: the children that can still matter are a prefix of the node's sorted row
-                // (scores only fall along the row); its length comes from a binary search, one atomic reserves the
-                // slots, and the writes are independent of each other
-                for (int x = b0 + tid; x < b1; x += TREE_THREADS) {
-                    const uint32_t kx = sm.nkey[x];
-                    if (kx < theta) continue;  // dead: none of its descendants can be selected
-                    const int row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
-                    const float sx = sm.nS[x];
-                    int lo_r = 0, hi_r = K;  // first r in [0, K] whose key falls below theta
-                    while (lo_r < hi_r) {
-                        const int mid = (lo_r + hi_r) >> 1;
-                        const uint32_t oc = ord_from_float(sx + sm.es[row + mid]);
-                        if ((oc < kx ? oc : kx) >= theta)
-                            lo_r = mid + 1;
-                        else
-                            hi_r = mid;
+                // The children that can still matter are a prefix of a node's sorted row (scores only fall along the
+                // row); its length comes from a binary search.  Full chunks of 1024 nodes (the dense early levels):
+                // one thread per node finds the length, a scan of the lengths places the chunk's children in the
+                // table, then one thread per child (found in the scan by binary search) writes it, so that neither a
+                // shared counter nor a node with many children holds the others up.  The remaining nodes (sparse
+                // levels): one thread per node reserves its slots with an atomic and writes its children itself.
+                int cur = ntot, c_tail = b0;
+                bool chunk_ovf = false;
+                for (; b1 - c_tail >= TREE_THREADS; c_tail += TREE_THREADS) {  // (uniform)
+                    const int c0 = c_tail, x = c0 + tid;
+                    int cnt = 0;
+                    {
+                        const uint32_t kx = sm.nkey[x];
+                        if (kx >= theta) {  // (else dead: none of its descendants can be selected)
+                            const int row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
+                            const float sx = sm.nS[x];
+                            int lo_r = 0, hi_r = K;  // first r in [0, K] whose key falls below theta
+                            while (lo_r < hi_r) {
+                                const int mid = (lo_r + hi_r) >> 1;
+                                const uint32_t oc = ord_from_float(sx + sm.es[row + mid]);
+                                if ((oc < kx ? oc : kx) >= theta)
+                                    lo_r = mid + 1;
+                                else
+                                    hi_r = mid;
+                            }
+                            cnt = lo_r;
+                        }
                     }
-                    const int cnt = lo_r;
-                    if (cnt == 0) continue;
-                    const int base = atomicAdd(&sm.scal[3], cnt);
-                    if (base + cnt > p.ncap) {
-                        sm.scal[4] = 1;
-                        continue;
+                    int incl = cnt;
+#pragma unroll
+                    for (int o2 = 1; o2 < 32; o2 <<= 1) {
+                        const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
+                        if (lane >= o2) incl += t;
                     }
-                    for (int r = 0; r < cnt; ++r) {
-                        const float sc = sx + sm.es[row + r];
+                    int* pre = (int*)sm.hist;  // [1024] inclusive scan of the chunk, then [32] warp totals
+                    if (lane == 31) pre[TREE_THREADS + warp] = incl;
+                    __syncthreads();
+                    const int wt = pre[TREE_THREADS + lane];
+                    int wincl = wt;
+#pragma unroll
+                    for (int o2 = 1; o2 < 32; o2 <<= 1) {
+                        const int t = __shfl_up_sync(0xFFFFFFFFu, wincl, o2);
+                        if (lane >= o2) wincl += t;
+                    }
+                    const int total = __shfl_sync(0xFFFFFFFFu, wincl, 31);
+                    pre[tid] = __shfl_sync(0xFFFFFFFFu, wincl - wt, warp) + incl;
+                    __syncthreads();
+                    if (cur + total > p.ncap) {  // (uniform)
+                        if (tid == 0) sm.scal[4] = 1;
+                        chunk_ovf = true;
+                        break;
+                    }
+                    for (int i = tid; i < total; i += TREE_THREADS) {
+                        int lo_t = 0, hi_t = TREE_THREADS - 1;  // owner: the first thread whose scan exceeds i
+                        while (lo_t < hi_t) {
+                            const int mid = (lo_t + hi_t) >> 1;
+                            if (pre[mid] > i)
+                                hi_t = mid;
+                            else
+                                lo_t = mid + 1;
+                        }
+                        const int r = i - (lo_t ? pre[lo_t - 1] : 0), xo = c0 + lo_t;
+                        const uint32_t kx = sm.nkey[xo];
+                        const int row = (d * K + (int)((sm.ninfo[xo] >> 13) & 31u)) * K;
+                        const float sc = sm.nS[xo] + sm.es[row + r];
                         const uint32_t oc = ord_from_float(sc);
-                        sm.nkey[base + r] = oc < kx ? oc : kx;
-                        sm.nS[base + r] = sc;
-                        sm.ninfo[base + r] = (uint32_t)x | ((uint32_t)sm.ei[row + r] << 13) | ((uint32_t)(d + 1) << 18);
+                        sm.nkey[cur + i] = oc < kx ? oc : kx;
+                        sm.nS[cur + i] = sc;
+                        sm.ninfo[cur + i] = (uint32_t)xo | ((uint32_t)sm.ei[row + r] << 13) | ((uint32_t)(d + 1) << 18);
+                    }
+                    cur += total;
+                    __syncthreads();  // the scan space is reused by the next chunk
+                }
+                if (c_tail > b0) {  // the counter takes over from here
+                    if (tid == 0) sm.scal[3] = cur;
+                    __syncthreads();
+                }
+                if (!chunk_ovf) {
+                    for (int x = c_tail + tid; x < b1; x += TREE_THREADS) {
+                        const uint32_t kx = sm.nkey[x];
+                        if (kx < theta) continue;  // dead: none of its descendants can be selected
+                        const int row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
+                        const float sx = sm.nS[x];
+                        int lo_r = 0, hi_r = K;  // first r in [0, K] whose key falls below theta
+                        while (lo_r < hi_r) {
+                            const int mid = (lo_r + hi_r) >> 1;
+                            const uint32_t oc = ord_from_float(sx + sm.es[row + mid]);
+                            if ((oc < kx ? oc : kx) >= theta)
+                                lo_r = mid + 1;
+                            else
+                                hi_r = mid;
+                        }
+                        const int cnt = lo_r;
+                        if (cnt == 0) continue;
+                        const int base = atomicAdd(&sm.scal[3], cnt);
+                        if (base + cnt > p.ncap) {
+                            sm.scal[4] = 1;
+                            continue;
+                        }
+                        for (int r = 0; r < cnt; ++r) {
+                            const float sc = sx + sm.es[row + r];
+                            const uint32_t oc = ord_from_float(sc);
+                            sm.nkey[base + r] = oc < kx ? oc : kx;
+                            sm.nS[base + r] = sc;
+                            sm.ninfo[base + r] = (uint32_t)x | ((uint32_t)sm.ei[row + r] << 13) | ((uint32_t)(d + 1) << 18);
+                        }
                     }
                 }
             }
@@ -568,7 +649,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             // theta only has to be a lower bound of its final value while the levels are built (it prunes), so
             // the exact B-th largest key is recomputed only when the table has grown noticeably
             if (ntot - 1 >= budget && (theta == 0u || ntot - n_at_select >= ntot / 2)) {
-                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 2, tid);  // a 16-bit lower bound is enough here
+                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 0, 2, 0u, sel_rem, tid);  // a 16-bit lower bound
                 n_at_select = ntot;
             }
             __syncthreads();
@@ -583,7 +664,13 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
 #endif
         }
         __syncthreads();
-        if (table_ok && ntot - 1 >= budget) theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 4, tid);  // exact
+        if (table_ok && ntot - 1 >= budget) {
+            // the exact value: the last 16-bit search still holds if nothing was appended after it
+            if (n_at_select == ntot && theta != 0u)
+                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 2, 4, theta, sel_rem, tid);
+            else
+                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 0, 4, 0u, sel_rem, tid);
+        }
         __syncthreads();
         if (table_ok) {
             // compact {key > theta} in table order (parents stay before their children)
