@@ -58,7 +58,7 @@ struct TreeSmem {
     uint8_t* depth;      // [nmax]
     // emission scratch, laid over the node table (dead by then)
     int16_t* lvl_list;   // [nmax]
-    int* cc;             // [nmax]   per-level child counts in level order, then their exclusive scan
+    int16_t* cc;         // [2][nmax] per-level child counts in level order, then their exclusive scan (two levels)
     uint32_t* stage;     // [8 warps * 32 rows * W] mask rows staged for coalesced stores
     uint32_t* hist;      // [2 * 4 * 256]
     int* lvl_count;      // [kMaxL + 2]
@@ -106,7 +106,7 @@ __host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, int n
         s->nS = (float*)(base + o_tab + (size_t)ncap * 4);
         s->ninfo = (uint32_t*)(base + o_tab + (size_t)ncap * 8);
         s->lvl_list = (int16_t*)(base + o_tab);
-        s->cc = (int*)(base + o_tab + (((size_t)nmax * 2 + 15) & ~(size_t)15));
+        s->cc = (int16_t*)(base + o_tab + (((size_t)nmax * 2 + 15) & ~(size_t)15));
         s->stage = (uint32_t*)(base + o_tab + (((size_t)nmax * 2 + 15) & ~(size_t)15) + (((size_t)nmax * 4 + 15) & ~(size_t)15));
         s->ent = (uint64_t*)(base + o_ent);
         s->S = (float*)(base + o_S);
@@ -673,6 +673,10 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         }
         __syncthreads();
         if (table_ok) {
+#ifdef GRAFT_TREE_PROF
+            __syncthreads();
+            if (tid == 0 && o.d_edge) o.d_edge[(size_t)b * L * K * K + 100 + 0] = (float)(clock64() - t_prof0);
+#endif
             // compact {key > theta} in table order (parents stay before their children)
             const int per = (ntot + TREE_THREADS - 1) / TREE_THREADS;
             const int i0 = tid * per < ntot ? tid * per : ntot, i1 = i0 + per < ntot ? i0 + per : ntot;
@@ -709,6 +713,10 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             }
             n_gt = total - 1;
             __syncthreads();
+#ifdef GRAFT_TREE_PROF
+            __syncthreads();
+            if (tid == 0 && o.d_edge) o.d_edge[(size_t)b * L * K * K + 100 + 1] = (float)(clock64() - t_prof0);
+#endif
             // frontier entries of the selected nodes: the first child of the sorted row that is not selected,
             // i.e. the first with ord(score) <= theta
             for (int n = tid; n <= n_gt; n += TREE_THREADS) {
@@ -717,8 +725,14 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 if (d < L) {
                     const int row = (d * K + sm.cand[n]) * K;
                     const float sn = sm.S[n];
-                    int pos = 0;
-                    while (pos < K && ord_from_float(sn + sm.es[row + pos]) > theta) ++pos;
+                    int pos = 0, hi_p = K;  // first entry of the (ordered) row whose key is not above theta
+                    while (pos < hi_p) {
+                        const int mid = (pos + hi_p) >> 1;
+                        if (ord_from_float(sn + sm.es[row + mid]) > theta)
+                            pos = mid + 1;
+                        else
+                            hi_p = mid;
+                    }
                     if (pos < K) e = pack_entry(sn + sm.es[row + pos], d + 1, pos, sm.cand[n], sm.ei[row + pos]);
                 }
                 sm.ent[n] = e;
@@ -831,20 +845,21 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         sm.lvl_list[sm.lvl_start[d] + atomicAdd(&sm.lvl_fill[d], 1)] = (int16_t)n;
     }
     __syncthreads();
+    // cc holds the child counts of the previous level in level order; it is double-buffered (two halves of nmax
+    // entries) so that a level's nodes can leave their own counts for the next level as soon as they know their place
+    if (tid == 0) sm.cc[0] = __popc(sm.chmask[0]);
+    __syncthreads();
     for (int d = 1; d <= L; ++d) {
         const int s_prev = sm.lvl_start[d - 1], n_prev = sm.lvl_count[d - 1];
         const int s_cur = sm.lvl_start[d], n_cur = sm.lvl_count[d];
         if (n_cur == 0) break;  // uniform: deeper levels are empty too
-        for (int i = tid; i < n_prev; i += TREE_THREADS) {
-            const int y = sm.lvl_list[s_prev + i];
-            sm.cc[sm.canon[y] - s_prev] = __popc(sm.chmask[y]);
-        }
-        __syncthreads();
-        if (warp == 0) {  // exclusive scan of cc[0..n_prev): a contiguous chunk per lane, then a warp scan
+        int16_t* ccp = sm.cc + ((d - 1) & 1) * nmax;
+        int16_t* ccn = sm.cc + (d & 1) * nmax;
+        if (warp == 0) {  // exclusive scan of ccp[0..n_prev): a contiguous chunk per lane, then a warp scan
             const int ch = (n_prev + 31) / 32;
             const int lo_i = lane * ch, hi_i = min(n_prev, lo_i + ch);
             int sum = 0;
-            for (int i = lo_i; i < hi_i; ++i) sum += sm.cc[i];
+            for (int i = lo_i; i < hi_i; ++i) sum += ccp[i];
             int incl = sum;
 #pragma unroll
             for (int o2 = 1; o2 < 32; o2 <<= 1) {
@@ -853,8 +868,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             }
             int run = incl - sum;
             for (int i = lo_i; i < hi_i; ++i) {
-                const int v = sm.cc[i];
-                sm.cc[i] = run;
+                const int v = ccp[i];
+                ccp[i] = (int16_t)run;
                 run += v;
             }
         }
@@ -862,11 +877,16 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         for (int i = tid; i < n_cur; i += TREE_THREADS) {
             const int x = sm.lvl_list[s_cur + i];
             const int y = sm.parent[x];
-            sm.canon[x] = (int16_t)(s_cur + sm.cc[sm.canon[y] - s_prev] +
-                                    __popc(sm.chmask[y] & ((1u << sm.cand[x]) - 1u)));
+            const int at = s_cur + ccp[sm.canon[y] - s_prev] + __popc(sm.chmask[y] & ((1u << sm.cand[x]) - 1u));
+            sm.canon[x] = (int16_t)at;
+            ccn[at - s_cur] = (int16_t)__popc(sm.chmask[x]);
         }
         __syncthreads();
     }
+#ifdef GRAFT_TREE_PROF
+    __syncthreads();
+    if (tid == 0 && o.d_edge) o.d_edge[(size_t)b * L * K * K + 100 + 2] = (float)(clock64() - t_prof0);
+#endif
     const int prefix = p.prefix_len[b];
     const size_t ob = (size_t)b * nmax;
     for (int n = tid; n < n_nodes; n += TREE_THREADS) {
@@ -887,6 +907,10 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         o.d_path_score[ob + i] = 0.f;
     }
     __syncthreads();
+#ifdef GRAFT_TREE_PROF
+    __syncthreads();
+    if (tid == 0 && o.d_edge) o.d_edge[(size_t)b * L * K * K + 100 + 3] = (float)(clock64() - t_prof0);
+#endif
     // ancestor masks: each thread builds one row in its warp's staging tile (walking up, level-order indices
     // only decrease, so the row is produced from its highest word down); the warp then stores its 32 rows,
     // which are contiguous in the output, with coalesced writes.  Padding rows are zero-filled directly.
