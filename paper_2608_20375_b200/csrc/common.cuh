@@ -76,6 +76,28 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// The same with a suspend-time hint (ns): the thread may sleep that long in hardware before it polls again, which
+// keeps the polls of a warp that has nothing else to do out of the issue slots of the warps beside it.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded_hint(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    for (uint32_t it = 0; it < GRAFT_SPIN_LIMIT; ++it) {
+        if (mbar_try_wait_hint(bar, parity, ns)) return true;
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
 // Bounded wait.  Returns false (and raises *abort_flag) when the limit is hit or another thread already
 // gave up; callers then carry on without waiting so that every thread still reaches the kernel's end.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag) {

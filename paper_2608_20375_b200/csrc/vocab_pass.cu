@@ -48,6 +48,7 @@ constexpr int WBLK = TILE / NW;               // bytes of a tile owned by one wa
 static_assert(WBLK == 2048, "one warp owns 2 KiB of every tile");
 constexpr int VEC_PER_LANE = WBLK / 16 / 32;  // 4
 static_assert(VEC_PER_LANE == 4, "chunk layout assumes four 16-byte vectors per lane per tile");
+constexpr uint32_t kVpIdleHintNs = 10000;  // suspend hint of the waits of the producer and epilogue warps
 constexpr int COS_WARP = PROD_WARP + 1;  // warp that computes the SABA cosines beside the stream
 static_assert(kVpThreads == NT + kVpEpiGroups * kVpEpiThreads + 64,
               "thread count = streaming warps + epilogue warps + producer warp + cosine warp");
@@ -453,7 +454,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             Seg sg;
             while (seg_iter_next<BF16>(p, it, sg)) {
                 for (int tile = 0; tile < sg.ntiles && p.dbg != 2; ++tile, ++t) {
-                    if (t >= nst) mbar_wait_bounded(empty0 + 8 * st, ph, &sh->abort_flag);
+                    if (t >= nst) mbar_wait_bounded_hint(empty0 + 8 * st, ph, &sh->abort_flag, kVpIdleHintNs);
                     uint32_t off = (uint32_t)tile * TILE;
                     uint32_t bytes = sg.body_bytes - off < (uint32_t)TILE ? sg.body_bytes - off : (uint32_t)TILE;
                     mbar_arrive_expect_tx(full0 + 8 * st, bytes);
@@ -496,7 +497,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 const int nfull = (int)(sg.body_bytes / TILE);
                 cm_t* slot = cmax + (size_t)pb * p.n_cmax + (size_t)tid * p.max_tiles;  // this thread's slots, by tile
                 for (int tile = 0; tile < sg.ntiles; ++tile, ++slot) {
-                    if (p.dbg != 2) mbar_wait_bounded(full0 + 8 * st, ph, &sh->abort_flag);
+                    if (p.dbg != 2) mbar_wait_bounded_hint(full0 + 8 * st, ph, &sh->abort_flag, 2000u);
                     const uint4* wb = (const uint4*)(ring + (size_t)st * TILE + (size_t)warp * WBLK);
                     if (p.dbg == 1) {
                         *slot = 0;
@@ -569,7 +570,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
 #ifdef GRAFT_VP_PROF
             long long tprof = clock64();
 #endif
-            if (ew == 0) mbar_wait_bounded(ready0 + 8 * pb, (k / kVpBufs) & 1u, &sh->abort_flag);
+            if (ew == 0) mbar_wait_bounded_hint(ready0 + 8 * pb, (k / kVpBufs) & 1u, &sh->abort_flag, kVpIdleHintNs);
             if (p.dbg) {
                 __syncwarp();
                 if (ew == 0 && lane == 0) mbar_arrive(done0 + 8 * pb);
