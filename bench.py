@@ -209,6 +209,16 @@ def run_graft(args):
     launches = g.launch_count() - launches0
     ms_total = ev0.elapsed_time(ev1)
     n_t, vocab_ms, tdes_ms, tree_ms = g.read_timing()
+    # what two event records cost the stream with nothing between them (the per-kernel figures above are intervals
+    # between such records, so each holds one of these; reported beside them, not subtracted from `frac`)
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(64)]
+    step(0)
+    for a, b_ in pairs:
+        a.record()
+        b_.record()
+        step(0)
+    torch.cuda.synchronize()
+    event_pair_ms = float(np.median([a.elapsed_time(b_) for a, b_ in pairs]))
     if world > 1:
         import torch.distributed as dist
         t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
@@ -279,10 +289,11 @@ def run_graft(args):
                    "l2_policy": f"{n_buf} rotating input sets of {logits_bytes / 1e6:.0f} MB each (> L2 of 126 MB)"},
         "gpu_launches": launches,
         "kernel_ms": {"vocab_pass": vocab_ms / max(1, n_t), "tdes_edges": tdes_ms / max(1, n_t),
-                      "tree": tree_ms / max(1, n_t), "calls_averaged": n_t},
+                      "tree": tree_ms / max(1, n_t), "calls_averaged": n_t, "empty_event_pair": event_pair_ms},
         "roofline": {"bound": "hbm", "kernel": "vocab_pass_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8000": achieved / 8000.0, "algorithmic_bytes": algo_bytes,
+                     "frac_net_of_event_pair": algo_bytes / max(1e-9, vocab_s - event_pair_ms * 1e-3) / 1e9 / peak,
                      "traffic": NCU_VOCAB_TRAFFIC_BYTES_M if w.name == "M" else None},
         "e2e": {"value": world * batch / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3, "steps": e2e_steps,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
