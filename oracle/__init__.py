@@ -200,6 +200,14 @@ def accept(n_nodes, token, parent, target_next, L):
     return a.value, path, bonus.value
 
 
+def hist_update(a_hist, w):
+    """hist for the next round from all accepted lengths so far, oldest first (Eq. 15)."""
+    a = np.ascontiguousarray(a_hist, dtype=np.int32)
+    f = lib().oracle_hist_update
+    f.restype = C.c_double
+    return float(f(_p(a), int(a.size), int(w)))
+
+
 def replay_check(edge, n_nodes, parent, cand, depth, eps):
     """Is the given node set a valid best-first outcome on the oracle's edge scores up to eps?"""
     edge = np.ascontiguousarray(edge, dtype=np.float32)

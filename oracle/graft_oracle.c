@@ -17,6 +17,7 @@
  *   O4  oracle_select         best-first expansion until B_t nodes         (Preliminaries "DDTree"; Sec. 3.1; Eq. 13)
  *   O5  oracle_emit           level-order tree, positions, ancestor mask   (Preliminaries "Tree-based speculative decoding")
  *   O6  oracle_accept         longest accepted path                        (Preliminaries, a_t)
+ *   O7  oracle_hist_update    hist_t over the last w accepted lengths      (Sec. 3.3, Eq. 15)
  *   --  oracle_replay_check   is a given node set a valid best-first outcome up to eps?
  *
  * Pins: every function here is pinned by tests that do not call it to produce their own
@@ -433,6 +434,22 @@ int oracle_accept(int n_nodes, const int32_t *token, const int32_t *parent, cons
     *accept_len = a;
     *bonus = target_next[cur];
     return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * O7.  Acceptance history (Eq. 15): hist_t = (1/w) sum_{i=1..w} a_{t-i}.  `a_hist` holds every
+ * accepted length so far, oldest first (n_rounds of them); the result is hist for the next round.
+ * Reading for the first rounds, where fewer than w lengths exist (the paper does not say): the
+ * mean of those that exist, and 0 before the first round.
+ * Pins: a constant history gives that constant; a step change crosses over in exactly w rounds;
+ * the definition recomputed with a library mean over the last w entries.
+ * ------------------------------------------------------------------------------------------ */
+double oracle_hist_update(const int32_t *a_hist, int n_rounds, int w) {
+    if (n_rounds <= 0 || w <= 0) return 0.0;
+    const int m = n_rounds < w ? n_rounds : w;
+    double s = 0.0;
+    for (int i = 1; i <= m; ++i) s += (double)a_hist[n_rounds - i];
+    return s / (double)m;
 }
 
 /* ------------------------------------------------------------------------------------------

@@ -525,3 +525,30 @@ def test_build_trees_bad_row_gives_root_only_tree():
     o = oracle.build_trees(x["logits"], None, x["root_token"], None, x["prefix_len"], x["fixed_budget"].numpy(),
                            oracle.SabaParams(), (8, 8, 8), tb["P"], tb["C"], tb["u"], 1.0, 0.2, w.K)
     assert o["status"].tolist() == [0, 1] and o["n_nodes"].tolist() == [9, 1]
+
+
+# --------------------------------------------------------------------------- O7 acceptance history (Eq. 15)
+def test_hist_constant_history_and_empty_history():
+    assert oracle.hist_update([], 4) == 0.0
+    for w in (1, 3, 8):
+        for n in (1, 2, 8, 20):
+            assert oracle.hist_update([5] * n, w) == 5.0
+
+
+def test_hist_step_change_crosses_over_in_w_rounds():
+    w = 4
+    a = [2] * 10
+    vals = []
+    for t in range(1, 7):
+        a.append(6)
+        vals.append(oracle.hist_update(a, w))
+    assert vals == [3.0, 4.0, 5.0, 6.0, 6.0, 6.0]  # one more new entry in the window each round, then saturated
+
+
+def test_hist_is_the_mean_of_the_last_w_entries():
+    rng = np.random.default_rng(15)
+    a = rng.integers(0, 17, size=40).astype(np.int32)
+    for w in (1, 5, 8, 64):
+        for n in (1, 3, 8, 40):
+            want = float(np.mean(a[:n][-w:].astype(np.float64)))
+            assert abs(oracle.hist_update(a[:n], w) - want) < 1e-12
