@@ -181,6 +181,25 @@ def run_graft(args):
     for i in range(args.warmup):
         step(i)
     torch.cuda.synchronize()
+    if args.cuda_graph:
+        # one captured round per input set, replayed in the timed loop (the per-kernel events then come from eager
+        # rounds: event records are not captured)
+        eager_step = step
+        side = torch.cuda.Stream()
+        graphs = []
+        for k in range(n_buf):
+            side.wait_stream(torch.cuda.current_stream())
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr, stream=side):
+                eager_step(k)
+            graphs.append(gr)
+        torch.cuda.synchronize()
+
+        def step(i, timed=False):  # noqa: F811
+            if timed:
+                eager_step(i)
+            else:
+                graphs[i % n_buf].replay()
 
     def barrier():
         if world > 1:
@@ -199,7 +218,10 @@ def run_graft(args):
         timed = (i % args.timing_every) == 0
         if timed:
             g.set_timing(1 if i == 0 else 2)  # 1 = reset the call count, 2 = go on counting
-        step(i)
+        if args.cuda_graph:
+            step(i, timed)
+        else:
+            step(i)
         if timed:
             g.set_timing(False)
     ev1.record()
@@ -384,6 +406,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--timing-every", type=int, default=8,
                     help="record the per-kernel events on every n-th timed step")
+    ap.add_argument("--cuda-graph", action="store_true", help="replay captured rounds in the timed loop")
     ap.add_argument("--edge-rows", type=int, default=None,
                     help="depths scored ahead of the expansion (default: the library's)")
     args = ap.parse_args()

@@ -186,6 +186,15 @@ graft_status graft_vocab_pass_static(int32_t batch, int32_t L, int32_t V, int32_
 graft_status graft_accept(graft_ctx* ctx, int32_t batch, const graft_tree_out* trees, const int32_t* d_target_next,
                           int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus_token, void* stream);
 
+/* Acceptance history on the device (Eq. 15: hist_t = mean of the last w accepted lengths), so that a decoding loop
+ * needs no host round trip between graft_accept and the next graft_build_trees.  After this call every
+ * graft_accept also appends a_t of sequence b to d_window[b] (a ring of w int32, caller-owned, start it zeroed),
+ * advances d_count[b] (int32 rounds seen, start at 0) and writes d_hist[b] = mean of the last min(count, w)
+ * lengths (the paper does not say what hist is before w rounds exist; 0 before the first).  Pass d_hist as the
+ * d_hist argument of the next graft_build_trees.  w in [1, 64]; w = 0 (pointers ignored) switches it off.
+ * Host-only call; the buffers are borrowed until it is called again or the context is destroyed. */
+graft_status graft_set_hist_window(graft_ctx* ctx, int32_t w, int32_t* d_window, int32_t* d_count, float* d_hist);
+
 /* Host-buffer form of graft_build_trees for end-to-end use: every pointer here is a HOST pointer (pinned
  * memory makes the copies asynchronous).  Copies the inputs host->device into context-owned staging buffers
  * (allocated on first use, sized for max_batch), runs the same kernels as graft_build_trees, copies

@@ -21,7 +21,7 @@ ST_BAD_LOGITS, ST_TAU_CLAMPED, ST_FRONTIER_EMPTY, ST_INTERNAL = 1, 2, 4, 8
 ENTRY_POINTS = [
     "graft_create", "graft_destroy", "graft_nmax", "graft_mask_words", "graft_set_saba", "graft_set_tdes_tables",
     "graft_tdes_precompute", "graft_build_trees", "graft_vocab_pass", "graft_vocab_pass_static", "graft_tdes_edges",
-    "graft_accept", "graft_set_edge_rows", "graft_edge_rows",
+    "graft_accept", "graft_set_edge_rows", "graft_edge_rows", "graft_set_hist_window",
     "graft_build_trees_host", "graft_launch_count", "graft_set_timing", "graft_read_timing", "graft_status_str",
     "graft_version",
 ]
@@ -80,6 +80,7 @@ def load_library():
     lib.graft_set_saba.argtypes = [vp, C.POINTER(_Saba)]
     lib.graft_set_tdes_tables.argtypes = [vp, vp, vp, vp, C.c_float, vp]
     lib.graft_set_edge_rows.argtypes = [vp, C.c_int32]
+    lib.graft_set_hist_window.argtypes = [vp, C.c_int32, vp, vp, vp]
     lib.graft_edge_rows.argtypes = [vp]
     lib.graft_edge_rows.restype = C.c_int32
     lib.graft_tdes_precompute.argtypes = [vp, vp, C.c_int, C.c_int32, vp, vp, vp, vp]
@@ -217,6 +218,18 @@ class Graft:
         p = _Saba(phi_conf, phi_degen, phi_hist, phi_bias, tau_min, cost_mode, c0, c1, c2, len(pts_n),
                   C.cast(n, C.POINTER(C.c_float)), C.cast(t, C.POINTER(C.c_float)))
         _check(self.lib, self.lib.graft_set_saba(self._ctx, C.byref(p)), "graft_set_saba")
+
+    def set_hist_window(self, w, window=None, count=None, hist=None):
+        """graft_accept keeps hist_t (Eq. 15) on the device: window [batch, w] int32, count [batch] int32,
+        hist [batch] float32 (pass `hist` to the next build_trees).  w = 0 switches it off."""
+        if w == 0:
+            _check(self.lib, self.lib.graft_set_hist_window(self._ctx, 0, None, None, None), "graft_set_hist_window")
+            self._hist_keep = None
+            return
+        _check(self.lib, self.lib.graft_set_hist_window(self._ctx, int(w), _ptr(window, torch.int32),
+                                                        _ptr(count, torch.int32), _ptr(hist, torch.float32)),
+               "graft_set_hist_window")
+        self._hist_keep = (window, count, hist)  # borrowed by the library
 
     def set_edge_rows(self, rows):
         """Depths [0, rows) are scored ahead of the expansion, deeper ones on demand (graft_set_edge_rows)."""

@@ -152,6 +152,10 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     ctx->w_esort = (float*)(base + o_es);
     ctx->w_eidx = (uint8_t*)(base + o_ei);
     ctx->d_u = (float*)(base + o_u);
+    ctx->hist_w = 0;
+    ctx->hist_window = nullptr;
+    ctx->hist_count = nullptr;
+    ctx->hist_out = nullptr;
     ctx->edge_rows = tree_lazy_fits(*cfg) ? (cfg->L < 8 ? cfg->L : 8) : cfg->L;
     ctx->w_errflag = (int32_t*)(base + o_err);
     ctx->w_cos = (double*)(base + o_cos);
@@ -366,6 +370,16 @@ graft_status graft_accept(graft_ctx* ctx, int32_t batch, const graft_tree_out* t
     if (accept_launch(ctx, batch, trees, d_target_next, d_accept_len, d_accept_path, d_bonus_token,
                       (cudaStream_t)stream) != cudaSuccess)
         return GRAFT_ERR_CUDA;
+    return GRAFT_OK;
+}
+
+graft_status graft_set_hist_window(graft_ctx* ctx, int32_t w, int32_t* d_window, int32_t* d_count, float* d_hist) {
+    if (!ctx || w < 0 || w > 64) return GRAFT_ERR_INVALID_ARG;
+    if (w > 0 && (!d_window || !d_count || !d_hist)) return GRAFT_ERR_INVALID_ARG;
+    ctx->hist_w = w;
+    ctx->hist_window = w ? d_window : nullptr;
+    ctx->hist_count = w ? d_count : nullptr;
+    ctx->hist_out = w ? d_hist : nullptr;
     return GRAFT_OK;
 }
 

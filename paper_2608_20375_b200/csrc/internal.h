@@ -61,6 +61,10 @@ struct graft_ctx {
     const float* d_C;
     float* d_u;  // owned copy [L, m]
     float tdes_s;
+    int hist_w;            // acceptance-history window (0 = off) and the caller's buffers for it
+    int32_t* hist_window;  // [max_batch, hist_w]
+    int32_t* hist_count;   // [max_batch]
+    float* hist_out;       // [max_batch]
     int edge_rows;  // depths [0, edge_rows) are scored by the edge-score kernel, deeper ones on demand in the tree kernel
     // scratch (one allocation)
     void* ws;

@@ -982,6 +982,11 @@ struct AcceptParams {
     int32_t* accept_len;
     int32_t* accept_path;
     int32_t* bonus;
+    // acceptance history (Eq. 15), updated here when hist_w > 0
+    int hist_w;
+    int32_t* hist_window;
+    int32_t* hist_count;
+    float* hist_out;
 };
 
 __global__ void __launch_bounds__(128) accept_kernel(const AcceptParams ap) {
@@ -1053,6 +1058,18 @@ __global__ void __launch_bounds__(128) accept_kernel(const AcceptParams ap) {
     if (lane == 0) {
         accept_len[b] = a;
         bonus[b] = tn[cur];
+        if (ap.hist_w > 0) {  // hist for the next round: mean of the last min(rounds, w) accepted lengths
+            const int w = ap.hist_w;
+            int n = ap.hist_count[b];
+            int32_t* ring = ap.hist_window + (size_t)b * w;
+            ring[n % w] = a;
+            n += 1;
+            ap.hist_count[b] = n;
+            const int cnt = n < w ? n : w;
+            int sum = 0;
+            for (int i = 0; i < cnt; ++i) sum += ring[i];
+            ap.hist_out[b] = (float)((double)sum / (double)cnt);
+        }
     }
 }
 
@@ -1132,6 +1149,10 @@ cudaError_t accept_launch(graft_ctx* ctx, int batch, const graft_tree_out* trees
     ap.accept_len = d_accept_len;
     ap.accept_path = d_accept_path;
     ap.bonus = d_bonus;
+    ap.hist_w = ctx->hist_w;
+    ap.hist_window = ctx->hist_window;
+    ap.hist_count = ctx->hist_count;
+    ap.hist_out = ctx->hist_out;
     const cudaError_t e = launch_pdl(accept_kernel, dim3(batch), dim3(128), (size_t)3 * ctx->nmax * sizeof(int32_t), st, ap);
     ctx->launches += 1;
     return e != cudaSuccess ? e : cudaGetLastError();
