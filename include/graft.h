@@ -176,6 +176,30 @@ graft_status graft_vocab_pass_static(int32_t batch, int32_t L, int32_t V, int32_
                                      const void* d_logits, int32_t* d_topk_id, float* d_topk_lp, float* d_lse,
                                      int32_t* d_row_status, void* stream);
 
+/* Vocabulary-parallel S1 (the logits of a tensor-parallel LM head are split over V across GPUs).  Each GPU runs
+ * graft_vocab_pass_partial on its shard: per row it leaves the log-sum-exp pieces and the K best keys of the shard
+ * (token ids local to the shard).  The partials of all shards, gathered into one buffer in shard order (one NCCL
+ * all-gather of 280 bytes per row and shard; they land in local memory first), are merged by graft_vocab_merge into
+ * the outputs graft_vocab_pass gives for the full row: the same candidates (value descending, global id
+ * ascending), log q over the whole vocabulary.  The context of graft_vocab_pass_partial is one created with V =
+ * the shard's width (and K = min(K, width) when a shard is narrower than K); graft_vocab_merge uses only K and L
+ * of its context.
+ *   d_out     [batch*L] partials of this shard
+ *   d_parts   [n_shards, batch*L] partials of all shards;  h_v_offset [n_shards] first global id of each shard
+ * (The paper has one drafter on one GPU; this is the one-exchange sharding of its dominant step.) */
+typedef struct {
+    double c;          /* reference exponent (log2 domain) */
+    double s;          /* sum_v 2^(z_v log2(e) - c) over the shard */
+    uint32_t vmax_ord; /* largest logit of the shard, as an order-preserving integer */
+    uint32_t nkeys;    /* valid keys (min(K, shard width)) */
+    uint64_t keys[32]; /* (order-preserving value << 32) | (0xFFFFFFFF - local id), descending */
+} graft_vocab_partial;
+graft_status graft_vocab_pass_partial(graft_ctx* ctx, int32_t batch, const void* d_logits_shard,
+                                      graft_vocab_partial* d_out, void* stream);
+graft_status graft_vocab_merge(graft_ctx* ctx, int32_t batch, int32_t n_shards, const graft_vocab_partial* d_parts,
+                               const int32_t* h_v_offset, int32_t* d_topk_id, float* d_topk_lp, float* d_lse,
+                               int32_t* d_row_status, void* stream);
+
 /* Acceptance walk (Preliminaries, "Speculative decoding": a_t; "Tree-based speculative decoding": the longest
  * accepted path is committed).  d_target_next[b, i] is the target model's next token after node i.  The tree
  * must be in the level order graft_build_trees emits (parent indices never decrease along the node index).

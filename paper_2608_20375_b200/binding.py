@@ -21,10 +21,13 @@ ST_BAD_LOGITS, ST_TAU_CLAMPED, ST_FRONTIER_EMPTY, ST_INTERNAL = 1, 2, 4, 8
 ENTRY_POINTS = [
     "graft_create", "graft_destroy", "graft_nmax", "graft_mask_words", "graft_set_saba", "graft_set_tdes_tables",
     "graft_tdes_precompute", "graft_build_trees", "graft_vocab_pass", "graft_vocab_pass_static", "graft_tdes_edges",
-    "graft_accept", "graft_set_edge_rows", "graft_edge_rows", "graft_set_hist_window",
+    "graft_accept", "graft_set_edge_rows", "graft_edge_rows", "graft_set_hist_window", "graft_vocab_pass_partial", "graft_vocab_merge",
     "graft_build_trees_host", "graft_launch_count", "graft_set_timing", "graft_read_timing", "graft_status_str",
     "graft_version",
 ]
+
+
+VOCAB_PARTIAL_BYTES = 280  # sizeof(graft_vocab_partial)
 
 
 class GraftError(RuntimeError):
@@ -81,6 +84,8 @@ def load_library():
     lib.graft_set_tdes_tables.argtypes = [vp, vp, vp, vp, C.c_float, vp]
     lib.graft_set_edge_rows.argtypes = [vp, C.c_int32]
     lib.graft_set_hist_window.argtypes = [vp, C.c_int32, vp, vp, vp]
+    lib.graft_vocab_pass_partial.argtypes = [vp, C.c_int32, vp, vp, vp]
+    lib.graft_vocab_merge.argtypes = [vp, C.c_int32, C.c_int32, vp, vp, vp, vp, vp, vp, vp]
     lib.graft_edge_rows.argtypes = [vp]
     lib.graft_edge_rows.restype = C.c_int32
     lib.graft_tdes_precompute.argtypes = [vp, vp, C.c_int, C.c_int32, vp, vp, vp, vp]
@@ -218,6 +223,25 @@ class Graft:
         p = _Saba(phi_conf, phi_degen, phi_hist, phi_bias, tau_min, cost_mode, c0, c1, c2, len(pts_n),
                   C.cast(n, C.POINTER(C.c_float)), C.cast(t, C.POINTER(C.c_float)))
         _check(self.lib, self.lib.graft_set_saba(self._ctx, C.byref(p)), "graft_set_saba")
+
+    # ---- vocabulary-parallel S1
+    def vocab_pass_partial(self, logits_shard, parts):
+        """parts: uint8 [batch*L, VOCAB_PARTIAL_BYTES] on the device (this shard's pieces of every row)."""
+        batch = logits_shard.shape[0]
+        if parts.dtype != torch.uint8 or parts.numel() != batch * self.cfg.L * VOCAB_PARTIAL_BYTES:
+            raise GraftError("parts must be uint8 [batch*L, VOCAB_PARTIAL_BYTES]")
+        _check(self.lib, self.lib.graft_vocab_pass_partial(self._ctx, batch, _ptr(logits_shard), _ptr(parts), _stream()),
+               "graft_vocab_pass_partial")
+
+    def vocab_merge(self, parts_all, v_offsets, ids, lp, lse, row_status):
+        """parts_all: uint8 [n_shards, batch*L, VOCAB_PARTIAL_BYTES]; v_offsets: first global id of each shard."""
+        n_shards = parts_all.shape[0]
+        batch = ids.shape[0]
+        off = (C.c_int32 * n_shards)(*[int(v) for v in v_offsets])
+        _check(self.lib, self.lib.graft_vocab_merge(self._ctx, batch, n_shards, _ptr(parts_all, torch.uint8), off,
+                                                    _ptr(ids, torch.int32), _ptr(lp, torch.float32),
+                                                    _ptr(lse, torch.float32), _ptr(row_status, torch.int32),
+                                                    _stream()), "graft_vocab_merge")
 
     def set_hist_window(self, w, window=None, count=None, hist=None):
         """graft_accept keeps hist_t (Eq. 15) on the device: window [batch, w] int32, count [batch] int32,

@@ -254,7 +254,7 @@ graft_status graft_vocab_pass(graft_ctx* ctx, int32_t batch, const void* d_logit
     const int esz = ctx->cfg.logits_dtype == GRAFT_BF16 ? 2 : 4;
     if ((uintptr_t)d_logits % esz) return GRAFT_ERR_INVALID_ARG;
     if (vp_launch(ctx, batch, d_logits, d_topk_id, d_topk_lp, d_lse, d_row_status ? d_row_status : ctx->w_row_status,
-                  nullptr, nullptr, (cudaStream_t)stream) != cudaSuccess)
+                  nullptr, nullptr, nullptr, (cudaStream_t)stream) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     return GRAFT_OK;
 }
@@ -339,7 +339,7 @@ graft_status graft_build_trees(graft_ctx* ctx, int32_t batch, const void* d_logi
 
     if (ev) cudaEventRecord(ev[0], st);
     if (vp_launch(ctx, batch, d_logits, ids, lps, lse, ctx->w_row_status, use_saba ? d_hidden : nullptr, ctx->w_cos,
-                  st) != cudaSuccess)
+                  nullptr, st) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     if (ev) cudaEventRecord(ev[1], st);
     // Edge scores of Eq. 4-6: the kernel scores the depths [0, edge_rows) for every sequence (all depths when the
@@ -369,6 +369,32 @@ graft_status graft_accept(graft_ctx* ctx, int32_t batch, const graft_tree_out* t
     if (batch < 1 || batch > ctx->cfg.max_batch) return GRAFT_ERR_INVALID_ARG;
     if (accept_launch(ctx, batch, trees, d_target_next, d_accept_len, d_accept_path, d_bonus_token,
                       (cudaStream_t)stream) != cudaSuccess)
+        return GRAFT_ERR_CUDA;
+    return GRAFT_OK;
+}
+
+graft_status graft_vocab_pass_partial(graft_ctx* ctx, int32_t batch, const void* d_logits_shard,
+                                      graft_vocab_partial* d_out, void* stream) {
+    if (!ctx || !d_logits_shard || !d_out) return GRAFT_ERR_INVALID_ARG;
+    if (batch < 1 || batch > ctx->cfg.max_batch) return GRAFT_ERR_INVALID_ARG;
+    const int esz = ctx->cfg.logits_dtype == GRAFT_BF16 ? 2 : 4;
+    if ((uintptr_t)d_logits_shard % esz || (uintptr_t)d_out % 8) return GRAFT_ERR_INVALID_ARG;
+    if (vp_launch(ctx, batch, d_logits_shard, ctx->w_topk_id, ctx->w_topk_lp, ctx->w_lse, ctx->w_row_status, nullptr,
+                  nullptr, d_out, (cudaStream_t)stream) != cudaSuccess)
+        return GRAFT_ERR_CUDA;
+    return GRAFT_OK;
+}
+
+graft_status graft_vocab_merge(graft_ctx* ctx, int32_t batch, int32_t n_shards, const graft_vocab_partial* d_parts,
+                               const int32_t* h_v_offset, int32_t* d_topk_id, float* d_topk_lp, float* d_lse,
+                               int32_t* d_row_status, void* stream) {
+    if (!ctx || !d_parts || !h_v_offset || !d_topk_id || !d_topk_lp || !d_lse || !d_row_status)
+        return GRAFT_ERR_INVALID_ARG;
+    if (batch < 1 || n_shards < 1 || n_shards > vp_merge_max_shards()) return GRAFT_ERR_INVALID_ARG;
+    for (int i = 0; i < n_shards; ++i)
+        if (h_v_offset[i] < 0 || (i > 0 && h_v_offset[i] <= h_v_offset[i - 1])) return GRAFT_ERR_INVALID_ARG;
+    if (vp_merge_launch(ctx, batch, n_shards, d_parts, h_v_offset, d_topk_id, d_topk_lp, d_lse, d_row_status,
+                        (cudaStream_t)stream) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     return GRAFT_OK;
 }

@@ -112,9 +112,14 @@ inline cudaError_t launch_pdl(void (*kernel)(P), dim3 grid, dim3 block, size_t s
 VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch);
 cudaError_t vp_configure(const graft_config& cfg, int num_sms, size_t* max_smem);
 cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* d_topk_id, float* d_topk_lp,
-                      float* d_lse, int32_t* d_row_status, const void* d_hidden, double* d_cos, cudaStream_t st);
+                      float* d_lse, int32_t* d_row_status, const void* d_hidden, double* d_cos,
+                      graft_vocab_partial* d_partial, cudaStream_t st);
 // d_hidden != NULL: one more warp per CTA also writes the adjacent-position cosines of the SABA state (Eq. 15)
-// to d_cos [batch, L]
+// to d_cos [batch, L]; d_partial != NULL: the rows' pieces go there instead of the outputs (vocabulary-parallel use)
+cudaError_t vp_merge_launch(graft_ctx* ctx, int batch, int n_shards, const graft_vocab_partial* d_parts,
+                            const int32_t* h_v_offset, int32_t* d_topk_id, float* d_topk_lp, float* d_lse,
+                            int32_t* d_row_status, cudaStream_t st);
+int vp_merge_max_shards();
 
 cudaError_t tdes_precompute_launch(graft_ctx* ctx, const void* d_emb, graft_dtype dt, int E, const float* d_W,
                                    const float* d_b, float* d_out, cudaStream_t st);

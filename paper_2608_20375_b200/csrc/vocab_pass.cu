@@ -83,6 +83,7 @@ struct VpParams {
     float* lse;
     int32_t* row_status;
     int32_t* errflag;
+    graft_vocab_partial* partial_out;  // vocabulary-parallel use: the row's pieces go here instead of the outputs
     // adjacent-position cosines of the SABA state (Eq. 15), computed by a warp of their own beside the stream;
     // cos_out == nullptr: not asked for
     const void* hidden;
@@ -406,6 +407,30 @@ __device__ int warp_fallback_select(EpiShared* sh, const VpParams& p, const Seg&
     }
     warp_select_topk(sh, nb, K, lane);
     return nb < K ? nb : K;
+}
+
+// The outputs of a finished row from its pieces: C, S with sum_v 2^(z_v c) = S 2^C (c = fp32(log2 e)), the largest
+// logit, and the K best keys.  One warp.
+__device__ __forceinline__ void vp_finalize(double Cd, double Sd, uint32_t Vm, int nk, int K, const uint64_t* keys,
+                                            int lane, int32_t* topk_id, float* topk_lp, float* lse,
+                                            int32_t* row_status) {
+    // The stream accumulates 2^(z c - ref) with c = fp32(log2 e), so (C + log2 S) ln 2 is the
+    // log-sum-exp of the logits scaled by a = c ln 2 = 1 + 1.3e-8.  To first order that adds
+    // (a - 1) E_q[z]; the largest logit stands in for the mean under q (the difference is a few
+    // units times 1e-8).
+    const float vmax = __uint_as_float(bits_from_ord(Vm));
+    const double a_minus_1 = (double)kLog2e * kLn2 - 1.0;
+    const double lse_d = (Cd + log2(Sd)) * kLn2 - a_minus_1 * (double)vmax;
+    const bool bad = !(Sd > 0.0) || !(Sd < 1e300) || Vm == 0u || vmax == INFINITY || vmax == -INFINITY || nk < K;
+    if (lane < K) {
+        const uint64_t key = lane < nk ? keys[lane] : 0ull;
+        topk_id[lane] = lane < nk ? (int32_t)key_id(key) : -1;
+        topk_lp[lane] = lane < nk ? (float)((double)key_value(key) - lse_d) : 0.f;
+    }
+    if (lane == 0) {
+        *lse = (float)lse_d;
+        *row_status = bad ? GRAFT_ST_BAD_LOGITS : 0;
+    }
 }
 
 template <bool BF16>
@@ -842,26 +867,19 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 }
             }
             VP_T(6);
-            if (finish) {
-                // The stream accumulates 2^(z c - ref) with c = fp32(log2 e), so (C + log2 S) ln 2 is the
-                // log-sum-exp of the logits scaled by a = c ln 2 = 1 + 1.3e-8.  To first order that adds
-                // (a - 1) E_q[z]; the largest logit stands in for the mean under q (the difference is a few
-                // units times 1e-8).
-                const float vmax = __uint_as_float(bits_from_ord(Vm));
-                const double a_minus_1 = (double)kLog2e * kLn2 - 1.0;
-                const double lse_d = (Cd + log2(Sd)) * kLn2 - a_minus_1 * (double)vmax;
-                const bool bad = !(Sd > 0.0) || !(Sd < 1e300) || Vm == 0u || vmax == INFINITY || vmax == -INFINITY ||
-                                 nk < p.K;
-                if (lane < p.K) {
-                    const uint64_t key = lane < nk ? es->outk[lane] : 0ull;
-                    p.topk_id[(size_t)sg.row * p.K + lane] = lane < nk ? (int32_t)key_id(key) : -1;
-                    p.topk_lp[(size_t)sg.row * p.K + lane] = lane < nk ? (float)((double)key_value(key) - lse_d) : 0.f;
-                }
-                VP_T(7);
+            if (finish && p.partial_out != nullptr) {
+                graft_vocab_partial* po = p.partial_out + sg.row;
+                if (lane < kMaxK) po->keys[lane] = lane < nk ? es->outk[lane] : 0ull;
                 if (lane == 0) {
-                    p.lse[sg.row] = (float)lse_d;
-                    p.row_status[sg.row] = bad ? GRAFT_ST_BAD_LOGITS : 0;
+                    po->c = Cd;
+                    po->s = Sd;
+                    po->vmax_ord = Vm;
+                    po->nkeys = (uint32_t)nk;
                 }
+            } else if (finish) {
+                vp_finalize(Cd, Sd, Vm, nk, p.K, es->outk, lane, p.topk_id + (size_t)sg.row * p.K,
+                            p.topk_lp + (size_t)sg.row * p.K, p.lse + sg.row, p.row_status + sg.row);
+                VP_T(7);
             }
             __syncwarp();
         }
@@ -881,6 +899,71 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
     }
 #endif
     if (tid == 0 && sh->abort_flag) atomicOr(p.errflag, 1);
+}
+
+// ---- vocabulary-parallel merge: one CTA of 128 threads per row ---------------------------------------------------
+constexpr int kMergeMaxShards = 64;
+struct MergeParams {
+    const graft_vocab_partial* parts;  // [n_shards, rows]
+    int n_shards, rows, K;
+    int32_t v_offset[kMergeMaxShards];
+    int32_t* topk_id;
+    float* topk_lp;
+    float* lse;
+    int32_t* row_status;
+};
+__global__ void __launch_bounds__(128) vocab_merge_kernel(const MergeParams p) {
+    __shared__ uint64_t cand[kMergeMaxShards * kMaxK];
+    __shared__ uint64_t outk[kMaxK];
+    __shared__ double sC[kMergeMaxShards], sS[kMergeMaxShards];
+    __shared__ uint32_t sV[kMergeMaxShards], sN[kMergeMaxShards];
+    const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+    const int n = p.n_shards * kMaxK;
+    // the shards' keys with global token ids (an empty slot stays 0 and ranks below every key)
+    for (int i = tid; i < n; i += 128) {
+        const int sidx = i / kMaxK, kk = i % kMaxK;
+        const graft_vocab_partial* r = p.parts + (size_t)sidx * p.rows + row;
+        uint64_t key = kk < (int)r->nkeys ? r->keys[kk] : 0ull;
+        if (key != 0ull) key = make_key(bits_from_ord((uint32_t)(key >> 32)), key_id(key) + (uint32_t)p.v_offset[sidx]);
+        cand[i] = key;
+    }
+    if (tid < p.n_shards) {
+        const graft_vocab_partial* r = p.parts + (size_t)tid * p.rows + row;
+        sC[tid] = r->c;
+        sS[tid] = r->s;
+        sV[tid] = r->vmax_ord;
+        sN[tid] = r->nkeys;
+    }
+    if (tid < kMaxK) outk[tid] = 0ull;
+    __syncthreads();
+    // exact top-K by rank counting (keys are distinct: ids are)
+    for (int i = tid; i < n; i += 128) {
+        const uint64_t key = cand[i];
+        if (key == 0ull) continue;
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += cand[j] > key ? 1 : 0;
+        if (rank < p.K) outk[rank] = key;
+    }
+    __syncthreads();
+    if (tid >= 32) return;
+    int have = 0;
+    for (int sidx = 0; sidx < p.n_shards; ++sidx) have += (int)sN[sidx];
+    const int nk = have < p.K ? have : p.K;
+    double Cm = -INFINITY;
+    uint32_t vm = 0u;
+    for (int sidx = 0; sidx < p.n_shards; ++sidx) {
+        Cm = fmax(Cm, sC[sidx]);
+        vm = vm > sV[sidx] ? vm : sV[sidx];
+    }
+    double S = 0.0;
+    for (int sidx = 0; sidx < p.n_shards; ++sidx) {
+        if (sC[sidx] != -INFINITY)
+            S += sS[sidx] * exp2(sC[sidx] - Cm);
+        else if (sS[sidx] != sS[sidx])
+            S += sS[sidx];
+    }
+    vp_finalize(Cm, S, vm, nk, p.K, outk, lane, p.topk_id + (size_t)row * p.K, p.topk_lp + (size_t)row * p.K,
+                p.lse + row, p.row_status + row);
 }
 
 }  // namespace
@@ -914,7 +997,8 @@ VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch) {
 }
 
 cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* d_topk_id, float* d_topk_lp,
-                      float* d_lse, int32_t* d_row_status, const void* d_hidden, double* d_cos, cudaStream_t st) {
+                      float* d_lse, int32_t* d_row_status, const void* d_hidden, double* d_cos,
+                      graft_vocab_partial* d_partial, cudaStream_t st) {
     const graft_config& cfg = ctx->cfg;
     const bool bf16 = cfg.logits_dtype == GRAFT_BF16;
     VpPlan pl = vp_make_plan(cfg, ctx->num_sms, batch);
@@ -935,6 +1019,7 @@ cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* 
     p.lse = d_lse;
     p.row_status = d_row_status;
     p.errflag = ctx->w_errflag;
+    p.partial_out = d_partial;
     p.hidden = d_hidden;
     p.hidden_bf16 = cfg.hidden_dtype == GRAFT_BF16 ? 1 : 0;
     p.hidden_dim = cfg.hidden_dim;
@@ -955,6 +1040,25 @@ cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* 
     ctx->launches += 1;
     return cudaGetLastError();
 }
+
+cudaError_t vp_merge_launch(graft_ctx* ctx, int batch, int n_shards, const graft_vocab_partial* d_parts,
+                            const int32_t* h_v_offset, int32_t* d_topk_id, float* d_topk_lp, float* d_lse,
+                            int32_t* d_row_status, cudaStream_t st) {
+    MergeParams p;
+    p.parts = d_parts;
+    p.n_shards = n_shards;
+    p.rows = batch * ctx->cfg.L;
+    p.K = ctx->cfg.K;
+    for (int i = 0; i < kMergeMaxShards; ++i) p.v_offset[i] = i < n_shards ? h_v_offset[i] : 0;
+    p.topk_id = d_topk_id;
+    p.topk_lp = d_topk_lp;
+    p.lse = d_lse;
+    p.row_status = d_row_status;
+    vocab_merge_kernel<<<p.rows, 128, 0, st>>>(p);
+    ctx->launches += 1;
+    return cudaGetLastError();
+}
+int vp_merge_max_shards() { return kMergeMaxShards; }
 
 cudaError_t vp_configure(const graft_config& cfg, int num_sms, size_t* max_smem) {
     // the largest dynamic shared-memory request any batch can produce (segment = a whole row)
@@ -1079,6 +1183,7 @@ extern "C" graft_status graft_vocab_pass_static(int32_t batch, int32_t L, int32_
     p.lse = d_lse;
     p.row_status = d_row_status;
     p.errflag = sd->scratch->errflag;
+    p.partial_out = nullptr;
     p.hidden = nullptr;
     p.hidden_bf16 = 0;
     p.hidden_dim = 0;

@@ -155,6 +155,53 @@ def test_tdes_edges_against_oracle(K, L, m, beta, root_edge):
             assert np.array_equal(edge[b], want)  # the DDTree score, bit for bit
 
 
+# --------------------------------------------------------------------------- vocabulary-parallel vocab pass
+@pytest.mark.parametrize("V,K,L,Bt,dtype,world", [
+    (50000, 16, 4, 3, "bf16", 2), (151936, 32, 2, 2, "bf16", 4), (32000, 8, 3, 2, "f32", 3), (9000, 32, 2, 2, "bf16", 8),
+    (70, 16, 2, 2, "f32", 5),  # shards narrower than K
+])
+def test_vocab_pass_parallel_matches_the_full_row_oracle(V, K, L, Bt, dtype, world):
+    """The ranks of a vocabulary-parallel run, emulated one after the other on this device: every shard's pieces,
+    then the merge, against the oracle on the full rows."""
+    from paper_2608_20375_b200 import Graft, VOCAB_PARTIAL_BYTES, vocab_range
+    w = gi.small(batch=Bt, L=L, V=V, K=K, logits_dtype=dtype)
+    z = gi.batch_inputs(w)["logits"]
+    z[0, 0, 5] = z[0, 0, V - 3] = z[0, 0, 7]  # equal values in different shards: ids decide
+    z[1, 1, ::2] = float("-inf")             # masked tokens
+    rows = Bt * L
+    parts, offs, keep = [], [], []
+    for r in range(world):
+        lo, hi = vocab_range(V, r, world)
+        offs.append(lo)
+        gs = Graft(hi - lo, L, min(K, hi - lo), 16, 8, Bt, 8, 8, 8, 0.0, 1, DT[dtype], 0)  # a narrow shard keeps all it has
+        p = torch.empty((rows, VOCAB_PARTIAL_BYTES), dtype=torch.uint8, device="cuda")
+        gs.vocab_pass_partial(z[:, :, lo:hi].contiguous().cuda(), p)
+        parts.append(p)
+        keep.append(gs)
+    allp = torch.stack(parts).contiguous()
+    ids = torch.empty((Bt, L, K), dtype=torch.int32, device="cuda")
+    lp = torch.empty((Bt, L, K), dtype=torch.float32, device="cuda")
+    lse = torch.empty((Bt, L), dtype=torch.float32, device="cuda")
+    rs = torch.empty((Bt, L), dtype=torch.int32, device="cuda")
+    gm = Graft(V, L, K, 16, 8, Bt, 8, 8, 8, 0.0, 1, DT[dtype], 0)  # the merge uses K and L of its context
+    keep.append(gm)
+    gm.vocab_merge(allp, offs, ids, lp, lse, rs)
+    torch.cuda.synchronize()
+    o_ids, o_lp, o_lse, o_st = oracle.vocab_pass(z.reshape(rows, V), K)
+    ids, lp, lse, rs = (t.cpu().numpy().reshape(rows, -1) for t in (ids, lp, lse, rs))
+    assert np.array_equal(rs[:, 0], o_st)
+    good = o_st == 0
+    assert good.all()
+    assert np.array_equal(ids[good], o_ids[good])
+    a, b = lp[good].astype(np.float64), o_lp[good].astype(np.float64)
+    assert np.array_equal(np.isneginf(a), np.isneginf(b))
+    fin = np.isfinite(b)
+    assert np.abs(a[fin] - b[fin]).max(initial=0) <= EPS
+    assert np.all(np.abs(lse[good, 0] - o_lse[good]) <= EPS + np.spacing(np.abs(lse[good, 0])))
+    for gs in keep:
+        gs.destroy()
+
+
 # --------------------------------------------------------------------------- whole round, small
 @pytest.mark.parametrize("kw", [
     dict(batch=4, L=4, V=1000, K=4, budget_min=8, budget_max=24, budget_step=8),

@@ -11,6 +11,7 @@ import torch.multiprocessing as mp
 
 import graft_inputs as gi
 from paper_2608_20375_b200.shard import shard_range
+from paper_2608_20375_b200.vocab_parallel import gather_partials, vocab_range
 
 
 def test_shard_ranges_tile_the_batch():
@@ -58,3 +59,50 @@ def test_two_ranks_gloo():
     full = gi.batch_inputs(w)
     assert abs(parts[0][0] + parts[1][0] - float(full["logits"].double().sum())) < 1e-6
     assert parts[0][1] + parts[1][1] == w.batch and tmax == 2.0
+
+
+def test_vocab_ranges_tile_the_vocabulary():
+    for V in (70, 9000, 32000, 151936):
+        for world in (1, 2, 3, 5, 8):
+            if V == 70 and world == 8:  # nine ids per rank cannot start on multiples of eight
+                try:
+                    vocab_range(V, 0, world)
+                    assert False, "expected ValueError"
+                except ValueError:
+                    continue
+            spans = [vocab_range(V, r, world) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == V and all(hi > lo for lo, hi in spans)
+            assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+            assert all(lo % 8 == 0 for lo, _ in spans)
+
+
+def _gather_worker(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rows = 6
+    parts = torch.full((rows, 280), rank + 1, dtype=torch.uint8)  # stand-in for this rank's partial records
+    parts[:, 0] = torch.arange(rows, dtype=torch.uint8)
+    allp = gather_partials(parts)
+    if rank == 1:
+        q.put(allp.numpy().copy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_partials_are_gathered_in_rank_order_gloo():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_gather_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    allp = q.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert allp.shape == (2, 6, 280)
+    for r in range(2):
+        assert (allp[r, :, 1:] == r + 1).all() and allp[r, :, 0].tolist() == list(range(6))
