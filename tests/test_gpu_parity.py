@@ -439,3 +439,11 @@ def test_config_full_size_sampled(name, nseq):
     assert excused <= max(1, len(sample) // 3)
     compare_accept(oracle, gi, g, w, out, gpu)
     assert len(set(gpu["budget"].tolist())) > 1 or name in ("C2",)
+    # the call the benchmark times (no debug outputs: the first depths by the edge-score kernel, deeper ones on
+    # demand) gives the same trees as the call checked above, bit for bit, for every sequence
+    out_p = g.alloc_out(w.batch, debug=False)
+    g.build_trees(z, h, root.cuda(), hist.cuda(), pref.cuda(), None, out_p)
+    torch.cuda.synchronize()
+    prod = out_p.cpu()
+    for k in ("n_nodes", "budget", "status", "token", "parent", "depth", "position", "path_score", "mask"):
+        assert np.array_equal(prod[k], gpu[k]), k
