@@ -3,6 +3,8 @@
 //   tdes_precompute_kernel   out[v] = W e_v + b            (text after Eq. 6: computed once per model)
 //   tdes_edges_kernel        edge[d][i][c] = log q_d(c) + beta * (f - mean_c f),
 //                            f = s (P[p_i] + u_d) . (C[c] + u_d) / sqrt(m)          (Eq. 4-6)
+//                            for the first depths of every sequence (the arithmetic is in edge_score.cuh,
+//                            which the tree kernel also uses for deeper depths)
 //
 // The per-round scorer is a gather of token-indexed table rows followed by K x K dot products of length
 // m per depth -- not a dense contraction over hidden states -- so it runs as fp32 FMAs out of shared

@@ -1,6 +1,7 @@
 // Per-sequence tail of the round: SABA budget (Sec. 3.3, Eq. 14-17), best-first expansion by TDES path
 // score until B_t nodes (Sec. 3.1; Eq. 13; the heap expansion described for DDTree), level-order emission
-// with the packed ancestor mask, and the acceptance walk.
+// with the packed ancestor mask, and the acceptance walk (which also keeps the acceptance history of Eq. 15).
+// Edge scores of depths that the edge-score kernel did not cover are worked out here when an expansion reaches them.
 #include "common.cuh"
 #include "internal.h"
 #include "edge_score.cuh"

@@ -3,19 +3,21 @@
 // (Preliminaries, "DFlash one-pass marginals": q_{t,d} and c^{(r)}_{t,d}; Eq. 3's log q).
 //
 // Shape of the kernel (sm_100a):
-//   * persistent grid, two CTAs per SM; the rows*V element stream is cut into equal contiguous shares,
+//   * persistent grid, one CTA per SM; the rows*V element stream is cut into equal contiguous shares,
 //     one per CTA, so a CTA sees at most two partial rows plus whole rows in between ("segments");
-//   * warp roles: one producer warp feeds a shared-memory ring with 16 KiB TMA bulk copies (cp.async.bulk +
-//     mbarrier complete_tx); eight streaming warps read the ring with 16-byte shared loads; one epilogue
-//     warp finishes segment k while the streaming warps are already in segment k+1;
+//   * warp roles: one producer warp feeds a four-stage shared-memory ring with 32 KiB TMA bulk copies
+//     (cp.async.bulk + mbarrier complete_tx); sixteen streaming warps read the ring with 16-byte shared loads;
+//     two epilogue groups of four warps finish alternate segments while the streaming warps are already in
+//     later ones; one warp computes the adjacent-position cosines of the SABA state (Eq. 15) beside the stream;
 //   * per 32-element chunk a streaming lane takes a packed max (stored for the second stage, 2 bytes per
 //     chunk), keeps a lazily rescaled reference exponent and adds 2^(z log2e - ref) with ex2.approx;
-//   * top-K needs no per-element work in the stream: after the segment, the K-th largest per-thread
-//     maximum is a lower bound T for the K-th largest element; only chunks whose stored max reaches T
+//   * top-K needs no per-element work in the stream: after the segment, the K-th largest of 64 group maxima
+//     is a lower bound T for the K-th largest element; only chunks whose stored max reaches T
 //     (about K of them) are re-read, their elements >= T become 64-bit keys (value desc, id asc) and the
 //     exact top-K is found by rank counting.  An overflow of the small key buffer (adversarial rows)
 //     falls back to an exact sliced selection;
-//   * rows shared by several CTAs are merged by the last CTA to arrive (a counter, no waiting).
+//   * rows shared by several CTAs are merged by the last CTA to arrive (a counter, no waiting);
+//   * vocabulary-parallel use: the row's pieces are left for a merge over shards instead (vocab_merge_kernel).
 // Every wait on an mbarrier is bounded; when one runs out the kernel raises an error flag and drains.
 #include <stdlib.h>
 #include <string.h>
@@ -58,13 +60,13 @@ struct VT;
 template <>
 struct VT<true> {
     using cm_t = uint16_t;
-    static constexpr int ESZ = 2, EPV = 8, CH = 32;
+    static constexpr int ESZ = 2, EPV = 8;
     static constexpr uint32_t NEG_INF_WORD = 0xFF80FF80u;
 };
 template <>
 struct VT<false> {
     using cm_t = uint16_t;  // the chunk maximum rounded UP to bf16 precision: an upper bound is all the scan needs
-    static constexpr int ESZ = 4, EPV = 4, CH = 16;
+    static constexpr int ESZ = 4, EPV = 4;
     static constexpr uint32_t NEG_INF_WORD = 0xFF800000u;
 };
 
