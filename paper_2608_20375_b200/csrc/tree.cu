@@ -390,9 +390,37 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         }
     }
     // adjacent-position cosines r_d = cos(h_d, h_{d+1}) (Eq. 15): written by the vocab pass
-    if (p.use_saba) {
-        if (tid < L - 1) sm.cosv[tid] = p.cos_pre[(size_t)b * L + tid];
-        __syncthreads();
+    if (p.use_saba && tid < L - 1) sm.cosv[tid] = p.cos_pre[(size_t)b * L + tid];
+    __syncthreads();
+    // While warp 0 works out the budget, the other warps expand levels 0 and 1 in full (1 + K + K^2 nodes), which
+    // needs no budget: with fewer than B nodes in the table every child is appended anyway, and if B is smaller
+    // than that the extra nodes only fall below the threshold found afterwards.
+    const bool spec = bulk && p.rows_pre >= 2 && L >= 2 && 1 + K + K * K <= p.ncap;
+    if (spec && warp >= 1) {
+        mbar_wait_bounded(smem_u32(&rows_bar), 0, &rows_abort);
+        const int t1 = tid - 32, nth = TREE_THREADS - 32;
+        if (t1 == 0) {
+            sm.nkey[0] = 0xFFFFFFFFu;
+            sm.nS[0] = 0.0f;
+            sm.ninfo[0] = 0u;
+        }
+        if (t1 < K) {  // level 0: the root's children, row (depth 0, parent rank 0)
+            const float sc = 0.0f + sm.es[t1];
+            sm.nkey[1 + t1] = ord_from_float(sc);
+            sm.nS[1 + t1] = sc;
+            sm.ninfo[1 + t1] = 0u | ((uint32_t)sm.ei[t1] << 13) | (1u << 18);
+        }
+        named_bar_sync(1, nth);
+        for (int j = t1; j < K * K; j += nth) {  // level 1
+            const int xi = j / K, r = j - xi * K, x = 1 + xi;
+            const uint32_t kx = sm.nkey[x];
+            const int row = (K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
+            const float sc = sm.nS[x] + sm.es[row + r];
+            const uint32_t oc = ord_from_float(sc);
+            sm.nkey[1 + K + j] = oc < kx ? oc : kx;
+            sm.nS[1 + K + j] = sc;
+            sm.ninfo[1 + K + j] = (uint32_t)x | ((uint32_t)sm.ei[row + r] << 13) | (2u << 18);
+        }
     }
     if (warp == 0) {
         int st = 0;
@@ -482,10 +510,14 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         sm.nkey[0] = 0xFFFFFFFFu;
         sm.nS[0] = 0.0f;
         sm.ninfo[0] = 0u;
-        sm.scal[3] = 1;
+        sm.scal[3] = spec ? 1 + K + K * K : 1;
         sm.scal[4] = 0;
         sm.lvl_start[0] = 0;
         sm.lvl_start[1] = 1;
+        if (spec) {
+            sm.lvl_start[2] = 1 + K;
+            sm.lvl_start[3] = 1 + K + K * K;
+        }
         sm.parent[0] = -1;
         sm.cand[0] = 0;
         sm.depth[0] = 0;
@@ -496,7 +528,15 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     uint32_t theta = 0u;
     if (budget > 0) {
         int ntot = 1, n_at_select = 1, sel_rem = 0;
-        for (int d = 0; d < L; ++d) {
+        if (spec) {  // levels 0 and 1 are in the table already: the threshold they give, then on from level 2
+            ntot = 1 + K + K * K;
+            if (ntot - 1 >= budget) {
+                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 0, 2, 0u, sel_rem, tid);
+                n_at_select = ntot;
+            }
+            __syncthreads();
+        }
+        for (int d = spec ? 2 : 0; d < L; ++d) {
 #ifdef GRAFT_TREE_PROF
             long long tl0 = clock64();
 #endif
