@@ -787,7 +787,21 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         for (; rows_done < L; ++rows_done) lazy_score_row(p, sm, rows_done, root, tid, inflight);
     }
     if (!table_ok && tid == 0) sm.ent[0] = budget > 0 ? pack_entry(0.0f + sm.es[0], 1, 0, 0, sm.ei[0]) : 0ull;
+    // emission needs every node's child mask and the node count of every level: cleared here, filled for the nodes
+    // selected so far by warps 1..31 while warp 0 runs the sequential tail, and for the tail's nodes by warp 0
+    if (tid < kMaxL + 2) {
+        sm.lvl_count[tid] = 0;
+        sm.lvl_fill[tid] = 0;
+    }
+    for (int n = tid; n < nmax; n += TREE_THREADS) sm.chmask[n] = 0u;
     __syncthreads();
+    const int n_pre = table_ok ? n_gt : 0;  // nodes 0..n_pre are final before the tail starts
+    if (warp >= 1) {
+        for (int n = tid - 32; n <= n_pre; n += TREE_THREADS - 32) {
+            if (n > 0) atomicOr(&sm.chmask[sm.parent[n]], 1u << sm.cand[n]);
+            atomicAdd(&sm.lvl_count[sm.depth[n]], 1);
+        }
+    }
     if (warp == 0) {
         // Phase 2: exact sequential expansion.  Every step scans all frontier entries (one per selected node)
         // for the best under the full order, including the lexicographic rule for equal scores.
@@ -846,14 +860,14 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             }
             __syncwarp();
         }
+        for (int n = n_pre + 1 + lane; n <= n_sel; n += 32) {  // the tail's nodes
+            atomicOr(&sm.chmask[sm.parent[n]], 1u << sm.cand[n]);
+            atomicAdd(&sm.lvl_count[sm.depth[n]], 1);
+        }
         if (lane == 0) {
             sm.scal[1] = n_sel + 1;
             sm.scal[2] = st;
         }
-    }
-    if (tid < kMaxL + 2) {
-        sm.lvl_count[tid] = 0;
-        sm.lvl_fill[tid] = 0;
     }
     __syncthreads();
 
@@ -865,20 +879,18 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     // the child counts of level d-1, laid out in level order, are scanned; a node of level d lands at
     // (start of level d) + (children of earlier parents) + (selected siblings of lower rank).
     const int n_nodes = sm.scal[1];
-    for (int n = tid; n < nmax; n += TREE_THREADS) sm.chmask[n] = 0u;
-    __syncthreads();
-    for (int n = tid; n < n_nodes; n += TREE_THREADS) {
-        if (n > 0) atomicOr(&sm.chmask[sm.parent[n]], 1u << sm.cand[n]);
-        atomicAdd(&sm.lvl_count[sm.depth[n]], 1);
-    }
-    __syncthreads();
-    if (tid == 0) {
-        int acc = 0;
-        for (int d = 0; d <= L; ++d) {
-            sm.lvl_start[d] = acc;
-            acc += sm.lvl_count[d];
+    if (warp == 0) {  // starts of the levels 0..L: an exclusive scan of the counts (L <= 32: lane = level, and one more)
+        const int c0 = lane <= L ? sm.lvl_count[lane] : 0;
+        int incl = c0;
+#pragma unroll
+        for (int o2 = 1; o2 < 32; o2 <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
+            if (lane >= o2) incl += t;
         }
-        sm.canon[0] = 0;
+        if (lane <= L) sm.lvl_start[lane] = incl - c0;
+        const int below32 = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        if (lane == 0 && L == 32) sm.lvl_start[32] = below32;
+        if (lane == 0) sm.canon[0] = 0;
     }
     __syncthreads();
     for (int n = tid; n < n_nodes; n += TREE_THREADS) {
