@@ -447,3 +447,52 @@ def test_config_full_size_sampled(name, nseq):
     prod = out_p.cpu()
     for k in ("n_nodes", "budget", "status", "token", "parent", "depth", "position", "path_score", "mask"):
         assert np.array_equal(prod[k], gpu[k]), k
+
+
+# --------------------------------------------------------------------------- seeded sweep of shapes
+def _fuzz_cases():
+    rng = np.random.default_rng(20375)
+    cases = []
+    for i in range(14):
+        K = int(rng.choice([1, 2, 3, 5, 8, 13, 16, 27, 32]))
+        L = int(rng.choice([1, 2, 3, 7, 16, 24, 32]))
+        if L * K * K * 4 > 128 * 1024:
+            L = 16
+        V = int(rng.choice([K + 1, 97, 1000, 4099, 30011]))
+        V = max(V, K)
+        bstep = int(rng.choice([1, 3, 8, 16]))
+        bmin = int(rng.choice([0, 1, 4, 16]))
+        bmax = bmin + bstep * int(rng.integers(0, 30))
+        bmax = min(bmax, 1023)
+        m = int(rng.choice([4, 8, 20, 64, 132]))
+        cases.append(dict(batch=int(rng.integers(1, 6)), L=L, V=V, K=K, budget_min=bmin, budget_max=bmax,
+                          budget_step=bstep, m=m, hidden_dim=int(rng.choice([1, 7, 8, 33, 256])),
+                          logits_dtype=str(rng.choice(["f32", "bf16"])), hidden_dtype=str(rng.choice(["f32", "bf16"])),
+                          beta=float(rng.choice([0.0, 0.2, 1.5])), seed=5000 + i,
+                          fixed_budget=(None if rng.random() < 0.6 else int(rng.integers(0, bmax + 1)))))
+    return cases
+
+
+@pytest.mark.parametrize("kw", _fuzz_cases())
+@pytest.mark.parametrize("rows", [None, 1])
+def test_round_seeded_sweep_of_shapes(kw, rows):
+    """Odd sizes (K and L from 1 to 32, tiny vocabularies, m = 4, hidden width 1, budgets from 0 to ~500 on coarse
+    and fine grids), every one against the oracle; once with the library's split of the edge scores, once with all
+    depths but the first scored inside the tree kernel."""
+    w = gi.small(**kw)
+    g = _graft(w)
+    if rows is not None:
+        from paper_2608_20375_b200 import GraftError
+        try:
+            g.set_edge_rows(min(rows, w.L))
+        except GraftError:
+            g.destroy()
+            pytest.skip("the split is fixed for this shape")
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    assert stats["excused_tree"] + stats["excused_budget"] <= max(1, w.batch // 2), stats
+    compare_accept(oracle, gi, g, w, out, gpu)
+    g.destroy()
