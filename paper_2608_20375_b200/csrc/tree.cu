@@ -272,9 +272,8 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 __device__ __forceinline__ void lazy_issue_gather(const TreeParams& p, const TreeSmem& sm, int j, int root_token, int tid) {
     if (j >= p.L || lazy_neutral(p, j)) return;
     const int K = p.K, m = p.m, ld = m + 4, q4 = m / 4, n_par = j == 0 ? 1 : K;
-    const int total = (n_par + K + 1) * q4;
-    for (int i = tid; i < total; i += TREE_THREADS) {
-        const int r = i / q4, k4 = i - r * q4;
+    const int warp = tid >> 5, lane = tid & 31;
+    for (int r = warp; r <= n_par + K; r += TREE_THREADS / 32) {  // a warp per table row, a lane per 16 bytes
         const float* src;
         float* dst;
         if (r == n_par + K) {
@@ -286,7 +285,7 @@ __device__ __forceinline__ void lazy_issue_gather(const TreeParams& p, const Tre
             src = (r < n_par ? p.P : p.C) + (size_t)tok * m;
             dst = r < n_par ? sm.gP + (size_t)r * ld : sm.gC + (size_t)(r - n_par) * ld;
         }
-        cp_async16(smem_u32(dst + 4 * k4), src + 4 * k4);
+        for (int k4 = lane; k4 < q4; k4 += 32) cp_async16(smem_u32(dst + 4 * k4), src + 4 * k4);
     }
     cp_async_commit();
 }
