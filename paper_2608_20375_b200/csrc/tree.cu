@@ -542,6 +542,9 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             const int b0 = sm.lvl_start[d], b1 = sm.lvl_start[d + 1];
             if (b1 == b0) break;
             if (d >= rows_done) {  // the edge rows of this depth: scored now, never if the expansion stops above it
+                int alive = 0;  // (nor if no node of the level can still have a selected child)
+                for (int x = b0 + tid; x < b1; x += TREE_THREADS) alive |= sm.nkey[x] >= theta ? 1 : 0;
+                if (!__syncthreads_or(alive)) break;
                 lazy_score_row(p, sm, d, root, tid, inflight);
                 rows_done = d + 1;
             }
