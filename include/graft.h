@@ -132,7 +132,11 @@ graft_status graft_set_edge_rows(graft_ctx* ctx, int32_t rows);
 int32_t graft_edge_rows(const graft_ctx* ctx);
 
 /* Table precompute (same passage): d_out[v] = W e_v + b for one tower.  d_emb [V, E] (dtype as given),
- * d_W [m, E] fp32, d_b [m] fp32 or NULL, d_out [V, m] fp32.  fp32 accumulation.  Call once per tower. */
+ * d_W [m, E] fp32, d_b [m] fp32 or NULL, d_out [V, m] fp32.  fp32 accumulation.  Call once per tower.
+ * With bf16 embeddings (16-byte aligned, E a multiple of 8) the products run on the tensor cores: the embeddings are
+ * exact operands and W enters as three bf16 parts, so the result differs from the fp32 one only by the order of
+ * the additions; the first such call allocates scratch in the context (3 m E bf16 values and the GEMM's
+ * workspace; GRAFT_ERR_WORKSPACE if that fails).  This is the once-per-model setup step, not the round. */
 graft_status graft_tdes_precompute(graft_ctx* ctx, const void* d_emb, graft_dtype emb_dtype, int32_t E,
                                    const float* d_W, const float* d_b, float* d_out, void* stream);
 

@@ -1,33 +1,86 @@
-"""Build libgraft.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a."""
+"""Build libgraft.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
+
+Every source becomes an object under _build/ (rebuilt when it or one of its headers is newer) and the objects are
+linked into libgraft.so.  The table-precompute GEMM (csrc/s0_gemm.cu) is built from the CUTLASS / CuTe sm100
+templates; their headers come from a CUTLASS tree vendored in the Python environment (GRAFT_CUTLASS_DIR overrides).
+"""
 from __future__ import annotations
 
+import importlib.util
 import os
 import subprocess
 import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libgraft.so")
-SOURCES = ["api.cu", "vocab_pass.cu", "tdes.cu", "tree.cu"]
-HEADERS = ["common.cuh", "internal.h", "edge_score.cuh", "cosine.cuh", os.path.join("..", "..", "include", "graft.h")]
+GRAFT_H = os.path.join("..", "..", "include", "graft.h")
+ALL_HEADERS = ["common.cuh", "internal.h", "edge_score.cuh", "cosine.cuh", GRAFT_H]
+# source -> headers it depends on
+SOURCES = {
+    "api.cu": ALL_HEADERS,
+    "vocab_pass.cu": ALL_HEADERS,
+    "tdes.cu": ALL_HEADERS,
+    "tree.cu": ALL_HEADERS,
+    "s0_gemm.cu": ["internal.h", GRAFT_H],
+}
 # no --use_fast_math: the fp64 pieces (log-sum-exp fold, SABA) and the fp32 divisions must stay IEEE
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "-shared"]
+              "-Xcompiler", "-fPIC"]
+
+
+def cutlass_dir() -> str:
+    """Root of a CUTLASS tree with include/ and tools/util/include/ (version 4.x: sm100 collective builders)."""
+    cands = []
+    if os.environ.get("GRAFT_CUTLASS_DIR"):
+        cands.append(os.environ["GRAFT_CUTLASS_DIR"])
+    for pkg, sub in (("flashinfer", os.path.join("data", "cutlass")), ("tilelang", os.path.join("3rdparty", "cutlass"))):
+        spec = importlib.util.find_spec(pkg)
+        if spec and spec.submodule_search_locations:
+            cands.append(os.path.join(list(spec.submodule_search_locations)[0], sub))
+    for c in cands:
+        if os.path.exists(os.path.join(c, "include", "cutlass", "gemm", "collective", "builders", "sm100_umma_builder.inl")):
+            return c
+    raise RuntimeError("no CUTLASS tree with the sm100 builders found (set GRAFT_CUTLASS_DIR)")
+
+
+def _stale(target: str, deps: list[str]) -> bool:
+    if not os.path.exists(target):
+        return True
+    t = os.path.getmtime(target)
+    return any(os.path.getmtime(d) > t for d in deps)
+
+
+def _obj(src: str) -> str:
+    return os.path.join(OBJ, src.replace(".cu", ".o"))
 
 
 def needs_build() -> bool:
-    if not os.path.exists(LIB):
-        return True
-    t = os.path.getmtime(LIB)
-    return any(os.path.getmtime(os.path.join(CSRC, f)) > t for f in SOURCES + HEADERS)
+    for src, hdrs in SOURCES.items():
+        if _stale(_obj(src), [os.path.join(CSRC, src)] + [os.path.join(CSRC, h) for h in hdrs]):
+            return True
+    return _stale(LIB, [_obj(s) for s in SOURCES])
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    if force or needs_build():
-        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-              [os.path.join(CSRC, f) for f in SOURCES] + ["-o", LIB, "-lcudart"]
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    os.makedirs(OBJ, exist_ok=True)
+    inc = ["-I", os.path.join(HERE, "..", "include")]
+    for src, hdrs in SOURCES.items():
+        deps = [os.path.join(CSRC, src)] + [os.path.join(CSRC, h) for h in hdrs]
+        if not (force or _stale(_obj(src), deps)):
+            continue
+        extra = []
+        if src == "s0_gemm.cu":
+            cut = cutlass_dir()
+            extra = ["--expt-relaxed-constexpr", "-diag-suppress", "20012", "-I", os.path.join(cut, "include"),
+                     "-I", os.path.join(cut, "tools", "util", "include")]
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + inc + extra + \
+              ["-c", os.path.join(CSRC, src), "-o", _obj(src)]
         subprocess.check_call(cmd)
+    if force or _stale(LIB, [_obj(s) for s in SOURCES]):
+        subprocess.check_call([nvcc, "-shared", "-o", LIB] + [_obj(s) for s in SOURCES] + ["-lcudart"])
     return LIB
 
 

@@ -152,6 +152,8 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     ctx->w_esort = (float*)(base + o_es);
     ctx->w_eidx = (uint8_t*)(base + o_ei);
     ctx->d_u = (float*)(base + o_u);
+    ctx->s0_scratch = nullptr;
+    ctx->s0_scratch_bytes = 0;
     ctx->hist_w = 0;
     ctx->hist_window = nullptr;
     ctx->hist_count = nullptr;
@@ -174,6 +176,7 @@ graft_status graft_destroy(graft_ctx* ctx) {
         if (ex->d_out) cudaFree(ex->d_out);
         delete ex;
     }
+    if (ctx->s0_scratch) cudaFree(ctx->s0_scratch);
     if (ctx->ws) cudaFree(ctx->ws);
     delete ctx;
     return GRAFT_OK;
@@ -242,6 +245,32 @@ graft_status graft_tdes_precompute(graft_ctx* ctx, const void* d_emb, graft_dtyp
                                    const float* d_W, const float* d_b, float* d_out, void* stream) {
     if (!ctx || !d_emb || !d_W || !d_out || E < 1) return GRAFT_ERR_INVALID_ARG;
     if (emb_dtype != GRAFT_F32 && emb_dtype != GRAFT_BF16) return GRAFT_ERR_INVALID_ARG;
+    // bf16 embeddings: the tensor cores (the embeddings are exact operands, W goes in as three bf16 parts); its
+    // scratch is allocated on the first such call (this is the once-per-model setup step, not the round)
+    if (emb_dtype == GRAFT_BF16) {
+        const size_t need = s0_tc_scratch_bytes(ctx->cfg.V, E, ctx->cfg.m);
+        if (need > 0) {
+            if (ctx->s0_scratch_bytes < need) {
+                if (ctx->s0_scratch) cudaFree(ctx->s0_scratch);
+                ctx->s0_scratch = nullptr;
+                ctx->s0_scratch_bytes = 0;
+                if (cudaMalloc(&ctx->s0_scratch, need) != cudaSuccess) {
+                    cudaGetLastError();
+                    return GRAFT_ERR_WORKSPACE;
+                }
+                ctx->s0_scratch_bytes = need;
+            }
+            int n = 0;
+            const cudaError_t e = s0_tc_launch(d_emb, ctx->cfg.V, E, ctx->cfg.m, d_W, d_b, d_out, ctx->s0_scratch, &n,
+                                               (cudaStream_t)stream);
+            ctx->launches += (uint64_t)n;
+            if (e == cudaSuccess) return GRAFT_OK;
+            if (e != cudaErrorNotSupported) {
+                cudaGetLastError();
+                return GRAFT_ERR_CUDA;
+            }
+        }
+    }
     if (tdes_precompute_launch(ctx, d_emb, emb_dtype, E, d_W, d_b, d_out, (cudaStream_t)stream) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     return GRAFT_OK;

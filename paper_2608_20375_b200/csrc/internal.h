@@ -81,6 +81,9 @@ struct graft_ctx {
     double* w_cos;                // [max_batch, L] adjacent-position cosines (Eq. 15)
     int32_t* w_errflag;           // [1] device-side internal error flag
     graft::VpPlan vp_plan;
+    // scratch of the tensor-core table precompute (allocated on its first use: three bf16 copies of W, GEMM workspace)
+    void* s0_scratch;
+    size_t s0_scratch_bytes;
     // host-buffer staging (allocated on first use of graft_build_trees_host)
     void* stage;
     size_t stage_bytes;
@@ -123,6 +126,10 @@ int vp_merge_max_shards();
 
 cudaError_t tdes_precompute_launch(graft_ctx* ctx, const void* d_emb, graft_dtype dt, int E, const float* d_W,
                                    const float* d_b, float* d_out, cudaStream_t st);
+// S0 on the tensor cores (bf16 embeddings): three bf16 GEMMs with fp32 accumulation (csrc/s0_gemm.cu)
+size_t s0_tc_scratch_bytes(int V, int E, int m);
+cudaError_t s0_tc_launch(const void* d_emb, int V, int E, int m, const float* d_W, const float* d_b, float* d_out,
+                         void* d_scratch, int* launches, cudaStream_t st);
 cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                               const int32_t* d_root_token, const int32_t* d_row_status, float* d_edge,
                               float* d_esort, uint8_t* d_eidx, int rows, cudaStream_t st);  // depths [0, rows)

@@ -120,9 +120,16 @@ def test_vocab_pass_is_reproducible_and_counters_reset():
 
 
 # --------------------------------------------------------------------------- TDES
-def test_tdes_precompute_against_oracle():
-    V, E, m, L = 777, 200, 24, 4
-    wts = gi.tdes_weights(V, E, m, L, seed=5, emb_dtype="bf16")
+@pytest.mark.parametrize("V,E,m,emb_dtype", [
+    (777, 200, 24, "bf16"),     # tensor-core path, ragged in every dimension
+    (4099, 512, 128, "bf16"),   # tensor-core path, several tiles
+    (300, 64, 4, "bf16"),       # tensor-core path, the narrowest scorer
+    (500, 100, 16, "bf16"),     # E not a multiple of 8: the FMA kernel
+    (777, 200, 24, "f32"),      # fp32 embeddings: the FMA kernel
+])
+def test_tdes_precompute_against_oracle(V, E, m, emb_dtype):
+    L = 4
+    wts = gi.tdes_weights(V, E, m, L, seed=5, emb_dtype=emb_dtype)
     w = gi.small(V=V, m=m, L=L)
     g = _graft(w)
     out = torch.empty((V, m), dtype=torch.float32, device="cuda")
@@ -131,6 +138,7 @@ def test_tdes_precompute_against_oracle():
         torch.cuda.synchronize()
         want = oracle.tdes_tables(wts["emb"], wts[Wk].numpy(), None if bk is None else wts[bk].numpy())
         np.testing.assert_allclose(out.cpu().numpy(), want, rtol=1e-5, atol=1e-5)
+    g.destroy()
 
 
 @pytest.mark.parametrize("K,L,m,beta,root_edge", [(4, 4, 16, 0.2, 1), (32, 16, 128, 0.2, 1), (7, 3, 36, 0.7, 0),
