@@ -67,6 +67,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     os.makedirs(OBJ, exist_ok=True)
     inc = ["-I", os.path.join(HERE, "..", "include")]
+    cmds = []
     for src, hdrs in SOURCES.items():
         deps = [os.path.join(CSRC, src)] + [os.path.join(CSRC, h) for h in hdrs]
         if not (force or _stale(_obj(src), deps)):
@@ -76,9 +77,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
             cut = cutlass_dir()
             extra = ["--expt-relaxed-constexpr", "-diag-suppress", "20012", "-I", os.path.join(cut, "include"),
                      "-I", os.path.join(cut, "tools", "util", "include")]
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + inc + extra + \
-              ["-c", os.path.join(CSRC, src), "-o", _obj(src)]
-        subprocess.check_call(cmd)
+        cmds.append([nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + inc + extra +
+                    ["-c", os.path.join(CSRC, src), "-o", _obj(src)])
+    procs = [subprocess.Popen(c) for c in cmds]  # the sources compile side by side
+    failed = [c for c, pr in zip(cmds, procs) if pr.wait() != 0]
+    if failed:
+        raise subprocess.CalledProcessError(1, failed[0])
     if force or _stale(LIB, [_obj(s) for s in SOURCES]):
         subprocess.check_call([nvcc, "-shared", "-o", LIB] + [_obj(s) for s in SOURCES] + ["-lcudart"])
     return LIB
