@@ -402,6 +402,8 @@ graft_status graft_accept(graft_ctx* ctx, int32_t batch, const graft_tree_out* t
     return GRAFT_OK;
 }
 
+static_assert(sizeof(graft_vocab_partial) == 280, "the Python binding gathers partials as 280-byte records");
+
 graft_status graft_vocab_pass_partial(graft_ctx* ctx, int32_t batch, const void* d_logits_shard,
                                       graft_vocab_partial* d_out, void* stream) {
     if (!ctx || !d_logits_shard || !d_out) return GRAFT_ERR_INVALID_ARG;
