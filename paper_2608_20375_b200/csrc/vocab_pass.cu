@@ -971,7 +971,7 @@ __global__ void __launch_bounds__(128) vocab_merge_kernel(const MergeParams p) {
 }  // namespace
 
 // ---- host side ----------------------------------------------------------------------------------
-static size_t vp_smem_bytes(int stages, int n_cmax, bool bf16) {
+static size_t vp_smem_bytes(int stages, int n_cmax) {
     return (size_t)stages * TILE + 24 * sizeof(uint64_t) + sizeof(VpShared) + (size_t)kVpBufs * n_cmax * 2 + 16;
 }
 
@@ -996,9 +996,9 @@ VpPlan vp_make_plan(const graft_config& cfg, int num_sms, int batch) {
     pl.max_seg_tiles = (int)((seg_elems * esz + TILE - 1) / TILE) + 1;
     const size_t budget = 224 * 1024;  // one CTA per SM
     int stages = 6;
-    while (stages > 2 && vp_smem_bytes(stages, pl.max_seg_tiles * NT, bf16) > budget) --stages;
+    while (stages > 2 && vp_smem_bytes(stages, pl.max_seg_tiles * NT) > budget) --stages;
     pl.stages = stages;
-    pl.smem_bytes = vp_smem_bytes(stages, pl.max_seg_tiles * NT, bf16);
+    pl.smem_bytes = vp_smem_bytes(stages, pl.max_seg_tiles * NT);
     return pl;
 }
 
