@@ -172,9 +172,10 @@ __device__ __forceinline__ uint64_t pack_entry(float score, int child_depth, int
 // Does the prefix of node n1 come before the prefix of node n2 in lexicographic order of candidate ranks?
 // Both at the same depth, n1 != n2.
 __device__ __forceinline__ bool path_less(const TreeSmem& sm, int n1, int n2) {
-    while (sm.parent[n1] != sm.parent[n2]) {
+    for (int step = 0; step < kMaxL && sm.parent[n1] != sm.parent[n2]; ++step) {  // (depth <= L: the bound is never hit)
         n1 = sm.parent[n1];
         n2 = sm.parent[n2];
+        if (n1 < 0 || n2 < 0) return n1 < n2;
     }
     return sm.cand[n1] < sm.cand[n2];
 }
@@ -982,7 +983,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             if (i < n_nodes) {
                 int w = W - 1;
                 uint32_t bits = 0u;
-                for (int a = i; a >= 0; a = sm.cparent[a]) {
+                int steps = 0;  // a node has at most L ancestors: the bound keeps the walk finite whatever the arrays hold
+                for (int a = i; a >= 0 && a < nmax && steps <= L; a = sm.cparent[a], ++steps) {
                     const int wa = a >> 5;
                     while (w > wa) {
                         row[w] = bits;
