@@ -364,7 +364,7 @@ graft_status graft_build_trees(graft_ctx* ctx, int32_t batch, const void* d_logi
     int32_t* ids = out->d_topk_id ? out->d_topk_id : ctx->w_topk_id;
     float* lps = out->d_topk_lp ? out->d_topk_lp : ctx->w_topk_lp;
     float* lse = out->d_lse ? out->d_lse : ctx->w_lse;
-    float* edge = out->d_edge ? out->d_edge : ctx->w_edge;
+    float* edge = out->d_edge;  // NULL: the edge kernel writes only the sorted rows the tree kernel reads
 
     if (ev) cudaEventRecord(ev[0], st);
     if (vp_launch(ctx, batch, d_logits, ids, lps, lse, ctx->w_row_status, use_saba ? d_hidden : nullptr, ctx->w_cos,

@@ -92,6 +92,8 @@ struct EdgeParams {
     int root_edge;
 };
 
+// WRITE_EDGE: also write the unsorted scores (the caller asked for the array); the tree kernel reads only the sorted rows
+template <bool WRITE_EDGE>
 __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
     extern __shared__ __align__(16) float smem[];
     pdl_launch_dependents();  // the tree kernel may move in as SMs free up; it waits for this grid before it reads
@@ -103,7 +105,6 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_par = (j == 0) ? 1 : K;
     const size_t row = (size_t)b * p.L + j;
-    float* out = p.edge + row * K * K;
     float* outs = p.esort + row * K * K;
     uint8_t* outi = p.eidx + row * K * K;
     const int32_t* ids = p.topk_id + row * K;
@@ -117,7 +118,7 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
         for (int i = threadIdx.x; i < K * K; i += 256) {
             int par = i / K, c = i % K;
             const float v = (bad || par >= n_par) ? 0.f : lps[c];
-            out[i] = v;
+            if (WRITE_EDGE) p.edge[row * K * K + i] = v;
             outs[i] = v;
             outi[i] = (uint8_t)c;
         }
@@ -168,7 +169,7 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
         edge_row_finish(par < n_par ? part + (size_t)par * K : nullptr, lps, p.scale, p.beta, K, wsc[warp], lane, val,
                         rank);
         if (lane < K) {
-            out[(size_t)par * K + lane] = val;
+            if (WRITE_EDGE) p.edge[(row * K + par) * K + lane] = val;
             outs[(size_t)par * K + rank] = val;
             outi[(size_t)par * K + rank] = (uint8_t)lane;
         }
@@ -194,7 +195,10 @@ size_t tdes_edges_smem(const graft_config& cfg) {
 }
 
 cudaError_t tdes_edges_configure(const graft_config& cfg) {
-    return cudaFuncSetAttribute(tdes_edges_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(tdes_edges_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)tdes_edges_smem(cfg));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(tdes_edges_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)tdes_edges_smem(cfg));
 }
 
@@ -221,7 +225,8 @@ cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_i
     p.beta = ctx->tdes_set ? cfg.beta : 0.0f;
     p.root_edge = cfg.root_edge;
     p.rows = rows;
-    const cudaError_t e = launch_pdl(tdes_edges_kernel, dim3(batch * rows), dim3(256), tdes_edges_smem(cfg), st, p);
+    const cudaError_t e = launch_pdl(d_edge ? tdes_edges_kernel<true> : tdes_edges_kernel<false>, dim3(batch * rows),
+                                     dim3(256), tdes_edges_smem(cfg), st, p);
     ctx->launches += 1;
     return e != cudaSuccess ? e : cudaGetLastError();
 }
