@@ -396,6 +396,91 @@ def run_reference(args):
     }))
 
 
+def run_overlap(args):
+    """--overlap-verifier-ms T: the batch as two micro-batches with contexts and streams of their own, a stub verifier
+    (a chain of GEMMs of about T ms) between build and walk; sequential schedule against overlapped one, on one GPU.
+    Prints its own JSON line (not the benchmark's metric)."""
+    from paper_2608_20375_b200 import Graft, MicroBatch, run_rounds, join
+
+    w = gi.WORKLOADS[args.workload]
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    n_micro, mb_batch = 2, w.batch // 2
+    dt = {"f32": 0, "bf16": 1}
+    tb = gi.tdes_tables(w)
+    P, Ct, u = tb["P"].to(dev), tb["C"].to(dev), tb["u"].to(dev)
+    micro = []
+    for i in range(n_micro):
+        g = Graft(w.V, w.L, w.K, w.m, w.hidden_dim, mb_batch, w.budget_min, w.budget_max, w.budget_step, w.beta, 1,
+                  dt[w.logits_dtype], dt[w.hidden_dtype])
+        g.set_tdes_tables(P, Ct, u, tb["s"])
+        g.set_saba(**gi.saba_defaults(w))
+        micro.append(MicroBatch(g, mb_batch, w.L))
+    n_buf = 4  # input sets per micro-batch: 8 x 156 MB of logits in rotation (> L2)
+    sets = [[{k: (v.to(dev) if torch.is_tensor(v) else v)
+              for k, v in _host_inputs(w, (i * n_buf + k) * mb_batch, (i * n_buf + k + 1) * mb_batch, 1)[0].items()}
+             for k in range(n_buf)] for i in range(n_micro)]
+    tn = torch.zeros((mb_batch, micro[0].graft.nmax), dtype=torch.int32, device=dev)
+    a = torch.randn(4096, 4096, device=dev, dtype=torch.bfloat16)
+    # size the stub: GEMMs of 4096^3 until one verification takes about the requested time
+    def chain(n):
+        y = a
+        for _ in range(n):
+            y = torch.mm(y, a)
+        return y
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    chain(8)
+    torch.cuda.synchronize()
+    e0.record()
+    chain(32)
+    e1.record()
+    torch.cuda.synchronize()
+    per_gemm = e0.elapsed_time(e1) / 32
+    n_gemm = max(1, int(round(args.overlap_verifier_ms / per_gemm)))
+
+    def draft(i, r):
+        return sets[i][r % n_buf]
+
+    def verify(i, r, out):
+        chain(n_gemm)
+        return tn
+
+    def build_only(i, r, out):
+        return tn
+
+    def timed(fn_verify, overlap, rounds):
+        run_rounds(micro, 8, draft, fn_verify, overlap=overlap)
+        join(micro)
+        torch.cuda.synchronize()
+        e0.record()
+        run_rounds(micro, rounds, draft, fn_verify, overlap=overlap)
+        join(micro)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / rounds
+
+    rounds = args.steps
+    res = {
+        "build_walk_only_ms": timed(build_only, False, rounds),
+        "sequential_ms": timed(verify, False, rounds),
+        "overlapped_ms": timed(verify, True, rounds),
+    }
+    e0.record()
+    for _ in range(rounds):
+        chain(n_gemm)
+        chain(n_gemm)
+    e1.record()
+    torch.cuda.synchronize()
+    res["verifier_only_ms"] = e0.elapsed_time(e1) / rounds
+    print(json.dumps({
+        "kind": "micro-batch overlap (two micro-batches, one round of each per step)", "workload": args.workload,
+        "micro_batches": n_micro, "batch_per_micro_batch": mb_batch, "rounds": rounds,
+        "stub_verifier": f"{n_gemm} bf16 GEMMs of 4096^3 per micro-batch round ({per_gemm * n_gemm:.3f} ms alone)",
+        **{k: round(v, 5) for k, v in res.items()},
+        "overlapped_over_sequential": round(res["overlapped_ms"] / res["sequential_ms"], 4),
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -409,7 +494,14 @@ def main():
     ap.add_argument("--cuda-graph", action="store_true", help="replay captured rounds in the timed loop")
     ap.add_argument("--edge-rows", type=int, default=None,
                     help="depths scored ahead of the expansion (default: the library's)")
+    ap.add_argument("--overlap-verifier-ms", type=float, default=None,
+                    help="instead of the benchmark: two micro-batches on two streams around a stub verifier of this "
+                         "duration, sequential against overlapped schedule")
     args = ap.parse_args()
+    if args.overlap_verifier_ms is not None and args.impl == "graft":
+        args.steps = 200 if args.steps is None else args.steps
+        run_overlap(args)
+        return
     if args.impl == "reference":
         args.steps = 10 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup

@@ -6,3 +6,4 @@ from .binding import (  # noqa: F401
 )
 from .shard import shard_range  # noqa: F401
 from .vocab_parallel import vocab_range, gather_partials, vocab_pass_parallel  # noqa: F401
+from .pipeline import MicroBatch, run_rounds, join  # noqa: F401

@@ -129,3 +129,87 @@ def test_round_in_a_cuda_graph():
             for k in ("n_nodes", "budget", "status", "token", "parent", "depth", "position", "path_score", "mask"):
                 assert np.array_equal(got[k], eager[i][k]), (rep, i, k)
     g.destroy()
+
+
+def test_micro_batches_on_streams_of_their_own():
+    """Two micro-batches, each with its own context and stream, so that one's tree building overlaps the other's
+    (stub) verification: every round's results are the sequential schedule's, bit for bit, and the sequential
+    schedule's first and last rounds are the oracle's."""
+    from paper_2608_20375_b200.pipeline import MicroBatch, join, run_rounds
+
+    rounds, hist_w, n_micro = 5, 3, 2
+    base = dict(batch=6, L=8, V=5000, K=8, budget_min=16, budget_max=96, budget_step=16, m=32, hidden_dim=64,
+                logits_dtype="bf16", hidden_dtype="bf16")
+    w0 = gi.small(**base)
+    keys = ("n_nodes", "budget", "status", "token", "parent", "depth", "position", "path_score", "mask", "topk_id",
+            "topk_lp", "lse", "edge", "state")
+    ctxs = [_graft(w0) for _ in range(n_micro)]
+    tb, saba_kw = ctxs[0][1], ctxs[0][2]
+    hist_bufs = []
+    for g, *_ in ctxs:
+        bufs = (torch.zeros((w0.batch, hist_w), dtype=torch.int32, device="cuda"),
+                torch.zeros(w0.batch, dtype=torch.int32, device="cuda"),
+                torch.zeros(w0.batch, dtype=torch.float32, device="cuda"))
+        g.set_hist_window(hist_w, *bufs)
+        hist_bufs.append(bufs)
+    micro = [MicroBatch(g, w0.batch, w0.L, out=g.alloc_out(w0.batch, debug=True)) for g, *_ in ctxs]
+    ws = [[gi.small(**base, seed=5200 + 10 * i + r) for r in range(rounds)] for i in range(n_micro)]
+    xs = [[gi.batch_inputs(w) for w in row] for row in ws]
+    dev_x = [[{k: x[k].cuda() for k in ("logits", "hidden", "root_token", "prefix_len")} for x in row] for row in xs]
+    burn = torch.randn(1024, 1024, device="cuda")
+    tn_dev = {}   # (i, r) -> target ids, fixed by the sequential pass
+    record = {}   # schedule -> (i, r) -> outputs
+    rng = np.random.default_rng(11)
+
+    def draft(i, r):
+        return dict(dev_x[i][r], hist=hist_bufs[i][2])
+
+    def run(schedule, overlap):
+        for bufs in hist_bufs:
+            for t in bufs:
+                t.zero_()
+        record[schedule] = {}
+
+        def verify(i, r, out):
+            y = burn
+            for _ in range(4):  # stands in for the target model's forward pass on this stream
+                y = torch.mm(y, burn) * 1e-3
+            if (i, r) not in tn_dev:  # sequential pass only: choose the target ids from the tree just built
+                torch.cuda.current_stream().synchronize()
+                t = out.cpu()
+                tn = np.stack([_target_next_from_tree(rng, {k: t[k][b] for k in ("n_nodes", "token", "parent")},
+                                                      w0.V) for b in range(w0.batch)])
+                tn_dev[(i, r)] = torch.from_numpy(tn).cuda()
+            return tn_dev[(i, r)]
+
+        def after(i, r, mb):
+            snap = {k: getattr(mb.out, k).clone() for k in keys}
+            snap["accept_len"] = mb.accept_len.clone()
+            snap["hist"] = hist_bufs[i][2].clone()
+            record[schedule][(i, r)] = snap
+
+        run_rounds(micro, rounds, draft, verify, overlap=overlap, after_round=after)
+        join(micro)
+        torch.cuda.synchronize()
+
+    run("sequential", False)
+    run("overlapped", True)
+    for key, snap in record["sequential"].items():
+        for k, v in snap.items():
+            assert torch.equal(v, record["overlapped"][key][k]), (key, k)
+    assert max(int(s["accept_len"].max()) for s in record["sequential"].values()) >= 2
+    # the sequential schedule against the oracle: the first round (no history yet) and the last (hist from the device)
+    for i in range(n_micro):
+        for r in (0, rounds - 1):
+            snap = record["sequential"][(i, r)]
+            x = dict(xs[i][r])
+            prev = record["sequential"][(i, r - 1)]["hist"] if r > 0 else torch.zeros(w0.batch)
+            x["hist"] = prev.cpu().float()
+            orc = oracle_round(oracle, ws[i][r], x, tb, saba_kw)
+            gpu = {k: snap[k].cpu().numpy() for k in keys}
+            gpu["mask"] = gpu["mask"].view("uint32")
+            stats = compare_round(oracle, ws[i][r], x, tb, saba_kw, gpu, orc)
+            assert stats["excused_tree"] == 0 and stats["excused_budget"] == 0, stats
+    for g, *_ in ctxs:
+        g.set_hist_window(0)
+        g.destroy()
