@@ -73,7 +73,7 @@ C5 = Workload("C5", 128, 16, 151936, 32, 4096, "bf16", "bf16", 16, 512, target_m
 M = Workload("M", 64, 16, 151936, 32, 4096, "bf16", "bf16", 16, 512, target_mode="decay", seed=20380)
 WORKLOADS = {w.name: w for w in (C1, C2, C3, C4, C5, M)}
 
-_TAGS = {"logits": 1, "hidden": 2, "boost_ids": 3, "boost_h": 4, "tables": 5, "scalars": 6, "target": 7, "emb": 8}
+_TAGS = {"logits": 1, "hidden": 2, "boost_ids": 3, "boost_h": 4, "tables": 5, "scalars": 6, "target": 7, "emb": 8, "traces": 9}
 
 
 def _rng(seed: int, tag: str, b: int = 0) -> np.random.Generator:
@@ -207,6 +207,44 @@ def target_next_from_depth(y: np.ndarray, depth: np.ndarray) -> np.ndarray:
     ok = d >= 0
     out[ok] = y[d[ok]]
     return out
+
+
+def tdes_traces(V: int, L: int, K: int, n_groups: int, n_pairs: int, n_edges: int, seed: int,
+                pos_rate: float = 0.15) -> dict:
+    """Synthetic TDES training traces (the paper's come from target-model runs that are not available).
+
+    Token ids are Zipf-distributed over a random permutation of the vocabulary (a few hot tokens, a long tail), depths
+    uniform in 1..L.  groups: a parent, a depth, K distinct children, their draft log-probabilities (descending, as
+    top-K candidates are) and target logits ~ N(0, 2^2); pairs: a compatible edge and an alternative that keeps
+    either its child (wrong parent) or its parent (competing child), half each; edges: (p, c, d, y) with about
+    `pos_rate` positives."""
+    g = _rng(seed, "traces")
+    perm = g.permutation(V)
+    w = 1.0 / np.arange(1, V + 1, dtype=np.float64) ** ZIPF_S
+    cdf = np.cumsum(w / w.sum())
+
+    def tokens(shape):
+        return perm[np.minimum(np.searchsorted(cdf, g.random(shape)), V - 1)].astype(np.int32)
+
+    child = np.empty((n_groups, K), np.int32)
+    for i in range(n_groups):  # K distinct children per group
+        got = np.unique(tokens(4 * K))
+        while got.size < K:
+            got = np.unique(np.concatenate([got, tokens(4 * K)]))
+        child[i] = g.permutation(got)[:K]
+    gaps = g.exponential(0.7, size=(n_groups, K)).astype(np.float32)
+    logq = -np.cumsum(gaps, axis=1, dtype=np.float32)
+    groups = dict(parent=tokens(n_groups), depth=g.integers(1, L + 1, n_groups).astype(np.int32), child=child,
+                  logq=logq.astype(np.float32), ztgt=(2.0 * g.standard_normal((n_groups, K))).astype(np.float32))
+    pos = np.stack([tokens(n_pairs), tokens(n_pairs), g.integers(1, L + 1, n_pairs).astype(np.int32)], axis=1)
+    neg = pos.copy()
+    swap_parent = g.random(n_pairs) < 0.5
+    neg[swap_parent, 0] = tokens(int(swap_parent.sum()))
+    neg[~swap_parent, 1] = tokens(int((~swap_parent).sum()))
+    pairs = np.concatenate([pos, neg], axis=1).astype(np.int32)
+    edges = np.stack([tokens(n_edges), tokens(n_edges), g.integers(1, L + 1, n_edges).astype(np.int32),
+                      (g.random(n_edges) < pos_rate).astype(np.int32)], axis=1).astype(np.int32)
+    return dict(groups=groups, pairs=pairs, edges=edges)
 
 
 def small(name: str = "T", **kw) -> Workload:

@@ -1,6 +1,6 @@
 """CPU oracle for the GRAFT draft-tree round -- TEST INFRASTRUCTURE, not product code.
 
-Thin ctypes marshalling around ``graft_oracle.c`` (plain C, fp64; each C function cites the
+Thin ctypes marshalling around ``graft_oracle.c`` and ``tdes_train_oracle.c`` (plain C, fp64; each C function cites the
 passage of the paper it restates).  Only the tests, the smoke check and the benchmark's
 CPU-baseline leg may import this package; the CUDA library never does, and this package never
 imports the CUDA package.  ``build()`` compiles the C file with gcc next to itself.
@@ -16,6 +16,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "graft_oracle.c")
+_SRCS = [_SRC, os.path.join(_HERE, "tdes_train_oracle.c")]
 _LIB = os.path.join(_HERE, "libgraft_oracle.so")
 _lib = None
 
@@ -25,9 +26,9 @@ ST_BAD_LOGITS, ST_TAU_CLAMPED, ST_FRONTIER_EMPTY = 1, 2, 4
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (no fast-math: fp64 semantics must be the plain ones)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(f) for f in _SRCS):
         subprocess.check_call(
-            ["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-ffp-contract=off", "-o", _LIB, _SRC, "-lm"]
+            ["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-ffp-contract=off", "-o", _LIB, *_SRCS, "-lm"]
         )
     return _LIB
 
@@ -206,6 +207,47 @@ def hist_update(a_hist, w):
     f = lib().oracle_hist_update
     f.restype = C.c_double
     return float(f(_p(a), int(a.size), int(w)))
+
+
+class _TdesLossCfg(C.Structure):
+    _fields_ = [("gamma", C.c_double), ("w1", C.c_double), ("lambda_kl", C.c_double), ("lambda_pair", C.c_double),
+                ("lambda_bce", C.c_double)]
+
+
+def tdes_loss(P, Ctab, u, s, groups, pairs, edges, gamma, w1, lambda_kl, lambda_pair, lambda_bce, grad=True):
+    """TDES training objective and its gradients (Eq. 7-12).
+
+    groups: dict(parent [G], depth [G], child [G,K], logq [G,K], ztgt [G,K]); pairs [N,6] = (p+, c+, d+, p-, c-, d-);
+    edges [N,4] = (p, c, d, y).  Returns dict(loss [4] = KL, pair, BCE, total; gP, gC, gu, gs in fp64)."""
+    P = np.ascontiguousarray(P, dtype=np.float32)
+    Ctab = np.ascontiguousarray(Ctab, dtype=np.float32)
+    u = np.ascontiguousarray(u, dtype=np.float32)
+    V, m = P.shape
+    L = u.shape[0]
+    gp = np.ascontiguousarray(groups["parent"], dtype=np.int32)
+    gd = np.ascontiguousarray(groups["depth"], dtype=np.int32)
+    gc = np.ascontiguousarray(groups["child"], dtype=np.int32)
+    gc = gc.reshape(gp.size, -1) if gp.size else gc.reshape(0, 1)
+    K = gc.shape[1]
+    gq = np.ascontiguousarray(groups["logq"], dtype=np.float32)
+    gz = np.ascontiguousarray(groups["ztgt"], dtype=np.float32)
+    pairs = np.ascontiguousarray(pairs, dtype=np.int32).reshape(-1, 6)
+    edges = np.ascontiguousarray(edges, dtype=np.int32).reshape(-1, 4)
+    for ids in (gp, gc, pairs[:, [0, 1, 3, 4]], edges[:, :2]):
+        if ids.size and (ids.min() < 0 or ids.max() >= V):
+            raise ValueError("token id out of range")
+    cfg = _TdesLossCfg(gamma, w1, lambda_kl, lambda_pair, lambda_bce)
+    loss = np.zeros(4, np.float64)
+    out = {"loss": loss}
+    if grad:
+        out.update(gP=np.zeros((V, m)), gC=np.zeros((V, m)), gu=np.zeros((L, m)), gs=np.zeros(1))
+    pp = (lambda k: _p(out[k])) if grad else (lambda k: None)
+    rc = lib().oracle_tdes_loss(_p(P), _p(Ctab), _p(u), C.c_double(s), V, L, m, K, int(gp.size), _p(gp), _p(gd), _p(gc),
+                                _p(gq), _p(gz), int(pairs.shape[0]), _p(pairs), int(edges.shape[0]), _p(edges),
+                                C.byref(cfg), _p(loss), pp("gP"), pp("gC"), pp("gu"), pp("gs"))
+    if rc != 0:
+        raise ValueError(f"oracle_tdes_loss failed ({rc})")
+    return out
 
 
 def replay_check(edge, n_nodes, parent, cand, depth, eps):
