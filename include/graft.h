@@ -223,6 +223,50 @@ graft_status graft_accept(graft_ctx* ctx, int32_t batch, const graft_tree_out* t
  * Host-only call; the buffers are borrowed until it is called again or the context is destroyed. */
 graft_status graft_set_hist_window(graft_ctx* ctx, int32_t w, int32_t* d_window, int32_t* d_count, float* d_hist);
 
+/* TDES training objective, forward and backward (Sec. 3.2 "Training", Eq. 7-12), on traces resident on the device.
+ * Every pointer of graft_tdes_traces is a DEVICE pointer (borrowed for the call); a list with n = 0 may be NULL.
+ *   groups (distribution level, Eq. 7-9): d_g_parent [n_groups] parent token, d_g_depth [n_groups] depth d in 1..L,
+ *     d_g_child [n_groups, K] the K children C_{p,d} (K = cfg.K), d_g_logq [n_groups, K] draft log q_d(c),
+ *     d_g_ztgt [n_groups, K] target-model logits z_tgt[p, c];
+ *   pairs (Eq. 10): d_pairs [n_pairs, 6] = (p+, c+, d+, p-, c-, d-), a target-compatible edge and an alternative;
+ *   edges (Eq. 11): d_edges [n_edges, 4] = (p, c, d, y), y = 1 when c is the target's next token under p. */
+typedef struct graft_tdes_traces {
+    int32_t n_groups;
+    const int32_t* d_g_parent;
+    const int32_t* d_g_depth;
+    const int32_t* d_g_child;
+    const float* d_g_logq;
+    const float* d_g_ztgt;
+    int32_t n_pairs;
+    const int32_t* d_pairs;
+    int32_t n_edges;
+    const int32_t* d_edges;
+} graft_tdes_traces;
+
+typedef struct graft_tdes_loss_config {
+    float gamma;       /* margin of Eq. 10 */
+    float w1;          /* weight of the positive edges in Eq. 11 */
+    float lambda_kl;   /* Eq. 12 */
+    float lambda_pair;
+    float lambda_bce;
+} graft_tdes_loss_config;
+
+/* With the scorer of Eq. 6 taken from the context (graft_set_tdes_tables: P, C, u, s):
+ *   d_loss [4] (fp64, overwritten) = L_KL, L_pair, L_BCE (each the mean over its items, 0 for an empty list) and
+ *     L = lambda_KL L_KL + lambda_pair L_pair + lambda_BCE L_BCE;
+ *   d_gP, d_gC [V, m], d_gu [L, m], d_gs [1] (fp32, 16-byte aligned): the gradient of L with respect to the table
+ *     rows P[v] = g_p(e_v), C[v] = g_c(e_v), the depth embeddings and the scale is ADDED to them (the caller zeroes
+ *     them; the additions are atomic and their order is not fixed, so results repeat only up to fp32 rounding).
+ *     All four NULL: losses only.  (The gradient for the weights of g_p is then gP^T E, one matrix product with
+ *     the frozen embeddings, left to the caller.)
+ *   d_skipped [1] or NULL (overwritten): items left out because a token id is outside [0, V) or a depth outside
+ *     [1, L]; they still count in the means' denominators.
+ * fp32 arithmetic, fp64 loss sums.  GRAFT_ERR_STATE before graft_set_tdes_tables; GRAFT_ERR_UNSUPPORTED for m > 512;
+ * GRAFT_ERR_INVALID_ARG for a NULL list with n > 0, a negative n, or only some of the gradient pointers NULL. */
+graft_status graft_tdes_loss(graft_ctx* ctx, const graft_tdes_traces* traces, const graft_tdes_loss_config* cfg,
+                             double* d_loss, int32_t* d_skipped, float* d_gP, float* d_gC, float* d_gu, float* d_gs,
+                             void* stream);
+
 /* Host-buffer form of graft_build_trees for end-to-end use: every pointer here is a HOST pointer (pinned
  * memory makes the copies asynchronous).  Copies the inputs host->device into context-owned staging buffers
  * (allocated on first use, sized for max_batch), runs the same kernels as graft_build_trees, copies

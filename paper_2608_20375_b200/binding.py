@@ -21,7 +21,7 @@ ST_BAD_LOGITS, ST_TAU_CLAMPED, ST_FRONTIER_EMPTY, ST_INTERNAL = 1, 2, 4, 8
 ENTRY_POINTS = [
     "graft_create", "graft_destroy", "graft_nmax", "graft_mask_words", "graft_set_saba", "graft_set_tdes_tables",
     "graft_tdes_precompute", "graft_build_trees", "graft_vocab_pass", "graft_vocab_pass_static", "graft_tdes_edges",
-    "graft_accept", "graft_set_edge_rows", "graft_edge_rows", "graft_set_hist_window", "graft_vocab_pass_partial", "graft_vocab_merge",
+    "graft_accept", "graft_tdes_loss", "graft_set_edge_rows", "graft_edge_rows", "graft_set_hist_window", "graft_vocab_pass_partial", "graft_vocab_merge",
     "graft_build_trees_host", "graft_launch_count", "graft_set_timing", "graft_read_timing", "graft_status_str",
     "graft_version",
 ]
@@ -52,6 +52,17 @@ class _TreeOut(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in (
         "d_n_nodes", "d_budget", "d_token", "d_parent", "d_depth", "d_position", "d_path_score", "d_mask", "d_status",
         "d_topk_id", "d_topk_lp", "d_lse", "d_edge", "d_state")]
+
+
+class _TdesTraces(C.Structure):
+    _fields_ = [("n_groups", C.c_int32), ("d_g_parent", C.c_void_p), ("d_g_depth", C.c_void_p),
+                ("d_g_child", C.c_void_p), ("d_g_logq", C.c_void_p), ("d_g_ztgt", C.c_void_p),
+                ("n_pairs", C.c_int32), ("d_pairs", C.c_void_p), ("n_edges", C.c_int32), ("d_edges", C.c_void_p)]
+
+
+class _TdesLossConfig(C.Structure):
+    _fields_ = [("gamma", C.c_float), ("w1", C.c_float), ("lambda_kl", C.c_float), ("lambda_pair", C.c_float),
+                ("lambda_bce", C.c_float)]
 
 
 _lib = None
@@ -95,6 +106,7 @@ def load_library():
     lib.graft_tdes_edges.argtypes = [vp, C.c_int32, vp, vp, vp, vp, vp]
     lib.graft_vocab_pass_static.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int, vp, vp, vp, vp, vp, vp]
     lib.graft_accept.argtypes = [vp, C.c_int32, C.POINTER(_TreeOut), vp, vp, vp, vp, vp]
+    lib.graft_tdes_loss.argtypes = [vp, C.POINTER(_TdesTraces), C.POINTER(_TdesLossConfig), vp, vp, vp, vp, vp, vp, vp]
     lib.graft_launch_count.argtypes = [vp]
     lib.graft_launch_count.restype = C.c_uint64
     lib.graft_set_timing.argtypes = [vp, C.c_int32]
@@ -330,6 +342,28 @@ class Graft:
         _check(self.lib, self.lib.graft_accept(self._ctx, batch, C.byref(oc), _ptr(target_next, i32),
                                                _ptr(accept_len, i32), _ptr(accept_path, i32),
                                                _ptr(bonus_token, i32), _stream()), "graft_accept")
+
+    def tdes_loss(self, groups, pairs, edges, gamma, w1, lambda_kl, lambda_pair, lambda_bce, loss, skipped=None,
+                  gP=None, gC=None, gu=None, gs=None):
+        """Training objective of the scorer and its gradients (Eq. 7-12) on device-resident traces.
+        groups: dict(parent [G], depth [G], child [G, K], logq [G, K], ztgt [G, K]) or None; pairs [N, 6] int32 or
+        None; edges [N, 4] int32 or None; loss: float64 [4] (overwritten); gP, gC [V, m], gu [L, m], gs [1] float32,
+        added to (all or none)."""
+        i32, f32 = torch.int32, torch.float32
+        t = _TdesTraces()
+        if groups is not None and groups["parent"].numel() > 0:
+            t.n_groups = groups["parent"].numel()
+            t.d_g_parent, t.d_g_depth = _ptr(groups["parent"], i32), _ptr(groups["depth"], i32)
+            t.d_g_child, t.d_g_logq, t.d_g_ztgt = (_ptr(groups["child"], i32), _ptr(groups["logq"], f32),
+                                                   _ptr(groups["ztgt"], f32))
+        if pairs is not None and pairs.numel() > 0:
+            t.n_pairs, t.d_pairs = pairs.shape[0], _ptr(pairs, i32)
+        if edges is not None and edges.numel() > 0:
+            t.n_edges, t.d_edges = edges.shape[0], _ptr(edges, i32)
+        lc = _TdesLossConfig(gamma, w1, lambda_kl, lambda_pair, lambda_bce)
+        _check(self.lib, self.lib.graft_tdes_loss(self._ctx, C.byref(t), C.byref(lc), _ptr(loss, torch.float64),
+                                                  _ptr(skipped, i32), _ptr(gP, f32), _ptr(gC, f32), _ptr(gu, f32),
+                                                  _ptr(gs, f32), _stream()), "graft_tdes_loss")
 
     # ---- bookkeeping
     def launch_count(self) -> int:

@@ -107,6 +107,7 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
 
     size_t vp_smem = 0;
     if (vp_configure(*cfg, ctx->num_sms, &vp_smem) != cudaSuccess || tdes_edges_configure(*cfg) != cudaSuccess ||
+        (tdes_loss_supported(*cfg) && tdes_loss_configure(*cfg) != cudaSuccess) ||
         tree_configure(*cfg) != cudaSuccess) {
         cudaGetLastError();
         delete extra_of(ctx);
@@ -284,6 +285,24 @@ graft_status graft_vocab_pass(graft_ctx* ctx, int32_t batch, const void* d_logit
     if ((uintptr_t)d_logits % esz) return GRAFT_ERR_INVALID_ARG;
     if (vp_launch(ctx, batch, d_logits, d_topk_id, d_topk_lp, d_lse, d_row_status ? d_row_status : ctx->w_row_status,
                   nullptr, nullptr, nullptr, (cudaStream_t)stream) != cudaSuccess)
+        return GRAFT_ERR_CUDA;
+    return GRAFT_OK;
+}
+
+graft_status graft_tdes_loss(graft_ctx* ctx, const graft_tdes_traces* tr, const graft_tdes_loss_config* lc,
+                             double* d_loss, int32_t* d_skipped, float* d_gP, float* d_gC, float* d_gu, float* d_gs,
+                             void* stream) {
+    if (!ctx || !tr || !lc || !d_loss) return GRAFT_ERR_INVALID_ARG;
+    if (!ctx->tdes_set) return GRAFT_ERR_STATE;
+    if (!tdes_loss_supported(ctx->cfg)) return GRAFT_ERR_UNSUPPORTED;
+    if (tr->n_groups < 0 || tr->n_pairs < 0 || tr->n_edges < 0) return GRAFT_ERR_INVALID_ARG;
+    if (tr->n_groups > 0 && (!tr->d_g_parent || !tr->d_g_depth || !tr->d_g_child || !tr->d_g_logq || !tr->d_g_ztgt))
+        return GRAFT_ERR_INVALID_ARG;
+    if ((tr->n_pairs > 0 && !tr->d_pairs) || (tr->n_edges > 0 && !tr->d_edges)) return GRAFT_ERR_INVALID_ARG;
+    const int n_grad = (d_gP != nullptr) + (d_gC != nullptr) + (d_gu != nullptr) + (d_gs != nullptr);
+    if (n_grad != 0 && n_grad != 4) return GRAFT_ERR_INVALID_ARG;
+    if (((uintptr_t)d_gP | (uintptr_t)d_gC | (uintptr_t)d_gu) & 15) return GRAFT_ERR_INVALID_ARG;
+    if (tdes_loss_launch(ctx, tr, lc, d_loss, d_skipped, d_gP, d_gC, d_gu, d_gs, (cudaStream_t)stream) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     return GRAFT_OK;
 }

@@ -139,6 +139,12 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
                         const int32_t* d_fixed_budget, const double* d_cos, const graft_tree_out* out, cudaStream_t st);
 cudaError_t accept_launch(graft_ctx* ctx, int batch, const graft_tree_out* trees, const int32_t* d_target_next,
                           int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus, cudaStream_t st);
+// TDES training objective, forward + backward (csrc/tdes_train.cu)
+cudaError_t tdes_loss_launch(graft_ctx* ctx, const graft_tdes_traces* tr, const graft_tdes_loss_config* lc,
+                             double* d_loss, int32_t* d_skipped, float* d_gP, float* d_gC, float* d_gu, float* d_gs,
+                             cudaStream_t st);
+cudaError_t tdes_loss_configure(const graft_config& cfg);
+bool tdes_loss_supported(const graft_config& cfg);
 size_t tree_smem_bytes(const graft_config& cfg);
 bool tree_lazy_fits(const graft_config& cfg);  // edge scores are computed inside the tree kernel
 
