@@ -481,6 +481,67 @@ def run_overlap(args):
     }))
 
 
+def run_tdes_loss(args):
+    """--tdes-loss: the TDES training objective forward + backward (graft_tdes_loss) on one synthetic batch of traces
+    at the paper's shapes; prints its own JSON line (not the benchmark's metric)."""
+    from paper_2608_20375_b200 import Graft
+    import oracle  # CPU-baseline leg only
+
+    V, L, K, m = 151936, 16, 32, 128
+    n_groups, n_pairs, n_edges = 32768, 131072, 262144
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    g = Graft(V, L, K, m, 32, 1, 16, 32, 16, 0.2, 1, 0, 0)
+    w = gi.small(V=V, L=L, K=K, m=m, seed=20381)
+    tb = gi.tdes_tables(w)
+    P, Ct, u = tb["P"].to(dev), tb["C"].to(dev), tb["u"].to(dev)
+    g.set_tdes_tables(P, Ct, u, tb["s"])
+    tr = gi.tdes_traces(V, L, K, n_groups, n_pairs, n_edges, seed=20382)
+    groups = {k: torch.from_numpy(np.ascontiguousarray(v)).to(dev) for k, v in tr["groups"].items()}
+    pairs, edges = torch.from_numpy(tr["pairs"]).to(dev), torch.from_numpy(tr["edges"]).to(dev)
+    cfg = dict(gamma=0.5, w1=4.0, lambda_kl=1.0, lambda_pair=1.0, lambda_bce=0.25)
+    loss = torch.zeros(4, dtype=torch.float64, device=dev)
+    gP, gC = torch.zeros((V, m), device=dev), torch.zeros((V, m), device=dev)
+    gu, gs = torch.zeros((L, m), device=dev), torch.zeros(1, device=dev)
+
+    def step():
+        g.tdes_loss(groups, pairs, edges, loss=loss, gP=gP, gC=gC, gu=gu, gs=gs, **cfg)
+
+    for _ in range(max(3, args.warmup or 3)):
+        step()
+    torch.cuda.synchronize()
+    steps = args.steps or 50
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    row = m * 4
+    # rows gathered + gradient rows added, once each: a group reads 1 + K rows and adds to 1 + K, an edge 2 and 2
+    alg = (n_groups * 2 * (1 + K) + n_pairs * 8 + n_edges * 4) * row
+    items = n_groups + n_pairs + n_edges
+    # the oracle on a slice of the same traces
+    n_s = 512
+    sub = {k: v[:n_s] for k, v in tr["groups"].items()}
+    t0 = time.perf_counter()
+    oracle.tdes_loss(tb["P"].numpy(), tb["C"].numpy(), tb["u"].numpy(), tb["s"], sub, tr["pairs"][:4 * n_s],
+                     tr["edges"][:8 * n_s], **cfg)
+    t_cpu = time.perf_counter() - t0
+    hbm_peak, peak_kind = _peaks()
+    print(json.dumps({
+        "kind": "TDES training objective, forward + backward (graft_tdes_loss)",
+        "shapes": {"V": V, "L": L, "K": K, "m": m, "groups": n_groups, "pairs": n_pairs, "edges": n_edges},
+        "ms_per_step": round(ms, 4), "items_per_s": round(items / (ms * 1e-3)),
+        "algorithmic_bytes": alg, "algorithmic_gbs": round(alg / (ms * 1e-3) / 1e9, 1),
+        "hbm_peak_gbs": hbm_peak, "peak_kind": "of " + peak_kind,
+        "note": "rows of hot tokens are served by L2, so the algorithmic rate is not bounded by the HBM peak",
+        "cpu_oracle": {"items": 13 * n_s, "seconds": round(t_cpu, 3),
+                       "items_per_s": round(13 * n_s / t_cpu)},
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -497,7 +558,12 @@ def main():
     ap.add_argument("--overlap-verifier-ms", type=float, default=None,
                     help="instead of the benchmark: two micro-batches on two streams around a stub verifier of this "
                          "duration, sequential against overlapped schedule")
+    ap.add_argument("--tdes-loss", action="store_true",
+                    help="instead of the benchmark: time the TDES training objective (forward + backward)")
     args = ap.parse_args()
+    if args.tdes_loss and args.impl == "graft":
+        run_tdes_loss(args)
+        return
     if args.overlap_verifier_ms is not None and args.impl == "graft":
         args.steps = 200 if args.steps is None else args.steps
         run_overlap(args)
