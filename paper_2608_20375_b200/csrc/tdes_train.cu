@@ -12,6 +12,10 @@
 // children, a pair, an edge): a lane holds four consecutive floats of every 128-float chunk of a row, dot products
 // are warp reductions, gradient rows go out as 16-byte vector atomics (`red.global.add.v4.f32`), the few u rows are
 // accumulated in shared memory per CTA and flushed once, losses and the scale's gradient are reduced per CTA.
+// Token frequencies are heavy-tailed, and atomic additions to one row serialise in L2: every warp therefore keeps
+// four gradient rows per table in shared memory (m <= 128), replaced by frequency (a hit raises a slot's credit, a
+// miss lowers the lowest one and takes the slot over when it reaches zero), so the few hottest tokens' rows reach
+// global memory once per warp instead of once per item.
 // The order of the atomic additions is not fixed, so the gradients are reproducible only up to fp32 rounding.
 #include <cuda_runtime.h>
 #include <math.h>
@@ -100,6 +104,73 @@ __device__ __forceinline__ void add_row_global(float* dst, int tok, int m, int l
                       make_float4(coef * r.v[ch].x, coef * r.v[ch].y, coef * r.v[ch].z, coef * r.v[ch].w));
     }
 }
+// A warp's four cached gradient rows of one table (m <= 128: one float4 per lane per row).
+constexpr int kTrSlots = 4;
+constexpr int kTrCreditMax = 64;
+struct WarpCache {
+    float* rows;  // [2][kTrSlots][128]
+    int* tags;    // [2][kTrSlots] token id or -1
+    int* credit;  // [2][kTrSlots]
+};
+// gradient row of token `tok` of table t (0: gP, 1: gC) += coef * r
+template <int NCH>
+__device__ __forceinline__ void add_row(const TrainParams& p, const WarpCache& wc, int t, int tok, int lane, float coef,
+                                        const Row<NCH>& r) {
+    float* dst = t == 0 ? p.gP : p.gC;
+    if (NCH != 1) {
+        add_row_global<NCH>(dst, tok, p.m, lane, coef, r);
+        return;
+    }
+    const int4 tg = *(const int4*)(wc.tags + kTrSlots * t);
+    const int slot = tg.x == tok ? 0 : tg.y == tok ? 1 : tg.z == tok ? 2 : tg.w == tok ? 3 : -1;
+    const float4 add = make_float4(coef * r.v[0].x, coef * r.v[0].y, coef * r.v[0].z, coef * r.v[0].w);
+    if (slot >= 0) {  // hit
+        float4* q = (float4*)(wc.rows + (size_t)(t * kTrSlots + slot) * 128) + lane;
+        float4 v = *q;
+        v.x += add.x;
+        v.y += add.y;
+        v.z += add.z;
+        v.w += add.w;
+        *q = v;
+        if (lane == 0) {
+            const int c = wc.credit[t * kTrSlots + slot];
+            if (c < kTrCreditMax) wc.credit[t * kTrSlots + slot] = c + 1;
+        }
+        __syncwarp();
+        return;
+    }
+    const int4 cr = *(const int4*)(wc.credit + kTrSlots * t);
+    int victim = 0, cmin = cr.x;
+    if (cr.y < cmin) victim = 1, cmin = cr.y;
+    if (cr.z < cmin) victim = 2, cmin = cr.z;
+    if (cr.w < cmin) victim = 3, cmin = cr.w;
+    if (cmin > 0) {  // the slot keeps its row for now; this addition goes to global memory
+        if (lane == 0) wc.credit[t * kTrSlots + victim] = cmin - 1;
+        __syncwarp();
+        if (lane < p.m / 4) atomicAdd((float4*)(dst + (size_t)tok * p.m) + lane, add);
+        return;
+    }
+    // take the slot over: its row goes to global memory, the new token's starts with this addition
+    const int old = wc.tags[t * kTrSlots + victim];
+    float4* q = (float4*)(wc.rows + (size_t)(t * kTrSlots + victim) * 128) + lane;
+    if (old >= 0 && lane < p.m / 4) atomicAdd((float4*)(dst + (size_t)old * p.m) + lane, *q);
+    *q = add;
+    __syncwarp();
+    if (lane == 0) {
+        wc.tags[t * kTrSlots + victim] = tok;
+        wc.credit[t * kTrSlots + victim] = 1;
+    }
+    __syncwarp();
+}
+__device__ __forceinline__ void cache_flush(const TrainParams& p, const WarpCache& wc, int lane) {
+    for (int t = 0; t < 2; ++t)
+        for (int sl = 0; sl < kTrSlots; ++sl) {
+            const int tok = wc.tags[t * kTrSlots + sl];
+            if (tok >= 0 && lane < p.m / 4)
+                atomicAdd((float4*)((t == 0 ? p.gP : p.gC) + (size_t)tok * p.m) + lane,
+                          *((const float4*)(wc.rows + (size_t)(t * kTrSlots + sl) * 128) + lane));
+        }
+}
 // the CTA's copy of gu: row d-1 += coef * (a + b)
 template <int NCH>
 __device__ __forceinline__ void add_u_shared(float* su, int d, int m, int lane, float coef, const Row<NCH>& a,
@@ -133,11 +204,12 @@ __device__ __forceinline__ float edge_forward(const TrainParams& p, int tp, int 
     return p.k0 * dot;
 }
 template <int NCH>
-__device__ __forceinline__ void edge_backward(const TrainParams& p, float* su, int tp, int tc, int d, int lane,
-                                              float gf, const Row<NCH>& a, const Row<NCH>& b, float dot, float& gs) {
+__device__ __forceinline__ void edge_backward(const TrainParams& p, const WarpCache& wc, float* su, int tp, int tc,
+                                              int d, int lane, float gf, const Row<NCH>& a, const Row<NCH>& b,
+                                              float dot, float& gs) {
     const float coef = gf * p.k0;
-    add_row_global<NCH>(p.gP, tp, p.m, lane, coef, b);
-    add_row_global<NCH>(p.gC, tc, p.m, lane, coef, a);
+    add_row<NCH>(p, wc, 0, tp, lane, coef, b);
+    add_row<NCH>(p, wc, 1, tc, lane, coef, a);
     add_u_shared<NCH>(su, d, p.m, lane, coef, a, b);
     gs += gf * dot * p.inv_sqrt_m;
 }
@@ -150,6 +222,17 @@ __global__ void __launch_bounds__(kTrThreads) tdes_loss_kernel(const TrainParams
     __shared__ int s_skip;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool grad = p.gP != nullptr;
+    WarpCache wc;  // behind su (NCH == 1 only): rows, then tags and credits, per warp
+    {
+        float* base = su + ((p.L * p.m + 3) & ~3);
+        wc.rows = base + (size_t)warp * 2 * kTrSlots * 128;
+        wc.tags = (int*)(base + (size_t)kTrWarps * 2 * kTrSlots * 128) + warp * 4 * kTrSlots;
+        wc.credit = wc.tags + 2 * kTrSlots;
+        if (NCH == 1 && lane < 2 * kTrSlots) {
+            wc.tags[lane] = -1;
+            wc.credit[lane] = 0;
+        }
+    }
     for (int i = threadIdx.x; i < p.L * p.m; i += kTrThreads) su[i] = 0.f;
     if (threadIdx.x < 3) s_loss[threadIdx.x] = 0.0;
     if (threadIdx.x == 0) {
@@ -213,7 +296,7 @@ __global__ void __launch_bounds__(kTrThreads) tdes_loss_kernel(const TrainParams
                 const int t = __shfl_sync(0xFFFFFFFFu, tc, c);
                 const float coef = __shfl_sync(0xFFFFFFFFu, gf_c, c) * p.k0;
                 const Row<NCH> b = load_row_plus_u<NCH>(p.C, urow, t, p.m, lane);
-                add_row_global<NCH>(p.gC, t, p.m, lane, coef, a);
+                add_row<NCH>(p, wc, 1, t, lane, coef, a);
 #pragma unroll
                 for (int ch = 0; ch < NCH; ++ch) {
                     accP.v[ch].x = fmaf(coef, b.v[ch].x, accP.v[ch].x);
@@ -226,7 +309,7 @@ __global__ void __launch_bounds__(kTrThreads) tdes_loss_kernel(const TrainParams
                     accU.v[ch].w = fmaf(coef, a.v[ch].w + b.v[ch].w, accU.v[ch].w);
                 }
             }
-            add_row_global<NCH>(p.gP, tp, p.m, lane, 1.f, accP);
+            add_row<NCH>(p, wc, 0, tp, lane, 1.f, accP);
             Row<NCH> zero;
 #pragma unroll
             for (int ch = 0; ch < NCH; ++ch) zero.v[ch] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -254,8 +337,8 @@ __global__ void __launch_bounds__(kTrThreads) tdes_loss_kernel(const TrainParams
         l_pair += (double)softplus_f(x);
         if (grad) {
             const float gx = p.w_pair * sigmoid_f(x);
-            edge_backward<NCH>(p, su, p1, c1, d1, lane, -gx, a1, b1, dot1, gs);
-            edge_backward<NCH>(p, su, p2, c2, d2, lane, gx, a2, b2, dot2, gs);
+            edge_backward<NCH>(p, wc, su, p1, c1, d1, lane, -gx, a1, b1, dot1, gs);
+            edge_backward<NCH>(p, wc, su, p2, c2, d2, lane, gx, a2, b2, dot2, gs);
         }
     }
     // ---- edge level (Eq. 11)
@@ -273,9 +356,10 @@ __global__ void __launch_bounds__(kTrThreads) tdes_loss_kernel(const TrainParams
         l_bce += (double)(p.w1 * y * softplus_f(-f) + (1.f - y) * softplus_f(f));
         if (grad) {
             const float gf = p.w_bce * (-p.w1 * y * sigmoid_f(-f) + (1.f - y) * sigmoid_f(f));
-            edge_backward<NCH>(p, su, tp, tc, d, lane, gf, a, b, dot, gs);
+            edge_backward<NCH>(p, wc, su, tp, tc, d, lane, gf, a, b, dot, gs);
         }
     }
+    if (NCH == 1 && grad) cache_flush(p, wc, lane);
     // ---- per-CTA reduction, then one round of global atomics
     if (lane == 0) {
         atomicAdd(&s_loss[0], l_kl);
@@ -302,6 +386,12 @@ __global__ void __launch_bounds__(kTrThreads) tdes_loss_kernel(const TrainParams
 }
 
 }  // namespace
+
+static size_t tdes_loss_smem(const graft_config& cfg) {
+    size_t b = (size_t)((cfg.L * cfg.m + 3) & ~3) * sizeof(float);  // gu
+    if (cfg.m <= 128) b += (size_t)kTrWarps * (2 * kTrSlots * 128 * sizeof(float) + 4 * kTrSlots * sizeof(int));
+    return b;
+}
 
 cudaError_t tdes_loss_launch(graft_ctx* ctx, const graft_tdes_traces* tr, const graft_tdes_loss_config* lc,
                              double* d_loss, int32_t* d_skipped, float* d_gP, float* d_gC, float* d_gu, float* d_gs,
@@ -352,8 +442,8 @@ cudaError_t tdes_loss_launch(graft_ctx* ctx, const graft_tdes_traces* tr, const 
     long long grid = (items + kTrWarps - 1) / kTrWarps;
     const long long cap = (long long)ctx->num_sms * 4;
     if (grid > cap) grid = cap;
-    const size_t smem = (size_t)cfg.L * cfg.m * sizeof(float);
     const int nch = (cfg.m / 4 + 31) / 32;
+    const size_t smem = tdes_loss_smem(cfg);
     if (nch <= 1)
         tdes_loss_kernel<1><<<(int)grid, kTrThreads, smem, st>>>(p);
     else if (nch == 2)
@@ -365,7 +455,7 @@ cudaError_t tdes_loss_launch(graft_ctx* ctx, const graft_tdes_traces* tr, const 
 }
 
 cudaError_t tdes_loss_configure(const graft_config& cfg) {
-    const int smem = cfg.L * cfg.m * (int)sizeof(float);
+    const int smem = (int)tdes_loss_smem(cfg);
     if (smem <= 48 * 1024) return cudaSuccess;
     cudaError_t e = cudaFuncSetAttribute(tdes_loss_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tdes_loss_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
