@@ -16,7 +16,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libgraft.so")
 GRAFT_H = os.path.join("..", "..", "include", "graft.h")
-ALL_HEADERS = ["common.cuh", "internal.h", "edge_score.cuh", "cosine.cuh", GRAFT_H]
+ALL_HEADERS = ["common.cuh", "internal.h", "edge_score.cuh", "cosine.cuh", "saba.cuh", GRAFT_H]
 # source -> headers it depends on
 SOURCES = {
     "api.cu": ALL_HEADERS,

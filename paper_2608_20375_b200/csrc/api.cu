@@ -127,7 +127,7 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     const size_t o_id = take(B * L * K * 4), o_lp = take(B * L * K * 4), o_lse = take(B * L * 4);
     const size_t o_rs = take(B * L * 4), o_edge = take(B * L * K * K * 4);
     const size_t o_es = take(B * L * K * K * 4), o_ei = take(B * L * K * K);
-    const size_t o_u = take(L * (size_t)cfg->m * 4), o_err = take(256), o_cos = take(B * L * 8);
+    const size_t o_u = take(L * (size_t)cfg->m * 4), o_err = take(256), o_cos = take(B * L * 8), o_saba = take(B * sizeof(SabaResult));
     ctx->ws_bytes = off;
     if (cudaMalloc(&ctx->ws, ctx->ws_bytes) != cudaSuccess) {
         cudaGetLastError();
@@ -162,6 +162,7 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     ctx->edge_rows = tree_lazy_fits(*cfg) ? (cfg->L < 8 ? cfg->L : 8) : cfg->L;
     ctx->w_errflag = (int32_t*)(base + o_err);
     ctx->w_cos = (double*)(base + o_cos);
+    ctx->w_saba = (SabaResult*)(base + o_saba);
     *out = ctx;
     return GRAFT_OK;
 }
@@ -313,7 +314,7 @@ graft_status graft_tdes_edges(graft_ctx* ctx, int32_t batch, const int32_t* d_to
     if (batch < 1 || batch > ctx->cfg.max_batch) return GRAFT_ERR_INVALID_ARG;
     if (ctx->cfg.beta != 0.0f && !ctx->tdes_set) return GRAFT_ERR_STATE;
     if (tdes_edges_launch(ctx, batch, d_topk_id, d_topk_lp, d_root_token, nullptr, d_edge, ctx->w_esort, ctx->w_eidx,
-                          ctx->cfg.L, (cudaStream_t)stream) != cudaSuccess)
+                          ctx->cfg.L, nullptr, nullptr, nullptr, nullptr, (cudaStream_t)stream) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     return GRAFT_OK;
 }
@@ -392,15 +393,16 @@ graft_status graft_build_trees(graft_ctx* ctx, int32_t batch, const void* d_logi
     if (ev) cudaEventRecord(ev[1], st);
     // Edge scores of Eq. 4-6: the kernel scores the depths [0, edge_rows) for every sequence (all depths when the
     // caller asks for the score array); the tree kernel scores deeper rows itself if an expansion gets that far.
-    {
-        const int rows = out->d_edge ? ctx->cfg.L : ctx->edge_rows;
-        if (rows > 0 && tdes_edges_launch(ctx, batch, ids, lps, d_root_token, ctx->w_row_status, edge, ctx->w_esort,
-                                          ctx->w_eidx, rows, st) != cudaSuccess)
-            return GRAFT_ERR_CUDA;
-    }
+    // The depth-0 CTA of each sequence in that kernel also works out the sequence's budget (Sec. 3.3), which the tree
+    // kernel then only reads; without an edge-score kernel the tree kernel does it itself.
+    const int rows = out->d_edge ? ctx->cfg.L : ctx->edge_rows;
+    if (rows > 0 && tdes_edges_launch(ctx, batch, ids, lps, d_root_token, ctx->w_row_status, edge, ctx->w_esort,
+                                      ctx->w_eidx, rows, ctx->w_saba, d_hist, d_prefix_len, d_fixed_budget,
+                                      st) != cudaSuccess)
+        return GRAFT_ERR_CUDA;
     if (ev) cudaEventRecord(ev[2], st);
-    if (tree_launch(ctx, batch, ids, lps, ctx->w_row_status, ctx->w_esort, ctx->w_eidx, d_hidden, d_root_token, d_hist, d_prefix_len,
-                    d_fixed_budget, ctx->w_cos, out, st) != cudaSuccess)
+    if (tree_launch(ctx, batch, ids, lps, ctx->w_row_status, ctx->w_esort, ctx->w_eidx, d_hidden, d_root_token, d_hist,
+                    d_prefix_len, d_fixed_budget, ctx->w_cos, rows > 0 ? ctx->w_saba : nullptr, out, st) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     if (ev) {
         cudaEventRecord(ev[3], st);

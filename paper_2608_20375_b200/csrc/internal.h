@@ -48,6 +48,13 @@ struct SabaDev {
     double pts_n[kMaxCostPts], pts_t[kMaxCostPts];
 };
 
+// Budget, status and decoding state of one sequence (Sec. 3.3), handed from the edge-score kernel to the tree kernel.
+struct SabaResult {
+    int32_t budget;
+    int32_t status;  // OR of the rows' status words, the vocab pass's error flag, GRAFT_ST_TAU_CLAMPED
+    float state[4];  // conf, degen, hist, tau
+};
+
 }  // namespace graft
 
 struct graft_ctx {
@@ -79,6 +86,7 @@ struct graft_ctx {
     float* w_esort;               // [max_batch, L, K, K] rows sorted by edge score
     uint8_t* w_eidx;              // [max_batch, L, K, K] child rank of each sorted entry
     double* w_cos;                // [max_batch, L] adjacent-position cosines (Eq. 15)
+    graft::SabaResult* w_saba;    // [max_batch] budgets worked out by the edge-score kernel
     int32_t* w_errflag;           // [1] device-side internal error flag
     graft::VpPlan vp_plan;
     // scratch of the tensor-core table precompute (allocated on its first use: three bf16 copies of W, GEMM workspace)
@@ -132,11 +140,15 @@ cudaError_t s0_tc_launch(const void* d_emb, int V, int E, int m, const float* d_
                          void* d_scratch, int* launches, cudaStream_t st);
 cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                               const int32_t* d_root_token, const int32_t* d_row_status, float* d_edge,
-                              float* d_esort, uint8_t* d_eidx, int rows, cudaStream_t st);  // depths [0, rows)
+                              float* d_esort, uint8_t* d_eidx, int rows, SabaResult* d_saba_out, const float* d_hist,
+                              const int32_t* d_prefix_len, const int32_t* d_fixed_budget, cudaStream_t st);
+// depths [0, rows); d_saba_out != NULL: the depth-0 CTA of every sequence also works out its budget (Sec. 3.3) from
+// the context's cosines, d_hist and d_prefix_len (or takes it from d_fixed_budget when that is not NULL)
 cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                         const int32_t* d_row_status, const float* d_esort, const uint8_t* d_eidx, const void* d_hidden,
                         const int32_t* d_root_token, const float* d_hist, const int32_t* d_prefix_len,
-                        const int32_t* d_fixed_budget, const double* d_cos, const graft_tree_out* out, cudaStream_t st);
+                        const int32_t* d_fixed_budget, const double* d_cos, const SabaResult* d_saba_pre,
+                        const graft_tree_out* out, cudaStream_t st);
 cudaError_t accept_launch(graft_ctx* ctx, int batch, const graft_tree_out* trees, const int32_t* d_target_next,
                           int32_t* d_accept_len, int32_t* d_accept_path, int32_t* d_bonus, cudaStream_t st);
 // TDES training objective, forward + backward (csrc/tdes_train.cu)

@@ -12,6 +12,7 @@
 #include "common.cuh"
 #include "internal.h"
 #include "edge_score.cuh"
+#include "saba.cuh"
 
 namespace graft {
 namespace {
@@ -90,11 +91,20 @@ struct EdgeParams {
     float scale;  // s / sqrt(m)
     float beta;
     int root_edge;
+    // the budget of every sequence (Sec. 3.3), worked out by its depth-0 CTA when saba_out is not NULL
+    SabaResult* saba_out;         // [batch]
+    const double* cos_pre;        // [batch, L] adjacent-position cosines from the vocab pass
+    const int32_t* vp_err;
+    const float* hist;            // [batch]
+    const int32_t* prefix_len;    // [batch]
+    const int32_t* fixed_budget;  // [batch], or NULL: SABA
+    int bmin, bmax, bstep;
+    SabaDev saba;
 };
 
 // WRITE_EDGE: also write the unsorted scores (the caller asked for the array); the tree kernel reads only the sorted rows
 template <bool WRITE_EDGE>
-__global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
+__global__ void __launch_bounds__(256, 4) tdes_edges_kernel(const EdgeParams p) {
     extern __shared__ __align__(16) float smem[];
     pdl_launch_dependents();  // the tree kernel may move in as SMs free up; it waits for this grid before it reads
     pdl_wait();               // the candidates come from the vocab pass
@@ -105,6 +115,14 @@ __global__ void __launch_bounds__(256) tdes_edges_kernel(const EdgeParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_par = (j == 0) ? 1 : K;
     const size_t row = (size_t)b * p.L + j;
+    if (j == 0 && p.saba_out != nullptr && warp == 7) {
+        // the depth-0 unit has one parent, so this CTA has time to spare: its last warp works out the sequence's budget,
+        // which the tree kernel would otherwise do in front of everything else
+        const SabaResult r = saba_warp(p.saba, p.bmin, p.bmax, p.bstep, p.L, K, p.row_status + (size_t)b * p.L, p.vp_err,
+                                       p.topk_lp + (size_t)b * p.L * K, p.cos_pre + (size_t)b * p.L, p.hist + b,
+                                       p.prefix_len + b, p.fixed_budget ? p.fixed_budget + b : nullptr, lane);
+        if (lane == 0) p.saba_out[b] = r;
+    }
     float* outs = p.esort + row * K * K;
     uint8_t* outi = p.eidx + row * K * K;
     const int32_t* ids = p.topk_id + row * K;
@@ -204,7 +222,8 @@ cudaError_t tdes_edges_configure(const graft_config& cfg) {
 
 cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                               const int32_t* d_root_token, const int32_t* d_row_status, float* d_edge,
-                              float* d_esort, uint8_t* d_eidx, int rows, cudaStream_t st) {
+                              float* d_esort, uint8_t* d_eidx, int rows, SabaResult* d_saba_out, const float* d_hist,
+                              const int32_t* d_prefix_len, const int32_t* d_fixed_budget, cudaStream_t st) {
     const graft_config& cfg = ctx->cfg;
     EdgeParams p;
     p.topk_id = d_topk_id;
@@ -225,6 +244,16 @@ cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_i
     p.beta = ctx->tdes_set ? cfg.beta : 0.0f;
     p.root_edge = cfg.root_edge;
     p.rows = rows;
+    p.saba_out = d_row_status ? d_saba_out : nullptr;
+    p.cos_pre = ctx->w_cos;
+    p.vp_err = ctx->w_errflag;
+    p.hist = d_hist;
+    p.prefix_len = d_prefix_len;
+    p.fixed_budget = d_fixed_budget;
+    p.bmin = cfg.budget_min;
+    p.bmax = cfg.budget_max;
+    p.bstep = cfg.budget_step;
+    p.saba = ctx->saba;
     const cudaError_t e = launch_pdl(d_edge ? tdes_edges_kernel<true> : tdes_edges_kernel<false>, dim3(batch * rows),
                                      dim3(256), tdes_edges_smem(cfg), st, p);
     ctx->launches += 1;

@@ -5,6 +5,7 @@
 #include "common.cuh"
 #include "internal.h"
 #include "edge_score.cuh"
+#include "saba.cuh"
 
 namespace graft {
 namespace {
@@ -37,6 +38,7 @@ struct TreeParams {
     int root_edge, m, V;
     int use_saba;
     SabaDev saba;
+    const SabaResult* saba_pre;  // [batch] budget, status and state worked out by the edge-score kernel, or NULL
 };
 
 constexpr int TREE_THREADS = 1024;  // one CTA per SM (shared memory bound): all warps serve the parallel phases
@@ -144,17 +146,6 @@ __host__ __device__ inline int tree_node_cap(int L, int K, int nmax, int lazy_m)
     if (cap > 6144) cap = 6144;
     if (cap < 2 * nmax) cap = 2 * nmax;
     return (int)cap;
-}
-
-__device__ __forceinline__ double saba_cost(const SabaDev& sp, double B, double prefix) {
-    if (sp.cost_mode == 0) return sp.c0 + sp.c1 * B + sp.c2 * B * prefix;
-    if (B <= sp.pts_n[0]) return sp.pts_t[0];
-    for (int i = 1; i < sp.n_pts; ++i)
-        if (B <= sp.pts_n[i]) {
-            double w = (B - sp.pts_n[i - 1]) / (sp.pts_n[i] - sp.pts_n[i - 1]);
-            return sp.pts_t[i - 1] + w * (sp.pts_t[i] - sp.pts_t[i - 1]);
-        }
-    return sp.pts_t[sp.n_pts - 1];
 }
 
 // Frontier entry of a selected node: its best child that is not selected yet.
@@ -390,7 +381,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         }
     }
     // adjacent-position cosines r_d = cos(h_d, h_{d+1}) (Eq. 15): written by the vocab pass
-    if (p.use_saba && tid < L - 1) sm.cosv[tid] = p.cos_pre[(size_t)b * L + tid];
+    if (p.use_saba && !p.saba_pre && tid < L - 1) sm.cosv[tid] = p.cos_pre[(size_t)b * L + tid];
     __syncthreads();
     // While warp 0 works out the budget, the other warps expand levels 0 and 1 in full (1 + K + K^2 nodes), which
     // needs no budget: with fewer than B nodes in the table every child is appended anyway, and if B is smaller
@@ -422,67 +413,19 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             sm.ninfo[1 + K + j] = (uint32_t)x | ((uint32_t)sm.ei[row + r] << 13) | (2u << 18);
         }
     }
-    if (warp == 0) {
-        int st = 0;
-        for (int j = lane; j < L; j += 32) st |= p.row_status[(size_t)b * L + j];
-        st = __reduce_or_sync(0xFFFFFFFFu, st);
-        if (p.vp_err[0] & 1) st |= GRAFT_ST_INTERNAL;
-        int budget = 0;
-        float state[4] = {0.f, 0.f, 0.f, 0.f};
-        if (!(st & GRAFT_ST_BAD_LOGITS)) {
-            if (!p.use_saba) {
-                budget = p.fixed_budget[b];
-                budget = budget < 0 ? 0 : (budget > p.bmax ? p.bmax : budget);
-            } else {
-                double conf = 0.0, rs = 0.0;
-                for (int j = lane; j < L; j += 32) conf += exp((double)p.topk_lp[((size_t)b * L + j) * K]);
-                for (int j = lane; j < L - 1; j += 32) rs += sm.cosv[j];
-#pragma unroll
-                for (int d = 16; d > 0; d >>= 1) {
-                    conf += __shfl_xor_sync(0xFFFFFFFFu, conf, d);
-                    rs += __shfl_xor_sync(0xFFFFFFFFu, rs, d);
-                }
-                conf /= (double)L;
-                double degen = 0.0;
-                if (L >= 2) degen = rs / (double)(L - 1) + (sm.cosv[L - 2] - sm.cosv[0]);
-                const double hist = (double)p.hist[b];
-                double tau = p.saba.phi_conf * conf + p.saba.phi_degen * degen + p.saba.phi_hist * hist + p.saba.phi_bias;
-                if (!(tau >= p.saba.tau_min)) {
-                    tau = p.saba.tau_min;
-                    st |= GRAFT_ST_TAU_CLAMPED;
-                }
-                const double prefix = (double)p.prefix_len[b];
-                double ubest = -INFINITY;
-                int bbest = p.bmin;
-                for (int B = p.bmin + lane * p.bstep; B <= p.bmax; B += 32 * p.bstep) {
-                    const double G = 1.0 - exp(-(double)B / tau);
-                    const double u = G / saba_cost(p.saba, (double)B, prefix);
-                    if (u > ubest) {
-                        ubest = u;
-                        bbest = B;
-                    }
-                }
-#pragma unroll
-                for (int d = 16; d > 0; d >>= 1) {
-                    const double u2 = __shfl_xor_sync(0xFFFFFFFFu, ubest, d);
-                    const int b2 = __shfl_xor_sync(0xFFFFFFFFu, bbest, d);
-                    if (u2 > ubest || (u2 == ubest && b2 < bbest)) {
-                        ubest = u2;
-                        bbest = b2;
-                    }
-                }
-                budget = bbest;
-                state[0] = (float)conf;
-                state[1] = (float)degen;
-                state[2] = (float)hist;
-                state[3] = (float)tau;
-            }
-        }
+    if (warp == 0) {  // status and budget: from the edge-score kernel if it ran ahead, else worked out here
+        SabaResult r;
+        if (p.saba_pre)
+            r = p.saba_pre[b];
+        else
+            r = saba_warp(p.saba, p.bmin, p.bmax, p.bstep, L, K, p.row_status + (size_t)b * L, p.vp_err,
+                          p.topk_lp + (size_t)b * L * K, sm.cosv, p.hist + b, p.prefix_len + b,
+                          p.use_saba ? nullptr : p.fixed_budget + b, lane);
         if (lane == 0) {
-            sm.scal[0] = budget;
-            sm.scal[2] = st;
+            sm.scal[0] = r.budget;
+            sm.scal[2] = r.status;
             if (o.d_state) {
-                for (int i = 0; i < 4; ++i) o.d_state[(size_t)b * 4 + i] = state[i];
+                for (int i = 0; i < 4; ++i) o.d_state[(size_t)b * 4 + i] = r.state[i];
             }
         }
     }
@@ -1151,7 +1094,8 @@ cudaError_t tree_configure(const graft_config& cfg) {
 cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                         const int32_t* d_row_status, const float* d_esort, const uint8_t* d_eidx, const void* d_hidden,
                         const int32_t* d_root_token, const float* d_hist, const int32_t* d_prefix_len,
-                        const int32_t* d_fixed_budget, const double* d_cos, const graft_tree_out* out, cudaStream_t st) {
+                        const int32_t* d_fixed_budget, const double* d_cos, const SabaResult* d_saba_pre,
+                        const graft_tree_out* out, cudaStream_t st) {
     const graft_config& cfg = ctx->cfg;
     TreeParams p;
     p.topk_id = d_topk_id;
@@ -1188,6 +1132,7 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     p.bstep = cfg.budget_step;
     p.use_saba = d_fixed_budget == nullptr;
     p.saba = ctx->saba;
+    p.saba_pre = d_saba_pre;
     const cudaError_t e = launch_pdl(tree_kernel, dim3(batch), dim3(TREE_THREADS), tree_smem_bytes(cfg), st, p);
     ctx->launches += 1;
     return e != cudaSuccess ? e : cudaGetLastError();
