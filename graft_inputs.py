@@ -73,7 +73,7 @@ C5 = Workload("C5", 128, 16, 151936, 32, 4096, "bf16", "bf16", 16, 512, target_m
 M = Workload("M", 64, 16, 151936, 32, 4096, "bf16", "bf16", 16, 512, target_mode="decay", seed=20380)
 WORKLOADS = {w.name: w for w in (C1, C2, C3, C4, C5, M)}
 
-_TAGS = {"logits": 1, "hidden": 2, "boost_ids": 3, "boost_h": 4, "tables": 5, "scalars": 6, "target": 7, "emb": 8, "traces": 9}
+_TAGS = {"logits": 1, "hidden": 2, "boost_ids": 3, "boost_h": 4, "tables": 5, "scalars": 6, "target": 7, "emb": 8, "traces": 9, "replay": 10}
 
 
 def _rng(seed: int, tag: str, b: int = 0) -> np.random.Generator:
@@ -245,6 +245,24 @@ def tdes_traces(V: int, L: int, K: int, n_groups: int, n_pairs: int, n_edges: in
     edges = np.stack([tokens(n_edges), tokens(n_edges), g.integers(1, L + 1, n_edges).astype(np.int32),
                       (g.random(n_edges) < pos_rate).astype(np.int32)], axis=1).astype(np.int32)
     return dict(groups=groups, pairs=pairs, edges=edges)
+
+
+def saba_replay_logs(n: int, seed: int, phi=(-160.0, 20.0, -5.0, 200.0), c=(6.0, 0.012, 2.0e-6), noise: float = 0.02,
+                     bmin: int = 32, bmax: int = 512, bstep: int = 16) -> dict:
+    """Synthetic same-prefix budget replay logs (the paper's come from held-out prompts run through the models).
+
+    Per logged round: a decoding state (conf ~ U(0.2, 0.95), degen ~ U(0.5, 1.4), hist ~ U(0, 8)), a budget from the
+    paper's grid, a prefix length ~ U{16..4096}; the gain and the latency follow the models of Eq. 16-17 with the
+    given parameters, times (1 + noise * N(0,1)) each; gains are clipped to [0, 1]."""
+    g = _rng(seed, "replay")
+    state = np.stack([g.uniform(0.2, 0.95, n), g.uniform(0.5, 1.4, n), g.uniform(0.0, 8.0, n)], axis=1)
+    budget = (bmin + bstep * g.integers(0, (bmax - bmin) // bstep + 1, n)).astype(np.int32)
+    prefix = g.integers(16, 4097, n).astype(np.int32)
+    tau = state @ np.asarray(phi[:3]) + phi[3]
+    gain = (1.0 - np.exp(-budget / np.maximum(tau, 1.0))) * (1.0 + noise * g.standard_normal(n))
+    lat = (c[0] + c[1] * budget + c[2] * budget * prefix.astype(np.float64)) * (1.0 + noise * g.standard_normal(n))
+    return dict(state=state.astype(np.float32), budget=budget, gain=np.clip(gain, 0.0, 1.0).astype(np.float32),
+                prefix_len=prefix, latency=lat.astype(np.float32))
 
 
 def small(name: str = "T", **kw) -> Workload:

@@ -250,6 +250,30 @@ def tdes_loss(P, Ctab, u, s, groups, pairs, edges, gamma, w1, lambda_kl, lambda_
     return out
 
 
+def saba_fit(state, budget, gain, prefix_len, latency):
+    """Least-squares fit of the SABA gain and cost models to replay logs (Sec. 3.3, Eq. 16-17).
+
+    The paper fits the parameters on held-out prompts by same-prefix budget replay and does not give the procedure;
+    the reading restated here is ordinary least squares, in fp64, with numpy's SVD-based solver as the one step:
+      gain: 0 < g_i < 1 at budget B_i  =>  tau_i = -B_i / ln(1 - g_i);  (phi, bias) = argmin sum (tau_i - phi.s_i - bias)^2
+      cost: (c0, c1, c2) = argmin sum (T_i - c0 - c1 B_i - c2 B_i prefix_i)^2
+    Returns dict(phi [4] = conf, degen, hist, bias; c [3]; n_gain; n_cost).
+    Pins (tests/test_oracle_saba_fit.py): exact recovery of known parameters from noise-free logs, the normal
+    equations' residual orthogonality, invariance under duplication and permutation of the rounds."""
+    s = np.asarray(state, dtype=np.float32).astype(np.float64).reshape(-1, 3)
+    B = np.asarray(budget, dtype=np.int32).astype(np.float64)
+    g = np.asarray(gain, dtype=np.float32).astype(np.float64)
+    pre = np.asarray(prefix_len, dtype=np.int32).astype(np.float64)
+    T = np.asarray(latency, dtype=np.float32).astype(np.float64)
+    use = (g > 0.0) & (g < 1.0)
+    tau = -B[use] / np.log1p(-g[use])
+    X = np.concatenate([s[use], np.ones((int(use.sum()), 1))], axis=1)
+    phi = np.linalg.lstsq(X, tau, rcond=None)[0] if use.sum() >= 4 else np.zeros(4)
+    H = np.stack([np.ones_like(B), B, B * pre], axis=1)
+    c = np.linalg.lstsq(H, T, rcond=None)[0] if B.size >= 3 else np.zeros(3)
+    return dict(phi=phi, c=c, n_gain=int(use.sum()), n_cost=int(B.size))
+
+
 def replay_check(edge, n_nodes, parent, cand, depth, eps):
     """Is the given node set a valid best-first outcome on the oracle's edge scores up to eps?"""
     edge = np.ascontiguousarray(edge, dtype=np.float32)
