@@ -542,6 +542,50 @@ def run_tdes_loss(args):
     }))
 
 
+def run_saba_fit(args):
+    """--saba-fit: the least-squares fit of the SABA models (graft_saba_fit) over synthetic replay logs; prints its own
+    JSON line (not the benchmark's metric)."""
+    from paper_2608_20375_b200 import Graft
+    import oracle  # CPU-baseline leg only
+
+    n = 16_000_000  # 36 bytes a round: 576 MB, well over L2
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    g = Graft(1000, 4, 4, 16, 8, 1, 8, 8, 8, 0.0, 1, 0, 0)
+    lg = gi.saba_replay_logs(n, seed=20383)
+    d = {k: torch.from_numpy(np.ascontiguousarray(v)).to(dev) for k, v in lg.items()}
+    out = torch.zeros(10, dtype=torch.float64, device=dev)
+
+    def step():
+        g.saba_fit(d["state"], d["budget"], d["gain"], d["prefix_len"], d["latency"], out)
+
+    for _ in range(max(3, args.warmup or 3)):
+        step()
+    torch.cuda.synchronize()
+    steps = args.steps or 20
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    n_s = 2_000_000
+    t0 = time.perf_counter()
+    ref = oracle.saba_fit(**{k: v[:n_s] for k, v in lg.items()})
+    t_cpu = time.perf_counter() - t0
+    hbm_peak, peak_kind = _peaks()
+    alg = n * 36
+    print(json.dumps({
+        "kind": "least-squares fit of the SABA gain and cost models (graft_saba_fit)", "rounds_logged": n,
+        "ms_per_fit": round(ms, 4), "algorithmic_bytes": alg, "achieved_gbs": round(alg / (ms * 1e-3) / 1e9, 1),
+        "hbm_peak_gbs": hbm_peak, "peak_kind": "of " + peak_kind, "frac": round(alg / (ms * 1e-3) / 1e9 / hbm_peak, 3),
+        "fit": [float(x) for x in out.cpu().numpy()],
+        "cpu_oracle": {"rounds": n_s, "seconds": round(t_cpu, 3), "rounds_per_s": round(n_s / t_cpu),
+                       "phi": [float(x) for x in ref["phi"]], "c": [float(x) for x in ref["c"]]},
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -560,7 +604,12 @@ def main():
                          "duration, sequential against overlapped schedule")
     ap.add_argument("--tdes-loss", action="store_true",
                     help="instead of the benchmark: time the TDES training objective (forward + backward)")
+    ap.add_argument("--saba-fit", action="store_true",
+                    help="instead of the benchmark: time the least-squares fit of the SABA models")
     args = ap.parse_args()
+    if args.saba_fit and args.impl == "graft":
+        run_saba_fit(args)
+        return
     if args.tdes_loss and args.impl == "graft":
         run_tdes_loss(args)
         return

@@ -267,6 +267,22 @@ graft_status graft_tdes_loss(graft_ctx* ctx, const graft_tdes_traces* traces, co
                              double* d_loss, int32_t* d_skipped, float* d_gP, float* d_gC, float* d_gu, float* d_gs,
                              void* stream);
 
+/* Least-squares fit of the SABA gain and cost models (Eq. 16, 17) to replay logs resident on the device.  The paper
+ * fits them on held-out prompts by same-prefix budget replay without giving the procedure; this is ordinary least
+ * squares on n logged rounds:
+ *   d_state [n, 3] fp32 (conf, degen, hist of Eq. 15), d_budget [n] int32 B, d_gain [n] fp32 (the share of the
+ *   attainable accepted length that budget B reached, in [0, 1]), d_prefix_len [n] int32, d_latency [n] fp32 (the
+ *   round's cost in the unit C_t is wanted in).
+ *   Gain: a logged 0 < g < 1 gives tau = -B / ln(1 - g); (phi, bias) minimise sum (tau - phi . s - bias)^2 (rounds
+ *   with g <= 0 or g >= 1 are left out).  Cost: (c0, c1, c2) minimise sum (T - c0 - c1 B - c2 B prefix)^2.
+ *   d_out [10] fp64 (overwritten): phi_conf, phi_degen, phi_hist, phi_bias, c0, c1, c2, rounds used for the gain
+ *   fit, rounds used for the cost fit, status (bit 0: gain system singular or fewer than 4 rounds, bit 1: cost
+ *   system singular or fewer than 3; the parameters of a failed fit are 0).  The values go into graft_saba_params
+ *   on the host (graft_set_saba).  fp64 arithmetic. */
+graft_status graft_saba_fit(graft_ctx* ctx, int64_t n, const float* d_state, const int32_t* d_budget,
+                            const float* d_gain, const int32_t* d_prefix_len, const float* d_latency, double* d_out,
+                            void* stream);
+
 /* Host-buffer form of graft_build_trees for end-to-end use: every pointer here is a HOST pointer (pinned
  * memory makes the copies asynchronous).  Copies the inputs host->device into context-owned staging buffers
  * (allocated on first use, sized for max_batch), runs the same kernels as graft_build_trees, copies

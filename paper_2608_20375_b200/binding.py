@@ -21,7 +21,7 @@ ST_BAD_LOGITS, ST_TAU_CLAMPED, ST_FRONTIER_EMPTY, ST_INTERNAL = 1, 2, 4, 8
 ENTRY_POINTS = [
     "graft_create", "graft_destroy", "graft_nmax", "graft_mask_words", "graft_set_saba", "graft_set_tdes_tables",
     "graft_tdes_precompute", "graft_build_trees", "graft_vocab_pass", "graft_vocab_pass_static", "graft_tdes_edges",
-    "graft_accept", "graft_tdes_loss", "graft_set_edge_rows", "graft_edge_rows", "graft_set_hist_window", "graft_vocab_pass_partial", "graft_vocab_merge",
+    "graft_accept", "graft_tdes_loss", "graft_saba_fit", "graft_set_edge_rows", "graft_edge_rows", "graft_set_hist_window", "graft_vocab_pass_partial", "graft_vocab_merge",
     "graft_build_trees_host", "graft_launch_count", "graft_set_timing", "graft_read_timing", "graft_status_str",
     "graft_version",
 ]
@@ -107,6 +107,7 @@ def load_library():
     lib.graft_vocab_pass_static.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int, vp, vp, vp, vp, vp, vp]
     lib.graft_accept.argtypes = [vp, C.c_int32, C.POINTER(_TreeOut), vp, vp, vp, vp, vp]
     lib.graft_tdes_loss.argtypes = [vp, C.POINTER(_TdesTraces), C.POINTER(_TdesLossConfig), vp, vp, vp, vp, vp, vp, vp]
+    lib.graft_saba_fit.argtypes = [vp, C.c_int64, vp, vp, vp, vp, vp, vp, vp]
     lib.graft_launch_count.argtypes = [vp]
     lib.graft_launch_count.restype = C.c_uint64
     lib.graft_set_timing.argtypes = [vp, C.c_int32]
@@ -364,6 +365,15 @@ class Graft:
         _check(self.lib, self.lib.graft_tdes_loss(self._ctx, C.byref(t), C.byref(lc), _ptr(loss, torch.float64),
                                                   _ptr(skipped, i32), _ptr(gP, f32), _ptr(gC, f32), _ptr(gu, f32),
                                                   _ptr(gs, f32), _stream()), "graft_tdes_loss")
+
+    def saba_fit(self, state, budget, gain, prefix_len, latency, out):
+        """Least-squares fit of the gain and cost models (Eq. 16-17) to n logged rounds on the device.
+        state [n, 3] float32, budget / prefix_len [n] int32, gain / latency [n] float32; out: float64 [10] =
+        phi_conf, phi_degen, phi_hist, phi_bias, c0, c1, c2, rounds in the gain fit, rounds in the cost fit, status."""
+        i32, f32 = torch.int32, torch.float32
+        _check(self.lib, self.lib.graft_saba_fit(self._ctx, int(budget.numel()), _ptr(state, f32), _ptr(budget, i32),
+                                                 _ptr(gain, f32), _ptr(prefix_len, i32), _ptr(latency, f32),
+                                                 _ptr(out, torch.float64), _stream()), "graft_saba_fit")
 
     # ---- bookkeeping
     def launch_count(self) -> int:

@@ -24,6 +24,7 @@ SOURCES = {
     "tdes.cu": ALL_HEADERS,
     "tree.cu": ALL_HEADERS,
     "tdes_train.cu": ["common.cuh", "internal.h", GRAFT_H],
+    "saba_fit.cu": ["common.cuh", "internal.h", GRAFT_H],
     "s0_gemm.cu": ["internal.h", GRAFT_H],
 }
 # no --use_fast_math: the fp64 pieces (log-sum-exp fold, SABA) and the fp32 divisions must stay IEEE

@@ -127,7 +127,7 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     const size_t o_id = take(B * L * K * 4), o_lp = take(B * L * K * 4), o_lse = take(B * L * 4);
     const size_t o_rs = take(B * L * 4), o_edge = take(B * L * K * K * 4);
     const size_t o_es = take(B * L * K * K * 4), o_ei = take(B * L * K * K);
-    const size_t o_u = take(L * (size_t)cfg->m * 4), o_err = take(256), o_cos = take(B * L * 8), o_saba = take(B * sizeof(SabaResult));
+    const size_t o_u = take(L * (size_t)cfg->m * 4), o_err = take(256), o_cos = take(B * L * 8), o_saba = take(B * sizeof(SabaResult)), o_fit = take(32 * 8);
     ctx->ws_bytes = off;
     if (cudaMalloc(&ctx->ws, ctx->ws_bytes) != cudaSuccess) {
         cudaGetLastError();
@@ -163,6 +163,7 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     ctx->w_errflag = (int32_t*)(base + o_err);
     ctx->w_cos = (double*)(base + o_cos);
     ctx->w_saba = (SabaResult*)(base + o_saba);
+    ctx->w_fit = (double*)(base + o_fit);
     *out = ctx;
     return GRAFT_OK;
 }
@@ -286,6 +287,17 @@ graft_status graft_vocab_pass(graft_ctx* ctx, int32_t batch, const void* d_logit
     if ((uintptr_t)d_logits % esz) return GRAFT_ERR_INVALID_ARG;
     if (vp_launch(ctx, batch, d_logits, d_topk_id, d_topk_lp, d_lse, d_row_status ? d_row_status : ctx->w_row_status,
                   nullptr, nullptr, nullptr, (cudaStream_t)stream) != cudaSuccess)
+        return GRAFT_ERR_CUDA;
+    return GRAFT_OK;
+}
+
+graft_status graft_saba_fit(graft_ctx* ctx, int64_t n, const float* d_state, const int32_t* d_budget,
+                            const float* d_gain, const int32_t* d_prefix_len, const float* d_latency, double* d_out,
+                            void* stream) {
+    if (!ctx || n < 1 || !d_state || !d_budget || !d_gain || !d_prefix_len || !d_latency || !d_out)
+        return GRAFT_ERR_INVALID_ARG;
+    if (saba_fit_launch(ctx, (long long)n, d_state, d_budget, d_gain, d_prefix_len, d_latency, d_out,
+                        (cudaStream_t)stream) != cudaSuccess)
         return GRAFT_ERR_CUDA;
     return GRAFT_OK;
 }

@@ -87,6 +87,7 @@ struct graft_ctx {
     uint8_t* w_eidx;              // [max_batch, L, K, K] child rank of each sorted entry
     double* w_cos;                // [max_batch, L] adjacent-position cosines (Eq. 15)
     graft::SabaResult* w_saba;    // [max_batch] budgets worked out by the edge-score kernel
+    double* w_fit;                // [32] normal equations of graft_saba_fit and its arrival counter, zero between calls
     int32_t* w_errflag;           // [1] device-side internal error flag
     graft::VpPlan vp_plan;
     // scratch of the tensor-core table precompute (allocated on its first use: three bf16 copies of W, GEMM workspace)
@@ -157,6 +158,9 @@ cudaError_t tdes_loss_launch(graft_ctx* ctx, const graft_tdes_traces* tr, const 
                              cudaStream_t st);
 cudaError_t tdes_loss_configure(const graft_config& cfg);
 bool tdes_loss_supported(const graft_config& cfg);
+cudaError_t saba_fit_launch(graft_ctx* ctx, long long n, const float* d_state, const int32_t* d_budget,
+                            const float* d_gain, const int32_t* d_prefix, const float* d_latency, double* d_out,
+                            cudaStream_t st);
 size_t tree_smem_bytes(const graft_config& cfg);
 bool tree_lazy_fits(const graft_config& cfg);  // edge scores are computed inside the tree kernel
 
