@@ -420,6 +420,12 @@ __device__ __forceinline__ void vp_finalize(double Cd, double Sd, uint32_t Vm, i
     // log-sum-exp of the logits scaled by a = c ln 2 = 1 + 1.3e-8.  To first order that adds
     // (a - 1) E_q[z]; the largest logit stands in for the mean under q (the difference is a few
     // units times 1e-8).
+    // every lane must use the same bits: the folds that produced C and S are butterflies of fused multiply-adds,
+    // which leave the lanes an ulp apart, and log-probabilities of equal logits (and their order) must not depend on
+    // the lane that writes them
+    Cd = __shfl_sync(0xFFFFFFFFu, Cd, 0);
+    Sd = __shfl_sync(0xFFFFFFFFu, Sd, 0);
+    Vm = __shfl_sync(0xFFFFFFFFu, Vm, 0);
     const float vmax = __uint_as_float(bits_from_ord(Vm));
     const double a_minus_1 = (double)kLog2e * kLn2 - 1.0;
     const double lse_d = (Cd + log2(Sd)) * kLn2 - a_minus_1 * (double)vmax;

@@ -49,6 +49,15 @@ def _vocab_case(z, K, dtype):
     fin = np.isfinite(b)
     assert np.array_equal(np.isneginf(a), np.isneginf(b))
     assert np.abs(a[fin] - b[fin]).max(initial=0) <= EPS
+    # candidates come in rank order, so their log-probabilities never increase along a row, and equal logits get the
+    # same bits (every candidate of a row is measured against one log-sum-exp)
+    with np.errstate(invalid="ignore"):
+        assert np.all(np.diff(a, axis=1) <= 0.0), "log-probabilities increase along a row"
+    zf = z.reshape(Bt * L, V).float().numpy()
+    for r in np.nonzero(good)[0][:64]:
+        vals = zf[r, ids[r]]
+        same = vals[1:] == vals[:-1]
+        assert np.array_equal(lp[r, 1:][same], lp[r, :-1][same]), f"row {r}: equal logits, different log-probabilities"
     # lse is returned as an fp32 number: allow its own rounding on top of EPS
     assert np.all(np.abs(lse[good, 0] - o_lse[good]) <= EPS + np.spacing(np.abs(lse[good, 0])))
     g.destroy()
@@ -332,6 +341,32 @@ def test_round_bad_rows_and_status_bits():
     orc = oracle_round(oracle, w, x, tb, saba_kw)
     assert gpu["status"].tolist() == [2, 1, 2, 1] == orc["status"].tolist()
     compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+
+
+@pytest.mark.parametrize("budget", [40, 600, 1000])
+def test_round_with_thousands_of_equal_path_scores(budget):
+    """Uniform rows and beta = 0: every prefix of a depth has the same score, so the threshold is decided among
+    thousands of equal keys (the exact select's list overflows and the radix passes take over) and the last nodes are
+    chosen by the order among equal scores alone.  One sequence has a single raised token per row, so that a few
+    hundred distinct scores sit beside the ties."""
+    w = gi.small(batch=3, L=5, V=2000, K=32, budget_min=budget, budget_max=budget, fixed_budget=budget, beta=0.0, m=16)
+    g = _graft(w)
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    x["logits"][:] = 0.0
+    x["logits"][1, :, 3] = 2.0
+    x["logits"][2, 1:, :] = torch.round(x["logits"][2, 1:, :] + torch.arange(w.V) % 3)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    # the sequences with a raised token add the same few fp32 numbers in different orders along different paths, so
+    # their near-ties may fall differently on log-probabilities that differ within the tolerance (checked as valid
+    # best-first outcomes by compare_round); the all-uniform sequence has exact ties and must match bit for bit
+    assert stats["excused_budget"] == 0 and stats["excused_tree"] <= 2, stats
+    for k in ("token", "parent", "depth", "mask"):
+        assert np.array_equal(gpu[k][0], orc[k][0]), k
+    assert gpu["n_nodes"].tolist() == [budget + 1] * 3
+    compare_accept(oracle, gi, g, w, out, gpu)
 
 
 def test_round_affine_cost_and_paper_grid():
