@@ -246,6 +246,46 @@ __device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, in
     return prefix;
 }
 
+// The exact B-th largest key once its top 16 bits are known (`prefix` and `remaining` as passes 0 and 1 of the radix
+// select left them).  The keys that share those 16 bits are few (path scores are spread over many more than 65536
+// values), so they are collected and ranked against each other directly, which takes three barriers instead of the
+// five of two more radix passes; if there are more than the list holds (heavy ties), the radix passes run after all.
+__device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, int lo, int hi, int kth, uint32_t prefix,
+                                      int& remaining, int tid) {
+    constexpr int kCap = 512;
+    uint32_t* list = sm.hist;           // [kCap] (the histogram space is idle between selects)
+    int* cnt = (int*)(sm.hist + 1024);  // [1]
+    if (tid == 0) *cnt = 0;
+    __syncthreads();
+    for (int i = lo + tid; i < hi; i += TREE_THREADS) {
+        const uint32_t k = keys[i];
+        if ((k & 0xFFFF0000u) == prefix) {
+            const int pos = atomicAdd(cnt, 1);
+            if (pos < kCap) list[pos] = k;
+        }
+    }
+    __syncthreads();
+    const int n = *cnt;
+    if (n > kCap) {  // (uniform)
+        __syncthreads();
+        return cta_kth_largest(sm, keys, lo, hi, kth, 2, 4, prefix, remaining, tid);
+    }
+    for (int i = tid; i < n; i += TREE_THREADS) {
+        const uint32_t k = list[i];
+        int gt = 0, ge = 0;
+        for (int j = 0; j < n; ++j) {
+            const uint32_t o = list[j];
+            gt += o > k ? 1 : 0;
+            ge += o >= k ? 1 : 0;
+        }
+        if (gt < remaining && remaining <= ge) sm.scal[6] = (int)k;  // (every writer writes the same value)
+    }
+    __syncthreads();
+    const uint32_t v = (uint32_t)sm.scal[6];
+    __syncthreads();  // the list and the result word are free again
+    return v;
+}
+
 // ---- edge scores on demand --------------------------------------------------------------------------------------
 // Row j of the edge scores (children at depth j+1), Eq. 4-6: the table rows P[parent token], C[child token] and
 // u_j are copied into shared memory asynchronously (16-byte cp.async chunks spread over the CTA, issued while the
@@ -653,10 +693,9 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         __syncthreads();
         if (table_ok && ntot - 1 >= budget) {
             // the exact value: the last 16-bit search still holds if nothing was appended after it
-            if (n_at_select == ntot && theta != 0u)
-                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 2, 4, theta, sel_rem, tid);
-            else
-                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 0, 4, 0u, sel_rem, tid);
+            if (!(n_at_select == ntot && theta != 0u))
+                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 0, 2, 0u, sel_rem, tid);
+            theta = cta_finish_select(sm, sm.nkey, 1, ntot, budget, theta, sel_rem, tid);
         }
         __syncthreads();
         if (table_ok) {
