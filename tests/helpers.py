@@ -75,7 +75,8 @@ def _close(a, b, tol):
     a = np.asarray(a, np.float64)
     b = np.asarray(b, np.float64)
     same_inf = np.isinf(a) & np.isinf(b) & (np.sign(a) == np.sign(b))
-    return bool(np.all(same_inf | (np.abs(a - b) <= tol)))
+    with np.errstate(invalid="ignore"):  # inf - inf where both sides are the same infinity
+        return bool(np.all(same_inf | (np.abs(a - b) <= tol)))
 
 
 def compare_round(oracle, w, x, tb, saba_kw, gpu, orc):

@@ -369,6 +369,28 @@ def test_round_with_thousands_of_equal_path_scores(budget):
     compare_accept(oracle, gi, g, w, out, gpu)
 
 
+@pytest.mark.parametrize("budget", [20, 50, 150])
+def test_round_with_equal_scores_across_depths_and_masked_tokens(budget):
+    """Sequence 0: below a uniform first position every later position has one token of probability 1 to fp32
+    precision, so a depth-1 prefix and the chain under it have exactly the same path score and the order among equal
+    scores (shallower first, then the order of the prefixes) decides across depths.  Sequence 1: only five tokens
+    of a K = 8 candidate set are finite at the deeper positions, so three children of every node score -inf."""
+    w = gi.small(batch=2, L=5, V=500, K=8, budget_min=budget, budget_max=budget, fixed_budget=budget, beta=0.0, m=16)
+    g = _graft(w)
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    x["logits"][0] = 0.0
+    x["logits"][0, 1:, 7] = 40.0
+    x["logits"][1, 1:, 5:] = float("-inf")
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    assert stats["excused_budget"] == 0 and stats["excused_tree"] <= 1, stats
+    for k in ("n_nodes", "token", "parent", "depth", "mask", "status"):
+        assert np.array_equal(gpu[k][0], orc[k][0]), k
+    compare_accept(oracle, gi, g, w, out, gpu)
+
+
 def test_round_affine_cost_and_paper_grid():
     w = gi.small(batch=6, L=8, V=4000, K=8, budget_min=32, budget_max=512, budget_step=16, hidden_dim=96)
     g = _graft(w)
