@@ -561,3 +561,24 @@ def test_round_seeded_sweep_of_shapes(kw, rows):
     assert stats["excused_tree"] + stats["excused_budget"] <= max(1, w.batch // 2), stats
     compare_accept(oracle, gi, g, w, out, gpu)
     g.destroy()
+
+
+@pytest.mark.parametrize("kw", _fuzz_cases()[:10])
+@pytest.mark.parametrize("step", [1.0, 0.25])
+def test_round_seeded_sweep_with_quantised_logits(kw, step):
+    """The same odd shapes with logits rounded to a coarse grid: the candidates of a row hold many equal values, so
+    log-probabilities, edge scores and path scores tie in bulk (exactly with beta = 0, up to the fp32 rounding of
+    different summation orders otherwise).  Every tree must still be the oracle's or a valid best-first outcome on
+    the oracle's scores, and with beta = 0 and exact ties it must be the oracle's."""
+    w = gi.small(**kw)
+    g = _graft(w)
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    z = x["logits"].float()
+    x["logits"] = (torch.round(z / step) * step).to(x["logits"].dtype)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    assert stats["excused_budget"] <= max(1, w.batch // 2), stats
+    compare_accept(oracle, gi, g, w, out, gpu)
+    g.destroy()
