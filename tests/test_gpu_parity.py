@@ -97,6 +97,29 @@ def test_vocab_pass_ties_uniform_masked_and_bad_rows():
     _vocab_case(z.to(torch.bfloat16), K, "bf16")
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_vocab_pass_full_width_rows_with_bulk_ties(dtype):
+    """Rows of the full vocabulary width, cut across CTAs, in which almost every element ties with the K-th largest:
+    the candidate filter lets everything through, so the exact selection over the whole segment takes over, and the
+    ids alone decide across the pieces of a row."""
+    V, K, L = 151936, 32, 8
+    g = torch.Generator().manual_seed(9)
+    z = torch.zeros((2, L, V))
+    z[0, 0] = 1.25                                                    # all equal
+    z[0, 1] = torch.round(torch.randn(V, generator=g))                # seven or so distinct values
+    z[0, 2] = -(torch.arange(V) // 4096).float()                      # descending plateaus of 4096
+    z[0, 3] = (torch.arange(V) // 4096).float()                       # ascending plateaus: the best sit at the end
+    z[0, 4, :] = float("-inf")
+    z[0, 4, V - 40:] = 3.0                                            # forty finite elements at the very end
+    z[0, 5, ::2] = 1.0                                                # alternating
+    z[0, 6] = torch.randn(V, generator=g)
+    z[0, 6, 1000:1000 + K + 5] = 9.0                                  # K + 5 tied winners inside one piece
+    z[0, 7] = torch.randn(V, generator=g)
+    z[0, 7, torch.arange(0, V, V // 40)] = 9.0                        # forty tied winners spread over every piece
+    z[1] = z[0].flip(0)
+    _vocab_case(z.to(torch.bfloat16) if dtype == "bf16" else z, K, dtype)
+
+
 def test_vocab_pass_large_magnitudes_and_negative_zero():
     V, K = 5000, 8
     g = torch.Generator().manual_seed(2)
@@ -580,5 +603,53 @@ def test_round_seeded_sweep_with_quantised_logits(kw, step):
     orc = oracle_round(oracle, w, x, tb, saba_kw)
     stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
     assert stats["excused_budget"] <= max(1, w.batch // 2), stats
+    compare_accept(oracle, gi, g, w, out, gpu)
+    g.destroy()
+
+
+@pytest.mark.parametrize("noise", [0.0, 1e-3])
+@pytest.mark.parametrize("beta", [0.0, 0.2])
+def test_round_when_the_node_table_overflows(noise, beta):
+    """Flat distributions with K = 20 and a budget of 1000: levels 0..2 hold 421 prefixes, fewer than the budget, so
+    level 3 would append 8000 more with no threshold to prune by, which is more than the node table of the parallel
+    phase holds; the sequential expansion then builds the whole tree."""
+    w = gi.small(batch=2, L=4, V=700, K=20, budget_min=1000, budget_max=1000, fixed_budget=1000, beta=beta, m=16)
+    g = _graft(w)
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    gen = torch.Generator().manual_seed(3)
+    x["logits"] = noise * torch.randn(x["logits"].shape, generator=gen)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    assert stats["excused_budget"] == 0, stats
+    assert gpu["n_nodes"].tolist() == [1001, 1001] and gpu["status"].tolist() == [0, 0]
+    if noise == 0.0 and beta == 0.0:
+        for k in ("token", "parent", "depth", "mask"):
+            assert np.array_equal(gpu[k], orc[k]), k
+    compare_accept(oracle, gi, g, w, out, gpu)
+    g.destroy()
+
+
+@pytest.mark.parametrize("K,L", [(5, 6), (32, 4)])
+def test_round_with_identical_table_rows_and_tied_candidates(K, L):
+    """Every token has the same projections, so f is the same for every edge of a depth and the centred score
+    vanishes up to rounding: edge scores tie wherever the candidates' log-probabilities tie (logits on a coarse
+    grid), and the rows' order falls back on the candidates' rank."""
+    w = gi.small(batch=3, L=L, V=900, K=K, budget_min=8, budget_max=200, budget_step=8, beta=0.7, m=24, seed=31)
+    from paper_2608_20375_b200 import Graft
+    g = Graft(w.V, w.L, w.K, w.m, w.hidden_dim, w.batch, w.budget_min, w.budget_max, w.budget_step, w.beta, 1, 0, 0)
+    tb = gi.tdes_tables(w)
+    tb["P"][:] = tb["P"][0]
+    tb["C"][:] = tb["C"][1]
+    saba_kw = gi.saba_defaults(w)
+    keep = [tb["P"].cuda(), tb["C"].cuda(), tb["u"].cuda()]
+    g.set_tdes_tables(keep[0], keep[1], keep[2], tb["s"])
+    g.set_saba(**saba_kw)
+    x = gi.batch_inputs(w)
+    x["logits"] = torch.round(x["logits"] * 2) / 2
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
     compare_accept(oracle, gi, g, w, out, gpu)
     g.destroy()
