@@ -653,3 +653,31 @@ def test_round_with_identical_table_rows_and_tied_candidates(K, L):
     compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
     compare_accept(oracle, gi, g, w, out, gpu)
     g.destroy()
+
+
+@pytest.mark.parametrize("beta", [0.0, 0.3])
+@pytest.mark.parametrize("rows", [None, 0, 3])
+def test_round_deep_trees_with_ties_scored_on_demand(beta, rows):
+    """Narrow candidate sets and peaked distributions on a coarse grid give trees sixteen levels deep with ties at
+    every level; the deeper edge rows are scored inside the tree kernel.  The call without debug outputs (the one
+    the benchmark times) must give the trees of the call that is checked against the oracle, bit for bit."""
+    w = gi.small(batch=4, L=16, V=3000, K=3, budget_min=16, budget_max=256, budget_step=16, beta=beta, m=32, seed=77,
+                 boost_lo=12.0, boost_hi=16.0)
+    g = _graft(w)
+    if rows is not None:
+        g.set_edge_rows(rows)
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    x["logits"] = torch.round(x["logits"])
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    assert int(gpu["depth"].max()) >= 10  # beyond the depths the edge-score kernel covers by default
+    out_p = g.alloc_out(w.batch, debug=False)
+    cu = lambda t: t.cuda()  # noqa: E731
+    g.build_trees(cu(x["logits"]), cu(x["hidden"]), cu(x["root_token"]), cu(x["hist"]), cu(x["prefix_len"]), None, out_p)
+    torch.cuda.synchronize()
+    prod = out_p.cpu()
+    for k in ("n_nodes", "budget", "status", "token", "parent", "depth", "position", "path_score", "mask"):
+        assert np.array_equal(prod[k], gpu[k]), k
+    g.destroy()
