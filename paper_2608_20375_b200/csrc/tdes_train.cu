@@ -113,7 +113,9 @@ struct WarpCache {
     int* credit;  // [2][kTrSlots]
 };
 // gradient row of token `tok` of table t (0: gP, 1: gC) += coef * r
-template <int NCH>
+// INSTALL = false: a token that is not cached goes straight to global memory without touching the slots' credits
+// (the K children of a group: one hot token among them would otherwise be chased out by the other K - 1)
+template <int NCH, bool INSTALL = true>
 __device__ __forceinline__ void add_row(const TrainParams& p, const WarpCache& wc, int t, int tok, int lane, float coef,
                                         const Row<NCH>& r) {
     float* dst = t == 0 ? p.gP : p.gC;
@@ -137,6 +139,10 @@ __device__ __forceinline__ void add_row(const TrainParams& p, const WarpCache& w
             if (c < kTrCreditMax) wc.credit[t * kTrSlots + slot] = c + 1;
         }
         __syncwarp();
+        return;
+    }
+    if (!INSTALL) {
+        if (lane < p.m / 4) atomicAdd((float4*)(dst + (size_t)tok * p.m) + lane, add);
         return;
     }
     const int4 cr = *(const int4*)(wc.credit + kTrSlots * t);
@@ -296,7 +302,7 @@ __global__ void __launch_bounds__(kTrThreads) tdes_loss_kernel(const TrainParams
                 const int t = __shfl_sync(0xFFFFFFFFu, tc, c);
                 const float coef = __shfl_sync(0xFFFFFFFFu, gf_c, c) * p.k0;
                 const Row<NCH> b = load_row_plus_u<NCH>(p.C, urow, t, p.m, lane);
-                add_row<NCH>(p, wc, 1, t, lane, coef, a);
+                add_row<NCH, false>(p, wc, 1, t, lane, coef, a);
 #pragma unroll
                 for (int ch = 0; ch < NCH; ++ch) {
                     accP.v[ch].x = fmaf(coef, b.v[ch].x, accP.v[ch].x);
