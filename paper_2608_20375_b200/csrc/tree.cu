@@ -246,20 +246,102 @@ __device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, in
     return prefix;
 }
 
-// The exact B-th largest key once its top 16 bits are known (`prefix` and `remaining` as passes 0 and 1 of the radix
-// select left them).  The keys that share those 16 bits are few (path scores are spread over many more than 65536
-// values), so they are collected and ranked against each other directly, which takes three barriers instead of the
-// five of two more radix passes; if there are more than the list holds (heavy ties), the radix passes run after all.
-__device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, int lo, int hi, int kth, uint32_t prefix,
-                                      int& remaining, int tid) {
+// Base and bin width of cta_select_bucket from the largest key: 1024 bins reach from the best score to 128 below it.
+__device__ __forceinline__ void select_range(uint32_t best_key, uint32_t& base, int& shift) {
+    base = best_key;
+    const float top = __uint_as_float(bits_from_ord(best_key));
+    const uint32_t low = ord_from_float(top - 128.0f);
+    const uint32_t range = base >= low ? base - low : 0u;
+    shift = 32 - __clz((int)(range >> 10));
+    if ((range >> 10) == 0u) shift = 0;
+}
+
+// Where the B-th largest key lies: a closed range of key values and the rank wanted inside it.
+struct SelBucket {
+    uint32_t lo, hi;  // lo is a lower bound of the B-th largest key
+    int rem;          // the B-th largest of all is the rem-th largest of the keys in [lo, hi]
+    bool valid;
+};
+
+// One histogram pass over keys[lo_i..hi_i): 1024 bins of equal width in key (ord) space, counted down from `base`,
+// an upper bound of every key (keys further than 1023 bins below it share the last bin).  With the bin width taken
+// from the key distance between the best score and that score minus 128, a bin spans about as much as a key's top
+// 16 bits do, so its lower edge prunes as well as two 8-bit radix passes would, for one pass and three barriers.
+// If the B-th largest falls into the shared last bin, two radix passes find its 16-bit bucket instead.
+// Bins are padded by one word per 32 so that warp 0's lanes, which own 32 consecutive bins each, read without
+// bank conflicts.  Every thread of the CTA calls this; hi_i - lo_i >= kth >= 1.
+__device__ uint32_t cta_select_bucket(const TreeSmem& sm, const uint32_t* keys, int lo_i, int hi_i, int kth,
+                                      uint32_t base, int shift, SelBucket& st, int tid) {
+    const int warp = tid >> 5, lane = tid & 31;
+    uint32_t* h = sm.hist;  // [1024 + 32]
+    h[tid] = 0u;
+    if (tid < 32) h[1024 + tid] = 0u;
+    __syncthreads();
+    for (int i = lo_i + tid; i < hi_i; i += TREE_THREADS) {
+        const uint32_t k = keys[i];
+        uint32_t d = base >= k ? (base - k) >> shift : 0u;
+        d = d > 1023u ? 1023u : d;
+        atomicAdd(&h[d + (d >> 5)], 1u);
+    }
+    __syncthreads();
+    if (warp == 0) {  // lane l owns bins 32 l .. 32 l + 31 (bin 0 holds the largest keys)
+        const uint32_t* mine = h + 33 * lane;
+        int sum = 0;
+#pragma unroll 8
+        for (int q = 0; q < 32; ++q) sum += (int)mine[q];
+        int incl = sum;
+#pragma unroll
+        for (int o2 = 1; o2 < 32; o2 <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
+            if (lane >= o2) incl += t;
+        }
+        const int excl = incl - sum;
+        if (excl < kth && kth <= incl) {
+            int acc = excl, bin = 32 * lane, rem = kth - excl;
+            for (int q = 0; q < 32; ++q) {
+                const int c = (int)mine[q];
+                if (acc < kth && kth <= acc + c) {
+                    bin = 32 * lane + q;
+                    rem = kth - acc;
+                }
+                acc += c;
+            }
+            sm.scal[6] = bin;
+            sm.scal[7] = rem;
+        }
+    }
+    __syncthreads();
+    const int bin = sm.scal[6];
+    st.rem = sm.scal[7];
+    st.valid = true;
+    if (bin >= 1023) {  // (uniform) below the range the bins resolve
+        __syncthreads();
+        int rem = 0;
+        const uint32_t prefix = cta_kth_largest(sm, keys, lo_i, hi_i, kth, 0, 2, 0u, rem, tid);
+        st.lo = prefix;
+        st.hi = prefix | 0xFFFFu;
+        st.rem = rem;
+        return st.lo;
+    }
+    const uint64_t below = ((uint64_t)bin + 1ull) << shift;  // keys of this bin are > base - below
+    st.lo = below > (uint64_t)base ? 0u : base - (uint32_t)below + 1u;
+    st.hi = base - ((uint32_t)bin << shift);
+    return st.lo;
+}
+
+// The exact B-th largest key once its bucket is known: the keys inside it are few (path scores are spread over
+// many more values than there are buckets), so they are collected and ranked against each other directly; if there
+// are more than the list holds (heavy ties), a full radix select runs instead.
+__device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, int lo_i, int hi_i, int kth,
+                                      const SelBucket& st, int tid) {
     constexpr int kCap = 512;
     uint32_t* list = sm.hist;           // [kCap] (the histogram space is idle between selects)
-    int* cnt = (int*)(sm.hist + 1024);  // [1]
+    int* cnt = (int*)(sm.hist + 1100);  // [1]
     if (tid == 0) *cnt = 0;
     __syncthreads();
-    for (int i = lo + tid; i < hi; i += TREE_THREADS) {
+    for (int i = lo_i + tid; i < hi_i; i += TREE_THREADS) {
         const uint32_t k = keys[i];
-        if ((k & 0xFFFF0000u) == prefix) {
+        if (k >= st.lo && k <= st.hi) {
             const int pos = atomicAdd(cnt, 1);
             if (pos < kCap) list[pos] = k;
         }
@@ -268,8 +350,10 @@ __device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, 
     const int n = *cnt;
     if (n > kCap) {  // (uniform)
         __syncthreads();
-        return cta_kth_largest(sm, keys, lo, hi, kth, 2, 4, prefix, remaining, tid);
+        int rem = 0;
+        return cta_kth_largest(sm, keys, lo_i, hi_i, kth, 0, 4, 0u, rem, tid);
     }
+    const int remaining = st.rem;
     for (int i = tid; i < n; i += TREE_THREADS) {
         const uint32_t k = list[i];
         int gt = 0, ge = 0;
@@ -510,11 +594,16 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     bool table_ok = budget > 0;
     uint32_t theta = 0u;
     if (budget > 0) {
-        int ntot = 1, n_at_select = 1, sel_rem = 0;
+        int ntot = 1, n_at_select = 1;
+        SelBucket sel;
+        sel.valid = false;
+        uint32_t sel_base = 0u;  // the largest key (the root's best child) and the bin width of the threshold searches
+        int sel_shift = 0;
         if (spec) {  // levels 0 and 1 are in the table already: the threshold they give, then on from level 2
             ntot = 1 + K + K * K;
             if (ntot - 1 >= budget) {
-                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 0, 2, 0u, sel_rem, tid);
+                select_range(sm.nkey[1], sel_base, sel_shift);
+                theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_base, sel_shift, sel, tid);
                 n_at_select = ntot;
             }
             __syncthreads();
@@ -676,7 +765,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             // theta only has to be a lower bound of its final value while the levels are built (it prunes), so
             // the exact B-th largest key is recomputed only when the table has grown noticeably
             if (ntot - 1 >= budget && (theta == 0u || ntot - n_at_select >= ntot / 2)) {
-                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 0, 2, 0u, sel_rem, tid);  // a 16-bit lower bound
+                select_range(sm.nkey[1], sel_base, sel_shift);
+                theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_base, sel_shift, sel, tid);  // a lower bound
                 n_at_select = ntot;
             }
             __syncthreads();
@@ -693,9 +783,11 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         __syncthreads();
         if (table_ok && ntot - 1 >= budget) {
             // the exact value: the last 16-bit search still holds if nothing was appended after it
-            if (!(n_at_select == ntot && theta != 0u))
-                theta = cta_kth_largest(sm, sm.nkey, 1, ntot, budget, 0, 2, 0u, sel_rem, tid);
-            theta = cta_finish_select(sm, sm.nkey, 1, ntot, budget, theta, sel_rem, tid);
+            if (!(n_at_select == ntot && sel.valid)) {
+                select_range(sm.nkey[1], sel_base, sel_shift);
+                cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_base, sel_shift, sel, tid);
+            }
+            theta = cta_finish_select(sm, sm.nkey, 1, ntot, budget, sel, tid);
         }
         __syncthreads();
         if (table_ok) {
