@@ -246,41 +246,42 @@ __device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, in
     return prefix;
 }
 
-// Base and bin width of cta_select_bucket from the largest key: 1024 bins reach from the best score to 128 below it.
-__device__ __forceinline__ void select_range(uint32_t best_key, uint32_t& base, int& shift) {
-    base = best_key;
-    const float top = __uint_as_float(bits_from_ord(best_key));
-    const uint32_t low = ord_from_float(top - 128.0f);
-    const uint32_t range = base >= low ? base - low : 0u;
-    shift = 32 - __clz((int)(range >> 10));
-    if ((range >> 10) == 0u) shift = 0;
+// Threshold searches work on 1024 bins of equal width in SCORE below the best score (the root's best child): bin b
+// holds the keys whose score lies in (top - (b + 1) w, top - b w], w = 1/32, so the bins reach 32 below the top; what
+// lies further down (or is -inf) shares the last bin.  The same expression gives a key's bin wherever it is needed.
+constexpr float kSelBinsPerUnit = 32.0f;
+__device__ __forceinline__ int select_bin(uint32_t key, float top) {
+    const float d = (top - __uint_as_float(bits_from_ord(key))) * kSelBinsPerUnit;
+    if (!(d < 1023.0f)) return 1023;  // (also NaN)
+    return d > 0.0f ? (int)d : 0;
 }
 
-// Where the B-th largest key lies: a closed range of key values and the rank wanted inside it.
+// Where the B-th largest key lies and the rank wanted there.
 struct SelBucket {
-    uint32_t lo, hi;  // lo is a lower bound of the B-th largest key
-    int rem;          // the B-th largest of all is the rem-th largest of the keys in [lo, hi]
+    int bin;          // the bin of select_bin, or -1: the closed key range [lo, hi] instead
+    uint32_t lo, hi;
+    int rem;          // the B-th largest of all is the rem-th largest of the keys in the bucket
     bool valid;
 };
+__device__ __forceinline__ bool select_in_bucket(const SelBucket& st, uint32_t key, float top) {
+    return st.bin >= 0 ? select_bin(key, top) == st.bin : (key >= st.lo && key <= st.hi);
+}
 
-// One histogram pass over keys[lo_i..hi_i): 1024 bins of equal width in key (ord) space, counted down from `base`,
-// an upper bound of every key (keys further than 1023 bins below it share the last bin).  With the bin width taken
-// from the key distance between the best score and that score minus 128, a bin spans about as much as a key's top
-// 16 bits do, so its lower edge prunes as well as two 8-bit radix passes would, for one pass and three barriers.
-// If the B-th largest falls into the shared last bin, two radix passes find its 16-bit bucket instead.
-// Bins are padded by one word per 32 so that warp 0's lanes, which own 32 consecutive bins each, read without
-// bank conflicts.  Every thread of the CTA calls this; hi_i - lo_i >= kth >= 1.
-__device__ uint32_t cta_select_bucket(const TreeSmem& sm, const uint32_t* keys, int lo_i, int hi_i, int kth,
-                                      uint32_t base, int shift, SelBucket& st, int tid) {
+// One histogram pass over keys[lo_i..hi_i) finds the bin that holds the B-th largest key, and a lower bound of that
+// key (the bin's lower edge less a hundredth of a bin: the rounding of select_bin is below 1e-4 of a bin).  A bin spans about as much
+// as a key's top 16 bits do at the scores met here, so the bound prunes as well as two 8-bit radix passes would,
+// for one pass and three barriers.  If the B-th largest falls into the shared last bin, two radix passes find its
+// 16-bit bucket instead.  Bins are padded by one word per 32 so that warp 0's lanes, which own 32 consecutive bins
+// each, read without bank conflicts.  Every thread of the CTA calls this; hi_i - lo_i >= kth >= 1.
+__device__ uint32_t cta_select_bucket(const TreeSmem& sm, const uint32_t* keys, int lo_i, int hi_i, int kth, float top,
+                                      SelBucket& st, int tid) {
     const int warp = tid >> 5, lane = tid & 31;
     uint32_t* h = sm.hist;  // [1024 + 32]
     h[tid] = 0u;
     if (tid < 32) h[1024 + tid] = 0u;
     __syncthreads();
     for (int i = lo_i + tid; i < hi_i; i += TREE_THREADS) {
-        const uint32_t k = keys[i];
-        uint32_t d = base >= k ? (base - k) >> shift : 0u;
-        d = d > 1023u ? 1023u : d;
+        const int d = select_bin(keys[i], top);
         atomicAdd(&h[d + (d >> 5)], 1u);
     }
     __syncthreads();
@@ -318,21 +319,21 @@ __device__ uint32_t cta_select_bucket(const TreeSmem& sm, const uint32_t* keys, 
         __syncthreads();
         int rem = 0;
         const uint32_t prefix = cta_kth_largest(sm, keys, lo_i, hi_i, kth, 0, 2, 0u, rem, tid);
+        st.bin = -1;
         st.lo = prefix;
         st.hi = prefix | 0xFFFFu;
         st.rem = rem;
         return st.lo;
     }
-    const uint64_t below = ((uint64_t)bin + 1ull) << shift;  // keys of this bin are > base - below
-    st.lo = below > (uint64_t)base ? 0u : base - (uint32_t)below + 1u;
-    st.hi = base - ((uint32_t)bin << shift);
-    return st.lo;
+    st.bin = bin;
+    st.lo = st.hi = 0u;
+    return ord_from_float(top - ((float)(bin + 1) + 0.01f) / kSelBinsPerUnit);
 }
 
 // The exact B-th largest key once its bucket is known: the keys inside it are few (path scores are spread over
 // many more values than there are buckets), so they are collected and ranked against each other directly; if there
 // are more than the list holds (heavy ties), a full radix select runs instead.
-__device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, int lo_i, int hi_i, int kth,
+__device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, int lo_i, int hi_i, int kth, float top,
                                       const SelBucket& st, int tid) {
     constexpr int kCap = 512;
     uint32_t* list = sm.hist;           // [kCap] (the histogram space is idle between selects)
@@ -341,7 +342,7 @@ __device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, 
     __syncthreads();
     for (int i = lo_i + tid; i < hi_i; i += TREE_THREADS) {
         const uint32_t k = keys[i];
-        if (k >= st.lo && k <= st.hi) {
+        if (select_in_bucket(st, k, top)) {
             const int pos = atomicAdd(cnt, 1);
             if (pos < kCap) list[pos] = k;
         }
@@ -597,13 +598,12 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         int ntot = 1, n_at_select = 1;
         SelBucket sel;
         sel.valid = false;
-        uint32_t sel_base = 0u;  // the largest key (the root's best child) and the bin width of the threshold searches
-        int sel_shift = 0;
+        float sel_top = 0.0f;  // the best score (the root's best child): where the bins of the threshold searches start
         if (spec) {  // levels 0 and 1 are in the table already: the threshold they give, then on from level 2
             ntot = 1 + K + K * K;
             if (ntot - 1 >= budget) {
-                select_range(sm.nkey[1], sel_base, sel_shift);
-                theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_base, sel_shift, sel, tid);
+                sel_top = __uint_as_float(bits_from_ord(sm.nkey[1]));
+                theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);
                 n_at_select = ntot;
             }
             __syncthreads();
@@ -765,8 +765,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             // theta only has to be a lower bound of its final value while the levels are built (it prunes), so
             // the exact B-th largest key is recomputed only when the table has grown noticeably
             if (ntot - 1 >= budget && (theta == 0u || ntot - n_at_select >= ntot / 2)) {
-                select_range(sm.nkey[1], sel_base, sel_shift);
-                theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_base, sel_shift, sel, tid);  // a lower bound
+                sel_top = __uint_as_float(bits_from_ord(sm.nkey[1]));
+                theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);  // a lower bound
                 n_at_select = ntot;
             }
             __syncthreads();
@@ -784,10 +784,10 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         if (table_ok && ntot - 1 >= budget) {
             // the exact value: the last 16-bit search still holds if nothing was appended after it
             if (!(n_at_select == ntot && sel.valid)) {
-                select_range(sm.nkey[1], sel_base, sel_shift);
-                cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_base, sel_shift, sel, tid);
+                sel_top = __uint_as_float(bits_from_ord(sm.nkey[1]));
+                cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);
             }
-            theta = cta_finish_select(sm, sm.nkey, 1, ntot, budget, sel, tid);
+            theta = cta_finish_select(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);
         }
         __syncthreads();
         if (table_ok) {
