@@ -397,14 +397,19 @@ def test_round_with_equal_scores_across_depths_and_masked_tokens(budget):
     """Sequence 0: below a uniform first position every later position has one token of probability 1 to fp32
     precision, so a depth-1 prefix and the chain under it have exactly the same path score and the order among equal
     scores (shallower first, then the order of the prefixes) decides across depths.  Sequence 1: only five tokens
-    of a K = 8 candidate set are finite at the deeper positions, so three children of every node score -inf."""
-    w = gi.small(batch=2, L=5, V=500, K=8, budget_min=budget, budget_max=budget, fixed_budget=budget, beta=0.0, m=16)
+    of a K = 8 candidate set are finite at the deeper positions, so three children of every node score -inf.
+    Sequence 2: see below."""
+    w = gi.small(batch=3, L=5, V=500, K=8, budget_min=budget, budget_max=budget, fixed_budget=budget, beta=0.0, m=16)
     g = _graft(w)
     tb, saba_kw, keep = _setup(w, g)
     x = gi.batch_inputs(w)
     x["logits"][0] = 0.0
     x["logits"][0, 1:, 7] = 40.0
     x["logits"][1, 1:, 5:] = float("-inf")
+    # sequence 2: one token of probability 1 at every position, the rest 46 below: the threshold lies far below the
+    # best score (beyond the range the threshold search's bins resolve)
+    x["logits"][2] = 0.0
+    x["logits"][2, :, 7] = 40.0
     out, gpu = gpu_round(g, w, x)
     orc = oracle_round(oracle, w, x, tb, saba_kw)
     stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
