@@ -630,7 +630,11 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                             const float x = load_elem_f32(rowp + (size_t)e * T::ESZ, BF16);
                             const uint32_t o = ord_from_float(x);
                             vmo = o > vmo ? o : vmo;
-                            float c1 = x * kLog2e, s1 = 1.0f;
+                            // x log2(e) = c1 + r with c1 the rounded product and r its exact remainder (one FMA):
+                            // 2^r = 1 + r ln 2 keeps what the rounding of c1 drops (up to 2e-6 of the term at
+                            // |x| = 30, which is the whole error of the row when its largest logit sits here)
+                            float c1 = __fmul_rn(x, kLog2e);
+                            float s1 = fmaf(fmaf(x, kLog2e, -c1), 0.69314718f, 1.0f);
                             if (x == -INFINITY) {
                                 c1 = -INFINITY;
                                 s1 = 0.f;

@@ -120,6 +120,31 @@ def test_vocab_pass_full_width_rows_with_bulk_ties(dtype):
     _vocab_case(z.to(torch.bfloat16) if dtype == "bf16" else z, K, dtype)
 
 
+@pytest.mark.parametrize("V,dtype", [(3, "bf16"), (6, "f32"), (14, "bf16"), (4099, "bf16"), (4097, "f32")])
+def test_vocab_pass_dominant_logit_outside_the_bulk_copies(V, dtype):
+    """One logit 30 above the rest, placed where the 16-byte bulk copies do not reach (tiny rows, the ragged first
+    and last elements of odd-length rows): the log-probability of that token is a rounding error away from 0, and
+    a path of 32 such tokens must stay within the tolerance of 1e-5, so each must be within about 1e-7."""
+    from paper_2608_20375_b200 import Graft
+    L, K = 8, min(V, 4)
+    z = torch.zeros((2, L, V))
+    for j in range(L):
+        z[0, j, (0, V - 1, 1, V - 2)[j % 4]] = 30.0 + j
+        z[1, j, (V - 1, 0)[j % 2]] = 30.0
+    zz = z.to(torch.bfloat16) if dtype == "bf16" else z
+    _vocab_case(zz, K, dtype)
+    g = Graft(V, L, K, 16, 8, 2, 8, 8, 8, 0.0, 1, DT[dtype], 0)
+    ids = torch.empty((2, L, K), dtype=torch.int32, device="cuda")
+    lp = torch.empty((2, L, K), dtype=torch.float32, device="cuda")
+    lse = torch.empty((2, L), dtype=torch.float32, device="cuda")
+    g.vocab_pass(zz.cuda(), ids, lp, lse)
+    torch.cuda.synchronize()
+    o_ids, o_lp, o_lse, o_st = oracle.vocab_pass(zz.reshape(2 * L, V), K)
+    top = lp.cpu().numpy().reshape(2 * L, K)[:, 0].astype(np.float64)
+    assert np.abs(top - o_lp[:, 0]).max() <= 1.5e-7, (top, o_lp[:, 0])  # 32 of them stay within 1e-5
+    g.destroy()
+
+
 def test_vocab_pass_large_magnitudes_and_negative_zero():
     V, K = 5000, 8
     g = torch.Generator().manual_seed(2)
