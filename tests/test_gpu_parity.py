@@ -711,3 +711,94 @@ def test_round_deep_trees_with_ties_scored_on_demand(beta, rows):
     for k in ("n_nodes", "budget", "status", "token", "parent", "depth", "position", "path_score", "mask"):
         assert np.array_equal(prod[k], gpu[k]), k
     g.destroy()
+
+
+# --------------------------------------------------------------------------- random sweep of input styles
+def _styled_logits(z, style, rng, gen, K):
+    """Logits of one of ten shapes, from ordinary to degenerate (z: fp32 [batch, L, V] drawn by graft_inputs)."""
+    Bt, L, V = z.shape
+    if style == "quant1":
+        return torch.round(z)
+    if style == "quant025":
+        return torch.round(z * 4) / 4
+    if style == "flat":
+        return 1e-3 * torch.randn(z.shape, generator=gen)
+    if style == "peaked":       # one token of probability 1 to fp32 precision
+        out = torch.zeros_like(z)
+        return out.scatter_(2, torch.randint(0, V, (Bt, L), generator=gen)[..., None], 30.0)
+    if style == "twopeaks":     # two equal winners (or one, where the draws coincide)
+        out = torch.zeros_like(z)
+        out.scatter_(2, torch.randint(0, V, (Bt, L), generator=gen)[..., None], 20.0)
+        return out.scatter_(2, torch.randint(0, V, (Bt, L), generator=gen)[..., None], 20.0)
+    if style == "mixed":
+        out = torch.round(z)
+        out[:, ::2] = 0.0
+        return out
+    if style == "huge":         # log-probabilities in the hundreds: one fp32 ulp is above the tolerance
+        return z * float(rng.choice([5.0, 10.0, 30.0]))
+    if style == "masked":       # between one and 2K finite tokens per row
+        keep_n = int(rng.integers(1, max(2, min(V, 2 * K))))
+        return z.masked_fill(torch.rand(z.shape, generator=gen).argsort(dim=2) >= keep_n, float("-inf"))
+    if style == "ramp":
+        return -torch.arange(V, dtype=torch.float32).expand(z.shape).clone() * float(rng.choice([1e-3, 0.1, 1.0]))
+    return z
+
+
+@pytest.mark.parametrize("seed", [101, 102, 103])
+def test_round_random_sweep_of_input_styles(seed):
+    """Fifty random rounds per seed: shapes from K = 1 to 32 and L = 1 to 32 over vocabularies of K + 1 to 30,011
+    tokens, budgets on odd grids, and logits of ten styles (ordinary, on coarse grids, flat, one or two dominant
+    tokens, mostly masked, in the hundreds, ramps).  Every round against the oracle under the comparison rule, the
+    acceptance walk too, and the call without debug outputs against the checked call, bit for bit."""
+    from paper_2608_20375_b200 import Graft, GraftError
+    rng = np.random.default_rng(seed)
+    styles = ["normal", "quant1", "quant025", "flat", "peaked", "mixed", "huge", "masked", "twopeaks", "ramp"]
+    done = 0
+    for ci in range(50):
+        K = int(rng.choice([1, 2, 3, 4, 5, 8, 13, 16, 20, 27, 32]))
+        L = int(rng.choice([1, 2, 3, 5, 7, 12, 16, 24, 32]))
+        if L * K * K * 4 > 128 * 1024:
+            L = 16
+        V = max(K, int(rng.choice([K + 1, 97, 1000, 4099, 30011])))
+        bstep = int(rng.choice([1, 3, 8, 16]))
+        bmin = int(rng.choice([0, 1, 4, 16, 64]))
+        bmax = min(bmin + bstep * int(rng.integers(0, 64)), 1023)
+        kw = dict(batch=int(rng.integers(1, 5)), L=L, V=V, K=K, budget_min=bmin, budget_max=bmax, budget_step=bstep,
+                  m=int(rng.choice([4, 8, 20, 64, 128])), hidden_dim=int(rng.choice([1, 8, 33, 256])),
+                  logits_dtype=str(rng.choice(["f32", "bf16"])), hidden_dtype=str(rng.choice(["f32", "bf16"])),
+                  beta=float(rng.choice([0.0, 0.0, 0.2, 1.5])), seed=int(rng.integers(1, 1 << 30)),
+                  fixed_budget=(None if rng.random() < 0.5 else int(rng.integers(0, bmax + 1))))
+        style = styles[ci % len(styles)]
+        rows = int(rng.choice([-1, 0, 1, 3]))
+        w = gi.small(**kw)
+        try:
+            g = _graft(w)
+        except GraftError:
+            continue  # a shape beyond the shared-memory limits
+        tb, saba_kw, keep = _setup(w, g)
+        if rows >= 0:
+            try:
+                g.set_edge_rows(min(rows, w.L))
+            except GraftError:
+                pass
+        x = gi.batch_inputs(w)
+        gen = torch.Generator().manual_seed(kw["seed"])
+        x["logits"] = _styled_logits(x["logits"].float(), style, rng, gen, K).to(x["logits"].dtype)
+        out, gpu = gpu_round(g, w, x)
+        orc = oracle_round(oracle, w, x, tb, saba_kw)
+        try:
+            compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+            compare_accept(oracle, gi, g, w, out, gpu)
+        except AssertionError as e:
+            raise AssertionError(f"case {ci} ({style}, edge rows {rows}, {kw}): {e}") from e
+        out_p = g.alloc_out(w.batch, debug=False)
+        cu = lambda t: None if t is None else t.cuda()  # noqa: E731
+        g.build_trees(cu(x["logits"]), cu(x["hidden"]), cu(x["root_token"]), cu(x["hist"]), cu(x["prefix_len"]),
+                      cu(x["fixed_budget"]), out_p)
+        torch.cuda.synchronize()
+        prod = out_p.cpu()
+        for k in ("n_nodes", "budget", "status", "token", "parent", "depth", "position", "path_score", "mask"):
+            assert np.array_equal(prod[k], gpu[k], equal_nan=prod[k].dtype.kind == "f"), (ci, style, k)
+        g.destroy()
+        done += 1
+    assert done >= 40
