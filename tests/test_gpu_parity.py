@@ -48,11 +48,11 @@ def _vocab_case(z, K, dtype):
     a, b = lp[good].astype(np.float64), o_lp[good].astype(np.float64)
     fin = np.isfinite(b)
     assert np.array_equal(np.isneginf(a), np.isneginf(b))
-    assert np.abs(a[fin] - b[fin]).max(initial=0) <= EPS
+    # (an fp32 result cannot be closer than its own spacing: one ulp beyond |x| = 128 already exceeds EPS)
+    assert np.all(np.abs(a[fin] - b[fin]) <= EPS + np.spacing(np.abs(b[fin]).astype(np.float32)))
     # candidates come in rank order, so their log-probabilities never increase along a row, and equal logits get the
     # same bits (every candidate of a row is measured against one log-sum-exp)
-    with np.errstate(invalid="ignore"):
-        assert np.all(np.diff(a, axis=1) <= 0.0), "log-probabilities increase along a row"
+    assert np.all(a[:, 1:] <= a[:, :-1]), "log-probabilities increase along a row"
     zf = z.reshape(Bt * L, V).float().numpy()
     for r in np.nonzero(good)[0][:64]:
         vals = zf[r, ids[r]]
