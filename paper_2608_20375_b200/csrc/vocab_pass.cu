@@ -50,6 +50,7 @@ constexpr int WBLK = TILE / NW;               // bytes of a tile owned by one wa
 static_assert(WBLK == 2048, "one warp owns 2 KiB of every tile");
 constexpr int VEC_PER_LANE = WBLK / 16 / 32;  // 4
 static_assert(VEC_PER_LANE == 4, "chunk layout assumes four 16-byte vectors per lane per tile");
+static_assert(WBLK == 32 * 4 * 16, "the exact fall-back selection reads one warp block per batch");
 constexpr uint32_t kVpIdleHintNs = 10000;  // suspend hint of the waits of the producer and epilogue warps
 constexpr int COS_WARP = PROD_WARP + 1;  // warp that computes the SABA cosines beside the stream
 static_assert(kVpThreads == NT + kVpEpiGroups * kVpEpiThreads + 64,
@@ -378,37 +379,81 @@ __device__ void warp_select_topk(EpiShared* sh, int n, int K, int lane) {
     __syncwarp();
 }
 
-// Exact selection over a whole segment straight from global memory, in slices small enough that the key
-// buffer cannot overflow.  Used only when the fast path's buffers overflowed.
+// Exact selection over a whole segment straight from global memory.  Used only when the fast path's buffers
+// overflowed, which means that most of the segment ties with its K-th largest element (rows that are flat, masked
+// to -inf, or all but one element equal).  The running K-th best key is the filter: an element enters the buffer
+// only if its key (value, then smaller id) beats it, and once the first K of a flat row are in, nothing else does.
+// The segment's 16-byte aligned body is read in batches of one streaming warp's 2 KiB of a tile; a batch whose
+// chunk maxima (left by the streaming warps) rule out a key above the filter is not read at all; the few elements
+// before and after the body go one by one.
+// When the buffer fills up, the best K are kept and the filter rises.
 template <bool BF16>
-__device__ int warp_fallback_select(EpiShared* sh, const VpParams& p, const Seg& sg, int lane) {
+__device__ int warp_fallback_select(EpiShared* sh, const VpParams& p, const Seg& sg,
+                                    const typename VT<BF16>::cm_t* cmx, int lane) {
     using T = VT<BF16>;
     const int K = p.K;
-    const int slice = kVpCandCap - kMaxK;
     const char* rowp = p.logits + (size_t)sg.row * p.V * T::ESZ;
-    uint64_t thr = 0;
-    int nb = 0, ovf = 0;
-    for (int base = sg.e0; base < sg.e1; base += slice) {
-        const int end = base + slice < sg.e1 ? base + slice : sg.e1;
-        int n = nb;
-        for (int e0 = base; e0 < end; e0 += 32) {
-            const int e = e0 + lane;
-            uint64_t key = 0;
-            if (e < end) key = make_key(__float_as_uint(load_elem_f32(rowp + (size_t)e * T::ESZ, BF16)), (uint32_t)e);
-            n = warp_append(sh->cand, n, kVpCandCap, e < end && key > thr, key, lane, &ovf);
-        }
+    uint64_t thr = 0;  // keys must beat this one
+    int n = 0, ovf = 0;
+    // ranking n keys against each other costs n^2 / 32 steps per lane: the buffer is cut back to its best K well
+    // before it is full (224 more keys at a time)
+    constexpr int kFallbackFill = 256 - 32;
+    auto shrink = [&]() {  // keep the best K of the buffer
         if (n > K) {
             warp_select_topk(sh, n, K, lane);
             if (lane < K) sh->cand[lane] = sh->outk[lane];
             thr = sh->outk[K - 1];
-            nb = K;
+            n = K;
             __syncwarp();
-        } else {
-            nb = n;
+        }
+    };
+    auto one_by_one = [&](int e_begin, int e_end) {
+        for (int e0 = e_begin; e0 < e_end; e0 += 32) {
+            const int e = e0 + lane;
+            uint64_t key = 0;
+            if (e < e_end) key = make_key(__float_as_uint(load_elem_f32(rowp + (size_t)e * T::ESZ, BF16)), (uint32_t)e);
+            n = warp_append(sh->cand, n, kVpCandCap, e < e_end && key > thr, key, lane, &ovf);
+            if (n > kFallbackFill) shrink();
+        }
+    };
+    one_by_one(sg.e0, sg.e_body0);
+    constexpr int U = 4;
+    const int nvec = (int)(sg.body_bytes / 16);
+    const uint4* body = (const uint4*)sg.body;
+    for (int v0 = 0; v0 < nvec; v0 += 32 * U) {
+        // The batch is one streaming warp's 2 KiB of a tile, and this lane's four vectors are the chunk whose
+        // maximum (rounded up to bf16) that warp's lane left in cmx.  A chunk cannot hold a key above the filter if
+        // its maximum is below the filter's value, or not above it while all its ids come after the filter's id.
+        if (thr != 0ull) {
+            const int tile = v0 / (TILE / 16), wb = (v0 % (TILE / 16)) / (32 * U);
+            const uint32_t mx = ord_from_bits((uint32_t)cmx[(size_t)(wb * 32 + lane) * p.max_tiles + tile] << 16);
+            const uint32_t v_thr = (uint32_t)(thr >> 32);
+            const uint32_t first_id = (uint32_t)(sg.e_body0 + (v0 + lane) * T::EPV);
+            const bool need = !(mx < v_thr || (mx <= v_thr && first_id > key_id(thr)));
+            if (!__any_sync(0xFFFFFFFFu, need)) continue;  // (uniform)
+        }
+#pragma unroll 1
+        for (int u = 0; u < U; ++u) {  // (one vector at a time: this path must not cost the kernel registers)
+            const int v = v0 + u * 32 + lane;
+            uint4 x = make_uint4(T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD);
+            if (v < nvec) x = body[v];
+            const uint32_t wv[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int q = 0; q < T::EPV; ++q) {
+                uint32_t xb;
+                if (BF16)
+                    xb = (q & 1) ? (wv[q >> 1] & 0xFFFF0000u) : (wv[q >> 1] << 16);
+                else
+                    xb = wv[q];
+                const uint64_t key = v < nvec ? make_key(xb, (uint32_t)(sg.e_body0 + v * T::EPV + q)) : 0ull;
+                n = warp_append(sh->cand, n, kVpCandCap, key > thr, key, lane, &ovf);
+                if (n > kFallbackFill) shrink();  // (uniform)
+            }
         }
     }
-    warp_select_topk(sh, nb, K, lane);
-    return nb < K ? nb : K;
+    one_by_one(sg.e_tail0, sg.e1);
+    warp_select_topk(sh, n, K, lane);
+    return n < K ? n : K;
 }
 
 // The outputs of a finished row from its pieces: C, S with sum_v 2^(z_v c) = S 2^C (c = fp32(log2 e)), the largest
@@ -716,7 +761,8 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     const uint32_t bits = (uint32_t)raw << 16;
                     if (ord_from_bits(bits) >= Tv) {
                         const int pos = atomicAdd(&es->nhits, 1);
-                        if (pos < kVpHitCap) es->hits[pos] = (uint32_t)tile * TILE + (t >> 5) * WBLK + (t & 31) * 16;
+                        if (pos >= kVpHitCap) break;  // too many: the exact selection over the segment takes over
+                        es->hits[pos] = (uint32_t)tile * TILE + (t >> 5) * WBLK + (t & 31) * 16;
                     }
                 }
             }
@@ -726,11 +772,15 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             //     A thread issues its loads of a round before it uses any: under a saturated memory system one
             //     round trip costs microseconds.
             {
-                const int nhits = es->nhits < kVpHitCap ? es->nhits : kVpHitCap;
-                if (etid == 0 && es->nhits > kVpHitCap) es->ovf = 1;
+                // (with too many hits nothing is re-read: a segment that is mostly ties would send every element
+                // through one shared counter)
+                const bool hit_ovf = es->nhits > kVpHitCap;
+                const int nhits = hit_ovf ? 0 : es->nhits;
+                if (etid == 0 && hit_ovf) es->ovf = 1;
                 constexpr int RU = 2;
                 const int nvec = nhits * VEC_PER_LANE;
-                for (int base = 0; base < nvec; base += kVpEpiThreads * RU) {
+                bool full = false;
+                for (int base = 0; base < nvec && !full; base += kVpEpiThreads * RU) {
                     uint4 vv[RU];
                     uint32_t offs[RU];
 #pragma unroll
@@ -757,10 +807,12 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                                 xb = (j & 1) ? (wv[j >> 1] & 0xFFFF0000u) : (wv[j >> 1] << 16);
                             else
                                 xb = wv[j];
-                            if (ord_from_bits(xb) >= Tv) {
+                            if (ord_from_bits(xb) >= Tv && !full) {
                                 const int pos = atomicAdd(&es->ncand, 1);
                                 if (pos < kVpCandCap)
                                     es->cand[pos] = make_key(xb, (uint32_t)(sg.e_body0 + offs[u] / T::ESZ + j));
+                                else
+                                    full = true;  // (the count stays above the capacity: the exact selection takes over)
                             }
                         }
                     }
@@ -780,7 +832,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     if (rank < p.K) es->outk[rank] = key;
                 }
             } else if (ew == 0) {
-                nk = warp_fallback_select<BF16>(es, p, sg, lane);
+                nk = warp_fallback_select<BF16>(es, p, sg, cmx, lane);
             }
             epi_bar(grp);
             if (ew != 0) continue;
