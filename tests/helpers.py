@@ -100,9 +100,10 @@ def compare_round(oracle, w, x, tb, saba_kw, gpu, orc):
         assert _close(gpu["topk_lp"][b], orc["topk_lp"][b], EPS), f"seq {b}: log-probs"
         assert _close(gpu["lse"][b], orc["lse"][b], EPS), f"seq {b}: lse"
         # edges
-        # (two ulps: an edge score is the rounded sum of a log-probability that may itself be an ulp off)
-        assert _close(gpu["edge"][b, 0, 0], orc["edge"][b, 0, 0], EPS, ulps=2), f"seq {b}: depth-1 edges"
-        assert _close(gpu["edge"][b, 1:], orc["edge"][b, 1:], EPS, ulps=2), f"seq {b}: edges"
+        # (three ulps: an edge score is the rounded sum of a log-probability that may itself be an ulp off, both
+        # sides round the sum once, and the fp32 dot product behind beta f has its own error)
+        assert _close(gpu["edge"][b, 0, 0], orc["edge"][b, 0, 0], EPS, ulps=3), f"seq {b}: depth-1 edges"
+        assert _close(gpu["edge"][b, 1:], orc["edge"][b, 1:], EPS, ulps=3), f"seq {b}: edges"
         # SABA
         o_budget = int(orc["budget"][b])
         ref = {k: orc[k][b] for k in ("n_nodes", "token", "parent", "depth", "position", "path_score", "mask")}
