@@ -51,6 +51,7 @@ static_assert(WBLK == 2048, "one warp owns 2 KiB of every tile");
 constexpr int VEC_PER_LANE = WBLK / 16 / 32;  // 4
 static_assert(VEC_PER_LANE == 4, "chunk layout assumes four 16-byte vectors per lane per tile");
 static_assert(WBLK == 32 * 4 * 16, "the exact fall-back selection reads one warp block per batch");
+constexpr uint32_t kOrdNegInf = 0x007FFFFFu;  // ord_from_bits of -inf: every finite value maps above it
 constexpr uint32_t kVpIdleHintNs = 10000;  // suspend hint of the waits of the producer and epilogue warps
 constexpr int COS_WARP = PROD_WARP + 1;  // warp that computes the SABA cosines beside the stream
 static_assert(kVpThreads == NT + kVpEpiGroups * kVpEpiThreads + 64,
@@ -332,6 +333,7 @@ struct __align__(16) EpiShared {  // private to one epilogue group
     uint32_t hits[kVpHitCap];
     uint16_t hthreads[NT];  // streaming threads whose maximum reaches T
     int nhits, ncand, nht, ovf;
+    int fill_ninf;  // the threshold fell on -inf: the candidates are the finite elements plus the first -inf ones
     uint32_t Tv;
 };
 struct __align__(16) VpShared {
@@ -733,7 +735,14 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 }
                 vmo = __reduce_max_sync(0xFFFFFFFFu, vmo);
                 overflow = __any_sync(0xFFFFFFFFu, overflow);
+                // A threshold at -inf (a vocabulary masked down to fewer finite tokens than the filter needs) would let
+                // every element through.  The K best are then the finite elements and, after them, the -inf elements
+                // of smallest id: the filter rises to the lowest finite value and the first K -inf elements of the
+                // segment are added below.
+                const bool ninf = Tv <= kOrdNegInf;
+                if (ninf) Tv = kOrdNegInf + 1u;
                 if (lane == 0) {
+                    es->fill_ninf = ninf ? 1 : 0;
                     es->Tv = Tv;
                     es->nhits = 0;
                     es->nht = 0;
@@ -819,6 +828,32 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 }
             }
             epi_bar(grp);
+            if (es->fill_ninf) {  // (uniform)
+                if (ew == 0) {
+                    // the first K elements equal to -inf of the segment's body, in id order (the few elements before
+                    // and after the body are candidates already); a segment that does not show K of them within
+                    // its first 8192 elements goes to the exact selection instead
+                    constexpr int kScan = 8192;
+                    int found = 0, e0 = sg.e_body0;
+                    for (; e0 < sg.e_tail0 && e0 - sg.e_body0 < kScan && found < p.K; e0 += 32) {
+                        const int e = e0 + lane;
+                        uint32_t xb = 0u;
+                        bool is = false;
+                        if (e < sg.e_tail0) {
+                            xb = __float_as_uint(load_elem_f32(rowp + (size_t)e * T::ESZ, BF16));
+                            is = xb == 0xFF800000u;
+                        }
+                        const uint32_t mk = __ballot_sync(0xFFFFFFFFu, is);
+                        if (is && found + __popc(mk & ((1u << lane) - 1u)) < p.K) {
+                            const int pos = atomicAdd(&es->ncand, 1);
+                            if (pos < kVpCandCap) es->cand[pos] = make_key(xb, (uint32_t)e);
+                        }
+                        found += __popc(mk);
+                    }
+                    if (found < p.K && e0 < sg.e_tail0 && lane == 0) es->ovf = 1;
+                }
+                epi_bar(grp);
+            }
             if (ew == 0) VP_T(4);
             // (f) exact top-K of the candidates by rank counting (keys are distinct, so ranks are a permutation)
             const bool overflow = es->ovf != 0 || es->ncand > kVpCandCap;
