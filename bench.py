@@ -624,7 +624,12 @@ def main():
     else:
         args.steps = 1000 if args.steps is None else args.steps
         args.warmup = max(3, 20 if args.warmup is None else args.warmup)
-        run_graft(args)
+        try:
+            run_graft(args)
+        finally:
+            import torch.distributed as dist
+            if dist.is_available() and dist.is_initialized():
+                dist.destroy_process_group()
 
 
 if __name__ == "__main__":
