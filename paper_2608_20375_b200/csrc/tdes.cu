@@ -153,6 +153,7 @@ __global__ void __launch_bounds__(256, 4) tdes_edges_kernel(const EdgeParams p) 
     __syncthreads();
     const float* urow = p.u + (size_t)j * m;
     constexpr int RPW = 2 * kMaxK / 8;  // rows per warp at most
+    const uint64_t keep = l2_policy_evict_last();
     for (int k40 = 0; k40 < m / 4; k40 += 32) {
         const int k4 = k40 + lane;
         float4 t[RPW];
@@ -161,7 +162,7 @@ __global__ void __launch_bounds__(256, 4) tdes_edges_kernel(const EdgeParams p) 
             const int r = warp + 8 * q;
             t[q] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (r < n_par + K && k4 < m / 4)
-                t[q] = __ldg((const float4*)((r < n_par ? p.P : p.C) + (size_t)toks[r] * m) + k4);
+                t[q] = ldg_f4_keep((const float4*)((r < n_par ? p.P : p.C) + (size_t)toks[r] * m) + k4, keep);
         }
         if (k4 < m / 4) {
             const float4 uu = *(const float4*)(urow + k4 * 4);

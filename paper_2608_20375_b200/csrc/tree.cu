@@ -379,8 +379,11 @@ __device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, 
 __device__ __forceinline__ bool lazy_neutral(const TreeParams& p, int j) {
     return p.beta == 0.0f || (j == 0 && !p.root_edge);
 }
+// (the table rows of frequent tokens are read round after round: L2 is asked to keep them, as in the edge-score kernel)
 __device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+    const uint64_t keep = l2_policy_evict_last();
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "l"(keep)
+                 : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
