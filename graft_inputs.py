@@ -1,7 +1,9 @@
 """Seeded synthetic inputs for the GRAFT draft-tree round.
 
 This module only *draws* inputs (random numbers, index sets, dtype rounding); it holds none of
-the method's arithmetic and is the one piece of code that both the CPU oracle's tests and the
+the method's arithmetic on the round's path (the one exception is data synthesis for the fitting step:
+`saba_replay_logs` evaluates the gain and latency models of Eq. 16-17 forward to fabricate the logs that
+the fit is then asked to recover) and is the one piece of code that both the CPU oracle's tests and the
 CUDA library's tests / benchmark use.  Every sequence is generated from its own counter-based
 stream (Philox keyed by (seed, tensor tag, sequence index)), so sequence b has the same bytes
 whatever the batch size or the rank that generates it.

@@ -124,7 +124,8 @@ graft_status graft_set_tdes_tables(graft_ctx* ctx, const float* d_P, const float
 /* How many depths the edge-score kernel covers ahead of the expansion.  The scores of Eq. 4-6 are needed only for
  * depths that the best-first expansion reaches, which is not known in advance: depths [0, rows) are scored for every
  * sequence by a kernel of their own, deeper ones inside the tree kernel when an expansion gets there.  The trees do
- * not depend on the split beyond fp32 rounding of the scores (the two scorers add in different orders).
+ * not depend on the split at all: both scorers run the same arithmetic in the same order, so a score has the same
+ * bits whichever kernel produced it.
  * rows in [0, L]; the default is min(L, 8), or L when the on-demand scorer's buffers do not fit in shared memory
  * (then any other value is GRAFT_ERR_INVALID_ARG).  Host-only call; takes effect from the next round.
  * (A tuning knob of this implementation; the paper scores all edges.) */
@@ -170,7 +171,8 @@ graft_status graft_tdes_edges(graft_ctx* ctx, int32_t batch, const int32_t* d_to
  * library until the process exits).  It is meant for callers that cannot let a library allocate -- a serving
  * process that gave all device memory to its own pool at start-up, or code that has to stay off the driver's
  * allocation lock on its latency path.
- *   Limits: batch * L <= 16384 rows and at most 512 CTAs (two per SM); beyond them GRAFT_ERR_UNSUPPORTED.
+ *   Limits: batch * L <= 16384 rows and at most 512 CTAs (the kernel launches one per SM); beyond them
+ *   GRAFT_ERR_UNSUPPORTED.
  *   d_row_status [batch * L] is required here.
  *   The first call on each device looks up the array's device address and sets the kernel's shared-memory
  *   attribute; make that first call before any stream capture begins.
@@ -180,7 +182,7 @@ graft_status graft_vocab_pass_static(int32_t batch, int32_t L, int32_t V, int32_
                                      const void* d_logits, int32_t* d_topk_id, float* d_topk_lp, float* d_lse,
                                      int32_t* d_row_status, void* stream);
 
-/* Vocabulary-parallel S1 (the logits of a tensor-parallel LM head are split over V across GPUs).  Each GPU runs
+/* Vocabulary-parallel vocab pass (the logits of a tensor-parallel LM head are split over V across GPUs).  Each GPU runs
  * graft_vocab_pass_partial on its shard: per row it leaves the log-sum-exp pieces and the K best keys of the shard
  * (token ids local to the shard).  The partials of all shards, gathered into one buffer in shard order (one NCCL
  * all-gather of 280 bytes per row and shard; they land in local memory first), are merged by graft_vocab_merge into

@@ -48,8 +48,8 @@ static float orc_load(const void *base, int dtype, size_t i) {
 }
 
 /* ------------------------------------------------------------------------------------------
- * O0.  P[v] = W_p e_v + b_p,  C[v] = W_c e_v + b_c   (the "two linear projections g_p, g_c"
- * of Sec. 3.2; "depend only on the token id, we compute them once").  fp64 accumulate,
+ * O0.  P[v] = W_p e_v + b_p,  C[v] = W_c e_v + b_c   (the two linear projections g_p and g_c
+ * of Sec. 3.2; a function of the token id alone, hence tabulated once per model).  fp64 accumulate,
  * rounded once to fp32.  bias may be NULL.
  * Pins: identity weights reproduce the embedding; agreement with a library matmul.
  * ------------------------------------------------------------------------------------------ */

@@ -148,7 +148,14 @@ def vocab_pass_static(logits, K, topk_id, topk_lp, lse, row_status):
     the scratch is a static device array inside the library).  logits [batch, L, V] on the GPU."""
     lib = load_library()
     batch, L, V = logits.shape
+    if logits.dtype not in (torch.bfloat16, torch.float32):
+        raise GraftError(f"logits must be bfloat16 or float32, got {logits.dtype}")
     dt = BF16 if logits.dtype == torch.bfloat16 else F32
+    # the library writes batch*L*K ids and log-probabilities and batch*L log-sum-exps and status words
+    for name, t, need in (("topk_id", topk_id, batch * L * K), ("topk_lp", topk_lp, batch * L * K),
+                          ("lse", lse, batch * L), ("row_status", row_status, batch * L)):
+        if t is None or t.numel() < need:
+            raise GraftError(f"{name} must hold at least {need} elements")
     _check(lib, lib.graft_vocab_pass_static(batch, L, V, K, dt, _ptr(logits), _ptr(topk_id, torch.int32),
                                             _ptr(topk_lp, torch.float32), _ptr(lse, torch.float32),
                                             _ptr(row_status, torch.int32), _stream()), "graft_vocab_pass_static")
@@ -237,7 +244,7 @@ class Graft:
                   C.cast(n, C.POINTER(C.c_float)), C.cast(t, C.POINTER(C.c_float)))
         _check(self.lib, self.lib.graft_set_saba(self._ctx, C.byref(p)), "graft_set_saba")
 
-    # ---- vocabulary-parallel S1
+    # ---- vocabulary-parallel vocab pass
     def vocab_pass_partial(self, logits_shard, parts):
         """parts: uint8 [batch*L, VOCAB_PARTIAL_BYTES] on the device (this shard's pieces of every row)."""
         batch = logits_shard.shape[0]

@@ -153,8 +153,8 @@ graft_status graft_create(const graft_config* cfg, graft_ctx** out) {
     ctx->w_esort = (float*)(base + o_es);
     ctx->w_eidx = (uint8_t*)(base + o_ei);
     ctx->d_u = (float*)(base + o_u);
-    ctx->s0_scratch = nullptr;
-    ctx->s0_scratch_bytes = 0;
+    ctx->tables_scratch = nullptr;
+    ctx->tables_scratch_bytes = 0;
     ctx->hist_w = 0;
     ctx->hist_window = nullptr;
     ctx->hist_count = nullptr;
@@ -179,7 +179,7 @@ graft_status graft_destroy(graft_ctx* ctx) {
         if (ex->d_out) cudaFree(ex->d_out);
         delete ex;
     }
-    if (ctx->s0_scratch) cudaFree(ctx->s0_scratch);
+    if (ctx->tables_scratch) cudaFree(ctx->tables_scratch);
     if (ctx->ws) cudaFree(ctx->ws);
     delete ctx;
     return GRAFT_OK;
@@ -251,20 +251,20 @@ graft_status graft_tdes_precompute(graft_ctx* ctx, const void* d_emb, graft_dtyp
     // bf16 embeddings: the tensor cores (the embeddings are exact operands, W goes in as three bf16 parts); its
     // scratch is allocated on the first such call (this is the once-per-model setup step, not the round)
     if (emb_dtype == GRAFT_BF16) {
-        const size_t need = s0_tc_scratch_bytes(ctx->cfg.V, E, ctx->cfg.m);
+        const size_t need = tables_tc_scratch_bytes(ctx->cfg.V, E, ctx->cfg.m);
         if (need > 0) {
-            if (ctx->s0_scratch_bytes < need) {
-                if (ctx->s0_scratch) cudaFree(ctx->s0_scratch);
-                ctx->s0_scratch = nullptr;
-                ctx->s0_scratch_bytes = 0;
-                if (cudaMalloc(&ctx->s0_scratch, need) != cudaSuccess) {
+            if (ctx->tables_scratch_bytes < need) {
+                if (ctx->tables_scratch) cudaFree(ctx->tables_scratch);
+                ctx->tables_scratch = nullptr;
+                ctx->tables_scratch_bytes = 0;
+                if (cudaMalloc(&ctx->tables_scratch, need) != cudaSuccess) {
                     cudaGetLastError();
                     return GRAFT_ERR_WORKSPACE;
                 }
-                ctx->s0_scratch_bytes = need;
+                ctx->tables_scratch_bytes = need;
             }
             int n = 0;
-            const cudaError_t e = s0_tc_launch(d_emb, ctx->cfg.V, E, ctx->cfg.m, d_W, d_b, d_out, ctx->s0_scratch, &n,
+            const cudaError_t e = tables_tc_launch(d_emb, ctx->cfg.V, E, ctx->cfg.m, d_W, d_b, d_out, ctx->tables_scratch, &n,
                                                (cudaStream_t)stream);
             ctx->launches += (uint64_t)n;
             if (e == cudaSuccess) return GRAFT_OK;
@@ -331,11 +331,6 @@ graft_status graft_tdes_edges(graft_ctx* ctx, int32_t batch, const int32_t* d_to
     return GRAFT_OK;
 }
 
-#if defined(GRAFT_VP_PROF) || defined(GRAFT_TREE_PROF)
-// profiling builds only (never in the shipped library): raw reads of the counters the instrumented kernels leave
-extern "C" int graft_debug_read(graft_ctx* ctx, int32_t* out64) { return (int)cudaMemcpy(out64, ctx->w_errflag, 256, cudaMemcpyDeviceToHost); }
-extern "C" int graft_debug_read2(graft_ctx* ctx, float* out, int n) { return (int)cudaMemcpy(out, ctx->w_edge, (size_t)n * 4, cudaMemcpyDeviceToHost); }
-#endif
 
 graft_status graft_set_timing(graft_ctx* ctx, int32_t enable) {
     if (!ctx) return GRAFT_ERR_INVALID_ARG;

@@ -91,8 +91,8 @@ struct graft_ctx {
     int32_t* w_errflag;           // [1] device-side internal error flag
     graft::VpPlan vp_plan;
     // scratch of the tensor-core table precompute (allocated on its first use: three bf16 copies of W, GEMM workspace)
-    void* s0_scratch;
-    size_t s0_scratch_bytes;
+    void* tables_scratch;
+    size_t tables_scratch_bytes;
     // host-buffer staging (allocated on first use of graft_build_trees_host)
     void* stage;
     size_t stage_bytes;
@@ -135,9 +135,11 @@ int vp_merge_max_shards();
 
 cudaError_t tdes_precompute_launch(graft_ctx* ctx, const void* d_emb, graft_dtype dt, int E, const float* d_W,
                                    const float* d_b, float* d_out, cudaStream_t st);
-// S0 on the tensor cores (bf16 embeddings): three bf16 GEMMs with fp32 accumulation (csrc/s0_gemm.cu)
-size_t s0_tc_scratch_bytes(int V, int E, int m);
-cudaError_t s0_tc_launch(const void* d_emb, int V, int E, int m, const float* d_W, const float* d_b, float* d_out,
+// table precompute on the tensor cores (bf16 embeddings): bf16 GEMMs with fp32 accumulation (csrc/tables_gemm.cu;
+// csrc/tables_gemm_stub.cu when the library is built without a CUTLASS tree: the scratch size is then 0 and
+// the FMA kernel runs instead)
+size_t tables_tc_scratch_bytes(int V, int E, int m);
+cudaError_t tables_tc_launch(const void* d_emb, int V, int E, int m, const float* d_W, const float* d_b, float* d_out,
                          void* d_scratch, int* launches, cudaStream_t st);
 cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
                               const int32_t* d_root_token, const int32_t* d_row_status, float* d_edge,

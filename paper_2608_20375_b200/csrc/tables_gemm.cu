@@ -1,4 +1,4 @@
-// S0 on the tensor cores: out[v] = W e_v + b for bf16 embeddings (text after Eq. 6: the projections depend only on the
+// Table precompute on the tensor cores: out[v] = W e_v + b for bf16 embeddings (text after Eq. 6: the projections depend only on the
 // token id and are computed once).  This is the one dense contraction of the method, [V, E] x [E, m].
 //
 // The embeddings are bf16, hence exact as tensor-core operands; the fp32 weights are split into three bf16 parts,
@@ -50,13 +50,13 @@ using CollectiveMainloop = typename cutlass::gemm::collective::CollectiveBuilder
 using GemmKernel =
     cutlass::gemm::kernel::GemmUniversal<cute::Shape<int, int, int, int>, CollectiveMainloop, CollectiveEpilogue, void>;
 using Gemm = cutlass::gemm::device::GemmUniversalAdapter<GemmKernel>;
-#ifndef GRAFT_S0_CHUNK_K
-#define GRAFT_S0_CHUNK_K 1024
+#ifndef GRAFT_TABLES_CHUNK_K
+#define GRAFT_TABLES_CHUNK_K 1024
 #endif
-constexpr int kS0ChunkK = GRAFT_S0_CHUNK_K;  // a multiple of 64 (the K extent of a tile)
+constexpr int kTablesChunkK = GRAFT_TABLES_CHUNK_K;  // a multiple of 64 (the K extent of a tile)
 
 // W (fp32, [m, E]) -> three bf16 parts; out rows <- bias
-__global__ void s0_split_kernel(const float* __restrict__ W, size_t n, __nv_bfloat16* __restrict__ w1,
+__global__ void weight_split_kernel(const float* __restrict__ W, size_t n, __nv_bfloat16* __restrict__ w1,
                                 __nv_bfloat16* __restrict__ w2, __nv_bfloat16* __restrict__ w3) {
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         const float w = W[i];
@@ -70,7 +70,7 @@ __global__ void s0_split_kernel(const float* __restrict__ W, size_t n, __nv_bflo
     }
 }
 // out[v][j] = bias[j] + tmp[v][j] + tmp[v][m + j] + tmp[v][2m + j] for the rows of one slab
-__global__ void s0_reduce_kernel(const float* __restrict__ tmp, const float* __restrict__ bias, float* __restrict__ out,
+__global__ void parts_reduce_kernel(const float* __restrict__ tmp, const float* __restrict__ bias, float* __restrict__ out,
                                  size_t rows, int m) {
     const size_t n = rows * (size_t)m;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
@@ -83,13 +83,13 @@ __global__ void s0_reduce_kernel(const float* __restrict__ tmp, const float* __r
 
 }  // namespace
 
-constexpr int kS0SlabRows = 65536;  // rows of V per slab: 65536 x 3m fp32 partial sums (100 MB at m = 128), mostly L2-resident
+constexpr int kTablesSlabRows = 65536;  // rows of V per slab: 65536 x 3m fp32 partial sums (100 MB at m = 128), mostly L2-resident
 
 // Scratch: three bf16 copies of W, a slab of partial sums, the GEMM's workspace.  Returns the bytes needed
 // (0: this path cannot be used).
-size_t s0_tc_scratch_bytes(int V, int E, int m) {
+size_t tables_tc_scratch_bytes(int V, int E, int m) {
     if ((E % 8) != 0 || (m % 4) != 0 || V < 1) return 0;
-    const int slab = V < kS0SlabRows ? V : kS0SlabRows;
+    const int slab = V < kTablesSlabRows ? V : kTablesSlabRows;
     Gemm::Arguments args{cutlass::gemm::GemmUniversalMode::kGemm,
                          {slab, 3 * m, E, 1},
                          {nullptr, {}, nullptr, {}},
@@ -99,16 +99,16 @@ size_t s0_tc_scratch_bytes(int V, int E, int m) {
            ((ws + 255) & ~(size_t)255) + 512;
 }
 
-// out [V, m] = emb [V, E] (bf16) . W^T + bias on the tensor cores.  d_scratch: s0_tc_scratch_bytes, 256-byte aligned.
+// out [V, m] = emb [V, E] (bf16) . W^T + bias on the tensor cores.  d_scratch: tables_tc_scratch_bytes, 256-byte aligned.
 // Returns cudaErrorNotSupported when the GEMM cannot take the problem (the caller then uses the FMA kernel).
-cudaError_t s0_tc_launch(const void* d_emb, int V, int E, int m, const float* d_W, const float* d_b, float* d_out,
+cudaError_t tables_tc_launch(const void* d_emb, int V, int E, int m, const float* d_W, const float* d_b, float* d_out,
                          void* d_scratch, int* launches, cudaStream_t st) {
     if (((uintptr_t)d_emb & 15) || ((uintptr_t)d_out & 15) || (E % 8) != 0 || (m % 4) != 0) return cudaErrorNotSupported;
-    const int slab = V < kS0SlabRows ? V : kS0SlabRows;
+    const int slab = V < kTablesSlabRows ? V : kTablesSlabRows;
     __nv_bfloat16* w3x = (__nv_bfloat16*)d_scratch;  // [3m, E]: W1 rows, then W2 rows, then W3 rows
     float* tmp = (float*)(((uintptr_t)(w3x + (size_t)3 * m * E) + 255) & ~(uintptr_t)255);  // [slab, 3m]
     void* ws = (void*)(((uintptr_t)(tmp + (size_t)slab * 3 * m) + 255) & ~(uintptr_t)255);
-    s0_split_kernel<<<256, 256, 0, st>>>(d_W, (size_t)m * E, w3x, w3x + (size_t)m * E, w3x + (size_t)2 * m * E);
+    weight_split_kernel<<<256, 256, 0, st>>>(d_W, (size_t)m * E, w3x, w3x + (size_t)m * E, w3x + (size_t)2 * m * E);
     *launches += 1;
     typename GemmKernel::StrideA sA{};
     typename GemmKernel::StrideB sB{};
@@ -118,8 +118,8 @@ cudaError_t s0_tc_launch(const void* d_emb, int V, int E, int m, const float* d_
         const int rows = V - v0 < slab ? V - v0 : slab;
         auto sC = cutlass::make_cute_packed_stride(typename GemmKernel::StrideC{}, cute::make_shape(rows, 3 * m, 1));
         auto sD = cutlass::make_cute_packed_stride(typename GemmKernel::StrideD{}, cute::make_shape(rows, 3 * m, 1));
-        for (int k0 = 0; k0 < E; k0 += kS0ChunkK) {
-            const int kc = E - k0 < kS0ChunkK ? E - k0 : kS0ChunkK;
+        for (int k0 = 0; k0 < E; k0 += kTablesChunkK) {
+            const int kc = E - k0 < kTablesChunkK ? E - k0 : kTablesChunkK;
             Gemm::Arguments args{cutlass::gemm::GemmUniversalMode::kGemm,
                                  {rows, 3 * m, kc, 1},
                                  {(const ElementA*)d_emb + (size_t)v0 * E + k0, sA, (const ElementB*)w3x + k0, sB},
@@ -130,7 +130,7 @@ cudaError_t s0_tc_launch(const void* d_emb, int V, int E, int m, const float* d_
             if (gemm.run(st) != cutlass::Status::kSuccess) return cudaErrorUnknown;
             *launches += 1;
         }
-        s0_reduce_kernel<<<1024, 256, 0, st>>>(tmp, d_b, d_out + (size_t)v0 * m, (size_t)rows, m);
+        parts_reduce_kernel<<<1024, 256, 0, st>>>(tmp, d_b, d_out + (size_t)v0 * m, (size_t)rows, m);
         *launches += 1;
     }
     return cudaGetLastError();

@@ -459,9 +459,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     pdl_wait();  // candidates, cosines and edge rows come from the kernels ahead in the stream
 
     // ---- status and budget ---------------------------------------------------------------------------
-#ifdef GRAFT_TREE_PROF
-    long long t_prof0 = clock64(), t_prof1 = 0, t_prof2 = 0, t_prof15 = 0;
-#endif
     // the sorted edge rows of this sequence: bulk copies through the TMA unit when the 16-byte rules allow it
     // (they land while warp 0 works out the budget), plain loads otherwise
     __shared__ __align__(8) uint64_t rows_bar;
@@ -564,9 +561,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         __syncthreads();
     }
 
-#ifdef GRAFT_TREE_PROF
-    t_prof1 = clock64();
-#endif
     // ---- best-first expansion ------------------------------------------------------------------------------
     // Best-first expansion selects prefixes in non-increasing order of their bottleneck key (the minimum path
     // score along the prefix), so after B selections the tree is the set of prefixes with key above the B-th
@@ -612,9 +606,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             __syncthreads();
         }
         for (int d = spec ? 2 : 0; d < L; ++d) {
-#ifdef GRAFT_TREE_PROF
-            long long tl0 = clock64();
-#endif
             const int b0 = sm.lvl_start[d], b1 = sm.lvl_start[d + 1];
             if (b1 == b0) break;
             if (d >= rows_done) {  // the edge rows of this depth: scored now, never if the expansion stops above it
@@ -754,9 +745,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 }
             }
             __syncthreads();
-#ifdef GRAFT_TREE_PROF
-            long long tl1 = clock64();
-#endif
             const int nt = sm.scal[3];
             if (sm.scal[4]) {
                 table_ok = false;
@@ -773,15 +761,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 n_at_select = ntot;
             }
             __syncthreads();
-#ifdef GRAFT_TREE_PROF
-            if (tid == 0 && o.d_edge) {
-                float* dbg = o.d_edge + (size_t)b * L * K * K;
-                dbg[4 * d] = (float)(tl1 - tl0);
-                dbg[4 * d + 1] = (float)(clock64() - tl1);
-                dbg[4 * d + 2] = (float)ntot;
-                dbg[4 * d + 3] = (float)(b1 - b0);
-            }
-#endif
         }
         __syncthreads();
         if (table_ok && ntot - 1 >= budget) {
@@ -794,10 +773,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         }
         __syncthreads();
         if (table_ok) {
-#ifdef GRAFT_TREE_PROF
-            __syncthreads();
-            if (tid == 0 && o.d_edge) o.d_edge[(size_t)b * L * K * K + 100 + 0] = (float)(clock64() - t_prof0);
-#endif
             // compact {key > theta} in table order (parents stay before their children)
             const int per = (ntot + TREE_THREADS - 1) / TREE_THREADS;
             const int i0 = tid * per < ntot ? tid * per : ntot, i1 = i0 + per < ntot ? i0 + per : ntot;
@@ -834,10 +809,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             }
             n_gt = total - 1;
             __syncthreads();
-#ifdef GRAFT_TREE_PROF
-            __syncthreads();
-            if (tid == 0 && o.d_edge) o.d_edge[(size_t)b * L * K * K + 100 + 1] = (float)(clock64() - t_prof0);
-#endif
             // frontier entries of the selected nodes: the first child of the sorted row that is not selected,
             // i.e. the first with ord(score) <= theta
             for (int n = tid; n <= n_gt; n += TREE_THREADS) {
@@ -860,9 +831,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             }
         }
     }
-#ifdef GRAFT_TREE_PROF
-    t_prof15 = clock64();
-#endif
     if (p.lazy && !table_ok && budget > 0) {  // the sequential fall-back may reach any depth
         for (; rows_done < L; ++rows_done) lazy_score_row(p, sm, rows_done, root, tid, inflight);
     }
@@ -951,9 +919,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     }
     __syncthreads();
 
-#ifdef GRAFT_TREE_PROF
-    t_prof2 = clock64();
-#endif
     // ---- emission in level order -------------------------------------------------------------------------
     // Level order = depth ascending, then the parent's level-order index, then candidate rank.  Level by level:
     // the child counts of level d-1, laid out in level order, are scanned; a node of level d lands at
@@ -1016,10 +981,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         }
         __syncthreads();
     }
-#ifdef GRAFT_TREE_PROF
-    __syncthreads();
-    if (tid == 0 && o.d_edge) o.d_edge[(size_t)b * L * K * K + 100 + 2] = (float)(clock64() - t_prof0);
-#endif
     const int prefix = p.prefix_len[b];
     const size_t ob = (size_t)b * nmax;
     for (int n = tid; n < n_nodes; n += TREE_THREADS) {
@@ -1040,10 +1001,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         o.d_path_score[ob + i] = 0.f;
     }
     __syncthreads();
-#ifdef GRAFT_TREE_PROF
-    __syncthreads();
-    if (tid == 0 && o.d_edge) o.d_edge[(size_t)b * L * K * K + 100 + 3] = (float)(clock64() - t_prof0);
-#endif
     // ancestor masks: each thread builds one row in its warp's staging tile (walking up, level-order indices
     // only decrease, so the row is produced from its highest word down); the warp then stores its 32 rows,
     // which are contiguous in the output, with coalesced writes.  Padding rows are zero-filled directly.
@@ -1085,15 +1042,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         const int z0 = ((n_nodes + 31) / 32) * 32;
         for (size_t k = (size_t)z0 * W + tid; k < (size_t)nmax * W; k += TREE_THREADS) o.d_mask[ob * W + k] = 0u;
     }
-#ifdef GRAFT_TREE_PROF
-    __syncthreads();
-    if (tid == 0 && o.d_state) {
-        o.d_state[(size_t)b * 4 + 0] = (float)(t_prof1 - t_prof0);
-        o.d_state[(size_t)b * 4 + 1] = (float)(t_prof15 - t_prof1);
-        o.d_state[(size_t)b * 4 + 2] = (float)(t_prof2 - t_prof15);
-        o.d_state[(size_t)b * 4 + 3] = (float)(clock64() - t_prof2);
-    }
-#endif
     if (p.lazy) cp_async_wait_all();  // table rows fetched ahead for a depth that was never scored
     if (tid == 0) {
         o.d_n_nodes[b] = n_nodes;

@@ -36,11 +36,6 @@ namespace graft {
 
 namespace {
 
-#ifdef GRAFT_VP_PROF
-#define VP_T(i) do { long long _t = clock64(); if (blockIdx.x == 1 && lane == 0) atomicAdd(p.errflag + 2 + (i), (int)((_t - tprof) >> 4)); tprof = _t; } while (0)
-#else
-#define VP_T(i) do { } while (0)
-#endif
 
 constexpr int NW = kVpConsumerWarps;          // streaming warps
 constexpr int NT = kVpConsumers;              // streaming threads
@@ -94,8 +89,6 @@ struct VpParams {
     int hidden_bf16, hidden_dim, L;
     double* cos_out;  // [rows / L, L]
     int use_hint;
-    float* dbg_out;  // profiling builds only
-    int dbg;  // experiments only: 1 = stream without arithmetic, 2 = arithmetic without streaming, 3 = no epilogue
 };
 
 struct Seg {
@@ -341,7 +334,6 @@ struct __align__(16) VpShared {
     uint32_t tmax[kVpBufs][NT];  // per-thread maxima of a finished segment, one buffer per segment in flight
     uint32_t gmax[kVpBufs][kVpGroups];  // the same maxima folded into 64 groups (lane, warp parity); zero when idle
     float wc[kVpBufs][NW], ws[kVpBufs][NW];
-    long long t_stream_end;      // profiling builds only
     volatile int abort_flag;
 };
 
@@ -500,9 +492,6 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
     cm_t* cmax = (cm_t*)(sh + 1);  // [kVpBufs][n_cmax]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-#ifdef GRAFT_VP_PROF
-    const long long t_kernel0 = clock64();
-#endif
     const long long G = gridDim.x;
     const long long q0 = cta_start(blockIdx.x, p.Q, G), q1 = cta_start(blockIdx.x + 1, p.Q, G);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 8);
@@ -533,7 +522,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             SegIter it = seg_iter_begin<BF16>(p, q0, q1);
             Seg sg;
             while (seg_iter_next<BF16>(p, it, sg)) {
-                for (int tile = 0; tile < sg.ntiles && p.dbg != 2; ++tile, ++t) {
+                for (int tile = 0; tile < sg.ntiles; ++tile, ++t) {
                     if (t >= nst) mbar_wait_bounded_hint(empty0 + 8 * st, ph, &sh->abort_flag, kVpIdleHintNs);
                     uint32_t off = (uint32_t)tile * TILE;
                     uint32_t bytes = sg.body_bytes - off < (uint32_t)TILE ? sg.body_bytes - off : (uint32_t)TILE;
@@ -577,11 +566,9 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 const int nfull = (int)(sg.body_bytes / TILE);
                 cm_t* slot = cmax + (size_t)pb * p.n_cmax + (size_t)tid * p.max_tiles;  // this thread's slots, by tile
                 for (int tile = 0; tile < sg.ntiles; ++tile, ++slot) {
-                    if (p.dbg != 2) mbar_wait_bounded_hint(full0 + 8 * st, ph, &sh->abort_flag, 2000u);
+                    mbar_wait_bounded_hint(full0 + 8 * st, ph, &sh->abort_flag, 2000u);
                     const uint4* wb = (const uint4*)(ring + (size_t)st * TILE + (size_t)warp * WBLK);
-                    if (p.dbg == 1) {
-                        *slot = 0;
-                    } else if (tile < nfull) {
+                    if (tile < nfull) {
                         process_chunk<BF16, false>(wb, lane, 0, a, slot);
                     } else {
                         int nv = ((int)(sg.body_bytes - (uint32_t)tile * TILE) - warp * WBLK) / 16;
@@ -615,14 +602,11 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             __syncwarp();
             if (lane == 0) mbar_arrive(ready0 + 8 * pb);
         }
-#ifdef GRAFT_VP_PROF
-        if (warp == 0 && lane == 0) sh->t_stream_end = clock64() - t_kernel0;
-#endif
     } else if (warp == COS_WARP) {
         // ------------------------------ cosine warp ----------------------------------------------
         // Adjacent-position cosines of the SABA state (Eq. 15): a few pairs of hidden-state rows per CTA, read
         // beside the logits stream (under 3 % of its bytes) so that nothing downstream waits for them.
-        if (p.cos_out != nullptr && !p.dbg) {
+        if (p.cos_out != nullptr) {
             const int npairs = (p.rows / p.L) * (p.L - 1);
             for (int q = (int)blockIdx.x; q < npairs; q += (int)gridDim.x) {
                 const int sb = q / (p.L - 1), d = q - sb * (p.L - 1);
@@ -647,19 +631,10 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             const uint32_t pb = k % kVpBufs;
             const char* rowp = p.logits + (size_t)sg.row * p.V * T::ESZ;
             const cm_t* cmx = cmax + (size_t)pb * p.n_cmax;
-#ifdef GRAFT_VP_PROF
-            long long tprof = clock64();
-#endif
             if (ew == 0) mbar_wait_bounded_hint(ready0 + 8 * pb, (k / kVpBufs) & 1u, &sh->abort_flag, kVpIdleHintNs);
-            if (p.dbg) {
-                __syncwarp();
-                if (ew == 0 && lane == 0) mbar_arrive(done0 + 8 * pb);
-                continue;
-            }
             float c = -INFINITY, s = 0.f;
             uint32_t vmo = 0;
             if (ew == 0) {
-                VP_T(0);
                 int overflow = 0, ncand = 0;
                 // (a) log-sum-exp pieces of the streaming warps
                 c = lane < NW ? sh->wc[pb][lane] : -INFINITY;
@@ -695,7 +670,6 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                         ncand = warp_append(es->cand, ncand, kVpCandCap, in, key, lane, &overflow);
                     }
                 }
-                VP_T(1);
                 // (c) T = the K-th largest group maximum, truncated to its top 16 bits: a lower bound of
                 //     the K-th largest element of the segment's body (0 when fewer than K threads saw data)
                 uint32_t Tv = 0;
@@ -749,7 +723,6 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     es->ncand = ncand;
                     es->ovf = overflow;
                 }
-                VP_T(2);
             }
             epi_bar(grp);
             const uint32_t Tv = es->Tv;
@@ -776,7 +749,6 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 }
             }
             epi_bar(grp);
-            if (ew == 0) VP_T(3);
             // (e) the 16-byte vectors of the hit chunks, re-read from global memory; elements >= T become keys.
             //     A thread issues its loads of a round before it uses any: under a saturated memory system one
             //     round trip costs microseconds.
@@ -854,7 +826,6 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 }
                 epi_bar(grp);
             }
-            if (ew == 0) VP_T(4);
             // (f) exact top-K of the candidates by rank counting (keys are distinct, so ranks are a permutation)
             const bool overflow = es->ovf != 0 || es->ncand > kVpCandCap;
             const int ncand = es->ncand < kVpCandCap ? es->ncand : kVpCandCap;
@@ -871,15 +842,6 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             }
             epi_bar(grp);
             if (ew != 0) continue;
-            VP_T(5);
-#ifdef GRAFT_VP_PROF
-            if (blockIdx.x == 1 && lane == 0) {
-                atomicAdd(p.errflag + 10, ncand);
-                atomicAdd(p.errflag + 11, es->nhits);
-                atomicAdd(p.errflag + 12, 1);
-                atomicAdd(p.errflag + 13, es->nht);
-            }
-#endif
             // the double-buffered arrays of parity pb may be reused from here on
             __syncwarp();
             if (lane == 0) mbar_arrive(done0 + 8 * pb);
@@ -965,7 +927,6 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     if (lane == 0) p.row_counter[sg.row] = 0;
                 }
             }
-            VP_T(6);
             if (finish && p.partial_out != nullptr) {
                 graft_vocab_partial* po = p.partial_out + sg.row;
                 if (lane < kMaxK) po->keys[lane] = lane < nk ? es->outk[lane] : 0ull;
@@ -978,25 +939,11 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             } else if (finish) {
                 vp_finalize(Cd, Sd, Vm, nk, p.K, es->outk, lane, p.topk_id + (size_t)sg.row * p.K,
                             p.topk_lp + (size_t)sg.row * p.K, p.lse + sg.row, p.row_status + sg.row);
-                VP_T(7);
             }
             __syncwarp();
         }
     }
     __syncthreads();
-#ifdef GRAFT_VP_PROF
-    if (tid == 0) {
-        unsigned smid;
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        long long gt;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
-        float* dbg = p.dbg_out + (size_t)blockIdx.x * 4;
-        dbg[0] = (float)sh->t_stream_end;
-        dbg[1] = (float)(clock64() - t_kernel0);
-        dbg[2] = (float)smid;
-        dbg[3] = (float)(gt & 0xFFFFFF);
-    }
-#endif
     if (tid == 0 && sh->abort_flag) atomicOr(p.errflag, 1);
 }
 
@@ -1129,13 +1076,6 @@ cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* 
     p.L = cfg.L;
     p.cos_out = (d_hidden != nullptr && cfg.L > 1) ? d_cos : nullptr;
     p.use_hint = 1;
-    p.dbg = 0;
-    p.dbg_out = ctx->w_edge;
-#ifdef GRAFT_VP_EXPERIMENT  // tuning switches, never compiled into the shipped library
-    if (getenv("GRAFT_VP_HINT")) p.use_hint = atoi(getenv("GRAFT_VP_HINT"));
-    if (getenv("GRAFT_VP_DEBUG")) p.dbg = atoi(getenv("GRAFT_VP_DEBUG"));
-    if (getenv("GRAFT_VP_STAGES")) p.stages = atoi(getenv("GRAFT_VP_STAGES"));
-#endif
     if (bf16)
         vocab_pass_kernel<true><<<pl.grid, kVpThreads, pl.smem_bytes, st>>>(p);
     else
@@ -1188,7 +1128,7 @@ cudaError_t vp_configure(const graft_config& cfg, int num_sms, size_t* max_smem)
 namespace graft {
 namespace {
 
-constexpr int kStaticMaxGrid = 512;     // CTAs: two per SM on up to 256 SMs
+constexpr int kStaticMaxGrid = 512;     // CTAs (one per SM is launched): room for any device
 constexpr int kStaticMaxRows = 16384;   // batch * L
 
 struct VpStaticScratch {
@@ -1293,8 +1233,6 @@ extern "C" graft_status graft_vocab_pass_static(int32_t batch, int32_t L, int32_
     p.L = L;
     p.cos_out = nullptr;
     p.use_hint = 1;
-    p.dbg = 0;
-    p.dbg_out = nullptr;
     if (logits_dtype == GRAFT_BF16)
         vocab_pass_kernel<true><<<pl.grid, kVpThreads, pl.smem_bytes, st>>>(p);
     else

@@ -5,7 +5,8 @@ import torch
 
 import graft_inputs as gi
 import oracle
-from helpers import EPS, check_tree_invariants, compare_accept, compare_round, gpu_round, oracle_round
+from helpers import (EPS, check_tree_invariants, compare_accept, compare_round, gpu_round, oracle_round,
+                     tolerance)
 
 pytestmark = pytest.mark.gpu
 
@@ -49,7 +50,7 @@ def _vocab_case(z, K, dtype):
     fin = np.isfinite(b)
     assert np.array_equal(np.isneginf(a), np.isneginf(b))
     # (an fp32 result cannot be closer than its own spacing: one ulp beyond |x| = 128 already exceeds EPS)
-    assert np.all(np.abs(a[fin] - b[fin]) <= EPS + np.spacing(np.abs(b[fin]).astype(np.float32)))
+    assert np.all(np.abs(a[fin] - b[fin]) <= tolerance(b[fin]))
     # candidates come in rank order, so their log-probabilities never increase along a row, and equal logits get the
     # same bits (every candidate of a row is measured against one log-sum-exp)
     assert np.all(a[:, 1:] <= a[:, :-1]), "log-probabilities increase along a row"
@@ -59,7 +60,7 @@ def _vocab_case(z, K, dtype):
         same = vals[1:] == vals[:-1]
         assert np.array_equal(lp[r, 1:][same], lp[r, :-1][same]), f"row {r}: equal logits, different log-probabilities"
     # lse is returned as an fp32 number: allow its own rounding on top of EPS
-    assert np.all(np.abs(lse[good, 0] - o_lse[good]) <= EPS + np.spacing(np.abs(lse[good, 0])))
+    assert np.all(np.abs(lse[good, 0] - o_lse[good]) <= tolerance(o_lse[good]))
     g.destroy()
     return float(np.abs(lse[good, 0] - o_lse[good]).max(initial=0))
 
@@ -183,6 +184,8 @@ def test_vocab_pass_is_reproducible_and_counters_reset():
     (300, 64, 4, "bf16"),       # tensor-core path, the narrowest scorer
     (500, 100, 16, "bf16"),     # E not a multiple of 8: the FMA kernel
     (777, 200, 24, "f32"),      # fp32 embeddings: the FMA kernel
+    (70001, 2048, 8, "bf16"),   # tensor-core path at the sizes it runs at: two slabs of rows, two chunks along E
+    (66000, 1096, 24, "bf16"),  # a second slab of 464 rows and a last chunk of 72 columns
 ])
 def test_tdes_precompute_against_oracle(V, E, m, emb_dtype):
     L = 4
@@ -262,7 +265,7 @@ def test_vocab_pass_parallel_matches_the_full_row_oracle(V, K, L, Bt, dtype, wor
     assert np.array_equal(np.isneginf(a), np.isneginf(b))
     fin = np.isfinite(b)
     assert np.abs(a[fin] - b[fin]).max(initial=0) <= EPS
-    assert np.all(np.abs(lse[good, 0] - o_lse[good]) <= EPS + np.spacing(np.abs(lse[good, 0])))
+    assert np.all(np.abs(lse[good, 0] - o_lse[good]) <= tolerance(o_lse[good]))
     for gs in keep:
         gs.destroy()
 
@@ -518,53 +521,89 @@ def test_config_C1_full():
     assert (gpu0["path_score"][0, 1:n] <= 0).all()
 
 
-@pytest.mark.parametrize("name,nseq", [("C2", 16), ("C3", 6), ("M", 6), ("C5", 4), ("C4", 3)])
-def test_config_full_size_sampled(name, nseq):
-    """Full-size launch configuration; the oracle checks a sample of sequences one by one, and the
-    invariants are checked on every sequence."""
+def _report(name, stats):
+    """The observed largest differences of a configured workload: printed, and appended as a JSON line to the file
+    that GRAFT_PARITY_REPORT names (if any)."""
+    import json
+    import os
+    line = json.dumps(dict(config=name, **{k: v for k, v in stats.items()}))
+    print("parity", line)
+    if os.environ.get("GRAFT_PARITY_REPORT"):
+        with open(os.environ["GRAFT_PARITY_REPORT"], "a") as f:
+            f.write(line + "\n")
+
+
+@pytest.mark.parametrize("name", ["C2", "C3", "M", "C5", "C4"])
+def test_config_full_size_every_sequence(name):
+    """Full-size launch configuration: EVERY sequence is compared with the oracle under the comparison rule and the
+    observed largest differences are reported.  No budget may differ; a tree may differ from the oracle's (as a valid
+    best-first outcome on a score gap below the tolerance, which compare_round verifies) in at most 1 % of the
+    sequences, i.e. in none below a batch of 100 (observed: one sequence of C4's 256, none elsewhere)."""
+    import os
     w = gi.WORKLOADS[name]
     g = _graft(w)
     tb, saba_kw, keep = _setup(w, g)
-    # every sequence's inputs come from its own stream, so a sample can be generated without the rest
-    sample = sorted(set(np.linspace(0, w.batch - 1, nseq).astype(int).tolist()))
-    z = torch.empty((w.batch, w.L, w.V), dtype=torch.bfloat16, device="cuda")
-    h = torch.empty((w.batch, w.L, w.hidden_dim), dtype=torch.bfloat16, device="cuda")
-    root = torch.empty(w.batch, dtype=torch.int32)
-    hist = torch.empty(w.batch, dtype=torch.float32)
-    pref = torch.empty(w.batch, dtype=torch.int32)
-    xs = {}
-    for b in range(w.batch):
-        xb = gi.batch_inputs(w, b, b + 1)
-        z[b], h[b] = xb["logits"][0].cuda(), xb["hidden"][0].cuda()
-        root[b], hist[b], pref[b] = xb["root_token"][0], xb["hist"][0], xb["prefix_len"][0]
-        if b in sample:
-            xs[b] = xb
+    x = gi.batch_inputs(w)
+    cu = lambda t: t.cuda()  # noqa: E731
+    z, h, root, hist, pref = (cu(x[k]) for k in ("logits", "hidden", "root_token", "hist", "prefix_len"))
     out = g.alloc_out(w.batch, debug=True)
-    g.build_trees(z, h, root.cuda(), hist.cuda(), pref.cuda(), None, out)
+    g.build_trees(z, h, root, hist, pref, None, out)
     torch.cuda.synchronize()
     gpu = out.cpu()
     assert (gpu["status"] == 0).all()
-    for b in range(w.batch):
-        tree = {k: gpu[k][b] for k in ("n_nodes", "token", "parent", "depth", "position", "path_score", "mask")}
-        check_tree_invariants(tree, int(gpu["budget"][b]), w.L, None, int(root[b]), int(pref[b]))
-        assert gpu["n_nodes"][b] == gpu["budget"][b] + 1
-    excused = 0
-    for b in sample:
-        orc = oracle_round(oracle, w, xs[b], tb, saba_kw, threads=1)
-        one = {k: v[b:b + 1] for k, v in gpu.items()}
-        st = compare_round(oracle, w, xs[b], tb, saba_kw, one, orc)
-        excused += st["excused_tree"] + st["excused_budget"]
-    assert excused <= max(1, len(sample) // 3)
+    assert np.array_equal(gpu["n_nodes"], gpu["budget"] + 1)
+    orc = oracle_round(oracle, w, x, tb, saba_kw, threads=os.cpu_count() or 8)
+    stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    _report(name, stats)
+    assert stats["sequences"] == w.batch
+    assert stats["excused_budget"] == 0 and stats["excused_tree"] <= w.batch // 100, stats
+    # at these magnitudes the rule is plain 1e-5 absolute: check the observed differences against it directly
+    for k in ("topk_lp", "lse", "edge", "path_score", "state"):
+        assert stats["max_delta"][k] <= EPS, (k, stats["max_delta"])
     compare_accept(oracle, gi, g, w, out, gpu)
     assert len(set(gpu["budget"].tolist())) > 1 or name in ("C2",)
     # the call the benchmark times (no debug outputs: the first depths by the edge-score kernel, deeper ones on
     # demand) gives the same trees as the call checked above, bit for bit, for every sequence
     out_p = g.alloc_out(w.batch, debug=False)
-    g.build_trees(z, h, root.cuda(), hist.cuda(), pref.cuda(), None, out_p)
+    g.build_trees(z, h, root, hist, pref, None, out_p)
     torch.cuda.synchronize()
     prod = out_p.cpu()
     for k in ("n_nodes", "budget", "status", "token", "parent", "depth", "position", "path_score", "mask"):
         assert np.array_equal(prod[k], gpu[k]), k
+    g.destroy()
+
+
+@pytest.mark.parametrize("K,L,budget", [(1, 5, 5), (1, 16, 16), (4, 8, 40), (32, 16, 512)])
+def test_acceptance_walk_reaches_full_depth(K, L, budget):
+    """Peaked rows (one token far above the rest at every position) and targets that follow the chain of best tokens:
+    the walk accepts all L draft tokens, the path is the chain, and the bonus token is the target's token after the
+    deepest node.  A second sequence's targets leave the chain at the last depth (a = L - 1)."""
+    w = gi.small(batch=2, L=L, V=2000, K=K, budget_min=budget, budget_max=budget, fixed_budget=budget, beta=0.0, m=16)
+    g = _graft(w)
+    _setup(w, g)
+    x = gi.batch_inputs(w)
+    best = torch.randint(0, w.V, (w.batch, L), generator=torch.Generator().manual_seed(11))
+    x["logits"].scatter_(2, best[..., None], 25.0)
+    out, gpu = gpu_round(g, w, x)
+    y = np.concatenate([best.numpy(), [[1234], [77]]], axis=1).astype(np.int32)  # y_1..y_L, then the bonus token
+    y[1, L - 1] = next(t for t in range(w.V) if t not in set(gpu["topk_id"][1, L - 1].tolist()))  # no child carries it
+    tn = np.stack([gi.target_next_from_depth(y[b], gpu["depth"][b]) for b in range(w.batch)])
+    a_len = torch.empty(w.batch, dtype=torch.int32, device="cuda")
+    a_path = torch.empty((w.batch, L), dtype=torch.int32, device="cuda")
+    bonus = torch.empty(w.batch, dtype=torch.int32, device="cuda")
+    g.accept(out, torch.from_numpy(tn).cuda(), a_len, a_path, bonus)
+    torch.cuda.synchronize()
+    a_len, a_path, bonus = a_len.cpu().numpy(), a_path.cpu().numpy(), bonus.cpu().numpy()
+    assert a_len.tolist() == [L, L - 1]
+    assert bonus.tolist() == [1234, int(y[1, L - 1])]
+    for b in range(w.batch):
+        a, path, bo = oracle.accept(int(gpu["n_nodes"][b]), gpu["token"][b], gpu["parent"][b], tn[b], L)
+        assert a == a_len[b] and np.array_equal(path, a_path[b]) and bo == bonus[b]
+        n = int(a_len[b])
+        assert np.array_equal(gpu["token"][b][a_path[b, :n]], y[b, :n])          # the path spells the targets
+        assert np.array_equal(gpu["depth"][b][a_path[b, :n]], np.arange(1, n + 1))
+        assert (a_path[b, n:] == -1).all()
+    g.destroy()
 
 
 # --------------------------------------------------------------------------- seeded sweep of shapes
@@ -632,7 +671,8 @@ def test_round_seeded_sweep_with_quantised_logits(kw, step):
     out, gpu = gpu_round(g, w, x)
     orc = oracle_round(oracle, w, x, tb, saba_kw)
     stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
-    assert stats["excused_budget"] <= max(1, w.batch // 2), stats
+    print("excused", stats)
+    assert stats["excused_budget"] <= max(1, w.batch // 2) and stats["excused_tree"] <= max(1, w.batch // 2), stats
     compare_accept(oracle, gi, g, w, out, gpu)
     g.destroy()
 
@@ -652,7 +692,8 @@ def test_round_when_the_node_table_overflows(noise, beta):
     out, gpu = gpu_round(g, w, x)
     orc = oracle_round(oracle, w, x, tb, saba_kw)
     stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
-    assert stats["excused_budget"] == 0, stats
+    print("excused", stats)
+    assert stats["excused_budget"] == 0 and stats["excused_tree"] <= (0 if noise == 0.0 and beta == 0.0 else 1), stats
     assert gpu["n_nodes"].tolist() == [1001, 1001] and gpu["status"].tolist() == [0, 0]
     if noise == 0.0 and beta == 0.0:
         for k in ("token", "parent", "depth", "mask"):
@@ -753,7 +794,7 @@ def test_round_random_sweep_of_input_styles(seed):
     from paper_2608_20375_b200 import Graft, GraftError
     rng = np.random.default_rng(seed)
     styles = ["normal", "quant1", "quant025", "flat", "peaked", "mixed", "huge", "masked", "twopeaks", "ramp"]
-    done = 0
+    done = seqs = excused = 0
     for ci in range(50):
         K = int(rng.choice([1, 2, 3, 4, 5, 8, 13, 16, 20, 27, 32]))
         L = int(rng.choice([1, 2, 3, 5, 7, 12, 16, 24, 32]))
@@ -787,7 +828,9 @@ def test_round_random_sweep_of_input_styles(seed):
         out, gpu = gpu_round(g, w, x)
         orc = oracle_round(oracle, w, x, tb, saba_kw)
         try:
-            compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+            st = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+            seqs += st["sequences"]
+            excused += st["excused_tree"] + st["excused_budget"]
             compare_accept(oracle, gi, g, w, out, gpu)
         except AssertionError as e:
             raise AssertionError(f"case {ci} ({style}, edge rows {rows}, {kw}): {e}") from e
@@ -802,3 +845,6 @@ def test_round_random_sweep_of_input_styles(seed):
         g.destroy()
         done += 1
     assert done >= 40
+    print("excused", excused, "of", seqs)
+    # (degenerate styles tie in bulk; the excused trees are valid best-first outcomes on near-ties)
+    assert excused <= max(1, seqs // 10), (excused, seqs)

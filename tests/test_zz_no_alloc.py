@@ -3,7 +3,8 @@
 Some hosts cannot let a library allocate device memory -- a server whose own pool owns the whole GPU after
 start-up, or a latency path that must not touch the driver's allocator -- so this entry point keeps its
 scratch in a static device array.  The test calls it through the C ABI twice in a row (the array is shared by
-all calls and keeps the previous call's contents) and checks both results against graft_vocab_pass.  It lives
+all calls and keeps the previous call's contents) and checks both results against graft_vocab_pass, and against
+the CPU oracle on the same rows.  It lives
 in a file that pytest collects last, and it must pass both alone in a fresh process and after the other tests.
 """
 import numpy as np
@@ -51,7 +52,15 @@ def test_static_entry_point_matches_context_entry_point_twice(shape, K, dtype):
         assert np.array_equal(rs.cpu().numpy(), want_rs)
         assert np.array_equal(ids.cpu().numpy()[good], want_ids[good])
         assert np.abs(lp.cpu().numpy()[good] - want_lp[good]).max() <= 1e-5
-        assert np.all(np.abs(lse.cpu().numpy()[good] - want_lse[good]) <= 1e-5 + np.spacing(np.abs(want_lse[good])))
+        assert np.abs(lse.cpu().numpy()[good] - want_lse[good]).max() <= 1e-5
+        # and against the oracle directly
+        import oracle
+        o_ids, o_lp, o_lse, o_st = oracle.vocab_pass(z.cpu().reshape(Bt * L, V), K)
+        ok = o_st == 0
+        assert np.array_equal(rs.cpu().numpy().reshape(-1), o_st)
+        assert np.array_equal(ids.cpu().numpy().reshape(Bt * L, K)[ok], o_ids[ok])
+        assert np.abs(lp.cpu().numpy().reshape(Bt * L, K)[ok].astype(np.float64) - o_lp[ok]).max() <= 1e-5
+        assert np.abs(lse.cpu().numpy().reshape(-1)[ok].astype(np.float64) - o_lse[ok]).max() <= 1e-5
 
 
 def test_static_entry_point_rejects_sizes_beyond_its_scratch():
