@@ -650,7 +650,7 @@ def test_round_seeded_sweep_of_shapes(kw, rows):
     out, gpu = gpu_round(g, w, x)
     orc = oracle_round(oracle, w, x, tb, saba_kw)
     stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
-    assert stats["excused_tree"] + stats["excused_budget"] <= max(1, w.batch // 2), stats
+    assert stats["excused_tree"] + stats["excused_budget"] <= 1, stats  # observed: none
     compare_accept(oracle, gi, g, w, out, gpu)
     g.destroy()
 
@@ -672,7 +672,7 @@ def test_round_seeded_sweep_with_quantised_logits(kw, step):
     orc = oracle_round(oracle, w, x, tb, saba_kw)
     stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
     print("excused", stats)
-    assert stats["excused_budget"] <= max(1, w.batch // 2) and stats["excused_tree"] <= max(1, w.batch // 2), stats
+    assert stats["excused_budget"] <= 1 and stats["excused_tree"] <= 1, stats  # observed: none
     compare_accept(oracle, gi, g, w, out, gpu)
     g.destroy()
 
@@ -847,4 +847,4 @@ def test_round_random_sweep_of_input_styles(seed):
     assert done >= 40
     print("excused", excused, "of", seqs)
     # (degenerate styles tie in bulk; the excused trees are valid best-first outcomes on near-ties)
-    assert excused <= max(1, seqs // 10), (excused, seqs)
+    assert excused <= seqs // 20, (excused, seqs)  # observed: 0 to 3 per hundred
