@@ -157,7 +157,10 @@ graft_status graft_build_trees(graft_ctx* ctx, int32_t batch, const void* d_logi
 /* The steps of the round on their own (the same kernels graft_build_trees runs), for per-step timing
  * and parity checks. */
 /* Vocab pass: per (sequence, position) log-sum-exp over V and the K top-ranked tokens with their log q.
- * d_row_status [batch*L] (may be NULL) receives GRAFT_ST_BAD_LOGITS or 0 per row. */
+ * d_row_status [batch*L] (may be NULL) receives per row 0, GRAFT_ST_BAD_LOGITS, and / or GRAFT_ST_INTERNAL when a
+ * bounded device-side wait ran out in a thread block that worked on the row (its outputs are then not valid; the
+ * call itself still returns GRAFT_OK and the context stays usable).  The same holds for graft_vocab_pass_static
+ * and, through the shards' pieces, for graft_vocab_pass_partial / graft_vocab_merge. */
 graft_status graft_vocab_pass(graft_ctx* ctx, int32_t batch, const void* d_logits, int32_t* d_topk_id,
                               float* d_topk_lp, float* d_lse, int32_t* d_row_status, void* stream);
 /* TDES edge scores (Eq. 4-6) from candidates: d_edge [batch, L, K, K]. */
@@ -197,7 +200,8 @@ typedef struct {
     double c;          /* reference exponent (log2 domain) */
     double s;          /* sum_v 2^(z_v log2(e) - c) over the shard */
     uint32_t vmax_ord; /* largest logit of the shard, as an order-preserving integer */
-    uint32_t nkeys;    /* valid keys (min(K, shard width)) */
+    uint32_t nkeys;    /* valid keys (min(K, shard width)); bit 31: a bounded device-side wait ran out while this
+                          shard was scanned (graft_vocab_merge reports it as GRAFT_ST_INTERNAL) */
     uint64_t keys[32]; /* (order-preserving value << 32) | (0xFFFFFFFF - local id), descending */
 } graft_vocab_partial;
 graft_status graft_vocab_pass_partial(graft_ctx* ctx, int32_t batch, const void* d_logits_shard,

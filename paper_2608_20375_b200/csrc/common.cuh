@@ -91,9 +91,10 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity
 }
 __device__ __forceinline__ bool mbar_wait_bounded_hint(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t ns) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;  // somebody gave up already: nobody waits any more
     for (uint32_t it = 0; it < GRAFT_SPIN_LIMIT; ++it) {
         if (mbar_try_wait_hint(bar, parity, ns)) return true;
-        if ((it & 255u) == 255u && *abort_flag) return false;
+        if ((it & 15u) == 15u && *abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
@@ -102,6 +103,7 @@ __device__ __forceinline__ bool mbar_wait_bounded_hint(uint32_t bar, uint32_t pa
 // gave up; callers then carry on without waiting so that every thread still reaches the kernel's end.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;  // somebody gave up already: nobody waits any more
     for (uint32_t it = 0; it < GRAFT_SPIN_LIMIT; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_flag) return false;

@@ -451,10 +451,10 @@ __device__ int warp_fallback_select(EpiShared* sh, const VpParams& p, const Seg&
 }
 
 // The outputs of a finished row from its pieces: C, S with sum_v 2^(z_v c) = S 2^C (c = fp32(log2 e)), the largest
-// logit, and the K best keys.  One warp.
+// logit, and the K best keys.  One warp.  `internal`: a bounded wait ran out in a CTA that worked on this row.
 __device__ __forceinline__ void vp_finalize(double Cd, double Sd, uint32_t Vm, int nk, int K, const uint64_t* keys,
                                             int lane, int32_t* topk_id, float* topk_lp, float* lse,
-                                            int32_t* row_status) {
+                                            int32_t* row_status, bool internal) {
     // The stream accumulates 2^(z c - ref) with c = fp32(log2 e), so (C + log2 S) ln 2 is the
     // log-sum-exp of the logits scaled by a = c ln 2 = 1 + 1.3e-8.  To first order that adds
     // (a - 1) E_q[z]; the largest logit stands in for the mean under q (the difference is a few
@@ -476,7 +476,7 @@ __device__ __forceinline__ void vp_finalize(double Cd, double Sd, uint32_t Vm, i
     }
     if (lane == 0) {
         *lse = (float)lse_d;
-        *row_status = bad ? GRAFT_ST_BAD_LOGITS : 0;
+        *row_status = (bad ? GRAFT_ST_BAD_LOGITS : 0) | (internal ? GRAFT_ST_INTERNAL : 0);
     }
 }
 
@@ -522,12 +522,27 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             SegIter it = seg_iter_begin<BF16>(p, q0, q1);
             Seg sg;
             while (seg_iter_next<BF16>(p, it, sg)) {
+                // the segment this CTA visits last is read the ordinary way instead of evict-first: the second
+                // stage of its epilogue, which nothing overlaps any more, then finds its chunks in L2
+                const bool hint = p.use_hint && !(it.qi >= it.q_last);
                 for (int tile = 0; tile < sg.ntiles; ++tile, ++t) {
                     if (t >= nst) mbar_wait_bounded_hint(empty0 + 8 * st, ph, &sh->abort_flag, kVpIdleHintNs);
+#ifdef GRAFT_TEST_WITHHOLD_TILE
+                    // Test builds only (the shipped library is never compiled with this): CTA 0 does not issue the
+                    // copy of one of its tiles, so that the streaming warps' bounded wait for it runs out and the
+                    // time-out path (error flag, status bit, drain) can be exercised without faulting anything.
+                    if (blockIdx.x == 0 && t == GRAFT_TEST_WITHHOLD_TILE) {
+                        if (++st == nst) {
+                            st = 0;
+                            ph ^= 1;
+                        }
+                        continue;
+                    }
+#endif
                     uint32_t off = (uint32_t)tile * TILE;
                     uint32_t bytes = sg.body_bytes - off < (uint32_t)TILE ? sg.body_bytes - off : (uint32_t)TILE;
                     mbar_arrive_expect_tx(full0 + 8 * st, bytes);
-                    if (p.use_hint)
+                    if (hint)
                         tma_load_1d_hint(smem_u32(ring + (size_t)st * TILE), sg.body + off, bytes, full0 + 8 * st, policy);
                     else
                         tma_load_1d(smem_u32(ring + (size_t)st * TILE), sg.body + off, bytes, full0 + 8 * st);
@@ -852,6 +867,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             double Cd = (double)c, Sd = (double)s;
             uint32_t Vm = vmo;
             bool finish = (nseg == 1);
+            int rec_internal = 0;  // a bounded wait ran out in one of the CTAs that left a record for this row
             if (nseg > 1) {
                 const int my_first_row = (int)(q0 / p.nq);
                 VpRecord* rec = p.records + (size_t)blockIdx.x * 2 + (sg.row == my_first_row ? 0 : 1);
@@ -860,7 +876,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     rec->c = c;
                     rec->s = s;
                     rec->vmax = __uint_as_float(vmo);
-                    rec->nkeys = (uint32_t)nk;
+                    rec->nkeys = (uint32_t)nk | (sh->abort_flag ? 0x80000000u : 0u);
                 }
                 __threadfence();
                 __syncwarp();
@@ -898,6 +914,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     for (int cc = c_first + lane; cc <= c_last; cc += 32) {
                         const int c_row0 = (int)(cta_start(cc, p.Q, G) / p.nq);
                         const VpRecord* r = p.records + (size_t)cc * 2 + (sg.row == c_row0 ? 0 : 1);
+                        if (__ldcg(&r->nkeys) & 0x80000000u) rec_internal = 1;
                         const float rc = __ldcg(&r->c);
                         const uint32_t rv = __float_as_uint(__ldcg(&r->vmax));
                         Cm = fmax(Cm, (double)rc);
@@ -921,6 +938,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     }
 #pragma unroll
                     for (int d = 16; d > 0; d >>= 1) S += __shfl_xor_sync(0xFFFFFFFFu, S, d);
+                    rec_internal = __any_sync(0xFFFFFFFFu, rec_internal);
                     Cd = Cm;
                     Sd = S;
                     Vm = vm;
@@ -934,11 +952,12 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     po->c = Cd;
                     po->s = Sd;
                     po->vmax_ord = Vm;
-                    po->nkeys = (uint32_t)nk;
+                    po->nkeys = (uint32_t)nk | ((rec_internal || sh->abort_flag) ? 0x80000000u : 0u);
                 }
             } else if (finish) {
                 vp_finalize(Cd, Sd, Vm, nk, p.K, es->outk, lane, p.topk_id + (size_t)sg.row * p.K,
-                            p.topk_lp + (size_t)sg.row * p.K, p.lse + sg.row, p.row_status + sg.row);
+                            p.topk_lp + (size_t)sg.row * p.K, p.lse + sg.row, p.row_status + sg.row,
+                            rec_internal || sh->abort_flag != 0);
             }
             __syncwarp();
         }
@@ -969,7 +988,7 @@ __global__ void __launch_bounds__(128) vocab_merge_kernel(const MergeParams p) {
     for (int i = tid; i < n; i += 128) {
         const int sidx = i / kMaxK, kk = i % kMaxK;
         const graft_vocab_partial* r = p.parts + (size_t)sidx * p.rows + row;
-        uint64_t key = kk < (int)r->nkeys ? r->keys[kk] : 0ull;
+        uint64_t key = kk < (int)(r->nkeys & 0x7FFFFFFFu) ? r->keys[kk] : 0ull;
         if (key != 0ull) key = make_key(bits_from_ord((uint32_t)(key >> 32)), key_id(key) + (uint32_t)p.v_offset[sidx]);
         cand[i] = key;
     }
@@ -978,7 +997,7 @@ __global__ void __launch_bounds__(128) vocab_merge_kernel(const MergeParams p) {
         sC[tid] = r->c;
         sS[tid] = r->s;
         sV[tid] = r->vmax_ord;
-        sN[tid] = r->nkeys;
+        sN[tid] = r->nkeys;  // bit 31: a bounded wait ran out while the shard was scanned
     }
     if (tid < kMaxK) outk[tid] = 0ull;
     __syncthreads();
@@ -993,7 +1012,11 @@ __global__ void __launch_bounds__(128) vocab_merge_kernel(const MergeParams p) {
     __syncthreads();
     if (tid >= 32) return;
     int have = 0;
-    for (int sidx = 0; sidx < p.n_shards; ++sidx) have += (int)sN[sidx];
+    bool internal = false;
+    for (int sidx = 0; sidx < p.n_shards; ++sidx) {
+        have += (int)(sN[sidx] & 0x7FFFFFFFu);
+        internal = internal || (sN[sidx] >> 31) != 0u;
+    }
     const int nk = have < p.K ? have : p.K;
     double Cm = -INFINITY;
     uint32_t vm = 0u;
@@ -1009,7 +1032,7 @@ __global__ void __launch_bounds__(128) vocab_merge_kernel(const MergeParams p) {
             S += sS[sidx];
     }
     vp_finalize(Cm, S, vm, nk, p.K, outk, lane, p.topk_id + (size_t)row * p.K, p.topk_lp + (size_t)row * p.K,
-                p.lse + row, p.row_status + row);
+                p.lse + row, p.row_status + row, internal);
 }
 
 }  // namespace
