@@ -46,7 +46,9 @@ constexpr int TREE_THREADS = 1024;  // one CTA per SM (shared memory bound): all
 struct TreeSmem {
     float* es;           // [L*K*K]  sorted edge rows
     uint8_t* ei;         // [L*K*K]  child rank of each sorted entry
-    // node table of the parallel phase (append-only; node 0 = root)
+    // node table of the parallel phase (append-only; node 0 = root).  Levels follow one another, and within a level
+    // the nodes stand in the order of their prefixes (the parent's place in its level, then the candidate rank), which
+    // is the level order of the emitted tree: a subset taken in table order is already in level order
     uint32_t* nkey;      // [ncap]   bottleneck key = min over the path of ord(path score); later: compact index
     float* nS;           // [ncap]   path score
     uint32_t* ninfo;     // [ncap]   parent's table index | candidate rank << 13 | depth << 18
@@ -63,7 +65,7 @@ struct TreeSmem {
     int16_t* lvl_list;   // [nmax]
     int16_t* cc;         // [2][nmax] per-level child counts in level order, then their exclusive scan (two levels)
     uint32_t* stage;     // [8 warps * 32 rows * W] mask rows staged for coalesced stores
-    uint32_t* hist;      // [2 * 4 * 256]
+    uint32_t* hist;      // [2208] histograms of the threshold searches; scan and child-mask scratch of the level expansion
     int* lvl_count;      // [kMaxL + 2]
     int* lvl_start;      // [kMaxL + 2]
     int* lvl_fill;       // [kMaxL + 2]
@@ -92,7 +94,7 @@ __host__ __device__ inline size_t tree_smem_layout(int L, int K, int nmax, int n
     size_t o_tab = take(table > emis ? table : emis);
     size_t o_ent = take((size_t)nmax * 8), o_S = take((size_t)nmax * 4), o_chm = take((size_t)nmax * 4),
            o_par = take((size_t)nmax * 2), o_can = take((size_t)nmax * 2), o_cp = take((size_t)nmax * 2),
-           o_cand = take(nmax), o_dep = take(nmax), o_hist = take(2048 * 4), o_lc = take((kMaxL + 2) * 4),
+           o_cand = take(nmax), o_dep = take(nmax), o_hist = take(2208 * 4), o_lc = take((kMaxL + 2) * 4),
            o_ls = take((kMaxL + 2) * 4), o_lf = take((kMaxL + 2) * 4), o_sc = take(16 * 4), o_cos = take(kMaxL * 8);
     size_t o_gp = 0, o_gc = 0, o_gu = 0, o_tk = 0, o_lp = 0;
     if (lazy_m > 0) {
@@ -520,11 +522,12 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             sm.nS[0] = 0.0f;
             sm.ninfo[0] = 0u;
         }
-        if (t1 < K) {  // level 0: the root's children, row (depth 0, parent rank 0)
+        if (t1 < K) {  // level 0: the root's children, row (depth 0, parent rank 0); a child's slot is its rank
             const float sc = 0.0f + sm.es[t1];
-            sm.nkey[1 + t1] = ord_from_float(sc);
-            sm.nS[1 + t1] = sc;
-            sm.ninfo[1 + t1] = 0u | ((uint32_t)sm.ei[t1] << 13) | (1u << 18);
+            const int c = sm.ei[t1];
+            sm.nkey[1 + c] = ord_from_float(sc);
+            sm.nS[1 + c] = sc;
+            sm.ninfo[1 + c] = 0u | ((uint32_t)c << 13) | (1u << 18);
         }
         named_bar_sync(1, nth);
         for (int j = t1; j < K * K; j += nth) {  // level 1
@@ -533,9 +536,10 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             const int row = (K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
             const float sc = sm.nS[x] + sm.es[row + r];
             const uint32_t oc = ord_from_float(sc);
-            sm.nkey[1 + K + j] = oc < kx ? oc : kx;
-            sm.nS[1 + K + j] = sc;
-            sm.ninfo[1 + K + j] = (uint32_t)x | ((uint32_t)sm.ei[row + r] << 13) | (2u << 18);
+            const int c = sm.ei[row + r], at = 1 + K + xi * K + c;
+            sm.nkey[at] = oc < kx ? oc : kx;
+            sm.nS[at] = sc;
+            sm.ninfo[at] = (uint32_t)x | ((uint32_t)c << 13) | (2u << 18);
         }
     }
     if (warp == 0) {  // status and budget: from the edge-score kernel if it ran ahead, else worked out here
@@ -590,6 +594,9 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     }
     __syncthreads();
     bool table_ok = budget > 0;
+    // ordered: the parallel phase selected the whole tree, and its nodes stand in level order already (no sequential
+    // tail, no placement): true unless several keys tie with the B-th largest or the node table overflowed
+    bool ordered = false;
     uint32_t theta = 0u;
     if (budget > 0) {
         int ntot = 1, n_at_select = 1;
@@ -599,7 +606,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         if (spec) {  // levels 0 and 1 are in the table already: the threshold they give, then on from level 2
             ntot = 1 + K + K * K;
             if (ntot - 1 >= budget) {
-                sel_top = __uint_as_float(bits_from_ord(sm.nkey[1]));
+                sel_top = 0.0f + sm.es[0];  // the root's best child
                 theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);
                 n_at_select = ntot;
             }
@@ -628,25 +635,28 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                         const int row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
                         const float sc = sm.nS[x] + sm.es[row + r];
                         const uint32_t oc = ord_from_float(sc);
-                        sm.nkey[ntot + j] = oc < kx ? oc : kx;
-                        sm.nS[ntot + j] = sc;
-                        sm.ninfo[ntot + j] = (uint32_t)x | ((uint32_t)sm.ei[row + r] << 13) | ((uint32_t)(d + 1) << 18);
+                        const int c = sm.ei[row + r], at = ntot + xi * K + c;  // (a full row: a child's slot is its rank)
+                        sm.nkey[at] = oc < kx ? oc : kx;
+                        sm.nS[at] = sc;
+                        sm.ninfo[at] = (uint32_t)x | ((uint32_t)c << 13) | ((uint32_t)(d + 1) << 18);
                     }
                     if (tid == 0) sm.scal[3] = ntot + total;
                 }
             } else {
                 // The children that can still matter are a prefix of a node's sorted row (scores only fall along the
-                // row); its length comes from a binary search.  Full chunks of 1024 nodes (the dense early levels):
-                // one thread per node finds the length, a scan of the lengths places the chunk's children in the
-                // table, then one thread per child (found in the scan by binary search) writes it, so that neither a
-                // shared counter nor a node with many children holds the others up.  The remaining nodes (sparse
-                // levels): one thread per node reserves its slots with an atomic and writes its children itself.
-                int cur = ntot, c_tail = b0;
-                bool chunk_ovf = false;
-                for (; b1 - c_tail >= TREE_THREADS; c_tail += TREE_THREADS) {  // (uniform)
-                    const int c0 = c_tail, x = c0 + tid;
+                // row); its length comes from a binary search.  The level is taken in chunks of 1024 nodes: one thread
+                // per node finds the length and the set of candidate ranks in that prefix, a scan of the lengths places
+                // the chunk's children in the table in the order of the nodes, then one thread per child (its node found
+                // in the scan by binary search) writes it, behind its siblings of lower rank.  No shared counter, a node
+                // with many children holds nobody up, and the table stays in level order.
+                int cur = ntot;
+                int* pre = (int*)sm.hist;            // [1024] inclusive scan of the chunk, then [32] warp totals
+                uint32_t* cmask = sm.hist + 1100;    // [1024] candidate ranks of the children a node appends
+                for (int c0 = b0; c0 < b1; c0 += TREE_THREADS) {  // (uniform)
+                    const int x = c0 + tid;
                     int cnt = 0;
-                    {
+                    uint32_t mask = 0u;
+                    if (x < b1) {
                         const uint32_t kx = sm.nkey[x];
                         if (kx >= theta) {  // (else dead: none of its descendants can be selected)
                             const int row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
@@ -661,15 +671,16 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                                     hi_r = mid;
                             }
                             cnt = lo_r;
+                            for (int r = 0; r < cnt; ++r) mask |= 1u << sm.ei[row + r];
                         }
                     }
+                    cmask[tid] = mask;
                     int incl = cnt;
 #pragma unroll
                     for (int o2 = 1; o2 < 32; o2 <<= 1) {
                         const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
                         if (lane >= o2) incl += t;
                     }
-                    int* pre = (int*)sm.hist;  // [1024] inclusive scan of the chunk, then [32] warp totals
                     if (lane == 31) pre[TREE_THREADS + warp] = incl;
                     __syncthreads();
                     const int wt = pre[TREE_THREADS + lane];
@@ -684,7 +695,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     __syncthreads();
                     if (cur + total > p.ncap) {  // (uniform)
                         if (tid == 0) sm.scal[4] = 1;
-                        chunk_ovf = true;
                         break;
                     }
                     for (int i = tid; i < total; i += TREE_THREADS) {
@@ -696,53 +706,22 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                             else
                                 lo_t = mid + 1;
                         }
-                        const int r = i - (lo_t ? pre[lo_t - 1] : 0), xo = c0 + lo_t;
+                        const int first = lo_t ? pre[lo_t - 1] : 0;
+                        const int r = i - first, xo = c0 + lo_t;
                         const uint32_t kx = sm.nkey[xo];
                         const int row = (d * K + (int)((sm.ninfo[xo] >> 13) & 31u)) * K;
                         const float sc = sm.nS[xo] + sm.es[row + r];
                         const uint32_t oc = ord_from_float(sc);
-                        sm.nkey[cur + i] = oc < kx ? oc : kx;
-                        sm.nS[cur + i] = sc;
-                        sm.ninfo[cur + i] = (uint32_t)xo | ((uint32_t)sm.ei[row + r] << 13) | ((uint32_t)(d + 1) << 18);
+                        const int c = sm.ei[row + r];
+                        const int at = cur + first + __popc(cmask[lo_t] & ((1u << c) - 1u));
+                        sm.nkey[at] = oc < kx ? oc : kx;
+                        sm.nS[at] = sc;
+                        sm.ninfo[at] = (uint32_t)xo | ((uint32_t)c << 13) | ((uint32_t)(d + 1) << 18);
                     }
                     cur += total;
                     __syncthreads();  // the scan space is reused by the next chunk
                 }
-                if (c_tail > b0) {  // the counter takes over from here
-                    if (tid == 0) sm.scal[3] = cur;
-                    __syncthreads();
-                }
-                if (!chunk_ovf) {
-                    for (int x = c_tail + tid; x < b1; x += TREE_THREADS) {
-                        const uint32_t kx = sm.nkey[x];
-                        if (kx < theta) continue;  // dead: none of its descendants can be selected
-                        const int row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
-                        const float sx = sm.nS[x];
-                        int lo_r = 0, hi_r = K;  // first r in [0, K] whose key falls below theta
-                        while (lo_r < hi_r) {
-                            const int mid = (lo_r + hi_r) >> 1;
-                            const uint32_t oc = ord_from_float(sx + sm.es[row + mid]);
-                            if ((oc < kx ? oc : kx) >= theta)
-                                lo_r = mid + 1;
-                            else
-                                hi_r = mid;
-                        }
-                        const int cnt = lo_r;
-                        if (cnt == 0) continue;
-                        const int base = atomicAdd(&sm.scal[3], cnt);
-                        if (base + cnt > p.ncap) {
-                            sm.scal[4] = 1;
-                            continue;
-                        }
-                        for (int r = 0; r < cnt; ++r) {
-                            const float sc = sx + sm.es[row + r];
-                            const uint32_t oc = ord_from_float(sc);
-                            sm.nkey[base + r] = oc < kx ? oc : kx;
-                            sm.nS[base + r] = sc;
-                            sm.ninfo[base + r] = (uint32_t)x | ((uint32_t)sm.ei[row + r] << 13) | ((uint32_t)(d + 1) << 18);
-                        }
-                    }
-                }
+                if (tid == 0) sm.scal[3] = cur;
             }
             __syncthreads();
             const int nt = sm.scal[3];
@@ -756,7 +735,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             // theta only has to be a lower bound of its final value while the levels are built (it prunes), so
             // the exact B-th largest key is recomputed only when the table has grown noticeably
             if (ntot - 1 >= budget && (theta == 0u || ntot - n_at_select >= ntot / 2)) {
-                sel_top = __uint_as_float(bits_from_ord(sm.nkey[1]));
+                sel_top = 0.0f + sm.es[0];  // the root's best child
                 theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);  // a lower bound
                 n_at_select = ntot;
             }
@@ -766,18 +745,36 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         if (table_ok && ntot - 1 >= budget) {
             // the exact value: the last 16-bit search still holds if nothing was appended after it
             if (!(n_at_select == ntot && sel.valid)) {
-                sel_top = __uint_as_float(bits_from_ord(sm.nkey[1]));
+                sel_top = 0.0f + sm.es[0];  // the root's best child
                 cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);
             }
             theta = cta_finish_select(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);
         }
         __syncthreads();
         if (table_ok) {
-            // compact {key > theta} in table order (parents stay before their children)
             const int per = (ntot + TREE_THREADS - 1) / TREE_THREADS;
             const int i0 = tid * per < ntot ? tid * per : ntot, i1 = i0 + per < ntot ? i0 + per : ntot;
+            // The tree is {key > theta} plus some of the keys equal to theta.  If exactly B keys reach theta (no other
+            // key ties with the B-th largest: the usual case), {key >= theta} is the whole tree; so is the table itself
+            // when it holds fewer than B nodes (theta = 0: every prefix there is has been appended).
+            uint32_t cut = theta;  // nodes with key > cut are taken here
+            if (theta != 0u) {
+                int ge = 0;
+                for (int i = i0 > 1 ? i0 : 1; i < i1; ++i) ge += sm.nkey[i] >= theta ? 1 : 0;
+                ge = __reduce_add_sync(0xFFFFFFFFu, ge);
+                if (tid == 0) sm.scal[8] = 0;
+                __syncthreads();
+                if (lane == 0 && ge) atomicAdd(&sm.scal[8], ge);
+                __syncthreads();
+                if (sm.scal[8] == budget) {  // (uniform)
+                    cut = theta - 1u;
+                    ordered = true;
+                }
+            } else if (ntot - 1 < budget) {
+                ordered = true;  // fewer prefixes than the budget: all of them
+            }
             int cnt = 0;
-            for (int i = i0; i < i1; ++i) cnt += (i == 0 || sm.nkey[i] > theta) ? 1 : 0;
+            for (int i = i0; i < i1; ++i) cnt += (i == 0 || sm.nkey[i] > cut) ? 1 : 0;
             int incl = cnt;
 #pragma unroll
             for (int o2 = 1; o2 < 32; o2 <<= 1) {
@@ -793,7 +790,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             int run = woff + incl - cnt;
             __syncthreads();
             for (int i = i0; i < i1; ++i) {
-                const bool sel = (i == 0 || sm.nkey[i] > theta);
+                const bool sel = (i == 0 || sm.nkey[i] > cut);
                 sm.nkey[i] = sel ? (uint32_t)run : 0xFFFFFFFFu;  // the key is no longer needed: keep the compact index
                 run += sel ? 1 : 0;
             }
@@ -809,9 +806,9 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             }
             n_gt = total - 1;
             __syncthreads();
-            // frontier entries of the selected nodes: the first child of the sorted row that is not selected,
-            // i.e. the first with ord(score) <= theta
-            for (int n = tid; n <= n_gt; n += TREE_THREADS) {
+            // (for the sequential tail only) frontier entries of the selected nodes: the first child of the sorted row
+            // that is not selected, i.e. the first with ord(score) <= theta
+            for (int n = tid; n <= n_gt && !ordered; n += TREE_THREADS) {
                 const int d = sm.depth[n];
                 uint64_t e = 0ull;
                 if (d < L) {
@@ -835,6 +832,12 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         for (; rows_done < L; ++rows_done) lazy_score_row(p, sm, rows_done, root, tid, inflight);
     }
     if (!table_ok && tid == 0) sm.ent[0] = budget > 0 ? pack_entry(0.0f + sm.es[0], 1, 0, 0, sm.ei[0]) : 0ull;
+    if (ordered) {  // (uniform) the tree is complete and in level order
+        if (tid == 0) {
+            sm.scal[1] = n_gt + 1;
+            if (n_gt < budget) sm.scal[2] |= GRAFT_ST_FRONTIER_EMPTY;
+        }
+    } else {
     // emission needs every node's child mask and the node count of every level: cleared here, filled for the nodes
     // selected so far by warps 1..31 while warp 0 runs the sequential tail, and for the tail's nodes by warp 0
     if (tid < kMaxL + 2) {
@@ -917,88 +920,96 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             sm.scal[2] = st;
         }
     }
+    }  // !ordered
     __syncthreads();
 
     // ---- emission in level order -------------------------------------------------------------------------
     // Level order = depth ascending, then the parent's level-order index, then candidate rank.  Level by level:
     // the child counts of level d-1, laid out in level order, are scanned; a node of level d lands at
     // (start of level d) + (children of earlier parents) + (selected siblings of lower rank).
+    // The placement is a chain of short steps over at most nmax nodes: one warp runs it with warp-level
+    // synchronisation only (a barrier of the whole CTA per step cost more than the steps), while the other warps
+    // write the padding of the outputs, which depends on the node count alone.
     const int n_nodes = sm.scal[1];
-    if (warp == 0) {  // starts of the levels 0..L: an exclusive scan of the counts (L <= 32: lane = level, and one more)
-        const int c0 = lane <= L ? sm.lvl_count[lane] : 0;
-        int incl = c0;
-#pragma unroll
-        for (int o2 = 1; o2 < 32; o2 <<= 1) {
-            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
-            if (lane >= o2) incl += t;
-        }
-        if (lane <= L) sm.lvl_start[lane] = incl - c0;
-        const int below32 = __shfl_sync(0xFFFFFFFFu, incl, 31);
-        if (lane == 0 && L == 32) sm.lvl_start[32] = below32;
-        if (lane == 0) sm.canon[0] = 0;
-    }
-    __syncthreads();
-    for (int n = tid; n < n_nodes; n += TREE_THREADS) {
-        const int d = sm.depth[n];
-        sm.lvl_list[sm.lvl_start[d] + atomicAdd(&sm.lvl_fill[d], 1)] = (int16_t)n;
-    }
-    __syncthreads();
-    // cc holds the child counts of the previous level in level order; it is double-buffered (two halves of nmax
-    // entries) so that a level's nodes can leave their own counts for the next level as soon as they know their place
-    if (tid == 0) sm.cc[0] = __popc(sm.chmask[0]);
-    __syncthreads();
-    for (int d = 1; d <= L; ++d) {
-        const int s_prev = sm.lvl_start[d - 1], n_prev = sm.lvl_count[d - 1];
-        const int s_cur = sm.lvl_start[d], n_cur = sm.lvl_count[d];
-        if (n_cur == 0) break;  // uniform: deeper levels are empty too
-        int16_t* ccp = sm.cc + ((d - 1) & 1) * nmax;
-        int16_t* ccn = sm.cc + (d & 1) * nmax;
-        if (warp == 0) {  // exclusive scan of ccp[0..n_prev): a contiguous chunk per lane, then a warp scan
-            const int ch = (n_prev + 31) / 32;
-            const int lo_i = lane * ch, hi_i = min(n_prev, lo_i + ch);
-            int sum = 0;
-            for (int i = lo_i; i < hi_i; ++i) sum += ccp[i];
-            int incl = sum;
+    const int prefix = p.prefix_len[b];
+    const size_t ob = (size_t)b * nmax;
+    if (warp == 0 && !ordered) {
+        // starts of the levels 0..L: an exclusive scan of the counts (L <= 32: lane = level, and one more)
+        {
+            const int c0 = lane <= L ? sm.lvl_count[lane] : 0;
+            int incl = c0;
 #pragma unroll
             for (int o2 = 1; o2 < 32; o2 <<= 1) {
                 const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
                 if (lane >= o2) incl += t;
             }
-            int run = incl - sum;
-            for (int i = lo_i; i < hi_i; ++i) {
-                const int v = ccp[i];
-                ccp[i] = (int16_t)run;
-                run += v;
+            if (lane <= L) sm.lvl_start[lane] = incl - c0;
+            const int below32 = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            if (lane == 0 && L == 32) sm.lvl_start[32] = below32;
+            if (lane == 0) {
+                sm.canon[0] = 0;
+                // cc holds the child counts of the previous level in level order; it is double-buffered (two halves
+                // of nmax entries) so that a level's nodes leave their own counts for the next level as they are placed
+                sm.cc[0] = (int16_t)__popc(sm.chmask[0]);
             }
         }
-        __syncthreads();
-        for (int i = tid; i < n_cur; i += TREE_THREADS) {
-            const int x = sm.lvl_list[s_cur + i];
-            const int y = sm.parent[x];
-            const int at = s_cur + ccp[sm.canon[y] - s_prev] + __popc(sm.chmask[y] & ((1u << sm.cand[x]) - 1u));
-            sm.canon[x] = (int16_t)at;
-            ccn[at - s_cur] = (int16_t)__popc(sm.chmask[x]);
+        __syncwarp();
+        for (int n = lane; n < n_nodes; n += 32) {  // the nodes of every level, in no particular order
+            const int d = sm.depth[n];
+            sm.lvl_list[sm.lvl_start[d] + atomicAdd(&sm.lvl_fill[d], 1)] = (int16_t)n;
         }
-        __syncthreads();
+        __syncwarp();
+        for (int d = 1; d <= L; ++d) {
+            const int s_prev = sm.lvl_start[d - 1], n_prev = sm.lvl_count[d - 1];
+            const int s_cur = sm.lvl_start[d], n_cur = sm.lvl_count[d];
+            if (n_cur == 0) break;  // deeper levels are empty too
+            int16_t* ccp = sm.cc + ((d - 1) & 1) * nmax;
+            int16_t* ccn = sm.cc + (d & 1) * nmax;
+            int carry = 0;  // exclusive scan of ccp[0..n_prev), 32 entries at a time
+            for (int base = 0; base < n_prev; base += 32) {
+                const int i = base + lane;
+                const int v = i < n_prev ? ccp[i] : 0;
+                int incl = v;
+#pragma unroll
+                for (int o2 = 1; o2 < 32; o2 <<= 1) {
+                    const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
+                    if (lane >= o2) incl += t;
+                }
+                if (i < n_prev) ccp[i] = (int16_t)(carry + incl - v);
+                carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+            }
+            __syncwarp();
+            for (int i = lane; i < n_cur; i += 32) {
+                const int x = sm.lvl_list[s_cur + i];
+                const int y = sm.parent[x];
+                const int at = s_cur + ccp[sm.canon[y] - s_prev] + __popc(sm.chmask[y] & ((1u << sm.cand[x]) - 1u));
+                sm.canon[x] = (int16_t)at;
+                ccn[at - s_cur] = (int16_t)__popc(sm.chmask[x]);
+            }
+            __syncwarp();
+        }
+    } else if (warp != 0) {
+        for (int i = n_nodes + tid - 32; i < nmax; i += TREE_THREADS - 32) {
+            o.d_token[ob + i] = -1;
+            o.d_parent[ob + i] = -1;
+            o.d_depth[ob + i] = -1;
+            o.d_position[ob + i] = -1;
+            o.d_path_score[ob + i] = 0.f;
+        }
+        // mask rows from the first multiple of 32 at or above n_nodes on are all padding
+        const int z0 = ((n_nodes + 31) / 32) * 32;
+        for (size_t k = (size_t)z0 * W + tid - 32; k < (size_t)nmax * W; k += TREE_THREADS - 32) o.d_mask[ob * W + k] = 0u;
     }
-    const int prefix = p.prefix_len[b];
-    const size_t ob = (size_t)b * nmax;
+    __syncthreads();
     for (int n = tid; n < n_nodes; n += TREE_THREADS) {
-        const int i = sm.canon[n], d = sm.depth[n];
-        const int par = n == 0 ? -1 : sm.canon[sm.parent[n]];
+        const int i = ordered ? n : sm.canon[n], d = sm.depth[n];
+        const int par = n == 0 ? -1 : (ordered ? sm.parent[n] : sm.canon[sm.parent[n]]);
         sm.cparent[i] = (int16_t)par;
         o.d_token[ob + i] = n == 0 ? root : p.topk_id[((size_t)b * L + d - 1) * K + sm.cand[n]];
         o.d_parent[ob + i] = par;
         o.d_depth[ob + i] = d;
         o.d_position[ob + i] = prefix - 1 + d;
         o.d_path_score[ob + i] = sm.S[n];
-    }
-    for (int i = n_nodes + tid; i < nmax; i += TREE_THREADS) {
-        o.d_token[ob + i] = -1;
-        o.d_parent[ob + i] = -1;
-        o.d_depth[ob + i] = -1;
-        o.d_position[ob + i] = -1;
-        o.d_path_score[ob + i] = 0.f;
     }
     __syncthreads();
     // ancestor masks: each thread builds one row in its warp's staging tile (walking up, level-order indices
@@ -1038,9 +1049,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             for (int k = lane; k < rows * W; k += 32) dst[k] = tile[k];
             __syncwarp();
         }
-        // rows from the first multiple of 32 at or above n_nodes on are all padding
-        const int z0 = ((n_nodes + 31) / 32) * 32;
-        for (size_t k = (size_t)z0 * W + tid; k < (size_t)nmax * W; k += TREE_THREADS) o.d_mask[ob * W + k] = 0u;
     }
     if (p.lazy) cp_async_wait_all();  // table rows fetched ahead for a depth that was never scored
     if (tid == 0) {
