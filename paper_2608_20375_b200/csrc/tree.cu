@@ -248,6 +248,69 @@ __device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, in
     return prefix;
 }
 
+// The same search over keys that are not stored anywhere: the keys of the children that the threads' nodes are
+// about to append (this thread's node: `cnt` children, key of child r = min(kx, ord(sx + es[row + r]))).  Two passes:
+// the leading 16 bits of the kth largest of them, the rest zero -- a lower bound of it.  At most kth nodes of one
+// level can end up in the tree, so this bound may replace a lower threshold before a level is appended; it keeps
+// a level from flooding the node table while few keys are known (sharply peaked rows: every deviation from the
+// best chain costs tens of units, and the B-th largest key of the table stays far down for several levels).
+// Every thread of the CTA calls it; the children number at least kth in all.
+__device__ uint32_t cta_kth_largest_of_children(const TreeSmem& sm, int cnt, uint32_t kx, float sx, int row, int kth,
+                                                int tid) {
+    const int warp = tid >> 5, lane = tid & 31;
+    uint32_t prefix = 0u, mask = 0u;
+    int remaining = kth;
+    sm.hist[tid] = 0u;
+    __syncthreads();
+    for (int pass = 0; pass < 2; ++pass) {
+        const int shift = 24 - 8 * pass;
+        uint32_t* h = sm.hist + (pass & 1) * 1024 + (warp & 3) * 256;
+        for (int r = 0; r < cnt; ++r) {
+            const uint32_t oc = ord_from_float(sx + sm.es[row + r]);
+            const uint32_t k = oc < kx ? oc : kx;
+            if ((k & mask) == prefix) atomicAdd(&h[(k >> shift) & 255u], 1u);
+        }
+        sm.hist[((pass + 1) & 1) * 1024 + tid] = 0u;  // the other generation, for the next pass
+        __syncthreads();
+        if (warp == 0) {  // lane l owns bins 255-8l .. 248-8l, from the top down
+            const uint32_t* hh = sm.hist + (pass & 1) * 1024;
+            int c[8], sum = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int bin = 255 - 8 * lane - j;
+                c[j] = (int)(hh[bin] + hh[256 + bin] + hh[512 + bin] + hh[768 + bin]);
+                sum += c[j];
+            }
+            int incl = sum;
+#pragma unroll
+            for (int o2 = 1; o2 < 32; o2 <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
+                if (lane >= o2) incl += t;
+            }
+            const int excl = incl - sum;
+            if (excl < remaining && remaining <= incl) {
+                int acc = excl, digit = 255 - 8 * lane, rem = remaining - excl;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (acc < remaining && remaining <= acc + c[j]) {
+                        digit = 255 - 8 * lane - j;
+                        rem = remaining - acc;
+                    }
+                    acc += c[j];
+                }
+                sm.scal[6] = digit;
+                sm.scal[7] = rem;
+            }
+        }
+        __syncthreads();
+        prefix |= (uint32_t)sm.scal[6] << shift;
+        mask |= 255u << shift;
+        remaining = sm.scal[7];
+    }
+    __syncthreads();
+    return prefix;
+}
+
 // Threshold searches work on 1024 bins of equal width in SCORE below the best score (the root's best child): bin b
 // holds the keys whose score lies in (top - (b + 1) w, top - b w], w = 1/32, so the bins reach 32 below the top; what
 // lies further down (or is -inf) shares the last bin.  The same expression gives a key's bin wherever it is needed.
@@ -652,15 +715,24 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 int cur = ntot;
                 int* pre = (int*)sm.hist;            // [1024] inclusive scan of the chunk, then [32] warp totals
                 uint32_t* cmask = sm.hist + 1100;    // [1024] candidate ranks of the children a node appends
+                // At most B nodes of a level end up in the tree: a chunk that would append many times more children than
+                // that (or more than the table has room for) first raises theta to (a lower bound of) the B-th largest
+                // key among those children.  (The search costs about as much as two ordinary levels: ordinary rounds,
+                // whose levels stay within a few times B, never run it.)
+                const int flood = 8 * budget > 1024 ? 8 * budget : 1024;
                 for (int c0 = b0; c0 < b1; c0 += TREE_THREADS) {  // (uniform)
-                    const int x = c0 + tid;
+                  const int x = c0 + tid;
+                  int total = 0;
+                  for (int attempt = 0;; ++attempt) {  // (uniform: at most two rounds)
                     int cnt = 0;
-                    uint32_t mask = 0u;
+                    uint32_t mask = 0u, kx = 0u;
+                    float sx = 0.0f;
+                    int row = 0;
                     if (x < b1) {
-                        const uint32_t kx = sm.nkey[x];
+                        kx = sm.nkey[x];
                         if (kx >= theta) {  // (else dead: none of its descendants can be selected)
-                            const int row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
-                            const float sx = sm.nS[x];
+                            row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
+                            sx = sm.nS[x];
                             int lo_r = 0, hi_r = K;  // first r in [0, K] whose key falls below theta
                             while (lo_r < hi_r) {
                                 const int mid = (lo_r + hi_r) >> 1;
@@ -671,7 +743,18 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                                     hi_r = mid;
                             }
                             cnt = lo_r;
-                            for (int r = 0; r < cnt; ++r) mask |= 1u << sm.ei[row + r];
+                            if ((K & 15) == 0) {  // rows of whole 16-byte vectors: the ranks come sixteen at a time
+                                for (int r0 = 0; r0 < cnt; r0 += 16) {
+                                    const uint4 q = *(const uint4*)(sm.ei + row + r0);
+                                    const uint32_t wq[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) {
+                                        if (r0 + j < cnt) mask |= 1u << ((wq[j >> 2] >> (8 * (j & 3))) & 31u);
+                                    }
+                                }
+                            } else {
+                                for (int r = 0; r < cnt; ++r) mask |= 1u << sm.ei[row + r];
+                            }
                         }
                     }
                     cmask[tid] = mask;
@@ -690,9 +773,16 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                         const int t = __shfl_up_sync(0xFFFFFFFFu, wincl, o2);
                         if (lane >= o2) wincl += t;
                     }
-                    const int total = __shfl_sync(0xFFFFFFFFu, wincl, 31);
+                    total = __shfl_sync(0xFFFFFFFFu, wincl, 31);
                     pre[tid] = __shfl_sync(0xFFFFFFFFu, wincl - wt, warp) + incl;
                     __syncthreads();
+                    if (attempt == 0 && total >= budget && (total > flood || cur + total > p.ncap)) {  // (uniform) the search below uses the scan's space: count again
+                        const uint32_t tl = cta_kth_largest_of_children(sm, cnt, kx, sx, row, budget, tid);
+                        theta = tl > theta ? tl : theta;
+                        continue;
+                    }
+                    break;
+                  }
                     if (cur + total > p.ncap) {  // (uniform)
                         if (tid == 0) sm.scal[4] = 1;
                         break;
@@ -783,10 +873,15 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             }
             if (lane == 31) sm.hist[warp] = (uint32_t)incl;
             __syncthreads();
-            int woff = 0;
-            for (int w = 0; w < warp; ++w) woff += (int)sm.hist[w];
-            int total = 0;
-            for (int w = 0; w < TREE_THREADS / 32; ++w) total += (int)sm.hist[w];
+            const int wt = (int)sm.hist[lane];  // (32 warps: a lane per warp total)
+            int wincl = wt;
+#pragma unroll
+            for (int o2 = 1; o2 < 32; o2 <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, wincl, o2);
+                if (lane >= o2) wincl += t;
+            }
+            const int woff = __shfl_sync(0xFFFFFFFFu, wincl - wt, warp);
+            const int total = __shfl_sync(0xFFFFFFFFu, wincl, 31);
             int run = woff + incl - cnt;
             __syncthreads();
             for (int i = i0; i < i1; ++i) {
