@@ -87,7 +87,8 @@ struct EdgeParams {
     float* esort;     // same rows, each sorted by (edge descending, child rank ascending)
     uint8_t* eidx;    // child rank of every sorted entry
     int L, K, m, V;
-    int rows;     // depths [0, rows) are scored: one CTA each
+    int rows;     // depths [0, rows) are scored for every sequence: one CTA each
+    int rows_all; // CTAs per sequence: depths [rows, rows_all) are scored only for sequences whose trees will run deep
     float scale;  // s / sqrt(m)
     float beta;
     int root_edge;
@@ -108,7 +109,8 @@ __global__ void __launch_bounds__(256, 4) tdes_edges_kernel(const EdgeParams p) 
     extern __shared__ __align__(16) float smem[];
     pdl_launch_dependents();  // the tree kernel may move in as SMs free up; it waits for this grid before it reads
     pdl_wait();               // the candidates come from the vocab pass
-    const int b = blockIdx.x / p.rows, j = blockIdx.x % p.rows;
+    const int b = blockIdx.x / p.rows_all, j = blockIdx.x % p.rows_all;
+    if (j >= p.rows && !deep_tree_likely(p.topk_lp + (size_t)b * p.L * p.K, p.L, p.K)) return;  // (uniform)
     const int K = p.K, m = p.m, ld = m + 4;  // padded row: 16-byte aligned, conflict-free float4 reads
     float* sP = smem;                        // [K][ld]  parent rows + u_d
     float* sC = smem + (size_t)kMaxK * ld;   // [K][ld]  child rows + u_d
@@ -245,6 +247,7 @@ cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_i
     p.beta = ctx->tdes_set ? cfg.beta : 0.0f;
     p.root_edge = cfg.root_edge;
     p.rows = rows;
+    p.rows_all = d_edge || rows == cfg.L ? rows : cfg.L;  // (rows < L only when the tree kernel can score on demand)
     p.saba_out = d_row_status ? d_saba_out : nullptr;
     p.cos_pre = ctx->w_cos;
     p.vp_err = ctx->w_errflag;
@@ -255,7 +258,7 @@ cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_i
     p.bmax = cfg.budget_max;
     p.bstep = cfg.budget_step;
     p.saba = ctx->saba;
-    const cudaError_t e = launch_pdl(d_edge ? tdes_edges_kernel<true> : tdes_edges_kernel<false>, dim3(batch * rows),
+    const cudaError_t e = launch_pdl(d_edge ? tdes_edges_kernel<true> : tdes_edges_kernel<false>, dim3(batch * p.rows_all),
                                      dim3(256), tdes_edges_smem(cfg), st, p);
     ctx->launches += 1;
     return e != cudaSuccess ? e : cudaGetLastError();

@@ -29,6 +29,7 @@ struct TreeParams {
     // Edge scores (Eq. 4-6): the rows of depths [0, rows_pre) come from the edge-score kernel through esort / eidx;
     // deeper rows are scored inside this kernel (lazy = 1), level by level, only if the expansion gets there.
     int rows_pre;
+    int rows_adaptive;  // the edge-score kernel also scored the deeper rows of sequences whose trees will run deep
     int lazy;
     int lazy_m;  // m when the shared-memory layout holds the buffers of the on-demand scorer, else 0
     const float* P;
@@ -528,10 +529,11 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     // (they land while warp 0 works out the budget), plain loads otherwise
     __shared__ __align__(8) uint64_t rows_bar;
     __shared__ int rows_abort;
-    const int ne = p.rows_pre * K * K;  // entries that come from the edge-score kernel
+    const int rows_pre = p.rows_pre;
+    const int ne = rows_pre * K * K;  // entries that come from the edge-score kernel for every sequence
     const bool bulk = ne > 0 && (ne % 16) == 0;
     const int root = p.root_token[b];
-    int rows_done = p.rows_pre;  // rows [0, rows_done) are in shared memory
+    int rows_done = rows_pre;  // rows [0, rows_done) are in shared memory
     int inflight = -1;           // on-demand scoring: depth whose table rows are being fetched
     if (tid == 0) {
         rows_abort = 0;
@@ -543,7 +545,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             sm.tokid[i] = p.topk_id[(size_t)b * L * K + i];
             sm.lpv[i] = p.topk_lp[(size_t)b * L * K + i];
         }
-        if (p.rows_pre == 0) {  // the table rows of depth 0 arrive while the budget is worked out
+        if (rows_pre == 0) {  // the table rows of depth 0 arrive while the budget is worked out
             __syncthreads();
             lazy_issue_gather(p, sm, 0, root, tid);
             inflight = 0;
@@ -570,13 +572,22 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             sm.ei[i] = p.eidx[seq_e + i];
         }
     }
+    // a sequence whose tree will run deep had its deeper rows scored by the edge-score kernel as well (they are needed
+    // several levels from here: plain loads, consumed after many barriers)
+    if (p.rows_adaptive && deep_tree_likely(p.topk_lp + (size_t)b * L * K, L, K)) {  // (uniform)
+        for (int i = ne + tid; i < L * K * K; i += TREE_THREADS) {
+            sm.es[i] = p.esort[seq_e + i];
+            sm.ei[i] = p.eidx[seq_e + i];
+        }
+        rows_done = L;
+    }
     // adjacent-position cosines r_d = cos(h_d, h_{d+1}) (Eq. 15): written by the vocab pass
     if (p.use_saba && !p.saba_pre && tid < L - 1) sm.cosv[tid] = p.cos_pre[(size_t)b * L + tid];
     __syncthreads();
     // While warp 0 works out the budget, the other warps expand levels 0 and 1 in full (1 + K + K^2 nodes), which
     // needs no budget: with fewer than B nodes in the table every child is appended anyway, and if B is smaller
     // than that the extra nodes only fall below the threshold found afterwards.
-    const bool spec = bulk && p.rows_pre >= 2 && L >= 2 && 1 + K + K * K <= p.ncap;
+    const bool spec = bulk && rows_pre >= 2 && L >= 2 && 1 + K + K * K <= p.ncap;
     if (spec && warp >= 1) {
         mbar_wait_bounded(smem_u32(&rows_bar), 0, &rows_abort);
         const int t1 = tid - 32, nth = TREE_THREADS - 32;
@@ -1302,6 +1313,7 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     p.W = ctx->mask_words;
     p.rows_pre = ctx->edge_rows;
     p.lazy = p.rows_pre < cfg.L ? 1 : 0;  // (only possible when tree_lazy_fits)
+    p.rows_adaptive = (p.lazy && p.rows_pre > 0 && d_saba_pre != nullptr) ? 1 : 0;
     p.lazy_m = tree_lazy_fits(cfg) ? cfg.m : 0;
     p.ncap = tree_node_cap(cfg.L, cfg.K, ctx->nmax, p.lazy_m);
     p.P = ctx->d_P;
