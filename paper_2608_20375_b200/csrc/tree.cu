@@ -1194,6 +1194,7 @@ __global__ void __launch_bounds__(128) accept_kernel(const AcceptParams ap) {
     int32_t* __restrict__ accept_len = ap.accept_len;
     int32_t* __restrict__ accept_path = ap.accept_path;
     int32_t* __restrict__ bonus = ap.bonus;
+    pdl_launch_dependents();  // the next round's vocab pass may set up its CTAs; it waits for this grid before it reads
     pdl_wait();  // the tree may come from a tree kernel that is still running ahead in the stream
     extern __shared__ __align__(16) int32_t acc_smem[];
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;

@@ -511,6 +511,11 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
     }
     if (tid < kVpBufs * kVpGroups) (&sh->gmax[0][0])[tid] = 0u;
     __syncthreads();
+    // Launched with programmatic stream serialization inside a round: the CTA is set up while the kernel ahead of it in
+    // the stream (the previous round's walk or tree kernel) drains; nothing is read or written before that kernel has
+    // completed (the logits may come from it, and the scratch this kernel writes is read by the previous round's
+    // kernels).  Launched the ordinary way this returns at once.
+    pdl_wait();
 
     if (warp == PROD_WARP) {
         // ------------------------------ producer warp --------------------------------------------
@@ -1099,12 +1104,10 @@ cudaError_t vp_launch(graft_ctx* ctx, int batch, const void* d_logits, int32_t* 
     p.L = cfg.L;
     p.cos_out = (d_hidden != nullptr && cfg.L > 1) ? d_cos : nullptr;
     p.use_hint = 1;
-    if (bf16)
-        vocab_pass_kernel<true><<<pl.grid, kVpThreads, pl.smem_bytes, st>>>(p);
-    else
-        vocab_pass_kernel<false><<<pl.grid, kVpThreads, pl.smem_bytes, st>>>(p);
+    const cudaError_t e = launch_pdl(bf16 ? vocab_pass_kernel<true> : vocab_pass_kernel<false>, dim3(pl.grid),
+                                     dim3(kVpThreads), pl.smem_bytes, st, p);
     ctx->launches += 1;
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t vp_merge_launch(graft_ctx* ctx, int batch, int n_shards, const graft_vocab_partial* d_parts,
