@@ -724,6 +724,49 @@ def run_sweep(args):
                       "fixed_budget": args.sweep_fixed_budget, "rows": rows}))
 
 
+def run_styles(args):
+    """`--styles`: the round's kernels (the library's own CUDA events) on degenerate inputs of the benchmark's shape:
+    ordinary logits, logits on coarse grids, flat rows, one or two dominant tokens over an exactly flat rest, sharply
+    peaked rows, masked vocabularies, ramps (graft_inputs.styled_logits).  One JSON line."""
+    from paper_2608_20375_b200 import Graft
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w0 = gi.WORKLOADS[args.workload]
+    rng = np.random.default_rng(5)
+    rows = []
+    for style in gi.STYLES:
+        w = gi.small(batch=w0.batch, L=w0.L, V=w0.V, K=w0.K, budget_min=w0.budget_min, budget_max=w0.budget_max,
+                     budget_step=w0.budget_step, m=w0.m, hidden_dim=256, logits_dtype=w0.logits_dtype,
+                     hidden_dtype=w0.hidden_dtype, beta=w0.beta, seed=123)
+        g = Graft(w.V, w.L, w.K, w.m, w.hidden_dim, w.batch, w.budget_min, w.budget_max, w.budget_step, w.beta, 1,
+                  1 if w.logits_dtype == "bf16" else 0, 1 if w.hidden_dtype == "bf16" else 0)
+        tb = gi.tdes_tables(w)
+        keep = [tb["P"].to(dev), tb["C"].to(dev), tb["u"].to(dev)]
+        g.set_tdes_tables(keep[0], keep[1], keep[2], tb["s"])
+        g.set_saba(**gi.saba_defaults(w))
+        x = gi.batch_inputs(w, 0, 8)  # eight sequences, repeated to the batch
+        gen = torch.Generator().manual_seed(w.seed)
+        rep = (w.batch + 7) // 8
+        z = gi.styled_logits(x["logits"].float(), style, rng, gen, w.K).to(x["logits"].dtype).repeat(rep, 1, 1)[:w.batch].to(dev)
+        h = x["hidden"].repeat(rep, 1, 1)[:w.batch].to(dev)
+        root, hist, pre = (x[k].repeat(rep)[:w.batch].to(dev) for k in ("root_token", "hist", "prefix_len"))
+        out = g.alloc_out(w.batch)
+        for _ in range(3):
+            g.build_trees(z, h, root, hist, pre, None, out)
+        torch.cuda.synchronize()
+        g.set_timing(1)
+        for _ in range(args.steps):
+            g.build_trees(z, h, root, hist, pre, None, out)
+        torch.cuda.synchronize()
+        n, a, b_, c = g.read_timing()
+        rows.append(dict(style=style, vocab_pass_us=round(a / n * 1e3, 1), tdes_edges_us=round(b_ / n * 1e3, 1),
+                         tree_us=round(c / n * 1e3, 1), budget_min=int(out.budget.min()), budget_max=int(out.budget.max()),
+                         status_or=int(out.status.max())))
+        g.destroy()
+    print(json.dumps({"styles": "per-kernel times of the round on degenerate inputs", "shape": w0.name,
+                      "rounds_timed": args.steps, "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -744,10 +787,16 @@ def main():
                     help="instead of the benchmark: time the TDES training objective (forward + backward)")
     ap.add_argument("--saba-fit", action="store_true",
                     help="instead of the benchmark: time the least-squares fit of the SABA models")
+    ap.add_argument("--styles", action="store_true",
+                    help="instead of the benchmark: the round's kernels timed on degenerate inputs (own JSON line)")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the benchmark: fixed-budget / beta sweeps on synthetic acceptance (own JSON line)")
     ap.add_argument("--sweep-fixed-budget", type=int, default=256, help="the fixed budget of the DDTree-style arms")
     args = ap.parse_args()
+    if args.styles and args.impl == "graft":
+        args.steps = 20 if args.steps is None else args.steps
+        run_styles(args)
+        return
     if args.sweep and args.impl == "graft":
         if "--workload" not in sys.argv:
             args.workload = "C5"

@@ -267,6 +267,39 @@ def saba_replay_logs(n: int, seed: int, phi=(-160.0, 20.0, -5.0, 200.0), c=(6.0,
                 prefix_len=prefix, latency=lat.astype(np.float32))
 
 
+STYLES = ("normal", "quant1", "quant025", "flat", "peaked", "mixed", "huge", "masked", "twopeaks", "ramp")
+
+
+def styled_logits(z, style, rng, gen, K):
+    """Logits of one of ten shapes, from ordinary to degenerate (z: fp32 [batch, L, V] drawn by graft_inputs)."""
+    Bt, L, V = z.shape
+    if style == "quant1":
+        return torch.round(z)
+    if style == "quant025":
+        return torch.round(z * 4) / 4
+    if style == "flat":
+        return 1e-3 * torch.randn(z.shape, generator=gen)
+    if style == "peaked":       # one token of probability 1 to fp32 precision
+        out = torch.zeros_like(z)
+        return out.scatter_(2, torch.randint(0, V, (Bt, L), generator=gen)[..., None], 30.0)
+    if style == "twopeaks":     # two equal winners (or one, where the draws coincide)
+        out = torch.zeros_like(z)
+        out.scatter_(2, torch.randint(0, V, (Bt, L), generator=gen)[..., None], 20.0)
+        return out.scatter_(2, torch.randint(0, V, (Bt, L), generator=gen)[..., None], 20.0)
+    if style == "mixed":
+        out = torch.round(z)
+        out[:, ::2] = 0.0
+        return out
+    if style == "huge":         # log-probabilities in the hundreds: one fp32 ulp is above the tolerance
+        return z * float(rng.choice([5.0, 10.0, 30.0]))
+    if style == "masked":       # between one and 2K finite tokens per row
+        keep_n = int(rng.integers(1, max(2, min(V, 2 * K))))
+        return z.masked_fill(torch.rand(z.shape, generator=gen).argsort(dim=2) >= keep_n, float("-inf"))
+    if style == "ramp":
+        return -torch.arange(V, dtype=torch.float32).expand(z.shape).clone() * float(rng.choice([1e-3, 0.1, 1.0]))
+    return z
+
+
 def small(name: str = "T", **kw) -> Workload:
     """A small workload for tests; override any field."""
     base = dict(name=name, batch=2, L=4, V=1000, K=4, hidden_dim=32, logits_dtype="f32", hidden_dtype="f32",
