@@ -104,16 +104,14 @@ __device__ __forceinline__ int cta_of(long long x, long long Q, long long G) {
     return (int)(((x + 1) * G + Q - 1) / Q - 1);
 }
 
+// The piece [qr0, qr1) (in quanta) of row `row`.  No division: segment boundaries are on the streaming warps' path.
 template <bool BF16>
-__device__ __forceinline__ Seg make_seg(const VpParams& p, long long qi, long long qend) {
+__device__ __forceinline__ Seg make_seg(const VpParams& p, int row, int qr0, int qr1) {
     using T = VT<BF16>;
     Seg s;
-    s.row = (int)(qi / p.nq);
-    long long qr0 = qi - (long long)s.row * p.nq;
-    long long qr1 = qr0 + (qend - qi);
-    if (qr1 > p.nq) qr1 = p.nq;
-    s.e0 = (int)(qr0 * kVpQuantum);
-    s.e1 = qr1 == p.nq ? p.V : (int)(qr1 * kVpQuantum);  // the last quantum of a row also takes the remainder
+    s.row = row;
+    s.e0 = qr0 * kVpQuantum;
+    s.e1 = qr1 == (int)p.nq ? p.V : qr1 * kVpQuantum;  // the last quantum of a row also takes the remainder
     const char* a0 = p.logits + ((size_t)s.row * p.V + s.e0) * T::ESZ;
     const char* a1 = p.logits + ((size_t)s.row * p.V + s.e1) * T::ESZ;
     uintptr_t b0 = ((uintptr_t)a0 + 15) & ~(uintptr_t)15;
@@ -129,45 +127,47 @@ __device__ __forceinline__ Seg make_seg(const VpParams& p, long long qi, long lo
     s.ntiles = (int)((s.body_bytes + TILE - 1) / TILE);
     return s;
 }
-__device__ __forceinline__ int seg_quanta(const Seg& s) {
-    const int n = (s.e1 - s.e0) / kVpQuantum;  // a row's last quantum holds up to 2 * kVpQuantum - 1 elements
-    return n < 1 ? 1 : n;
-}
-
 
 // A CTA's share of the stream as a list of segments.  The share's last segment (usually a partial row that is
 // shared with the next CTA) is visited FIRST, so that the cross-CTA merge of shared rows happens early instead
-// of at the kernel's tail; the remaining segments follow in stream order.
+// of at the kernel's tail; the remaining segments follow in stream order.  Two divisions when the walk begins, none
+// per segment.
 struct SegIter {
-    long long q0, q1, qi, q_last;  // q_last: first quantum of the share's last segment
-    int state;                     // 0: emit the last segment, 1: walk [q0, q_last)
+    int r_first, r_last;  // rows of the share's first and last quantum
+    int qr_first;         // where the share begins within r_first
+    int qr_last0, qr_last1;  // the last segment's piece of r_last
+    int row;              // next row of the walk over [r_first, r_last)
+    int state;            // 0: emit the last segment, 1: walk, 2: nothing at all
+    bool whole_last;      // the last segment is the only one (it starts where the share starts)
 };
 template <bool BF16>
 __device__ __forceinline__ SegIter seg_iter_begin(const VpParams& p, long long q0, long long q1) {
     SegIter it;
-    it.q0 = q0;
-    it.q1 = q1;
-    it.qi = q0;
-    // the last segment starts at the last row boundary inside the share (or at q0)
-    const long long r_last = (q1 - 1) / p.nq;
-    const long long b = r_last * p.nq;
-    it.q_last = b > q0 ? b : q0;
-    it.state = 0;
+    it.state = q0 < q1 ? 0 : 2;
+    it.r_first = (int)(q0 / p.nq);
+    it.qr_first = (int)(q0 - (long long)it.r_first * p.nq);
+    it.r_last = (int)((q1 - 1) / p.nq);
+    // the last segment starts at the last row boundary inside the share (or where the share starts)
+    it.whole_last = it.r_last == it.r_first;
+    it.qr_last0 = it.whole_last ? it.qr_first : 0;
+    it.qr_last1 = (int)(q1 - (long long)it.r_last * p.nq);
+    it.row = it.r_first;
     return it;
 }
 template <bool BF16>
 __device__ __forceinline__ bool seg_iter_next(const VpParams& p, SegIter& it, Seg& sg) {
-    if (it.q0 >= it.q1) return false;
     if (it.state == 0) {
-        sg = make_seg<BF16>(p, it.q_last, it.q1);
+        sg = make_seg<BF16>(p, it.r_last, it.qr_last0, it.qr_last1);
         it.state = 1;
         return true;
     }
-    if (it.qi >= it.q_last) return false;
-    sg = make_seg<BF16>(p, it.qi, it.q_last);
-    it.qi += seg_quanta(sg);
+    if (it.state == 2 || it.row >= it.r_last) return false;
+    sg = make_seg<BF16>(p, it.row, it.row == it.r_first ? it.qr_first : 0, (int)p.nq);
+    ++it.row;
     return true;
 }
+// After seg_iter_next returned a segment: is it the one this CTA visits last?
+__device__ __forceinline__ bool seg_iter_at_end(const SegIter& it) { return it.row >= it.r_last; }
 
 __device__ __forceinline__ float load_elem_f32(const char* p, bool bf16) {
     if (bf16) return __uint_as_float(((uint32_t) * (const uint16_t*)p) << 16);
@@ -175,32 +175,6 @@ __device__ __forceinline__ float load_elem_f32(const char* p, bool bf16) {
 }
 
 // ---- per-thread streaming state -----------------------------------------------------------------
-struct Acc {
-    float ref;     // reference exponent, log2 domain; -inf before the first finite value
-    float s;       // sum of 2^(z log2e - ref)
-    uint32_t tmo;  // ord() of the largest value seen; 0 = nothing seen
-};
-
-__device__ __forceinline__ float acc_begin_chunk(Acc& a, float cm) {
-    // Raise the reference only when the chunk maximum exceeds it by more than 2^16: rescaling is then
-    // rare, and every term stays below 2^16.
-    float cms = cm * kLog2e;
-    if (cms > a.ref + 16.0f) {
-        a.s *= ex2_approx(a.ref - cms);
-        a.ref = cms;
-    }
-    return (a.ref == -INFINITY) ? 0.0f : -a.ref;
-}
-
-// (c, s) pairs stand for s * 2^c; merge two of them
-__device__ __forceinline__ void merge_cs(float& c, float& s, float c2, float s2) {
-    const float cn = fmaxf(c, c2);
-    const float f1 = (c == -INFINITY) ? 0.f : ex2_approx(c - cn);
-    const float f2 = (c2 == -INFINITY) ? 0.f : ex2_approx(c2 - cn);
-    s = s * f1 + s2 * f2;
-    c = cn;
-}
-
 #if GRAFT_VP_F32X2
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
     uint64_t r;
@@ -220,13 +194,78 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
 }
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
 #endif
 
+// The running log-sum-exp of one streaming thread over a segment: sum of 2^(z log2e - ref) in four fp32
+// accumulators (two packed pairs), a reference exponent that is raised lazily (only when a chunk's maximum exceeds
+// it by more than 2^16, so that rescaling is rare and every term stays far from overflow), and the largest value.
+struct Acc {
+    float ref;      // reference exponent, log2 domain; -inf before the first finite value
+    float nref;     // -ref (0 while ref is -inf): the addend of the fused multiply-add
+    uint32_t thr;   // a chunk maximum above this value raises the reference: bf16 logits: the value in both halves
+                    // of a packed pair; fp32 logits: float bits
+    uint32_t rmax;  // largest value so far: bf16 logits: a packed pair of running maxima; fp32 logits: float bits
+#if GRAFT_VP_F32X2
+    uint64_t a0, a1;
+#else
+    float s0, s1, s2, s3;
+#endif
+};
+
+template <bool BF16>
+__device__ __forceinline__ void acc_init(Acc& a) {
+    a.ref = -INFINITY;
+    a.nref = 0.f;
+    a.thr = BF16 ? 0xFF80FF80u : 0xFF800000u;  // -inf: the first finite value sets the reference
+    a.rmax = a.thr;
+#if GRAFT_VP_F32X2
+    a.a0 = a.a1 = 0ull;
+#else
+    a.s0 = a.s1 = a.s2 = a.s3 = 0.f;
+#endif
+}
+
+// The chunk maximum cm exceeded the threshold: raise the reference to cm (rare).
+template <bool BF16>
+__device__ __forceinline__ void acc_raise(Acc& a, float cm) {
+    const float cms = cm * kLog2e;
+    if (!(cms > a.ref + 16.0f)) return;  // (the threshold is a truncated copy of ref + 16: it may fire a little early)
+    const float f = ex2_approx(a.ref - cms);  // 0 when ref is -inf (nothing added yet) or cm is +inf
+#if GRAFT_VP_F32X2
+    const uint64_t f2 = pack2(f, f);
+    a.a0 = mul2(a.a0, f2);
+    a.a1 = mul2(a.a1, f2);
+#else
+    a.s0 *= f;
+    a.s1 *= f;
+    a.s2 *= f;
+    a.s3 *= f;
+#endif
+    a.ref = cms;
+    a.nref = -cms;
+    // values above (ref + 16) / log2e raise the reference again; the bound need not be exact (terms overflow only
+    // 2^111 above it), so it is kept as its leading 16 bits for the packed comparison of bf16 chunks
+    const uint32_t zb = __float_as_uint((cms + 16.0f) * 0.6931471805599453f);
+    a.thr = BF16 ? ((zb >> 16) | (zb & 0xFFFF0000u)) : zb;
+}
+
+__device__ __forceinline__ float pair_max_bf16(uint32_t pm) {  // the larger half of a packed bf16 pair, as fp32
+    return fmaxf(__uint_as_float(pm << 16), __uint_as_float(pm & 0xFFFF0000u));
+}
+
+// One chunk of a streaming lane: four 16-byte vectors of a tile (32 bf16 or 16 fp32 logits).  The chunk maximum goes
+// to *cmax_slot for the second stage (2 bytes: the bf16 value, or the fp32 maximum rounded up to bf16).
 template <bool BF16, bool GUARD>
 __device__ __forceinline__ void process_chunk(const uint4* __restrict__ wb, int lane, int nvalid_vec, Acc& a,
                                               typename VT<BF16>::cm_t* cmax_slot) {
     using T = VT<BF16>;
     uint4 v[VEC_PER_LANE];
+    uint32_t vm[VEC_PER_LANE];
 #pragma unroll
     for (int i = 0; i < VEC_PER_LANE; ++i) {
         if (!GUARD || (i * 32 + lane) < nvalid_vec)
@@ -234,35 +273,39 @@ __device__ __forceinline__ void process_chunk(const uint4* __restrict__ wb, int 
         else
             v[i] = make_uint4(T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD);
     }
-    float cm;
+    uint32_t cmk;
     if (BF16) {
-        uint32_t m0 = hmax2_bf16(hmax2_bf16(v[0].x, v[0].y), hmax2_bf16(v[0].z, v[0].w));
-        uint32_t m1 = hmax2_bf16(hmax2_bf16(v[1].x, v[1].y), hmax2_bf16(v[1].z, v[1].w));
-        uint32_t m2 = hmax2_bf16(hmax2_bf16(v[2].x, v[2].y), hmax2_bf16(v[2].z, v[2].w));
-        uint32_t m3 = hmax2_bf16(hmax2_bf16(v[3].x, v[3].y), hmax2_bf16(v[3].z, v[3].w));
-        uint32_t pm = hmax2_bf16(hmax2_bf16(m0, m1), hmax2_bf16(m2, m3));
-        cm = fmaxf(__uint_as_float(pm << 16), __uint_as_float(pm & 0xFFFF0000u));
-        *cmax_slot = (typename T::cm_t)(__float_as_uint(cm) >> 16);
+#pragma unroll
+        for (int i = 0; i < VEC_PER_LANE; ++i) vm[i] = hmax2_bf16(hmax2_bf16(v[i].x, v[i].y), hmax2_bf16(v[i].z, v[i].w));
+        cmk = hmax2_bf16(hmax2_bf16(vm[0], vm[1]), hmax2_bf16(vm[2], vm[3]));
+        a.rmax = hmax2_bf16(a.rmax, cmk);
+        {
+            // the larger half of the pair, as 16 bits: the halves swapped (one byte permute), one more packed maximum
+            uint32_t sw;
+            asm("prmt.b32 %0, %1, %1, 0x1032;" : "=r"(sw) : "r"(cmk));
+            *cmax_slot = (typename T::cm_t)(hmax2_bf16(cmk, sw) & 0xFFFFu);
+        }
+        if (hmax2_bf16(cmk, a.thr) != a.thr) acc_raise<BF16>(a, pair_max_bf16(cmk));  // some half above the threshold
     } else {
         float m = -INFINITY;
 #pragma unroll
         for (int i = 0; i < VEC_PER_LANE; ++i) {
-            m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(v[i].x), __uint_as_float(v[i].y)),
-                               fmaxf(__uint_as_float(v[i].z), __uint_as_float(v[i].w))));
+            const float mi = fmaxf(fmaxf(__uint_as_float(v[i].x), __uint_as_float(v[i].y)),
+                                   fmaxf(__uint_as_float(v[i].z), __uint_as_float(v[i].w)));
+            vm[i] = __float_as_uint(mi);
+            m = fmaxf(m, mi);
         }
-        cm = m;
+        cmk = __float_as_uint(m);
+        a.rmax = __float_as_uint(fmaxf(__uint_as_float(a.rmax), m));
         {
             // round toward +inf onto the bf16 grid: positive values round their magnitude up, negative ones truncate
-            const uint32_t mb = __float_as_uint(cm);
+            const uint32_t mb = cmk;
             *cmax_slot = (typename T::cm_t)((mb >> 31) ? (mb >> 16) : ((mb + 0xFFFFu) >> 16));
         }
+        if (m > __uint_as_float(a.thr)) acc_raise<BF16>(a, m);
     }
-    uint32_t o = ord_from_float(cm);
-    a.tmo = o > a.tmo ? o : a.tmo;
-    const float nref = acc_begin_chunk(a, cm);
 #if GRAFT_VP_F32X2
-    const uint64_t c2 = pack2(kLog2e, kLog2e), r2 = pack2(nref, nref);
-    uint64_t acc0 = 0ull, acc1 = 0ull;  // two (+0, +0) pairs
+    const uint64_t c2 = pack2(kLog2e, kLog2e), r2 = pack2(a.nref, a.nref);
 #pragma unroll
     for (int i = 0; i < VEC_PER_LANE; ++i) {
         const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
@@ -274,50 +317,66 @@ __device__ __forceinline__ void process_chunk(const uint4* __restrict__ wb, int 
                 unpack2(fma2(x2, c2, r2), t0, t1);
                 const uint64_t e2 = pack2(ex2_approx(t0), ex2_approx(t1));
                 if (k & 1)
-                    acc1 = add2(acc1, e2);
+                    a.a1 = add2(a.a1, e2);
                 else
-                    acc0 = add2(acc0, e2);
+                    a.a0 = add2(a.a0, e2);
             }
         } else {
             float t0, t1, t2, t3;
             unpack2(fma2(pack2(__uint_as_float(w[0]), __uint_as_float(w[1])), c2, r2), t0, t1);
             unpack2(fma2(pack2(__uint_as_float(w[2]), __uint_as_float(w[3])), c2, r2), t2, t3);
-            acc0 = add2(acc0, pack2(ex2_approx(t0), ex2_approx(t1)));
-            acc1 = add2(acc1, pack2(ex2_approx(t2), ex2_approx(t3)));
+            a.a0 = add2(a.a0, pack2(ex2_approx(t0), ex2_approx(t1)));
+            a.a1 = add2(a.a1, pack2(ex2_approx(t2), ex2_approx(t3)));
         }
     }
-    float s0, s1, s2, s3;
-    unpack2(acc0, s0, s1);
-    unpack2(acc1, s2, s3);
-    a.s += (s0 + s1) + (s2 + s3);
 #else
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
     for (int i = 0; i < VEC_PER_LANE; ++i) {
         const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
         if (BF16) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                float lo = __uint_as_float(w[k] << 16), hi = __uint_as_float(w[k] & 0xFFFF0000u);
-                float e0 = ex2_approx(fmaf(lo, kLog2e, nref)), e1 = ex2_approx(fmaf(hi, kLog2e, nref));
+                const float lo = __uint_as_float(w[k] << 16), hi = __uint_as_float(w[k] & 0xFFFF0000u);
+                const float e0 = ex2_approx(fmaf(lo, kLog2e, a.nref)), e1 = ex2_approx(fmaf(hi, kLog2e, a.nref));
                 if (k & 1) {
-                    s2 += e0;
-                    s3 += e1;
+                    a.s2 += e0;
+                    a.s3 += e1;
                 } else {
-                    s0 += e0;
-                    s1 += e1;
+                    a.s0 += e0;
+                    a.s1 += e1;
                 }
             }
         } else {
-            s0 += ex2_approx(fmaf(__uint_as_float(w[0]), kLog2e, nref));
-            s1 += ex2_approx(fmaf(__uint_as_float(w[1]), kLog2e, nref));
-            s2 += ex2_approx(fmaf(__uint_as_float(w[2]), kLog2e, nref));
-            s3 += ex2_approx(fmaf(__uint_as_float(w[3]), kLog2e, nref));
+            a.s0 += ex2_approx(fmaf(__uint_as_float(w[0]), kLog2e, a.nref));
+            a.s1 += ex2_approx(fmaf(__uint_as_float(w[1]), kLog2e, a.nref));
+            a.s2 += ex2_approx(fmaf(__uint_as_float(w[2]), kLog2e, a.nref));
+            a.s3 += ex2_approx(fmaf(__uint_as_float(w[3]), kLog2e, a.nref));
         }
     }
-    a.s += (s0 + s1) + (s2 + s3);
 #endif
 }
+
+template <bool BF16>
+__device__ __forceinline__ float acc_sum(const Acc& a) {
+#if GRAFT_VP_F32X2
+    float s0, s1, s2, s3;
+    unpack2(a.a0, s0, s1);
+    unpack2(a.a1, s2, s3);
+    return (s0 + s1) + (s2 + s3);
+#else
+    return (a.s0 + a.s1) + (a.s2 + a.s3);
+#endif
+}
+
+// (c, s) pairs stand for s * 2^c; merge two of them
+__device__ __forceinline__ void merge_cs(float& c, float& s, float c2, float s2) {
+    const float cn = fmaxf(c, c2);
+    const float f1 = (c == -INFINITY) ? 0.f : ex2_approx(c - cn);
+    const float f2 = (c2 == -INFINITY) ? 0.f : ex2_approx(c2 - cn);
+    s = s * f1 + s2 * f2;
+    c = cn;
+}
+
 
 // ---- shared-memory control block ---------------------------------------------------------------
 struct __align__(16) EpiShared {  // private to one epilogue group
@@ -529,7 +588,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             while (seg_iter_next<BF16>(p, it, sg)) {
                 // the segment this CTA visits last is read the ordinary way instead of evict-first: the second
                 // stage of its epilogue, which nothing overlaps any more, then finds its chunks in L2
-                const bool hint = p.use_hint && !(it.qi >= it.q_last);
+                const bool hint = p.use_hint && !seg_iter_at_end(it);
                 for (int tile = 0; tile < sg.ntiles; ++tile, ++t) {
                     if (t >= nst) mbar_wait_bounded_hint(empty0 + 8 * st, ph, &sh->abort_flag, kVpIdleHintNs);
 #ifdef GRAFT_TEST_WITHHOLD_TILE
@@ -577,9 +636,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
         for (; seg_iter_next<BF16>(p, it, sg); ++k) {
             const uint32_t pb = k % kVpBufs;
             Acc a;
-            a.ref = -INFINITY;
-            a.s = 0.f;
-            a.tmo = 0u;
+            acc_init<BF16>(a);
             // buffer pb is free once the epilogue of segment k - kVpBufs is done
             if (k >= kVpBufs) mbar_wait_bounded(done0 + 8 * pb, ((k / kVpBufs) - 1u) & 1u, &sh->abort_flag);
             {
@@ -604,16 +661,19 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 }
             }
             // hand the segment over to the epilogue warp
-            sh->tmax[pb][tid] = a.tmo;
-            atomicMax(&sh->gmax[pb][(warp & 1) * 32 + lane], a.tmo);
+            // (a thread that saw no data keeps 0 = nothing seen)
+            const uint32_t tmo = sg.ntiles > 0 ? ord_from_float(BF16 ? pair_max_bf16(a.rmax) : __uint_as_float(a.rmax)) : 0u;
+            sh->tmax[pb][tid] = tmo;
+            atomicMax(&sh->gmax[pb][(warp & 1) * 32 + lane], tmo);
             {
-                float c = a.ref, s = a.s;
+                // the warp's piece of the log-sum-exp: the largest reference of its lanes (one integer reduction over
+                // the order-preserving images), every lane's sum rescaled to it once, then a butterfly of plain adds
+                // (a fixed order: the result does not depend on timing)
+                const uint32_t co = __reduce_max_sync(0xFFFFFFFFu, ord_from_float(a.ref));
+                const float c = __uint_as_float(bits_from_ord(co));
+                float s = (a.ref == -INFINITY) ? 0.f : acc_sum<BF16>(a) * ex2_approx(a.ref - c);
 #pragma unroll
-                for (int d = 16; d > 0; d >>= 1) {
-                    const float c2 = __shfl_xor_sync(0xFFFFFFFFu, c, d);
-                    const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, d);
-                    merge_cs(c, s, c2, s2);
-                }
+                for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
                 if (lane == 0) {
                     sh->wc[pb][warp] = c;
                     sh->ws[pb][warp] = s;
@@ -866,8 +926,11 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             __syncwarp();
             if (lane == 0) mbar_arrive(done0 + 8 * pb);
             // (g) finish the row, or leave a record for the CTA that arrives last
+            // (a whole row is nobody else's: the divisions that find a shared row's CTAs are for partial rows only)
+            const bool whole_row = sg.e0 == 0 && sg.e1 == p.V;
             const long long x0 = (long long)sg.row * p.nq;
-            const int c_first = cta_of(x0, p.Q, G), c_last = cta_of(x0 + p.nq - 1, p.Q, G);
+            const int c_first = whole_row ? (int)blockIdx.x : cta_of(x0, p.Q, G);
+            const int c_last = whole_row ? (int)blockIdx.x : cta_of(x0 + p.nq - 1, p.Q, G);
             const int nseg = c_last - c_first + 1;
             double Cd = (double)c, Sd = (double)s;
             uint32_t Vm = vmo;
