@@ -399,8 +399,9 @@ __device__ uint32_t cta_select_bucket(const TreeSmem& sm, const uint32_t* keys, 
 // The exact B-th largest key once its bucket is known: the keys inside it are few (path scores are spread over
 // many more values than there are buckets), so they are collected and ranked against each other directly; if there
 // are more than the list holds (heavy ties), a full radix select runs instead.
+// *n_reach: how many of all the keys reach the value returned (kth if no other key ties with it), or -1 if unknown.
 __device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, int lo_i, int hi_i, int kth, float top,
-                                      const SelBucket& st, int tid) {
+                                      const SelBucket& st, int tid, int* n_reach) {
     constexpr int kCap = 512;
     uint32_t* list = sm.hist;           // [kCap] (the histogram space is idle between selects)
     int* cnt = (int*)(sm.hist + 1100);  // [1]
@@ -418,6 +419,7 @@ __device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, 
     if (n > kCap) {  // (uniform)
         __syncthreads();
         int rem = 0;
+        *n_reach = -1;
         return cta_kth_largest(sm, keys, lo_i, hi_i, kth, 0, 4, 0u, rem, tid);
     }
     const int remaining = st.rem;
@@ -429,10 +431,14 @@ __device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, 
             gt += o > k ? 1 : 0;
             ge += o >= k ? 1 : 0;
         }
-        if (gt < remaining && remaining <= ge) sm.scal[6] = (int)k;  // (every writer writes the same value)
+        if (gt < remaining && remaining <= ge) {  // (every writer writes the same values)
+            sm.scal[6] = (int)k;
+            sm.scal[7] = kth - remaining + ge;  // the keys above the bucket, and those of the bucket that reach k
+        }
     }
     __syncthreads();
     const uint32_t v = (uint32_t)sm.scal[6];
+    *n_reach = sm.scal[7];
     __syncthreads();  // the list and the result word are free again
     return v;
 }
@@ -671,6 +677,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     // ordered: the parallel phase selected the whole tree, and its nodes stand in level order already (no sequential
     // tail, no placement): true unless several keys tie with the B-th largest or the node table overflowed
     bool ordered = false;
+    int n_reach = -1;  // keys that reach the final theta, if the search that found it counted them
     uint32_t theta = 0u;
     if (budget > 0) {
         int ntot = 1, n_at_select = 1;
@@ -849,7 +856,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 sel_top = 0.0f + sm.es[0];  // the root's best child
                 cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);
             }
-            theta = cta_finish_select(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);
+            theta = cta_finish_select(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid, &n_reach);
         }
         __syncthreads();
         if (table_ok) {
@@ -860,14 +867,17 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             // when it holds fewer than B nodes (theta = 0: every prefix there is has been appended).
             uint32_t cut = theta;  // nodes with key > cut are taken here
             if (theta != 0u) {
-                int ge = 0;
-                for (int i = i0 > 1 ? i0 : 1; i < i1; ++i) ge += sm.nkey[i] >= theta ? 1 : 0;
-                ge = __reduce_add_sync(0xFFFFFFFFu, ge);
-                if (tid == 0) sm.scal[8] = 0;
-                __syncthreads();
-                if (lane == 0 && ge) atomicAdd(&sm.scal[8], ge);
-                __syncthreads();
-                if (sm.scal[8] == budget) {  // (uniform)
+                if (n_reach < 0) {  // (uniform) the radix search does not count them: one pass over the table
+                    int ge = 0;
+                    for (int i = i0 > 1 ? i0 : 1; i < i1; ++i) ge += sm.nkey[i] >= theta ? 1 : 0;
+                    ge = __reduce_add_sync(0xFFFFFFFFu, ge);
+                    if (tid == 0) sm.scal[8] = 0;
+                    __syncthreads();
+                    if (lane == 0 && ge) atomicAdd(&sm.scal[8], ge);
+                    __syncthreads();
+                    n_reach = sm.scal[8];
+                }
+                if (n_reach == budget) {  // (uniform)
                     cut = theta - 1u;
                     ordered = true;
                 }
