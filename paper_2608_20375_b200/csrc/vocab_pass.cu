@@ -268,8 +268,13 @@ __device__ __forceinline__ void process_chunk(const uint4* __restrict__ wb, int 
     uint32_t vm[VEC_PER_LANE];
 #pragma unroll
     for (int i = 0; i < VEC_PER_LANE; ++i) {
-        if (!GUARD || (i * 32 + lane) < nvalid_vec)
-            v[i] = wb[i * 32 + lane];
+        // A lane's chunk is 64 contiguous bytes (vectors 4 lane .. 4 lane + 3 of the warp's block), so that the second
+        // stage re-reads a hit chunk as one 64-byte piece of one line instead of four sectors of four lines (random
+        // DRAM accesses beside the stream cost it bandwidth).  The lanes take their four vectors in rotated order,
+        // (i + lane / 2) mod 4, which spreads the eight lanes of a shared-memory phase over all bank groups.
+        const int vi = 4 * lane + ((i + (lane >> 1)) & 3);
+        if (!GUARD || vi < nvalid_vec)
+            v[i] = wb[vi];
         else
             v[i] = make_uint4(T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD);
     }
@@ -474,14 +479,14 @@ __device__ int warp_fallback_select(EpiShared* sh, const VpParams& p, const Seg&
     const int nvec = (int)(sg.body_bytes / 16);
     const uint4* body = (const uint4*)sg.body;
     for (int v0 = 0; v0 < nvec; v0 += 32 * U) {
-        // The batch is one streaming warp's 2 KiB of a tile, and this lane's four vectors are the chunk whose
+        // The batch is one streaming warp's 2 KiB of a tile, and this lane's four consecutive vectors are the chunk whose
         // maximum (rounded up to bf16) that warp's lane left in cmx.  A chunk cannot hold a key above the filter if
         // its maximum is below the filter's value, or not above it while all its ids come after the filter's id.
         if (thr != 0ull) {
             const int tile = v0 / (TILE / 16), wb = (v0 % (TILE / 16)) / (32 * U);
             const uint32_t mx = ord_from_bits((uint32_t)cmx[(size_t)(wb * 32 + lane) * p.max_tiles + tile] << 16);
             const uint32_t v_thr = (uint32_t)(thr >> 32);
-            const uint32_t first_id = (uint32_t)(sg.e_body0 + (v0 + lane) * T::EPV);
+            const uint32_t first_id = (uint32_t)(sg.e_body0 + (v0 + 4 * lane) * T::EPV);
             const bool need = !(mx < v_thr || (mx <= v_thr && first_id > key_id(thr)));
             if (!__any_sync(0xFFFFFFFFu, need)) continue;  // (uniform)
         }
@@ -824,7 +829,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     if (ord_from_bits(bits) >= Tv) {
                         const int pos = atomicAdd(&es->nhits, 1);
                         if (pos >= kVpHitCap) break;  // too many: the exact selection over the segment takes over
-                        es->hits[pos] = (uint32_t)tile * TILE + (t >> 5) * WBLK + (t & 31) * 16;
+                        es->hits[pos] = (uint32_t)tile * TILE + (t >> 5) * WBLK + (t & 31) * 64;
                     }
                 }
             }
@@ -850,7 +855,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                         vv[u] = make_uint4(T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD, T::NEG_INF_WORD);
                         offs[u] = 0xFFFFFFFFu;
                         if (i < nvec) {
-                            const uint32_t off = es->hits[i / VEC_PER_LANE] + (uint32_t)(i % VEC_PER_LANE) * 512u;
+                            const uint32_t off = es->hits[i / VEC_PER_LANE] + (uint32_t)(i % VEC_PER_LANE) * 16u;
                             if (off < sg.body_bytes) {
                                 offs[u] = off;
                                 vv[u] = *(const uint4*)(sg.body + off);
