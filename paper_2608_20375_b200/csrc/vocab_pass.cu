@@ -437,6 +437,14 @@ __device__ void warp_select_topk(EpiShared* sh, int n, int K, int lane) {
     __syncwarp();
 }
 
+// ord() of the largest element of a 16-byte vector
+template <bool BF16>
+__device__ __forceinline__ uint32_t vec_max_ord(const uint4& x) {
+    if (BF16) return ord_from_float(pair_max_bf16(hmax2_bf16(hmax2_bf16(x.x, x.y), hmax2_bf16(x.z, x.w))));
+    return ord_from_float(fmaxf(fmaxf(__uint_as_float(x.x), __uint_as_float(x.y)),
+                                fmaxf(__uint_as_float(x.z), __uint_as_float(x.w))));
+}
+
 // Exact selection over a whole segment straight from global memory.  Used only when the fast path's buffers
 // overflowed, which means that most of the segment ties with its K-th largest element (rows that are flat, masked
 // to -inf, or all but one element equal).  The running K-th best key is the filter: an element enters the buffer
@@ -865,6 +873,8 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
 #pragma unroll
                     for (int u = 0; u < RU; ++u) {
                         if (offs[u] == 0xFFFFFFFFu) continue;
+                        // (three of a hit chunk's four vectors hold nothing that reaches T: one test for the vector)
+                        if (vec_max_ord<BF16>(vv[u]) < Tv) continue;
                         const uint32_t wv[4] = {vv[u].x, vv[u].y, vv[u].z, vv[u].w};
 #pragma unroll
                         for (int j = 0; j < T::EPV; ++j) {
