@@ -212,6 +212,9 @@ def run_graft(args):
 
     # per-kernel CUDA events (recorded by the library on the launching stream around each of its kernels) are taken
     # on every TIMING_EVERY-th step of the timed region: four event records cost the stream a few microseconds
+    # (a round with its four event records takes about 16 us longer than one without: in a long run every
+    # steps/32-th round carries them, which still gives 32 samples and keeps their cost under 1 % of ms_per_step)
+    timing_every = max(args.timing_every, args.steps // MIN_KERNEL_SAMPLES)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     torch.cuda.synchronize()
@@ -219,7 +222,7 @@ def run_graft(args):
     t_wall0 = time.perf_counter()
     ev0.record()
     for i in range(args.steps):
-        timed = (i % args.timing_every) == 0
+        timed = (i % timing_every) == 0
         if timed:
             g.set_timing(1 if i == 0 else 2)  # 1 = reset the call count, 2 = go on counting
         if args.cuda_graph:
@@ -237,7 +240,9 @@ def run_graft(args):
     # sampler's window takes them in
     n_t = g.read_timing()[0]
     extra = 0
-    while n_t + extra < MIN_KERNEL_SAMPLES:
+    evx0, evx1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    evx0.record()
+    while n_t + extra < MIN_KERNEL_SAMPLES or extra < 8:
         g.set_timing(2 if (n_t + extra) > 0 else 1)
         if args.cuda_graph:
             step(extra, True)
@@ -245,7 +250,11 @@ def run_graft(args):
             step(extra)
         g.set_timing(False)
         extra += 1
+    evx1.record()
     torch.cuda.synchronize()
+    # a round that carries the per-kernel event records: longer than an ordinary one (the records cost time and keep a
+    # kernel from setting up while the one ahead of it drains); the per-kernel intervals add up to this, not to ms_per_step
+    instrumented_round_ms = evx0.elapsed_time(evx1) / extra
     # ... and a short run leaves the clock sampler (a reading every few milliseconds) nothing to read: the same rounds
     # go on, untimed, until the window under load holds a handful of readings
     i_more = 0
@@ -340,7 +349,8 @@ def run_graft(args):
                    "l2_policy": f"{n_buf} rotating input sets of {logits_bytes / 1e6:.0f} MB each (> L2 of 126 MB)"},
         "gpu_launches": launches,
         "kernel_ms": {"vocab_pass": vocab_ms / max(1, n_t), "tdes_edges": tdes_ms / max(1, n_t),
-                      "tree": tree_ms / max(1, n_t), "calls_averaged": n_t, "empty_event_pair": event_pair_ms},
+                      "tree": tree_ms / max(1, n_t), "calls_averaged": n_t, "empty_event_pair": event_pair_ms,
+                      "round_with_these_events": instrumented_round_ms},
         "roofline": {"bound": "hbm", "kernel": "vocab_pass_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8000": achieved / 8000.0, "algorithmic_bytes": algo_bytes,
@@ -776,7 +786,7 @@ def main():
     ap.add_argument("--impl", default="graft", choices=["graft", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--timing-every", type=int, default=8,
-                    help="record the per-kernel events on every n-th timed step")
+                    help="record the per-kernel events on every n-th timed step (at least; steps/32 in a long run)")
     ap.add_argument("--cuda-graph", action="store_true", help="replay captured rounds in the timed loop")
     ap.add_argument("--edge-rows", type=int, default=None,
                     help="depths scored ahead of the expansion (default: the library's)")
