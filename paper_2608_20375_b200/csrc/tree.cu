@@ -256,8 +256,8 @@ __device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, in
 // a level from flooding the node table while few keys are known (sharply peaked rows: every deviation from the
 // best chain costs tens of units, and the B-th largest key of the table stays far down for several levels).
 // Every thread of the CTA calls it; the children number at least kth in all.
-__device__ uint32_t cta_kth_largest_of_children(const TreeSmem& sm, int cnt, uint32_t kx, float sx, int row, int kth,
-                                                int tid) {
+__device__ uint32_t cta_kth_largest_of_children_radix(const TreeSmem& sm, int cnt, uint32_t kx, float sx, int row,
+                                                      int kth, int tid) {
     const int warp = tid >> 5, lane = tid & 31;
     uint32_t prefix = 0u, mask = 0u;
     int remaining = kth;
@@ -320,6 +320,72 @@ __device__ __forceinline__ int select_bin(uint32_t key, float top) {
     const float d = (top - __uint_as_float(bits_from_ord(key))) * kSelBinsPerUnit;
     if (!(d < 1023.0f)) return 1023;  // (also NaN)
     return d > 0.0f ? (int)d : 0;
+}
+
+// A lower bound of the kth largest key among the children that the threads' nodes are about to append (see
+// cta_kth_largest_of_children_radix): one pass over 1024 bins of equal width in score between the current threshold
+// (every child counted reaches it) and the best child, whose lower edge is the bound; the radix passes only if that
+// range is not finite (their top bits crowd into a few counters, which thousands of atomics then queue on; bins in
+// score spread them).
+__device__ uint32_t cta_kth_largest_of_children(const TreeSmem& sm, int cnt, uint32_t kx, float sx, int row, int kth,
+                                                uint32_t theta, int tid) {
+    const int warp = tid >> 5, lane = tid & 31;
+    uint32_t* h = sm.hist;  // [1024 + 32], then [1] the best child key
+    h[tid] = 0u;
+    if (tid < 33) h[1024 + tid] = 0u;
+    __syncthreads();
+    {
+        uint32_t best = 0u;  // a node's first child has its largest key
+        if (cnt > 0) {
+            const uint32_t oc = ord_from_float(sx + sm.es[row]);
+            best = oc < kx ? oc : kx;
+        }
+        best = __reduce_max_sync(0xFFFFFFFFu, best);
+        if (lane == 0 && best) atomicMax(&h[1056], best);
+    }
+    __syncthreads();
+    const float top = __uint_as_float(bits_from_ord(h[1056])), low = __uint_as_float(bits_from_ord(theta));
+    const float scale = 1023.0f / (top - low);
+    if (!(scale > 0.0f) || !(scale < 1e30f)) {  // (uniform) no finite range: -inf scores, or all children equal
+        __syncthreads();
+        return cta_kth_largest_of_children_radix(sm, cnt, kx, sx, row, kth, tid);
+    }
+    for (int r = 0; r < cnt; ++r) {
+        const uint32_t oc = ord_from_float(sx + sm.es[row + r]);
+        const float sc = __uint_as_float(bits_from_ord(oc < kx ? oc : kx));
+        const float df = (top - sc) * scale;
+        const int d = df > 0.0f ? (df < 1023.0f ? (int)df : 1023) : 0;
+        atomicAdd(&h[d + (d >> 5)], 1u);
+    }
+    __syncthreads();
+    if (warp == 0) {  // lane l owns bins 32 l .. 32 l + 31 (bin 0 holds the largest keys)
+        const uint32_t* mine = h + 33 * lane;
+        int sum = 0;
+#pragma unroll 8
+        for (int q = 0; q < 32; ++q) sum += (int)mine[q];
+        int incl = sum;
+#pragma unroll
+        for (int o2 = 1; o2 < 32; o2 <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
+            if (lane >= o2) incl += t;
+        }
+        const int excl = incl - sum;
+        if (excl < kth && kth <= incl) {
+            int acc = excl, bin = 32 * lane;
+            for (int q = 0; q < 32; ++q) {
+                const int c = (int)mine[q];
+                if (acc < kth && kth <= acc + c) bin = 32 * lane + q;
+                acc += c;
+            }
+            sm.scal[6] = bin;
+        }
+    }
+    __syncthreads();
+    const int bin = sm.scal[6];
+    __syncthreads();
+    // the lower edge of the bin, less a hundredth of a bin for the rounding of the bin index; never below theta
+    const uint32_t bound = ord_from_float(top - ((float)(bin + 1) + 0.01f) / scale);
+    return bound > theta ? bound : theta;
 }
 
 // Where the B-th largest key lies and the rank wanted there.
@@ -795,7 +861,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     pre[tid] = __shfl_sync(0xFFFFFFFFu, wincl - wt, warp) + incl;
                     __syncthreads();
                     if (attempt == 0 && total >= budget && (total > flood || cur + total > p.ncap)) {  // (uniform) the search below uses the scan's space: count again
-                        const uint32_t tl = cta_kth_largest_of_children(sm, cnt, kx, sx, row, budget, tid);
+                        const uint32_t tl = cta_kth_largest_of_children(sm, cnt, kx, sx, row, budget, theta, tid);
                         theta = tl > theta ? tl : theta;
                         continue;
                     }
