@@ -26,6 +26,15 @@ __device__ __forceinline__ bool deep_tree_likely(const float* __restrict__ topk_
 }
 
 
+// Where the r-th entry of the sorted row of parent rank c stands inside the row (scores only; the child ranks stand
+// in order): rotated by the parent's rank.  The tree kernel's threads look at the same place r of different parents'
+// rows far more often than at different places of one row, and with K = 32 a row is one pass over the shared-memory
+// banks: unrotated, such a look is a 32-way bank conflict.
+__device__ __forceinline__ int es_col(int r, int c, int K) {
+    const int x = r + c;
+    return x < K ? x : x - K;
+}
+
 // K x K dot products by 8 warps.  Warp ty takes parents ty, ty+8, ty+16, ty+24; lane = (ks, tx): children tx and
 // tx+16, and every second float4 of the m axis starting at ks.  A lane keeps a 4 x 2 tile of running sums, each as
 // a packed fp32 pair (even and odd elements of the m axis; `fma.rn.f32x2`, so 16 packed FMAs per six 16-byte

@@ -84,7 +84,7 @@ struct EdgeParams {
     const float* C;
     const float* u;
     float* edge;      // [batch, L, K, K] by (parent rank, child rank)
-    float* esort;     // same rows, each sorted by (edge descending, child rank ascending)
+    float* esort;     // same rows, each sorted by (edge descending, child rank ascending), stored rotated (es_col)
     uint8_t* eidx;    // child rank of every sorted entry
     int L, K, m, V;
     int rows;     // depths [0, rows) are scored for every sequence: one CTA each
@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(256, 4) tdes_edges_kernel(const EdgeParams p) 
             int par = i / K, c = i % K;
             const float v = (bad || par >= n_par) ? 0.f : lps[c];
             if (WRITE_EDGE) p.edge[row * K * K + i] = v;
-            outs[i] = v;
+            outs[par * K + es_col(c, par, K)] = v;
             outi[i] = (uint8_t)c;
         }
         return;
@@ -191,7 +191,7 @@ __global__ void __launch_bounds__(256, 4) tdes_edges_kernel(const EdgeParams p) 
                         rank);
         if (lane < K) {
             if (WRITE_EDGE) p.edge[(row * K + par) * K + lane] = val;
-            outs[(size_t)par * K + rank] = val;
+            outs[(size_t)par * K + es_col(rank, par, K)] = val;
             outi[(size_t)par * K + rank] = (uint8_t)lane;
         }
     }

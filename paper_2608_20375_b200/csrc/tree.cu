@@ -17,7 +17,7 @@ struct TreeParams {
     const int32_t* row_status;
     const double* cos_pre;  // [batch, L] adjacent-position cosines (Eq. 15), written by the vocab pass
     const int32_t* vp_err;  // word 0: a bounded wait of the vocab pass ran out (sticky)
-    const float* esort;   // [batch, L, K, K] edge rows sorted by (edge desc, child rank asc)
+    const float* esort;   // [batch, L, K, K] edge rows sorted by (edge desc, child rank asc), each rotated by its parent rank (es_col)
     const uint8_t* eidx;  // child rank of each sorted entry
     const int32_t* root_token;
     const float* hist;
@@ -257,7 +257,7 @@ __device__ uint32_t cta_kth_largest(const TreeSmem& sm, const uint32_t* keys, in
 // best chain costs tens of units, and the B-th largest key of the table stays far down for several levels).
 // Every thread of the CTA calls it; the children number at least kth in all.
 __device__ uint32_t cta_kth_largest_of_children_radix(const TreeSmem& sm, int cnt, uint32_t kx, float sx, int row,
-                                                      int kth, int tid) {
+                                                      int cx, int K, int kth, int tid) {
     const int warp = tid >> 5, lane = tid & 31;
     uint32_t prefix = 0u, mask = 0u;
     int remaining = kth;
@@ -267,7 +267,7 @@ __device__ uint32_t cta_kth_largest_of_children_radix(const TreeSmem& sm, int cn
         const int shift = 24 - 8 * pass;
         uint32_t* h = sm.hist + (pass & 1) * 1024 + (warp & 3) * 256;
         for (int r = 0; r < cnt; ++r) {
-            const uint32_t oc = ord_from_float(sx + sm.es[row + r]);
+            const uint32_t oc = ord_from_float(sx + sm.es[row + es_col(r, cx, K)]);
             const uint32_t k = oc < kx ? oc : kx;
             if ((k & mask) == prefix) atomicAdd(&h[(k >> shift) & 255u], 1u);
         }
@@ -327,8 +327,8 @@ __device__ __forceinline__ int select_bin(uint32_t key, float top) {
 // (every child counted reaches it) and the best child, whose lower edge is the bound; the radix passes only if that
 // range is not finite (their top bits crowd into a few counters, which thousands of atomics then queue on; bins in
 // score spread them).
-__device__ uint32_t cta_kth_largest_of_children(const TreeSmem& sm, int cnt, uint32_t kx, float sx, int row, int kth,
-                                                uint32_t theta, int tid) {
+__device__ uint32_t cta_kth_largest_of_children(const TreeSmem& sm, int cnt, uint32_t kx, float sx, int row, int cx,
+                                                int K, int kth, uint32_t theta, int tid) {
     const int warp = tid >> 5, lane = tid & 31;
     uint32_t* h = sm.hist;  // [1024 + 32], then [1] the best child key
     h[tid] = 0u;
@@ -337,7 +337,7 @@ __device__ uint32_t cta_kth_largest_of_children(const TreeSmem& sm, int cnt, uin
     {
         uint32_t best = 0u;  // a node's first child has its largest key
         if (cnt > 0) {
-            const uint32_t oc = ord_from_float(sx + sm.es[row]);
+            const uint32_t oc = ord_from_float(sx + sm.es[row + cx]);  // (entry 0 stands at column cx)
             best = oc < kx ? oc : kx;
         }
         best = __reduce_max_sync(0xFFFFFFFFu, best);
@@ -348,10 +348,10 @@ __device__ uint32_t cta_kth_largest_of_children(const TreeSmem& sm, int cnt, uin
     const float scale = 1023.0f / (top - low);
     if (!(scale > 0.0f) || !(scale < 1e30f)) {  // (uniform) no finite range: -inf scores, or all children equal
         __syncthreads();
-        return cta_kth_largest_of_children_radix(sm, cnt, kx, sx, row, kth, tid);
+        return cta_kth_largest_of_children_radix(sm, cnt, kx, sx, row, cx, K, kth, tid);
     }
     for (int r = 0; r < cnt; ++r) {
-        const uint32_t oc = ord_from_float(sx + sm.es[row + r]);
+        const uint32_t oc = ord_from_float(sx + sm.es[row + es_col(r, cx, K)]);
         const float sc = __uint_as_float(bits_from_ord(oc < kx ? oc : kx));
         const float df = (top - sc) * scale;
         const int d = df > 0.0f ? (df < 1023.0f ? (int)df : 1023) : 0;
@@ -559,7 +559,7 @@ __device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSm
     if (lazy_neutral(p, j)) {
         // edge = log q exactly (the DDTree score of Eq. 3); log q is already ordered by rank
         for (int i = tid; i < K * K; i += TREE_THREADS) {
-            es[i] = (i / K) < n_par ? lps[i % K] : 0.f;
+            es[(i / K) * K + es_col(i % K, i / K, K)] = (i / K) < n_par ? lps[i % K] : 0.f;
             ei[i] = (uint8_t)(i % K);
         }
         __syncthreads();
@@ -579,7 +579,7 @@ __device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSm
         int rank;
         edge_row_finish(par < n_par ? part + (size_t)par * K : nullptr, lps, p.scale, p.beta, K, wsc, lane, val, rank);
         if (lane < K) {
-            es[(size_t)par * K + rank] = val;
+            es[(size_t)par * K + es_col(rank, par, K)] = val;
             ei[(size_t)par * K + rank] = (uint8_t)lane;
         }
     }
@@ -612,17 +612,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         mbar_init(smem_u32(&rows_bar), 1);
         mbar_fence_init();
     }
-    if (p.lazy) {  // the candidates of every depth, for the rows that may have to be scored here
-        for (int i = tid; i < L * K; i += TREE_THREADS) {
-            sm.tokid[i] = p.topk_id[(size_t)b * L * K + i];
-            sm.lpv[i] = p.topk_lp[(size_t)b * L * K + i];
-        }
-        if (rows_pre == 0) {  // the table rows of depth 0 arrive while the budget is worked out
-            __syncthreads();
-            lazy_issue_gather(p, sm, 0, root, tid);
-            inflight = 0;
-        }
-    }
     const size_t seq_e = (size_t)b * L * K * K;  // this sequence's rows in esort / eidx
     if (bulk) {
         if (tid == 0) {
@@ -642,6 +631,17 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         for (int i = tid; i < ne; i += TREE_THREADS) {
             sm.es[i] = p.esort[seq_e + i];
             sm.ei[i] = p.eidx[seq_e + i];
+        }
+    }
+    if (p.lazy) {  // the candidates of every depth, for the rows that may have to be scored here
+        for (int i = tid; i < L * K; i += TREE_THREADS) {
+            sm.tokid[i] = p.topk_id[(size_t)b * L * K + i];
+            sm.lpv[i] = p.topk_lp[(size_t)b * L * K + i];
+        }
+        if (rows_pre == 0) {  // the table rows of depth 0 arrive while the budget is worked out
+            __syncthreads();
+            lazy_issue_gather(p, sm, 0, root, tid);
+            inflight = 0;
         }
     }
     // a sequence whose tree will run deep had its deeper rows scored by the edge-score kernel as well (they are needed
@@ -679,8 +679,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         for (int j = t1; j < K * K; j += nth) {  // level 1
             const int xi = j / K, r = j - xi * K, x = 1 + xi;
             const uint32_t kx = sm.nkey[x];
-            const int row = (K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
-            const float sc = sm.nS[x] + sm.es[row + r];
+            const int cx = (int)((sm.ninfo[x] >> 13) & 31u), row = (K + cx) * K;
+            const float sc = sm.nS[x] + sm.es[row + es_col(r, cx, K)];
             const uint32_t oc = ord_from_float(sc);
             const int c = sm.ei[row + r], at = 1 + K + xi * K + c;
             sm.nkey[at] = oc < kx ? oc : kx;
@@ -779,8 +779,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     for (int j = tid; j < total; j += TREE_THREADS) {
                         const int xi = j / K, r = j - xi * K, x = b0 + xi;
                         const uint32_t kx = sm.nkey[x];
-                        const int row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
-                        const float sc = sm.nS[x] + sm.es[row + r];
+                        const int cx = (int)((sm.ninfo[x] >> 13) & 31u), row = (d * K + cx) * K;
+                        const float sc = sm.nS[x] + sm.es[row + es_col(r, cx, K)];
                         const uint32_t oc = ord_from_float(sc);
                         const int c = sm.ei[row + r], at = ntot + xi * K + c;  // (a full row: a child's slot is its rank)
                         sm.nkey[at] = oc < kx ? oc : kx;
@@ -811,16 +811,17 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     int cnt = 0;
                     uint32_t mask = 0u, kx = 0u;
                     float sx = 0.0f;
-                    int row = 0;
+                    int row = 0, cx = 0;
                     if (x < b1) {
                         kx = sm.nkey[x];
                         if (kx >= theta) {  // (else dead: none of its descendants can be selected)
-                            row = (d * K + (int)((sm.ninfo[x] >> 13) & 31u)) * K;
+                            cx = (int)((sm.ninfo[x] >> 13) & 31u);
+                            row = (d * K + cx) * K;
                             sx = sm.nS[x];
                             int lo_r = 0, hi_r = K;  // first r in [0, K] whose key falls below theta
                             while (lo_r < hi_r) {
                                 const int mid = (lo_r + hi_r) >> 1;
-                                const uint32_t oc = ord_from_float(sx + sm.es[row + mid]);
+                                const uint32_t oc = ord_from_float(sx + sm.es[row + es_col(mid, cx, K)]);
                                 if ((oc < kx ? oc : kx) >= theta)
                                     lo_r = mid + 1;
                                 else
@@ -861,7 +862,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     pre[tid] = __shfl_sync(0xFFFFFFFFu, wincl - wt, warp) + incl;
                     __syncthreads();
                     if (attempt == 0 && total >= budget && (total > flood || cur + total > p.ncap)) {  // (uniform) the search below uses the scan's space: count again
-                        const uint32_t tl = cta_kth_largest_of_children(sm, cnt, kx, sx, row, budget, theta, tid);
+                        const uint32_t tl = cta_kth_largest_of_children(sm, cnt, kx, sx, row, cx, K, budget, theta, tid);
                         theta = tl > theta ? tl : theta;
                         continue;
                     }
@@ -883,8 +884,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                         const int first = lo_t ? pre[lo_t - 1] : 0;
                         const int r = i - first, xo = c0 + lo_t;
                         const uint32_t kx = sm.nkey[xo];
-                        const int row = (d * K + (int)((sm.ninfo[xo] >> 13) & 31u)) * K;
-                        const float sc = sm.nS[xo] + sm.es[row + r];
+                        const int co = (int)((sm.ninfo[xo] >> 13) & 31u), row = (d * K + co) * K;
+                        const float sc = sm.nS[xo] + sm.es[row + es_col(r, co, K)];
                         const uint32_t oc = ord_from_float(sc);
                         const int c = sm.ei[row + r];
                         const int at = cur + first + __popc(cmask[lo_t] & ((1u << c) - 1u));
@@ -999,12 +1000,12 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     int pos = 0, hi_p = K;  // first entry of the (ordered) row whose key is not above theta
                     while (pos < hi_p) {
                         const int mid = (pos + hi_p) >> 1;
-                        if (ord_from_float(sn + sm.es[row + mid]) > theta)
+                        if (ord_from_float(sn + sm.es[row + es_col(mid, sm.cand[n], K)]) > theta)
                             pos = mid + 1;
                         else
                             hi_p = mid;
                     }
-                    if (pos < K) e = pack_entry(sn + sm.es[row + pos], d + 1, pos, sm.cand[n], sm.ei[row + pos]);
+                    if (pos < K) e = pack_entry(sn + sm.es[row + es_col(pos, sm.cand[n], K)], d + 1, pos, sm.cand[n], sm.ei[row + pos]);
                 }
                 sm.ent[n] = e;
             }
@@ -1075,8 +1076,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 sm.S[n_new] = s_new;
                 uint64_t e_adv = 0ull, e_new = 0ull;
                 if (pos + 1 < K) {
-                    const int at = ((d - 1) * K + cpar) * K + pos + 1;
-                    e_adv = pack_entry(sm.S[bn] + sm.es[at], d, pos + 1, cpar, sm.ei[at]);
+                    const int at = ((d - 1) * K + cpar) * K;
+                    e_adv = pack_entry(sm.S[bn] + sm.es[at + es_col(pos + 1, cpar, K)], d, pos + 1, cpar, sm.ei[at + pos + 1]);
                 }
                 if (d < L && n_sel < budget) {  // (after the last selection the entry is never read)
                     // a node selected here has a key >= theta, so it sits in the table and the row of its depth
@@ -1085,7 +1086,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                         st |= GRAFT_ST_INTERNAL;
                     } else {
                         const int at = (d * K + c) * K;
-                        e_new = pack_entry(s_new + sm.es[at], d + 1, 0, c, sm.ei[at]);
+                        e_new = pack_entry(s_new + sm.es[at + c], d + 1, 0, c, sm.ei[at]);  // (entry 0 stands at column c)
                     }
                 }
                 sm.ent[bn] = e_adv;
@@ -1187,15 +1188,16 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         const int i = ordered ? n : sm.canon[n], d = sm.depth[n];
         const int par = n == 0 ? -1 : (ordered ? sm.parent[n] : sm.canon[sm.parent[n]]);
         sm.cparent[i] = (int16_t)par;
-        o.d_token[ob + i] = n == 0 ? root : p.topk_id[((size_t)b * L + d - 1) * K + sm.cand[n]];
+        o.d_token[ob + i] = n == 0 ? root
+                                   : (p.lazy ? sm.tokid[(d - 1) * K + sm.cand[n]]  // (staged in the prologue)
+                                             : p.topk_id[((size_t)b * L + d - 1) * K + sm.cand[n]]);
         o.d_parent[ob + i] = par;
         o.d_depth[ob + i] = d;
         o.d_position[ob + i] = prefix - 1 + d;
         o.d_path_score[ob + i] = sm.S[n];
     }
     __syncthreads();
-    // ancestor masks: each thread builds one row in its warp's staging tile (walking up, level-order indices
-    // only decrease, so the row is produced from its highest word down); the warp then stores its 32 rows,
+    // ancestor masks: each thread builds one row in its warp's staging tile; the warp then stores its 32 rows,
     // which are contiguous in the output, with coalesced writes.  Padding rows are zero-filled directly.
     {
         const size_t stage_off = (((size_t)nmax * 2 + 15) & ~(size_t)15) + (((size_t)nmax * 4 + 15) & ~(size_t)15);
@@ -1207,23 +1209,12 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         for (int i0 = warp * 32; i0 < n_nodes && warp < mw; i0 += mw * 32) {
             const int i = i0 + lane;
             uint32_t* row = tile + lane * W;
+            // the tile is cleared by the warp together, then a lane sets the bits of its node's ancestors (itself included)
+            for (int k = lane; k < 32 * W; k += 32) tile[k] = 0u;
+            __syncwarp();
             if (i < n_nodes) {
-                int w = W - 1;
-                uint32_t bits = 0u;
                 int steps = 0;  // a node has at most L ancestors: the bound keeps the walk finite whatever the arrays hold
-                for (int a = i; a >= 0 && a < nmax && steps <= L; a = sm.cparent[a], ++steps) {
-                    const int wa = a >> 5;
-                    while (w > wa) {
-                        row[w] = bits;
-                        bits = 0u;
-                        --w;
-                    }
-                    bits |= 1u << (a & 31);
-                }
-                row[w] = bits;
-                for (--w; w >= 0; --w) row[w] = 0u;
-            } else {
-                for (int w = 0; w < W; ++w) row[w] = 0u;
+                for (int a = i; a >= 0 && a < nmax && steps <= L; a = sm.cparent[a], ++steps) row[a >> 5] |= 1u << (a & 31);
             }
             __syncwarp();
             const int rows = min(32, nmax - i0);
