@@ -400,15 +400,15 @@ __device__ __forceinline__ bool select_in_bucket(const SelBucket& st, uint32_t k
 }
 
 // One histogram pass over keys[lo_i..hi_i) finds the bin that holds the B-th largest key, and a lower bound of that
-// key (the bin's lower edge less a hundredth of a bin: the rounding of select_bin is below 1e-4 of a bin).  A bin spans about as much
-// as a key's top 16 bits do at the scores met here, so the bound prunes as well as two 8-bit radix passes would,
-// for one pass and three barriers.  If the B-th largest falls into the shared last bin, two radix passes find its
-// 16-bit bucket instead.  Bins are padded by one word per 32 so that warp 0's lanes, which own 32 consecutive bins
-// each, read without bank conflicts.  Every thread of the CTA calls this; hi_i - lo_i >= kth >= 1.
+// key (the bin's lower edge less a hundredth of a bin: the rounding of select_bin is below 1e-4 of a bin).  A bin
+// spans about as much as a key's top 16 bits do at the scores met here, so the bound prunes as well as two 8-bit
+// radix passes would, for one pass.  If the B-th largest falls into the shared last bin, two radix passes find its
+// 16-bit bucket instead.  Bins are padded by one word per 32 (the flood search's lanes own 32 consecutive bins each
+// and read them without bank conflicts).  Every thread of the CTA calls this; hi_i - lo_i >= kth >= 1.
 __device__ uint32_t cta_select_bucket(const TreeSmem& sm, const uint32_t* keys, int lo_i, int hi_i, int kth, float top,
                                       SelBucket& st, int tid) {
     const int warp = tid >> 5, lane = tid & 31;
-    uint32_t* h = sm.hist;  // [1024 + 32]
+    uint32_t* h = sm.hist;  // [1024 + 32] bins, [1060 + 32] sums of 32 bins
     h[tid] = 0u;
     if (tid < 32) h[1024 + tid] = 0u;
     __syncthreads();
@@ -417,30 +417,34 @@ __device__ uint32_t cta_select_bucket(const TreeSmem& sm, const uint32_t* keys, 
         atomicAdd(&h[d + (d >> 5)], 1u);
     }
     __syncthreads();
-    if (warp == 0) {  // lane l owns bins 32 l .. 32 l + 31 (bin 0 holds the largest keys)
-        const uint32_t* mine = h + 33 * lane;
-        int sum = 0;
-#pragma unroll 8
-        for (int q = 0; q < 32; ++q) sum += (int)mine[q];
-        int incl = sum;
+    // warp w adds up bins 32 w .. 32 w + 31 (bin 0 holds the largest keys); warp 0 then finds the group of 32 bins that
+    // holds the kth largest key in a scan of the 32 sums, and the bin in a scan of that group: two short steps
+    {
+        const uint32_t wsum = __reduce_add_sync(0xFFFFFFFFu, h[33 * warp + lane]);
+        if (lane == 0) h[1060 + warp] = wsum;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const int ws = (int)h[1060 + lane];
+        int incl = ws;
 #pragma unroll
         for (int o2 = 1; o2 < 32; o2 <<= 1) {
             const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o2);
             if (lane >= o2) incl += t;
         }
-        const int excl = incl - sum;
-        if (excl < kth && kth <= incl) {
-            int acc = excl, bin = 32 * lane, rem = kth - excl;
-            for (int q = 0; q < 32; ++q) {
-                const int c = (int)mine[q];
-                if (acc < kth && kth <= acc + c) {
-                    bin = 32 * lane + q;
-                    rem = kth - acc;
-                }
-                acc += c;
-            }
-            sm.scal[6] = bin;
-            sm.scal[7] = rem;
+        const uint32_t gm = __ballot_sync(0xFFFFFFFFu, incl - ws < kth && kth <= incl);  // (one lane: kth <= keys in all)
+        const int g = gm ? __ffs(gm) - 1 : 31;
+        const int base = __shfl_sync(0xFFFFFFFFu, incl - ws, g);
+        const int c = (int)h[33 * g + lane];
+        int inc2 = c;
+#pragma unroll
+        for (int o2 = 1; o2 < 32; o2 <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, inc2, o2);
+            if (lane >= o2) inc2 += t;
+        }
+        if (base + inc2 - c < kth && kth <= base + inc2) {
+            sm.scal[6] = 32 * g + lane;
+            sm.scal[7] = kth - (base + inc2 - c);
         }
     }
     __syncthreads();
@@ -769,7 +773,12 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 lazy_score_row(p, sm, d, root, tid, inflight);
                 rows_done = d + 1;
             }
+            // grow: can a node appended here have a child that reaches theta?  (Its best child stands first in its sorted
+            // row.)  If none can, the next level would append nothing: the loop ends here instead of finding that out
+            // with a whole pass.  theta only rises, so "cannot now" stays true.
+            int grow = 0;
             if (theta == 0u) {
+                grow = d + 1 < L ? 1 : 0;
                 // no threshold yet (fewer than B nodes so far): every child of every node of the level is appended,
                 // one thread per (node, child), at a position that needs no atomic
                 const int total = (b1 - b0) * K;
@@ -822,20 +831,21 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                             while (lo_r < hi_r) {
                                 const int mid = (lo_r + hi_r) >> 1;
                                 const uint32_t oc = ord_from_float(sx + sm.es[row + es_col(mid, cx, K)]);
-                                if ((oc < kx ? oc : kx) >= theta)
+                                if (oc >= theta)  // (kx >= theta already: the child's key min(kx, oc) reaches theta iff oc does)
                                     lo_r = mid + 1;
                                 else
                                     hi_r = mid;
                             }
                             cnt = lo_r;
-                            if ((K & 15) == 0) {  // rows of whole 16-byte vectors: the ranks come sixteen at a time
-                                for (int r0 = 0; r0 < cnt; r0 += 16) {
-                                    const uint4 q = *(const uint4*)(sm.ei + row + r0);
-                                    const uint32_t wq[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                                    for (int j = 0; j < 16; ++j) {
-                                        if (r0 + j < cnt) mask |= 1u << ((wq[j >> 2] >> (8 * (j & 3))) & 31u);
-                                    }
+                            if ((K & 3) == 0) {  // rows of whole words: the ranks come four at a time
+                                const uint32_t* eiw = (const uint32_t*)(sm.ei + row);
+                                for (int r0 = 0; r0 < cnt; r0 += 4) {
+                                    const uint32_t q = eiw[r0 >> 2];
+                                    const int left = cnt - r0;
+                                    mask |= 1u << (q & 31u);
+                                    if (left > 1) mask |= 1u << ((q >> 8) & 31u);
+                                    if (left > 2) mask |= 1u << ((q >> 16) & 31u);
+                                    if (left > 3) mask |= 1u << ((q >> 24) & 31u);
                                 }
                             } else {
                                 for (int r = 0; r < cnt; ++r) mask |= 1u << sm.ei[row + r];
@@ -889,6 +899,14 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                         const uint32_t oc = ord_from_float(sc);
                         const int c = sm.ei[row + r];
                         const int at = cur + first + __popc(cmask[lo_t] & ((1u << c) - 1u));
+                        if (d + 1 < L) {
+                            if (d + 1 < rows_done) {
+                                const uint32_t ob = ord_from_float(sc + sm.es[((d + 1) * K + c) * K + c]);  // (entry 0: column c)
+                                grow |= (ob >= theta && oc >= theta) ? 1 : 0;
+                            } else {
+                                grow = 1;  // (that row is not scored yet)
+                            }
+                        }
                         sm.nkey[at] = oc < kx ? oc : kx;
                         sm.nS[at] = sc;
                         sm.ninfo[at] = (uint32_t)xo | ((uint32_t)c << 13) | ((uint32_t)(d + 1) << 18);
@@ -898,7 +916,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 }
                 if (tid == 0) sm.scal[3] = cur;
             }
-            __syncthreads();
+            const int any_grow = __syncthreads_or(grow);
             const int nt = sm.scal[3];
             if (sm.scal[4]) {
                 table_ok = false;
@@ -907,9 +925,10 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             if (tid == 0) sm.lvl_start[d + 2] = nt;
             if (nt == ntot) break;  // nothing appended: no deeper level
             ntot = nt;
+            if (!any_grow) break;  // no node of the new level can have a child in the tree
             // theta only has to be a lower bound of its final value while the levels are built (it prunes), so
             // the exact B-th largest key is recomputed only when the table has grown noticeably
-            if (ntot - 1 >= budget && (theta == 0u || ntot - n_at_select >= ntot / 2)) {
+            if (ntot - 1 >= budget && (theta == 0u || ntot - n_at_select >= ntot / 8)) {
                 sel_top = 0.0f + sm.es[0];  // the root's best child
                 theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);  // a lower bound
                 n_at_select = ntot;
