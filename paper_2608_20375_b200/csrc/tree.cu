@@ -837,19 +837,23 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                                     hi_r = mid;
                             }
                             cnt = lo_r;
-                            if ((K & 3) == 0) {  // rows of whole words: the ranks come four at a time
+                            // the candidate ranks of the first cnt entries, four at a time where the rows are whole words;
+                            // a long prefix is taken as all ranks less those of the entries behind it
+                            const bool tail = 2 * cnt > K;
+                            const int r_lo = tail ? cnt : 0, r_hi = tail ? K : cnt;
+                            if ((K & 3) == 0) {
                                 const uint32_t* eiw = (const uint32_t*)(sm.ei + row);
-                                for (int r0 = 0; r0 < cnt; r0 += 4) {
+                                for (int r0 = r_lo & ~3; r0 < r_hi; r0 += 4) {
                                     const uint32_t q = eiw[r0 >> 2];
-                                    const int left = cnt - r0;
-                                    mask |= 1u << (q & 31u);
-                                    if (left > 1) mask |= 1u << ((q >> 8) & 31u);
-                                    if (left > 2) mask |= 1u << ((q >> 16) & 31u);
-                                    if (left > 3) mask |= 1u << ((q >> 24) & 31u);
+                                    if (r0 >= r_lo) mask |= 1u << (q & 31u);
+                                    if (r0 + 1 >= r_lo && r0 + 1 < r_hi) mask |= 1u << ((q >> 8) & 31u);
+                                    if (r0 + 2 >= r_lo && r0 + 2 < r_hi) mask |= 1u << ((q >> 16) & 31u);
+                                    if (r0 + 3 >= r_lo && r0 + 3 < r_hi) mask |= 1u << ((q >> 24) & 31u);
                                 }
                             } else {
-                                for (int r = 0; r < cnt; ++r) mask |= 1u << sm.ei[row + r];
+                                for (int r = r_lo; r < r_hi; ++r) mask |= 1u << sm.ei[row + r];
                             }
+                            if (tail) mask = (K == 32 ? 0xFFFFFFFFu : (1u << K) - 1u) & ~mask;
                         }
                     }
                     cmask[tid] = mask;
