@@ -54,6 +54,7 @@ __device__ __forceinline__ void edge_dots(const float* rP, const float* rC, cons
         for (int i2 = 0; i2 < 2; ++i2) acc[i][i2] = make_float2(0.f, 0.f);
     const float* c0 = rC + (size_t)min(tx, K - 1) * ld;  // (rows past K: read, never used)
     const float* c1 = rC + (size_t)min(tx + 16, K - 1) * ld;
+#pragma unroll 2
     for (int k4 = ks; k4 < q4; k4 += 2) {
         float4 uu = make_float4(0.f, 0.f, 0.f, 0.f);
         if (ADD_U) uu = *(const float4*)(rU + 4 * k4);
@@ -108,7 +109,7 @@ __device__ __forceinline__ void edge_dots(const float* rP, const float* rC, cons
 // before it.  dots: the parent's K dot products, or nullptr for a parent that does not exist (a row of zeros).
 // wsc: 32 words of shared memory of this warp.  Returns the score in `val` and the place in `rank` (lanes < K).
 __device__ __forceinline__ void edge_row_finish(const float* dots, const float* lps, float scale, float beta, int K,
-                                                uint32_t* wsc, int lane, float& val, int& rank) {
+                                                float inv_K, uint32_t* wsc, int lane, float& val, int& rank) {
     const int c = lane;
     val = 0.f;
     if (dots != nullptr) {
@@ -116,7 +117,10 @@ __device__ __forceinline__ void edge_row_finish(const float* dots, const float* 
         float sum = ft;
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
-        const float mean = sum / (float)K;
+        // sum / K: the product with 1 / K (worked out once by the caller) and one correction step with the exact
+        // remainder, which gives the rounded quotient without the division's special-case code
+        const float q0 = sum * inv_K;
+        const float mean = fmaf(fmaf(-q0, (float)K, sum), inv_K, q0);
         val = fmaf(beta, ft - mean, c < K ? lps[c] : 0.f);
     }
     const uint32_t mine = c < K ? ord_from_float(val) : 0u;  // 0 is below the image of every float
@@ -129,8 +133,13 @@ __device__ __forceinline__ void edge_row_finish(const float* dots, const float* 
         const uint4 o4 = *(const uint4*)(wsc + 4 * i4);
         rank += (o4.x > mine ? 1 : 0) + (o4.y > mine ? 1 : 0) + (o4.z > mine ? 1 : 0) + (o4.w > mine ? 1 : 0);
     }
-    const uint32_t same = __match_any_sync(0xFFFFFFFFu, mine);
-    rank += __popc(same & ((1u << lane) - 1u));
+    // equal scores (rare) go by child rank: the counts above are a permutation of 0..K-1 unless some scores are equal,
+    // and only then are the lanes with the same score looked up (a slow instruction)
+    const uint32_t seen = __reduce_or_sync(0xFFFFFFFFu, c < K ? 1u << rank : 0u);
+    if (seen != (K == 32 ? 0xFFFFFFFFu : (1u << K) - 1u)) {  // (uniform)
+        const uint32_t same = __match_any_sync(0xFFFFFFFFu, mine);
+        rank += __popc(same & ((1u << lane) - 1u));
+    }
 }
 
 }  // namespace graft

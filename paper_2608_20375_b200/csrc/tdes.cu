@@ -184,11 +184,12 @@ __global__ void __launch_bounds__(256, 4) tdes_edges_kernel(const EdgeParams p) 
     __shared__ uint32_t wsc[8][32];
     edge_dots<false>(sP, sC, nullptr, m, K, n_par, part, warp, lane);
     __syncthreads();
+    const float inv_K = 1.0f / (float)K;
     for (int par = warp; par < K; par += 8) {
         float val;
         int rank;
-        edge_row_finish(par < n_par ? part + (size_t)par * K : nullptr, lps, p.scale, p.beta, K, wsc[warp], lane, val,
-                        rank);
+        edge_row_finish(par < n_par ? part + (size_t)par * K : nullptr, lps, p.scale, p.beta, K, inv_K, wsc[warp], lane,
+                        val, rank);
         if (lane < K) {
             if (WRITE_EDGE) p.edge[(row * K + par) * K + lane] = val;
             outs[(size_t)par * K + es_col(rank, par, K)] = val;

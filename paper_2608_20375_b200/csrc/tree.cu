@@ -578,10 +578,12 @@ __device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSm
     __syncthreads();
     lazy_issue_gather(p, sm, j + 1, root_token, tid);  // the table rows of this depth are no longer read
     inflight = j + 1;
+    const float inv_K = 1.0f / (float)K;
     for (int par = warp; par < K; par += TREE_THREADS / 32) {  // one warp per parent
         float val;
         int rank;
-        edge_row_finish(par < n_par ? part + (size_t)par * K : nullptr, lps, p.scale, p.beta, K, wsc, lane, val, rank);
+        edge_row_finish(par < n_par ? part + (size_t)par * K : nullptr, lps, p.scale, p.beta, K, inv_K, wsc, lane, val,
+                        rank);
         if (lane < K) {
             es[(size_t)par * K + es_col(rank, par, K)] = val;
             ei[(size_t)par * K + rank] = (uint8_t)lane;
