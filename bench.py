@@ -276,6 +276,23 @@ def run_graft(args):
         step(0)
     torch.cuda.synchronize()
     event_pair_ms = float(np.median([a.elapsed_time(b_) for a, b_ in pairs]))
+    # the vocab pass alone, launched back to back over the same rotating inputs through its own entry point
+    # (graft_vocab_pass) with one event pair around the whole series: its throughput with no event record between
+    # launches, i.e. with each launch setting up while the one ahead drains, as inside an ordinary round
+    vb_ids = torch.empty((batch, w.L, w.K), dtype=torch.int32, device=dev)
+    vb_lp = torch.empty((batch, w.L, w.K), dtype=torch.float32, device=dev)
+    vb_lse = torch.empty((batch, w.L), dtype=torch.float32, device=dev)
+    vb_st = torch.empty((batch, w.L), dtype=torch.int32, device=dev)
+    n_b2b = 200
+    for i in range(8):
+        g.vocab_pass(dev_sets[i % n_buf]["logits"], vb_ids, vb_lp, vb_lse, vb_st)
+    evb0, evb1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    evb0.record()
+    for i in range(n_b2b):
+        g.vocab_pass(dev_sets[i % n_buf]["logits"], vb_ids, vb_lp, vb_lse, vb_st)
+    evb1.record()
+    torch.cuda.synchronize()
+    vocab_b2b_ms = evb0.elapsed_time(evb1) / n_b2b
     if world > 1:
         import torch.distributed as dist
         t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
@@ -350,13 +367,15 @@ def run_graft(args):
         "gpu_launches": launches,
         "kernel_ms": {"vocab_pass": vocab_ms / max(1, n_t), "tdes_edges": tdes_ms / max(1, n_t),
                       "tree": tree_ms / max(1, n_t), "calls_averaged": n_t, "empty_event_pair": event_pair_ms,
-                      "round_with_these_events": instrumented_round_ms},
+                      "round_with_these_events": instrumented_round_ms,
+                      "vocab_pass_back_to_back": vocab_b2b_ms},
         "roofline": {"bound": "hbm", "kernel": "vocab_pass_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8000": achieved / 8000.0, "algorithmic_bytes": algo_bytes,
                      "achieved_with_hidden": achieved_h, "frac_with_hidden": achieved_h / peak,
                      "algorithmic_bytes_with_hidden": logits_bytes + hidden_bytes,
                      "frac_net_of_event_pair": algo_bytes / max(1e-9, vocab_s - event_pair_ms * 1e-3) / 1e9 / peak,
+                     "frac_back_to_back": algo_bytes / (vocab_b2b_ms * 1e-3) / 1e9 / peak,
                      "traffic": NCU_VOCAB_TRAFFIC_BYTES_M if w.name == "M" else None},
         "e2e": {"value": world * batch / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3, "steps": e2e_steps,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
