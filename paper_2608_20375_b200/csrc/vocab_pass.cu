@@ -828,16 +828,35 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             }
             epi_bar(grp);
             {
+                // (listed thread, tile) pairs, four per thread at a time with their loads in flight together; the pair's
+                // thread comes from a multiplication (idx / ntiles for idx < 2^16 and ntiles < 2^16, exactly)
                 const int npairs = es->nht * sg.ntiles;
-                for (int idx = etid; idx < npairs; idx += kVpEpiThreads) {
-                    const int h = idx / sg.ntiles, tile = idx - h * sg.ntiles;
-                    const uint32_t t = es->hthreads[h];
-                    const cm_t raw = cmx[(size_t)t * p.max_tiles + tile];
-                    const uint32_t bits = (uint32_t)raw << 16;
-                    if (ord_from_bits(bits) >= Tv) {
-                        const int pos = atomicAdd(&es->nhits, 1);
-                        if (pos >= kVpHitCap) break;  // too many: the exact selection over the segment takes over
-                        es->hits[pos] = (uint32_t)tile * TILE + (t >> 5) * WBLK + (t & 31) * 64;
+                const uint32_t magic = sg.ntiles > 1 ? 0xFFFFFFFFu / (uint32_t)sg.ntiles + 1u : 0u;  // ceil(2^32 / ntiles)
+                constexpr int PU = 4;
+                bool stop = false;
+                for (int base = 0; base < npairs && !stop; base += kVpEpiThreads * PU) {
+                    uint32_t raw[PU], off[PU];
+#pragma unroll
+                    for (int u = 0; u < PU; ++u) {
+                        const int idx = base + u * kVpEpiThreads + etid;
+                        raw[u] = 0u;
+                        off[u] = 0u;
+                        if (idx < npairs) {
+                            const int h = sg.ntiles > 1 ? (int)__umulhi((uint32_t)idx, magic) : idx, tile = idx - h * sg.ntiles;
+                            const uint32_t t = es->hthreads[h];
+                            raw[u] = cmx[(size_t)t * p.max_tiles + tile];
+                            off[u] = (uint32_t)tile * TILE + (t >> 5) * WBLK + (t & 31) * 64;
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < PU; ++u) {
+                        if (ord_from_bits(raw[u] << 16) >= Tv && base + u * kVpEpiThreads + etid < npairs && !stop) {
+                            const int pos = atomicAdd(&es->nhits, 1);
+                            if (pos >= kVpHitCap)
+                                stop = true;  // too many: the exact selection over the segment takes over
+                            else
+                                es->hits[pos] = off[u];
+                        }
                     }
                 }
             }
@@ -926,11 +945,18 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             const int ncand = es->ncand < kVpCandCap ? es->ncand : kVpCandCap;
             int nk = ncand < p.K ? ncand : p.K;
             if (!overflow) {
-                for (int i = etid; i < ncand; i += kVpEpiThreads) {
-                    const uint64_t key = es->cand[i];
-                    int rank = 0;
-                    for (int j = 0; j < ncand; ++j) rank += (es->cand[j] > key) ? 1 : 0;
-                    if (rank < p.K) es->outk[rank] = key;
+                // two neighbouring lanes per candidate, each over every other key, two running counts each
+                for (int i0 = 0; i0 < ncand; i0 += kVpEpiThreads / 2) {
+                    const int i = i0 + (etid >> 1);
+                    const uint64_t key = i < ncand ? es->cand[i] : ~0ull;
+                    int r0 = 0, r1 = 0;
+                    for (int j = etid & 1; j < ncand; j += 4) {
+                        r0 += (es->cand[j] > key) ? 1 : 0;
+                        r1 += (j + 2 < ncand && es->cand[j + 2] > key) ? 1 : 0;
+                    }
+                    int rank = r0 + r1;
+                    rank += __shfl_xor_sync(0xFFFFFFFFu, rank, 1);
+                    if (i < ncand && (etid & 1) == 0 && rank < p.K) es->outk[rank] = key;
                 }
             } else if (ew == 0) {
                 nk = warp_fallback_select<BF16>(es, p, sg, cmx, lane);
