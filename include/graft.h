@@ -211,7 +211,8 @@ graft_status graft_vocab_merge(graft_ctx* ctx, int32_t batch, int32_t n_shards, 
                                int32_t* d_row_status, void* stream);
 
 /* Acceptance walk (Preliminaries, "Speculative decoding": a_t; "Tree-based speculative decoding": the longest
- * accepted path is committed).  d_target_next[b, i] is the target model's next token after node i.  The tree
+ * accepted path is committed).  d_target_next [batch, Nmax]: d_target_next[b, i] is the target model's next token
+ * after node i (all Nmax entries of a sequence are read; those at or beyond its node count may hold anything).  The tree
  * must be in the level order graft_build_trees emits (parent indices never decrease along the node index).
  * Starting at the root, follow the child whose token equals target_next of the current node.
  *   d_accept_len  [batch]     number of accepted draft tokens a_t (bonus token not counted)

@@ -1294,28 +1294,30 @@ __global__ void __launch_bounds__(128) accept_kernel(const AcceptParams ap) {
     int32_t* tok = par + nmax;
     int32_t* tn = tok + nmax;
     const size_t ob = (size_t)b * nmax;
+    // every slot of the three arrays is staged, padding included, so that these loads do not wait for the node count
+    // (one round trip to global memory instead of two); the walk below never looks beyond the count
     int nn = n_nodes[b];
-    nn = nn < 1 ? 1 : (nn > nmax ? nmax : nn);
     {
         constexpr int U = 8;  // 128 threads x 8 covers the largest tree (1024 nodes) in one round
         int32_t vp[U], vt[U], vn[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int i = tid + 128 * u;
-            vp[u] = i < nn ? parent[ob + i] : 0;
-            vt[u] = i < nn ? token[ob + i] : 0;
-            vn[u] = i < nn ? target_next[ob + i] : 0;
+            vp[u] = i < nmax ? parent[ob + i] : 0;
+            vt[u] = i < nmax ? token[ob + i] : 0;
+            vn[u] = i < nmax ? target_next[ob + i] : 0;
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int i = tid + 128 * u;
-            if (i < nn) {
+            if (i < nmax) {
                 par[i] = vp[u];
                 tok[i] = vt[u];
                 tn[i] = vn[u];
             }
         }
     }
+    nn = nn < 1 ? 1 : (nn > nmax ? nmax : nn);
     __syncthreads();
     if (tid >= 32) return;
     int cur = 0, a = 0;
