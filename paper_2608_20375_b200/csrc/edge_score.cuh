@@ -16,13 +16,22 @@ namespace graft {
 // top-1 probability of the block >= 0.2: on the configured workloads trees reach depth 8 from about there); the tree
 // kernel, which takes the same decision from the same numbers, scores what is missing on demand.  A matter of speed
 // only: a row has the same bits whoever scores it.
-__device__ __forceinline__ bool deep_tree_likely(const float* __restrict__ topk_lp_seq, int L, int K) {
-    // every warp calls this with all its lanes: lane d takes position d (L <= 32), then a butterfly sum in a fixed order
+// (In two steps, so that a caller can have the load in flight beside its other loads: lane d's top-1 log-probability
+// of position d, 0 for d >= L; then the decision, taken by every lane of a warp together.)
+__device__ __forceinline__ float deep_tree_load(const float* __restrict__ topk_lp_seq, int L, int K) {
     const int lane = threadIdx.x & 31;
-    float s = lane < L ? ex2_approx(topk_lp_seq[(size_t)lane * K] * kLog2e) : 0.f;
+    return lane < L ? topk_lp_seq[(size_t)lane * K] : 0.f;
+}
+__device__ __forceinline__ bool deep_tree_decide(float lp_top, int L) {
+    // lane d holds position d (L <= 32); a butterfly sum in a fixed order
+    const int lane = threadIdx.x & 31;
+    float s = lane < L ? ex2_approx(lp_top * kLog2e) : 0.f;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
     return s >= 0.2f * (float)L;
+}
+__device__ __forceinline__ bool deep_tree_likely(const float* __restrict__ topk_lp_seq, int L, int K) {
+    return deep_tree_decide(deep_tree_load(topk_lp_seq, L, K), L);
 }
 
 

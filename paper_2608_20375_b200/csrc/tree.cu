@@ -610,7 +610,20 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     const int rows_pre = p.rows_pre;
     const int ne = rows_pre * K * K;  // entries that come from the edge-score kernel for every sequence
     const bool bulk = ne > 0 && (ne % 16) == 0;
+    // the prologue's loads from global memory are all issued before the first of them is used: one round trip
     const int root = p.root_token[b];
+    const float lp_top = p.rows_adaptive ? deep_tree_load(p.topk_lp + (size_t)b * L * K, L, K) : 0.f;
+    SabaResult pre_r;
+    pre_r.budget = 0;
+    pre_r.status = 0;
+    pre_r.state[0] = pre_r.state[1] = pre_r.state[2] = pre_r.state[3] = 0.f;
+    if (p.saba_pre && tid == 0) pre_r = p.saba_pre[b];
+    int32_t lz_tok = 0;
+    float lz_lp = 0.f;
+    if (p.lazy && tid < L * K) {  // (L K <= 1024: a thread per candidate)
+        lz_tok = p.topk_id[(size_t)b * L * K + tid];
+        lz_lp = p.topk_lp[(size_t)b * L * K + tid];
+    }
     int rows_done = rows_pre;  // rows [0, rows_done) are in shared memory
     int inflight = -1;           // on-demand scoring: depth whose table rows are being fetched
     if (tid == 0) {
@@ -640,9 +653,9 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         }
     }
     if (p.lazy) {  // the candidates of every depth, for the rows that may have to be scored here
-        for (int i = tid; i < L * K; i += TREE_THREADS) {
-            sm.tokid[i] = p.topk_id[(size_t)b * L * K + i];
-            sm.lpv[i] = p.topk_lp[(size_t)b * L * K + i];
+        if (tid < L * K) {
+            sm.tokid[tid] = lz_tok;
+            sm.lpv[tid] = lz_lp;
         }
         if (rows_pre == 0) {  // the table rows of depth 0 arrive while the budget is worked out
             __syncthreads();
@@ -652,7 +665,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     }
     // a sequence whose tree will run deep had its deeper rows scored by the edge-score kernel as well (they are needed
     // several levels from here: plain loads, consumed after many barriers)
-    if (p.rows_adaptive && deep_tree_likely(p.topk_lp + (size_t)b * L * K, L, K)) {  // (uniform)
+    if (p.rows_adaptive && deep_tree_decide(lp_top, L)) {  // (uniform)
         for (int i = ne + tid; i < L * K * K; i += TREE_THREADS) {
             sm.es[i] = p.esort[seq_e + i];
             sm.ei[i] = p.eidx[seq_e + i];
@@ -697,7 +710,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     if (warp == 0) {  // status and budget: from the edge-score kernel if it ran ahead, else worked out here
         SabaResult r;
         if (p.saba_pre)
-            r = p.saba_pre[b];
+            r = pre_r;  // (lane 0's copy is the one used below)
         else
             r = saba_warp(p.saba, p.bmin, p.bmax, p.bstep, L, K, p.row_status + (size_t)b * L, p.vp_err,
                           p.topk_lp + (size_t)b * L * K, sm.cosv, p.hist + b, p.prefix_len + b,
