@@ -32,7 +32,7 @@ METRIC = "draft trees built and verified-walked per second (batch 64, L=16, V=15
 UNIT = "trees/s"
 # DRAM bytes (read + write) of one vocab-pass launch on workload M: the mean of the two launches of the ncu
 # capture summarised in profiles/vocab_pass_kernel_M.md.
-NCU_VOCAB_TRAFFIC_BYTES_M = 330_030_000  # profiles/vocab_pass_kernel_M.md: mean of two launches, read + write
+NCU_VOCAB_TRAFFIC_BYTES_M = 324_300_000  # profiles/vocab_pass_kernel_M.md: mean of two launches, read + write
 L2_BYTES = 126 * 1024 * 1024
 
 
