@@ -52,7 +52,7 @@ struct TreeSmem {
     // is the level order of the emitted tree: a subset taken in table order is already in level order
     uint32_t* nkey;      // [ncap]   bottleneck key = min over the path of ord(path score); later: compact index
     float* nS;           // [ncap]   path score
-    uint32_t* ninfo;     // [ncap]   parent's table index | candidate rank << 13 | depth << 18
+    uint32_t* ninfo;     // [ncap]   parent's table index | candidate rank << 13 | depth << 18 | place in the parent's sorted row << 24
     // compact arrays by selection index n (0 = root; a parent's index is smaller than its children's)
     uint64_t* ent;       // [nmax]   frontier entry of node n: its best unselected child, 0 = none
     float* S;            // [nmax]   path score
@@ -692,7 +692,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             const int c = sm.ei[t1];
             sm.nkey[1 + c] = ord_from_float(sc);
             sm.nS[1 + c] = sc;
-            sm.ninfo[1 + c] = 0u | ((uint32_t)c << 13) | (1u << 18);
+            sm.ninfo[1 + c] = 0u | ((uint32_t)c << 13) | (1u << 18) | ((uint32_t)t1 << 24);
         }
         named_bar_sync(1, nth);
         for (int j = t1; j < K * K; j += nth) {  // level 1
@@ -704,7 +704,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             const int c = sm.ei[row + r], at = 1 + K + xi * K + c;
             sm.nkey[at] = oc < kx ? oc : kx;
             sm.nS[at] = sc;
-            sm.ninfo[at] = (uint32_t)x | ((uint32_t)c << 13) | (2u << 18);
+            sm.ninfo[at] = (uint32_t)x | ((uint32_t)c << 13) | (2u << 18) | ((uint32_t)r << 24);
         }
     }
     if (warp == 0) {  // status and budget: from the edge-score kernel if it ran ahead, else worked out here
@@ -744,14 +744,6 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         sm.nkey[0] = 0xFFFFFFFFu;
         sm.nS[0] = 0.0f;
         sm.ninfo[0] = 0u;
-        sm.scal[3] = spec ? 1 + K + K * K : 1;
-        sm.scal[4] = 0;
-        sm.lvl_start[0] = 0;
-        sm.lvl_start[1] = 1;
-        if (spec) {
-            sm.lvl_start[2] = 1 + K;
-            sm.lvl_start[3] = 1 + K + K * K;
-        }
         sm.parent[0] = -1;
         sm.cand[0] = 0;
         sm.depth[0] = 0;
@@ -778,9 +770,14 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             }
             __syncthreads();
         }
+        // (the bounds of the level being expanded and the end of the table are the same in every thread: no thread has to
+        // publish them, and a level costs three barriers -- two in the scan, one at its end)
+        int lv0 = spec ? 1 + K : 0, lv1 = spec ? 1 + K + K * K : 1;
         for (int d = spec ? 2 : 0; d < L; ++d) {
-            const int b0 = sm.lvl_start[d], b1 = sm.lvl_start[d + 1];
+            const int b0 = lv0, b1 = lv1;
             if (b1 == b0) break;
+            int lvl_end = ntot;
+            bool over = false;  // the node table is full
             if (d >= rows_done) {  // the edge rows of this depth: scored now, never if the expansion stops above it
                 int alive = 0;  // (nor if no node of the level can still have a selected child)
                 for (int x = b0 + tid; x < b1; x += TREE_THREADS) alive |= sm.nkey[x] >= theta ? 1 : 0;
@@ -798,7 +795,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 // one thread per (node, child), at a position that needs no atomic
                 const int total = (b1 - b0) * K;
                 if (ntot + total > p.ncap) {
-                    if (tid == 0) sm.scal[4] = 1;
+                    over = true;
                 } else {
                     for (int j = tid; j < total; j += TREE_THREADS) {
                         const int xi = j / K, r = j - xi * K, x = b0 + xi;
@@ -809,9 +806,9 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                         const int c = sm.ei[row + r], at = ntot + xi * K + c;  // (a full row: a child's slot is its rank)
                         sm.nkey[at] = oc < kx ? oc : kx;
                         sm.nS[at] = sc;
-                        sm.ninfo[at] = (uint32_t)x | ((uint32_t)c << 13) | ((uint32_t)(d + 1) << 18);
+                        sm.ninfo[at] = (uint32_t)x | ((uint32_t)c << 13) | ((uint32_t)(d + 1) << 18) | ((uint32_t)r << 24);
                     }
-                    if (tid == 0) sm.scal[3] = ntot + total;
+                    lvl_end = ntot + total;
                 }
             } else {
                 // The children that can still matter are a prefix of a node's sorted row (scores only fall along the
@@ -898,7 +895,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     break;
                   }
                     if (cur + total > p.ncap) {  // (uniform)
-                        if (tid == 0) sm.scal[4] = 1;
+                        over = true;
                         break;
                     }
                     for (int i = tid; i < total; i += TREE_THREADS) {
@@ -928,21 +925,22 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                         }
                         sm.nkey[at] = oc < kx ? oc : kx;
                         sm.nS[at] = sc;
-                        sm.ninfo[at] = (uint32_t)xo | ((uint32_t)c << 13) | ((uint32_t)(d + 1) << 18);
+                        sm.ninfo[at] = (uint32_t)xo | ((uint32_t)c << 13) | ((uint32_t)(d + 1) << 18) | ((uint32_t)r << 24);
                     }
                     cur += total;
-                    __syncthreads();  // the scan space is reused by the next chunk
+                    if (c0 + TREE_THREADS < b1) __syncthreads();  // the scan space is reused by the next chunk
                 }
-                if (tid == 0) sm.scal[3] = cur;
+                lvl_end = cur;
             }
-            const int any_grow = __syncthreads_or(grow);
-            const int nt = sm.scal[3];
-            if (sm.scal[4]) {
+            const int any_grow = __syncthreads_or(grow);  // (the level's nodes are in the table for every thread)
+            const int nt = lvl_end;
+            if (over) {
                 table_ok = false;
                 break;
             }
-            if (tid == 0) sm.lvl_start[d + 2] = nt;
             if (nt == ntot) break;  // nothing appended: no deeper level
+            lv0 = ntot;
+            lv1 = nt;
             ntot = nt;
             if (!any_grow) break;  // no node of the new level can have a child in the tree
             // theta only has to be a lower bound of its final value while the levels are built (it prunes), so
@@ -951,8 +949,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 sel_top = 0.0f + sm.es[0];  // the root's best child
                 theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);  // a lower bound
                 n_at_select = ntot;
+                __syncthreads();  // (its bins share the space of the next level's scan)
             }
-            __syncthreads();
         }
         __syncthreads();
         if (table_ok && ntot - 1 >= budget) {
@@ -985,6 +983,49 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 if (n_reach == budget) {  // (uniform)
                     cut = theta - 1u;
                     ordered = true;
+                } else if (n_reach > budget) {  // (uniform)
+                    // A few keys tie with the B-th largest.  Best-first takes prefixes of equal path score in the order
+                    // (shallower first, then the parent's place in its level, then the place in the parent's sorted row),
+                    // and a prefix only after its parent; among the tied nodes -- all in the table -- that is a short
+                    // simulation by one warp, a lane per tied node (up to 32 of them; more go to the sequential
+                    // expansion below).  The nodes it takes get a key above theta, and the tree is again a subset of the
+                    // table in table order.
+                    int* tlist = (int*)sm.hist;  // [32] table indices of the tied nodes, [32]: their number
+                    if (tid == 0) tlist[32] = 0;
+                    __syncthreads();
+                    for (int i = i0 > 1 ? i0 : 1; i < i1; ++i) {
+                        if (sm.nkey[i] == theta) {
+                            const int pos = atomicAdd(&tlist[32], 1);
+                            if (pos < 32) tlist[pos] = i;
+                        }
+                    }
+                    __syncthreads();
+                    const int nt = tlist[32];
+                    if (nt <= 32) {  // (uniform)
+                        if (warp == 0) {
+                            const int want = budget - (n_reach - nt);  // how many of the tied nodes belong to the tree
+                            const int me = lane < nt ? tlist[lane] : 0;
+                            const uint32_t info = lane < nt ? sm.ninfo[me] : 0u;
+                            const int par = (int)(info & 8191u);
+                            const uint32_t hi = lane < nt ? ord_from_float(sm.nS[me]) : 0u;
+                            const uint32_t lo = ((63u - ((info >> 18) & 63u)) << 18) | ((8191u - (uint32_t)par) << 5) |
+                                                (31u - ((info >> 24) & 31u));
+                            bool avail = lane < nt && sm.nkey[par] > theta;  // (else the parent is a tied node itself)
+                            bool picked = false;
+                            for (int step = 0; step < want; ++step) {
+                                const uint32_t bh = __reduce_max_sync(0xFFFFFFFFu, avail && !picked ? hi : 0u);
+                                const uint32_t bl = __reduce_max_sync(0xFFFFFFFFu, avail && !picked && hi == bh ? lo + 1u : 0u);
+                                if (bl == 0u) break;  // (nothing to take: cannot happen while want <= nt)
+                                const bool mine = avail && !picked && hi == bh && lo + 1u == bl;
+                                const int taken = __shfl_sync(0xFFFFFFFFu, me, __ffs(__ballot_sync(0xFFFFFFFFu, mine)) - 1);
+                                if (mine) picked = true;
+                                if (lane < nt && par == taken) avail = true;
+                            }
+                            if (picked) sm.nkey[me] = theta + 1u;
+                        }
+                        __syncthreads();
+                        ordered = true;
+                    }
                 }
             } else if (ntot - 1 < budget) {
                 ordered = true;  // fewer prefixes than the budget: all of them
@@ -1022,7 +1063,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 const uint32_t info = sm.ninfo[i];
                 sm.parent[n] = (int16_t)sm.nkey[info & 8191u];
                 sm.cand[n] = (uint8_t)((info >> 13) & 31u);
-                sm.depth[n] = (uint8_t)(info >> 18);
+                sm.depth[n] = (uint8_t)((info >> 18) & 63u);
                 sm.S[n] = sm.nS[i];
             }
             n_gt = total - 1;
