@@ -1183,7 +1183,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         }
     }
     }  // !ordered
-    __syncthreads();
+    if (!ordered) __syncthreads();  // (uniform; an ordered tree needs nothing from the block above)
 
     // ---- emission in level order -------------------------------------------------------------------------
     // Level order = depth ascending, then the parent's level-order index, then candidate rank.  Level by level:
@@ -1192,7 +1192,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     // The placement is a chain of short steps over at most nmax nodes: one warp runs it with warp-level
     // synchronisation only (a barrier of the whole CTA per step cost more than the steps), while the other warps
     // write the padding of the outputs, which depends on the node count alone.
-    const int n_nodes = sm.scal[1];
+    const int n_nodes = ordered ? n_gt + 1 : sm.scal[1];
     const int prefix = p.prefix_len[b];
     const size_t ob = (size_t)b * nmax;
     if (warp == 0 && !ordered) {
@@ -1262,7 +1262,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         const int z0 = ((n_nodes + 31) / 32) * 32;
         for (size_t k = (size_t)z0 * W + tid - 32; k < (size_t)nmax * W; k += TREE_THREADS - 32) o.d_mask[ob * W + k] = 0u;
     }
-    __syncthreads();
+    if (!ordered) __syncthreads();  // (the placement above; the padding is nobody's input)
     for (int n = tid; n < n_nodes; n += TREE_THREADS) {
         const int i = ordered ? n : sm.canon[n], d = sm.depth[n];
         const int par = n == 0 ? -1 : (ordered ? sm.parent[n] : sm.canon[sm.parent[n]]);
