@@ -391,6 +391,8 @@ struct __align__(16) EpiShared {  // private to one epilogue group
     uint16_t hthreads[NT];  // streaming threads whose maximum reaches T
     int nhits, ncand, nht, ovf;
     int fill_ninf;  // the threshold fell on -inf: the candidates are the finite elements plus the first -inf ones
+    int fill_tie;   // too many chunks reach the threshold T (bulk ties at T): the candidates are the elements above T
+                    // plus the first elements equal to T
     uint32_t Tv;
 };
 struct __align__(16) VpShared {
@@ -810,6 +812,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 if (ninf) Tv = kOrdNegInf + 1u;
                 if (lane == 0) {
                     es->fill_ninf = ninf ? 1 : 0;
+                    es->fill_tie = 0;
                     es->Tv = Tv;
                     es->nhits = 0;
                     es->nht = 0;
@@ -827,7 +830,11 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 if (x >= Tv && x != 0u) es->hthreads[atomicAdd(&es->nht, 1)] = (uint16_t)t;
             }
             epi_bar(grp);
-            {
+            // Te: what a chunk's maximum (and, below, an element) must reach.  T itself at first; if more chunks reach T
+            // than the list holds -- thousands of elements tie with T -- the scan is repeated for what lies above T, and
+            // the elements equal to T are taken in id order from the front of the segment further down.
+            uint32_t Te = Tv;
+            for (int mode = 0; mode < 2; ++mode) {  // (uniform)
                 // (listed thread, tile) pairs, four per thread at a time with their loads in flight together; the pair's
                 // thread comes from a multiplication (idx / ntiles for idx < 2^16 and ntiles < 2^16, exactly)
                 const int npairs = es->nht * sg.ntiles;
@@ -850,7 +857,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     }
 #pragma unroll
                     for (int u = 0; u < PU; ++u) {
-                        if (ord_from_bits(raw[u] << 16) >= Tv && base + u * kVpEpiThreads + etid < npairs && !stop) {
+                        if (ord_from_bits(raw[u] << 16) >= Te && base + u * kVpEpiThreads + etid < npairs && !stop) {
                             const int pos = atomicAdd(&es->nhits, 1);
                             if (pos >= kVpHitCap)
                                 stop = true;  // too many: the exact selection over the segment takes over
@@ -859,8 +866,16 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                         }
                     }
                 }
+                epi_bar(grp);
+                if (mode == 1 || !BF16 || es->fill_ninf || es->nhits <= kVpHitCap) break;  // (uniform)
+                epi_bar(grp);  // (everybody has read the count)
+                if (etid == 0) {
+                    es->nhits = 0;
+                    es->fill_tie = 1;
+                }
+                Te = Tv + 1u;
+                epi_bar(grp);
             }
-            epi_bar(grp);
             // (e) the 16-byte vectors of the hit chunks, re-read from global memory; elements >= T become keys.
             //     A thread issues its loads of a round before it uses any: under a saturated memory system one
             //     round trip costs microseconds.
@@ -893,7 +908,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     for (int u = 0; u < RU; ++u) {
                         if (offs[u] == 0xFFFFFFFFu) continue;
                         // (three of a hit chunk's four vectors hold nothing that reaches T: one test for the vector)
-                        if (vec_max_ord<BF16>(vv[u]) < Tv) continue;
+                        if (vec_max_ord<BF16>(vv[u]) < Te) continue;
                         const uint32_t wv[4] = {vv[u].x, vv[u].y, vv[u].z, vv[u].w};
 #pragma unroll
                         for (int j = 0; j < T::EPV; ++j) {
@@ -902,7 +917,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                                 xb = (j & 1) ? (wv[j >> 1] & 0xFFFF0000u) : (wv[j >> 1] << 16);
                             else
                                 xb = wv[j];
-                            if (ord_from_bits(xb) >= Tv && !full) {
+                            if (ord_from_bits(xb) >= Te && !full) {
                                 const int pos = atomicAdd(&es->ncand, 1);
                                 if (pos < kVpCandCap)
                                     es->cand[pos] = make_key(xb, (uint32_t)(sg.e_body0 + offs[u] / T::ESZ + j));
@@ -914,12 +929,16 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 }
             }
             epi_bar(grp);
-            if (es->fill_ninf) {  // (uniform)
+            if (es->fill_ninf || es->fill_tie) {  // (uniform)
                 if (ew == 0) {
+                    // (the same walk serves bulk ties at T: the first K elements equal to T, looked for in the segment's
+                    // first 2048 elements only -- where ties are that many they are found at once)
+                    const bool tie = es->fill_tie != 0;
+                    const uint32_t want_bits = tie ? bits_from_ord(Tv) : 0xFF800000u;
                     // the first K elements equal to -inf of the segment's body, in id order (the few elements before
                     // and after the body are candidates already); a segment that does not show K of them within
                     // its first 8192 elements goes to the exact selection instead
-                    constexpr int kScan = 8192;
+                    const int kScan = tie ? 2048 : 8192;
                     int found = 0, e0 = sg.e_body0;
                     for (; e0 < sg.e_tail0 && e0 - sg.e_body0 < kScan && found < p.K; e0 += 32) {
                         const int e = e0 + lane;
@@ -927,7 +946,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                         bool is = false;
                         if (e < sg.e_tail0) {
                             xb = __float_as_uint(load_elem_f32(rowp + (size_t)e * T::ESZ, BF16));
-                            is = xb == 0xFF800000u;
+                            is = xb == want_bits;
                         }
                         const uint32_t mk = __ballot_sync(0xFFFFFFFFu, is);
                         if (is && found + __popc(mk & ((1u << lane) - 1u)) < p.K) {
