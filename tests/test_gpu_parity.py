@@ -121,6 +121,33 @@ def test_vocab_pass_full_width_rows_with_bulk_ties(dtype):
     _vocab_case(z.to(torch.bfloat16) if dtype == "bf16" else z, K, dtype)
 
 
+@pytest.mark.parametrize("V", [151936, 40003])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_vocab_pass_bulk_ties_beside_larger_values(V, dtype):
+    """Thousands of elements tie with the K-th largest value while a few lie above it: the top-K are the larger
+    ones, wherever they are, then the tied ones of smallest id -- also when tied elements share a chunk with a larger
+    one, when only one tied element is wanted, when the tied value is negative, and when the tied elements do not
+    start at the front of the row."""
+    K, L = 32, 8
+    g = torch.Generator().manual_seed(V)
+    z = torch.zeros((2, L, V))
+    z[0, 0, torch.randint(0, V, (5,), generator=g)] = 4.0            # five winners anywhere, the rest ties at 0
+    z[0, 1, 5000] = 5.0                                               # a winner whose chunk is otherwise ties
+    z[0, 1, 17] = 2.5                                                 # ... and one among the first tied elements
+    idx = torch.randperm(V, generator=g)[:K - 1]
+    z[0, 2, idx] = 1.0 + torch.arange(K - 1).float() / 64             # K - 1 distinct winners: one tied element wanted
+    z[0, 3] = -7.5                                                    # ties at a negative value
+    z[0, 3, V - 3] = -7.0
+    z[0, 4, :3000] = -1.0 - torch.rand(3000, generator=g)             # the tied elements start behind 3000 lower ones
+    z[0, 4, V // 2] = 2.0
+    z[0, 5, torch.arange(0, V, 997)] = 3.0                            # more than K winners above the ties
+    z[0, 6, :10] = torch.arange(10).float()                           # winners and ties together at the front
+    z[0, 7] = torch.where(torch.rand(V, generator=g) < 0.5, 0.0, -0.5)  # two values, half each
+    z[0, 7, V - 1] = 0.25
+    z[1] = z[0].flip(0)
+    _vocab_case(z.to(torch.bfloat16) if dtype == "bf16" else z, K, dtype)
+
+
 @pytest.mark.parametrize("V,dtype", [(3, "bf16"), (6, "f32"), (14, "bf16"), (4099, "bf16"), (4097, "f32")])
 def test_vocab_pass_dominant_logit_outside_the_bulk_copies(V, dtype):
     """One logit 30 above the rest, placed where the 16-byte bulk copies do not reach (tiny rows, the ragged first
