@@ -934,7 +934,6 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     // (the same walk serves bulk ties at T: the first K elements equal to T, looked for in the segment's
                     // first 2048 elements only -- where ties are that many they are found at once)
                     const bool tie = es->fill_tie != 0;
-                    const uint32_t want_bits = tie ? bits_from_ord(Tv) : 0xFF800000u;
                     // the first K elements equal to -inf of the segment's body, in id order (the few elements before
                     // and after the body are candidates already); a segment that does not show K of them within
                     // its first 8192 elements goes to the exact selection instead
@@ -946,7 +945,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                         bool is = false;
                         if (e < sg.e_tail0) {
                             xb = __float_as_uint(load_elem_f32(rowp + (size_t)e * T::ESZ, BF16));
-                            is = xb == want_bits;
+                            is = tie ? ord_from_bits(xb) == Tv : xb == 0xFF800000u;  // (-0 and +0 are one value)
                         }
                         const uint32_t mk = __ballot_sync(0xFFFFFFFFu, is);
                         if (is && found + __popc(mk & ((1u << lane) - 1u)) < p.K) {

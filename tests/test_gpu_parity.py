@@ -146,6 +146,11 @@ def test_vocab_pass_bulk_ties_beside_larger_values(V, dtype):
     z[0, 7, V - 1] = 0.25
     z[1] = z[0].flip(0)
     _vocab_case(z.to(torch.bfloat16) if dtype == "bf16" else z, K, dtype)
+    # rows of +0 and -0 (one value, two bit patterns) under one winner: the tied elements are the first of either
+    zs = torch.zeros((1, L, V))
+    zs[0, :, 1::2] = -0.0
+    zs[0, :, 700] = 1.0
+    _vocab_case(zs.to(torch.bfloat16) if dtype == "bf16" else zs, K, dtype)
 
 
 @pytest.mark.parametrize("V,dtype", [(3, "bf16"), (6, "f32"), (14, "bf16"), (4099, "bf16"), (4097, "f32")])
