@@ -765,7 +765,24 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             ntot = 1 + K + K * K;
             if (ntot - 1 >= budget) {
                 sel_top = 0.0f + sm.es[0];  // the root's best child
-                theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);
+                // The threshold of levels 0 and 1 alone is loose: the best child of every level-1 node is a prefix too, and
+                // its key costs one look at the node's sorted row.  Those K^2 keys stand behind the table for the search
+                // (the level's real children overwrite them), which then gives a bound closer to the final one and a
+                // level 2 that appends a third of what it would.
+                int nsel = ntot;
+                if (L > 2 && rows_done > 2 && ntot + K * K <= p.ncap) {  // (uniform)
+                    for (int j = tid; j < K * K; j += TREE_THREADS) {
+                        const int x = 1 + K + j;
+                        const uint32_t kx = sm.nkey[x];
+                        const int cx = (int)((sm.ninfo[x] >> 13) & 31u);
+                        const uint32_t oc = ord_from_float(sm.nS[x] + sm.es[(2 * K + cx) * K + cx]);  // (entry 0: column cx)
+                        sm.nkey[ntot + j] = oc < kx ? oc : kx;
+                    }
+                    nsel = ntot + K * K;
+                    __syncthreads();
+                }
+                theta = cta_select_bucket(sm, sm.nkey, 1, nsel, budget, sel_top, sel, tid);
+                if (nsel != ntot) sel.valid = false;  // (the bucket counts keys that are not in the table)
                 n_at_select = ntot;
             }
             __syncthreads();
