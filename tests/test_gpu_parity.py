@@ -452,6 +452,44 @@ def test_round_with_thousands_of_equal_path_scores(budget):
     compare_accept(oracle, gi, g, w, out, gpu)
 
 
+@pytest.mark.parametrize("beta", [0.0, 0.25])
+def test_round_every_cut_through_small_groups_of_tied_prefixes(beta):
+    """The same sequence under every fixed budget from 1 to 96: its logits sit on a grid of 1/2 with pairs and triples of
+    equal values among the best candidates of every position, and exact powers of two as probabilities' ratios, so
+    prefixes tie in twos to tens -- siblings, cousins under different parents, a parent with the chain below it -- and
+    every budget cuts such a group somewhere.  A few tied keys at the threshold are resolved among the tied nodes of
+    the table (more than 32 by the sequential expansion): either way the tree must be the oracle's, node for node."""
+    nb = 96
+    w = gi.small(batch=nb, L=5, V=64, K=8, budget_min=1, budget_max=nb, budget_step=1, fixed_budget=1, beta=beta, m=8,
+                 seed=5)
+    g = _graft(w)
+    tb, saba_kw, keep = _setup(w, g)
+    if beta != 0.0:  # equal rows for tokens that share a logit, so that their edge scores tie as well
+        for t in (tb["P"], tb["C"]):
+            t[1::2] = t[0::2][: t[1::2].shape[0]]
+        keep = [tb["P"].cuda(), tb["C"].cuda(), tb["u"].cuda()]
+        g.set_tdes_tables(keep[0], keep[1], keep[2], tb["s"])
+    x = gi.batch_inputs(w)
+    row = torch.full((w.L, w.V), -20.0)
+    for d in range(w.L):
+        vals = [4.0, 4.0, 3.5, 3.5, 3.5, 3.0, 2.5, 2.5][:: 1 if d % 2 == 0 else -1]
+        row[d, 2 * d: 2 * d + 8] = torch.tensor(vals)
+    x["logits"][:] = row.to(x["logits"].dtype)
+    x["root_token"][:] = x["root_token"][0]
+    x["hist"][:] = x["hist"][0]
+    x["prefix_len"][:] = x["prefix_len"][0]
+    x["hidden"][:] = x["hidden"][0]
+    x["fixed_budget"] = torch.arange(1, nb + 1, dtype=torch.int32)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    assert stats["excused_budget"] == 0 and stats["excused_tree"] == 0, stats
+    for k in ("n_nodes", "token", "parent", "depth", "mask", "status"):
+        assert np.array_equal(gpu[k], orc[k]), k
+    assert gpu["n_nodes"].tolist() == [b + 1 for b in range(1, nb + 1)]
+    compare_accept(oracle, gi, g, w, out, gpu)
+
+
 @pytest.mark.parametrize("budget", [20, 50, 150])
 def test_round_with_equal_scores_across_depths_and_masked_tokens(budget):
     """Sequence 0: below a uniform first position every later position has one token of probability 1 to fp32
