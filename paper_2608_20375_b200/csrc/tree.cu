@@ -531,9 +531,10 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 // Every thread calls this; the copies of one row form one group per thread.
-__device__ __forceinline__ void lazy_issue_gather(const TreeParams& p, const TreeSmem& sm, int j, int root_token, int tid) {
+__device__ __forceinline__ void lazy_issue_gather(const TreeParams& p, const TreeSmem& sm, int j, int root_token, int tid,
+                                                  const int K, const int m) {
     if (j >= p.L || lazy_neutral(p, j)) return;
-    const int K = p.K, m = p.m, ld = m + 4, q4 = m / 4, n_par = j == 0 ? 1 : K;
+    const int ld = m + 4, q4 = m / 4, n_par = j == 0 ? 1 : K;
     const int warp = tid >> 5, lane = tid & 31;
     for (int r = warp; r <= n_par + K; r += TREE_THREADS / 32) {  // a warp per table row, a lane per 16 bytes
         const float* src;
@@ -554,8 +555,8 @@ __device__ __forceinline__ void lazy_issue_gather(const TreeParams& p, const Tre
 // Every thread of the CTA calls this.
 // `inflight` is the depth whose table rows are on their way (or -1).
 __device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSmem& sm, int j, int root_token, int tid,
-                                               int& inflight) {
-    const int K = p.K, m = p.m, n_par = j == 0 ? 1 : K;
+                                               int& inflight, const int K, const int m) {
+    const int n_par = j == 0 ? 1 : K;
     const int warp = tid >> 5, lane = tid & 31;
     float* es = sm.es + (size_t)j * K * K;
     uint8_t* ei = sm.ei + (size_t)j * K * K;
@@ -569,14 +570,14 @@ __device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSm
         __syncthreads();
         return;
     }
-    if (inflight != j) lazy_issue_gather(p, sm, j, root_token, tid);
+    if (inflight != j) lazy_issue_gather(p, sm, j, root_token, tid, K, m);
     cp_async_wait_all();
     __syncthreads();
     float* part = (float*)sm.hist;                // [K][K] dot products (the histogram space is idle here)
     uint32_t* wsc = sm.hist + 1024 + warp * 32;   // [32] per warp
     if (warp < 8) edge_dots<true>(sm.gP, sm.gC, sm.gU, m, K, n_par, part, warp, lane);
     __syncthreads();
-    lazy_issue_gather(p, sm, j + 1, root_token, tid);  // the table rows of this depth are no longer read
+    lazy_issue_gather(p, sm, j + 1, root_token, tid, K, m);  // the table rows of this depth are no longer read
     inflight = j + 1;
     const float inv_K = 1.0f / (float)K;
     for (int par = warp; par < K; par += TREE_THREADS / 32) {  // one warp per parent
@@ -592,12 +593,16 @@ __device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSm
     __syncthreads();
 }
 
+// KC, MC: the number of candidates per position and the width of the TDES tables as compile-time constants (the
+// configured workloads' K = 32, m = 128: every index computation with K becomes a shift), or 0: taken from the parameters
+template <int KC, int MC>
 __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int K = KC ? KC : p.K, p_m = MC ? MC : p.m;
     TreeSmem sm;
-    tree_smem_layout(p.L, p.K, p.nmax, p.ncap, p.lazy_m, &sm, smem_raw);
+    tree_smem_layout(p.L, K, p.nmax, p.ncap, p.lazy_m, &sm, smem_raw);
     const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int L = p.L, K = p.K, nmax = p.nmax, W = p.W;
+    const int L = p.L, nmax = p.nmax, W = p.W;
     const graft_tree_out& o = p.out;
     pdl_launch_dependents();  // an acceptance walk queued behind this kernel may move in; it waits for this grid
     pdl_wait();  // candidates, cosines and edge rows come from the kernels ahead in the stream
@@ -659,7 +664,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         }
         if (rows_pre == 0) {  // the table rows of depth 0 arrive while the budget is worked out
             __syncthreads();
-            lazy_issue_gather(p, sm, 0, root, tid);
+            lazy_issue_gather(p, sm, 0, root, tid, K, p_m);
             inflight = 0;
         }
     }
@@ -799,7 +804,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 int alive = 0;  // (nor if no node of the level can still have a selected child)
                 for (int x = b0 + tid; x < b1; x += TREE_THREADS) alive |= sm.nkey[x] >= theta ? 1 : 0;
                 if (!__syncthreads_or(alive)) break;
-                lazy_score_row(p, sm, d, root, tid, inflight);
+                lazy_score_row(p, sm, d, root, tid, inflight, K, p_m);
                 rows_done = d + 1;
             }
             // grow: can a node appended here have a child that reaches theta?  (Its best child stands first in its sorted
@@ -1108,7 +1113,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         }
     }
     if (p.lazy && !table_ok && budget > 0) {  // the sequential fall-back may reach any depth
-        for (; rows_done < L; ++rows_done) lazy_score_row(p, sm, rows_done, root, tid, inflight);
+        for (; rows_done < L; ++rows_done) lazy_score_row(p, sm, rows_done, root, tid, inflight, K, p_m);
     }
     if (!table_ok && tid == 0) sm.ent[0] = budget > 0 ? pack_entry(0.0f + sm.es[0], 1, 0, 0, sm.ei[0]) : 0ull;
     if (ordered) {  // (uniform) the tree is complete and in level order
@@ -1450,7 +1455,9 @@ size_t tree_smem_bytes(const graft_config& cfg) {
 }
 
 cudaError_t tree_configure(const graft_config& cfg) {
-    return cudaFuncSetAttribute(tree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tree_smem_bytes(cfg));
+    cudaError_t e = cudaFuncSetAttribute(tree_kernel<0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tree_smem_bytes(cfg));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(tree_kernel<32, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tree_smem_bytes(cfg));
 }
 
 cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
@@ -1496,7 +1503,9 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     p.use_saba = d_fixed_budget == nullptr;
     p.saba = ctx->saba;
     p.saba_pre = d_saba_pre;
-    const cudaError_t e = launch_pdl(tree_kernel, dim3(batch), dim3(TREE_THREADS), tree_smem_bytes(cfg), st, p);
+    const bool common = cfg.K == 32 && cfg.m == 128;
+    const cudaError_t e = launch_pdl(common ? tree_kernel<32, 128> : tree_kernel<0, 0>, dim3(batch), dim3(TREE_THREADS),
+                                     tree_smem_bytes(cfg), st, p);
     ctx->launches += 1;
     return e != cudaSuccess ? e : cudaGetLastError();
 }
