@@ -104,14 +104,15 @@ struct EdgeParams {
 };
 
 // WRITE_EDGE: also write the unsorted scores (the caller asked for the array); the tree kernel reads only the sorted rows
-template <bool WRITE_EDGE>
+// KC, MC: K and m as compile-time constants (the configured workloads' 32 and 128), or 0: taken from the parameters
+template <bool WRITE_EDGE, int KC, int MC>
 __global__ void __launch_bounds__(256, 4) tdes_edges_kernel(const EdgeParams p) {
     extern __shared__ __align__(16) float smem[];
     pdl_launch_dependents();  // the tree kernel may move in as SMs free up; it waits for this grid before it reads
     pdl_wait();               // the candidates come from the vocab pass
     const int b = blockIdx.x / p.rows_all, j = blockIdx.x % p.rows_all;
     if (j >= p.rows && !deep_tree_likely(p.topk_lp + (size_t)b * p.L * p.K, p.L, p.K)) return;  // (uniform)
-    const int K = p.K, m = p.m, ld = m + 4;  // padded row: 16-byte aligned, conflict-free float4 reads
+    const int K = KC ? KC : p.K, m = MC ? MC : p.m, ld = m + 4;  // padded row: 16-byte aligned, conflict-free float4 reads
     float* sP = smem;                        // [K][ld]  parent rows + u_d
     float* sC = smem + (size_t)kMaxK * ld;   // [K][ld]  child rows + u_d
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -217,11 +218,13 @@ size_t tdes_edges_smem(const graft_config& cfg) {
 }
 
 cudaError_t tdes_edges_configure(const graft_config& cfg) {
-    cudaError_t e = cudaFuncSetAttribute(tdes_edges_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)tdes_edges_smem(cfg));
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(tdes_edges_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)tdes_edges_smem(cfg));
+    const int bytes = (int)tdes_edges_smem(cfg);
+    cudaError_t e = cudaFuncSetAttribute(tdes_edges_kernel<true, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tdes_edges_kernel<false, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tdes_edges_kernel<false, 32, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return e;
 }
 
 cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
@@ -259,8 +262,10 @@ cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_i
     p.bmax = cfg.budget_max;
     p.bstep = cfg.budget_step;
     p.saba = ctx->saba;
-    const cudaError_t e = launch_pdl(d_edge ? tdes_edges_kernel<true> : tdes_edges_kernel<false>, dim3(batch * p.rows_all),
-                                     dim3(256), tdes_edges_smem(cfg), st, p);
+    const bool common = cfg.K == 32 && cfg.m == 128;
+    const cudaError_t e = launch_pdl(d_edge ? tdes_edges_kernel<true, 0, 0>
+                                            : (common ? tdes_edges_kernel<false, 32, 128> : tdes_edges_kernel<false, 0, 0>),
+                                     dim3(batch * p.rows_all), dim3(256), tdes_edges_smem(cfg), st, p);
     ctx->launches += 1;
     return e != cudaSuccess ? e : cudaGetLastError();
 }
