@@ -595,10 +595,13 @@ __device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSm
 
 // KC, MC: the number of candidates per position and the width of the TDES tables as compile-time constants (the
 // configured workloads' K = 32, m = 128: every index computation with K becomes a shift), or 0: taken from the parameters
-template <int KC, int MC>
+// FAST: the usual round is known at compile time as well -- the budget comes from the edge-score kernel (no SABA
+// arithmetic in this instance) and deeper rows are scored on demand
+template <int KC, int MC, bool FAST>
 __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int K = KC ? KC : p.K, p_m = MC ? MC : p.m;
+    const bool p_lazy = FAST ? true : p.lazy != 0;
     TreeSmem sm;
     tree_smem_layout(p.L, K, p.nmax, p.ncap, p.lazy_m, &sm, smem_raw);
     const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -622,10 +625,10 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     pre_r.budget = 0;
     pre_r.status = 0;
     pre_r.state[0] = pre_r.state[1] = pre_r.state[2] = pre_r.state[3] = 0.f;
-    if (p.saba_pre && tid == 0) pre_r = p.saba_pre[b];
+    if ((FAST || p.saba_pre) && tid == 0) pre_r = p.saba_pre[b];
     int32_t lz_tok = 0;
     float lz_lp = 0.f;
-    if (p.lazy && tid < L * K) {  // (L K <= 1024: a thread per candidate)
+    if (p_lazy && tid < L * K) {  // (L K <= 1024: a thread per candidate)
         lz_tok = p.topk_id[(size_t)b * L * K + tid];
         lz_lp = p.topk_lp[(size_t)b * L * K + tid];
     }
@@ -657,7 +660,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             sm.ei[i] = p.eidx[seq_e + i];
         }
     }
-    if (p.lazy) {  // the candidates of every depth, for the rows that may have to be scored here
+    if (p_lazy) {  // the candidates of every depth, for the rows that may have to be scored here
         if (tid < L * K) {
             sm.tokid[tid] = lz_tok;
             sm.lpv[tid] = lz_lp;
@@ -678,7 +681,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         rows_done = L;
     }
     // adjacent-position cosines r_d = cos(h_d, h_{d+1}) (Eq. 15): written by the vocab pass
-    if (p.use_saba && !p.saba_pre && tid < L - 1) sm.cosv[tid] = p.cos_pre[(size_t)b * L + tid];
+    if (!FAST && p.use_saba && !p.saba_pre && tid < L - 1) sm.cosv[tid] = p.cos_pre[(size_t)b * L + tid];
     __syncthreads();
     // While warp 0 works out the budget, the other warps expand levels 0 and 1 in full (1 + K + K^2 nodes), which
     // needs no budget: with fewer than B nodes in the table every child is appended anyway, and if B is smaller
@@ -714,7 +717,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     }
     if (warp == 0) {  // status and budget: from the edge-score kernel if it ran ahead, else worked out here
         SabaResult r;
-        if (p.saba_pre)
+        if (FAST || p.saba_pre)
             r = pre_r;  // (lane 0's copy is the one used below)
         else
             r = saba_warp(p.saba, p.bmin, p.bmax, p.bstep, L, K, p.row_status + (size_t)b * L, p.vp_err,
@@ -1112,7 +1115,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             }
         }
     }
-    if (p.lazy && !table_ok && budget > 0) {  // the sequential fall-back may reach any depth
+    if (p_lazy && !table_ok && budget > 0) {  // the sequential fall-back may reach any depth
         for (; rows_done < L; ++rows_done) lazy_score_row(p, sm, rows_done, root, tid, inflight, K, p_m);
     }
     if (!table_ok && tid == 0) sm.ent[0] = budget > 0 ? pack_entry(0.0f + sm.es[0], 1, 0, 0, sm.ei[0]) : 0ull;
@@ -1290,7 +1293,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
         const int par = n == 0 ? -1 : (ordered ? sm.parent[n] : sm.canon[sm.parent[n]]);
         sm.cparent[i] = (int16_t)par;
         o.d_token[ob + i] = n == 0 ? root
-                                   : (p.lazy ? sm.tokid[(d - 1) * K + sm.cand[n]]  // (staged in the prologue)
+                                   : (p_lazy ? sm.tokid[(d - 1) * K + sm.cand[n]]  // (staged in the prologue)
                                              : p.topk_id[((size_t)b * L + d - 1) * K + sm.cand[n]]);
         o.d_parent[ob + i] = par;
         o.d_depth[ob + i] = d;
@@ -1324,7 +1327,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             __syncwarp();
         }
     }
-    if (p.lazy) cp_async_wait_all();  // table rows fetched ahead for a depth that was never scored
+    if (p_lazy) cp_async_wait_all();  // table rows fetched ahead for a depth that was never scored
     if (tid == 0) {
         o.d_n_nodes[b] = n_nodes;
         o.d_budget[b] = sm.scal[0];
@@ -1455,9 +1458,9 @@ size_t tree_smem_bytes(const graft_config& cfg) {
 }
 
 cudaError_t tree_configure(const graft_config& cfg) {
-    cudaError_t e = cudaFuncSetAttribute(tree_kernel<0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tree_smem_bytes(cfg));
+    cudaError_t e = cudaFuncSetAttribute(tree_kernel<0, 0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tree_smem_bytes(cfg));
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(tree_kernel<32, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tree_smem_bytes(cfg));
+    return cudaFuncSetAttribute(tree_kernel<32, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tree_smem_bytes(cfg));
 }
 
 cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
@@ -1503,8 +1506,8 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     p.use_saba = d_fixed_budget == nullptr;
     p.saba = ctx->saba;
     p.saba_pre = d_saba_pre;
-    const bool common = cfg.K == 32 && cfg.m == 128;
-    const cudaError_t e = launch_pdl(common ? tree_kernel<32, 128> : tree_kernel<0, 0>, dim3(batch), dim3(TREE_THREADS),
+    const bool common = cfg.K == 32 && cfg.m == 128 && p.lazy && p.saba_pre != nullptr;
+    const cudaError_t e = launch_pdl(common ? tree_kernel<32, 128, true> : tree_kernel<0, 0, false>, dim3(batch), dim3(TREE_THREADS),
                                      tree_smem_bytes(cfg), st, p);
     ctx->launches += 1;
     return e != cudaSuccess ? e : cudaGetLastError();
