@@ -224,6 +224,10 @@ cudaError_t tdes_edges_configure(const graft_config& cfg) {
         e = cudaFuncSetAttribute(tdes_edges_kernel<false, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(tdes_edges_kernel<false, 32, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tdes_edges_kernel<false, 16, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tdes_edges_kernel<false, 8, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     return e;
 }
 
@@ -262,10 +266,13 @@ cudaError_t tdes_edges_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_i
     p.bmax = cfg.budget_max;
     p.bstep = cfg.budget_step;
     p.saba = ctx->saba;
-    const bool common = cfg.K == 32 && cfg.m == 128;
-    const cudaError_t e = launch_pdl(d_edge ? tdes_edges_kernel<true, 0, 0>
-                                            : (common ? tdes_edges_kernel<false, 32, 128> : tdes_edges_kernel<false, 0, 0>),
-                                     dim3(batch * p.rows_all), dim3(256), tdes_edges_smem(cfg), st, p);
+    void (*kern)(const EdgeParams) = d_edge ? tdes_edges_kernel<true, 0, 0> : tdes_edges_kernel<false, 0, 0>;
+    if (!d_edge && cfg.m == 128) {  // K and m known at compile time
+        if (cfg.K == 32) kern = tdes_edges_kernel<false, 32, 128>;
+        if (cfg.K == 16) kern = tdes_edges_kernel<false, 16, 128>;
+        if (cfg.K == 8) kern = tdes_edges_kernel<false, 8, 128>;
+    }
+    const cudaError_t e = launch_pdl(kern, dim3(batch * p.rows_all), dim3(256), tdes_edges_smem(cfg), st, p);
     ctx->launches += 1;
     return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -1458,9 +1458,12 @@ size_t tree_smem_bytes(const graft_config& cfg) {
 }
 
 cudaError_t tree_configure(const graft_config& cfg) {
-    cudaError_t e = cudaFuncSetAttribute(tree_kernel<0, 0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tree_smem_bytes(cfg));
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(tree_kernel<32, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tree_smem_bytes(cfg));
+    const int bytes = (int)tree_smem_bytes(cfg);
+    cudaError_t e = cudaFuncSetAttribute(tree_kernel<0, 0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<32, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<16, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<8, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return e;
 }
 
 cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, const float* d_topk_lp,
@@ -1506,9 +1509,14 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     p.use_saba = d_fixed_budget == nullptr;
     p.saba = ctx->saba;
     p.saba_pre = d_saba_pre;
-    const bool common = cfg.K == 32 && cfg.m == 128 && p.lazy && p.saba_pre != nullptr;
-    const cudaError_t e = launch_pdl(common ? tree_kernel<32, 128, true> : tree_kernel<0, 0, false>, dim3(batch), dim3(TREE_THREADS),
-                                     tree_smem_bytes(cfg), st, p);
+    // the instances with K and m known at compile time serve the usual round (the budget from the edge-score kernel,
+    // deeper rows on demand)
+    const bool usual = cfg.m == 128 && p.lazy && p.saba_pre != nullptr;
+    void (*kern)(const TreeParams) = tree_kernel<0, 0, false>;
+    if (usual && cfg.K == 32) kern = tree_kernel<32, 128, true>;
+    if (usual && cfg.K == 16) kern = tree_kernel<16, 128, true>;
+    if (usual && cfg.K == 8) kern = tree_kernel<8, 128, true>;
+    const cudaError_t e = launch_pdl(kern, dim3(batch), dim3(TREE_THREADS), tree_smem_bytes(cfg), st, p);
     ctx->launches += 1;
     return e != cudaSuccess ? e : cudaGetLastError();
 }
