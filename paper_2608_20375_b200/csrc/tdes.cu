@@ -110,7 +110,18 @@ __global__ void __launch_bounds__(256, 4) tdes_edges_kernel(const EdgeParams p) 
     extern __shared__ __align__(16) float smem[];
     pdl_launch_dependents();  // the tree kernel may move in as SMs free up; it waits for this grid before it reads
     pdl_wait();               // the candidates come from the vocab pass
-    const int b = blockIdx.x / p.rows_all, j = blockIdx.x % p.rows_all;
+    // the depths scored for every sequence come first in the grid, the depths that only deep trees need behind them: the
+    // CTAs of the latter mostly exit at once and should not take the places of CTAs with work
+    const int n_all = (int)gridDim.x / p.rows_all * p.rows;  // units that every sequence needs
+    int b, j;
+    if ((int)blockIdx.x < n_all) {
+        b = (int)blockIdx.x / p.rows;
+        j = (int)blockIdx.x - b * p.rows;
+    } else {
+        const int r = (int)blockIdx.x - n_all, nd = p.rows_all - p.rows;
+        b = r / nd;
+        j = p.rows + (r - b * nd);
+    }
     if (j >= p.rows && !deep_tree_likely(p.topk_lp + (size_t)b * p.L * p.K, p.L, p.K)) return;  // (uniform)
     const int K = KC ? KC : p.K, m = MC ? MC : p.m, ld = m + 4;  // padded row: 16-byte aligned, conflict-free float4 reads
     float* sP = smem;                        // [K][ld]  parent rows + u_d
