@@ -597,15 +597,15 @@ __device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSm
 // configured workloads' K = 32, m = 128: every index computation with K becomes a shift), or 0: taken from the parameters
 // FAST: the usual round is known at compile time as well -- the budget comes from the edge-score kernel (no SABA
 // arithmetic in this instance) and deeper rows are scored on demand
-template <int KC, int MC, bool FAST>
+template <int KC, int MC, bool FAST, int NMAXC = 0>
 __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int K = KC ? KC : p.K, p_m = MC ? MC : p.m;
     const bool p_lazy = FAST ? true : p.lazy != 0;
     TreeSmem sm;
-    tree_smem_layout(p.L, K, p.nmax, p.ncap, p.lazy_m, &sm, smem_raw);
+    tree_smem_layout(p.L, K, NMAXC ? NMAXC : p.nmax, p.ncap, p.lazy_m, &sm, smem_raw);
     const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int L = p.L, nmax = p.nmax, W = p.W;
+    const int L = p.L, nmax = NMAXC ? NMAXC : p.nmax, W = NMAXC ? (NMAXC + 31) / 32 : p.W;
     const graft_tree_out& o = p.out;
     pdl_launch_dependents();  // an acceptance walk queued behind this kernel may move in; it waits for this grid
     pdl_wait();  // candidates, cosines and edge rows come from the kernels ahead in the stream
@@ -1461,6 +1461,7 @@ cudaError_t tree_configure(const graft_config& cfg) {
     const int bytes = (int)tree_smem_bytes(cfg);
     cudaError_t e = cudaFuncSetAttribute(tree_kernel<0, 0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<32, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<32, 128, true, 513>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<16, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<8, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     return e;
@@ -1513,7 +1514,7 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     // deeper rows on demand)
     const bool usual = cfg.m == 128 && p.lazy && p.saba_pre != nullptr;
     void (*kern)(const TreeParams) = tree_kernel<0, 0, false>;
-    if (usual && cfg.K == 32) kern = tree_kernel<32, 128, true>;
+    if (usual && cfg.K == 32) kern = ctx->nmax == 513 ? tree_kernel<32, 128, true, 513> : tree_kernel<32, 128, true>;
     if (usual && cfg.K == 16) kern = tree_kernel<16, 128, true>;
     if (usual && cfg.K == 8) kern = tree_kernel<8, 128, true>;
     const cudaError_t e = launch_pdl(kern, dim3(batch), dim3(TREE_THREADS), tree_smem_bytes(cfg), st, p);
