@@ -603,7 +603,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     const int K = KC ? KC : p.K, p_m = MC ? MC : p.m;
     const bool p_lazy = FAST ? true : p.lazy != 0;
     TreeSmem sm;
-    tree_smem_layout(p.L, K, NMAXC ? NMAXC : p.nmax, p.ncap, p.lazy_m, &sm, smem_raw);
+    const int ncap = NMAXC ? 6144 : p.ncap;  // (the instance with the outputs' size known is used at full capacity only)
+    tree_smem_layout(p.L, K, NMAXC ? NMAXC : p.nmax, ncap, p.lazy_m, &sm, smem_raw);
     const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int L = p.L, nmax = NMAXC ? NMAXC : p.nmax, W = NMAXC ? (NMAXC + 31) / 32 : p.W;
     const graft_tree_out& o = p.out;
@@ -686,7 +687,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     // While warp 0 works out the budget, the other warps expand levels 0 and 1 in full (1 + K + K^2 nodes), which
     // needs no budget: with fewer than B nodes in the table every child is appended anyway, and if B is smaller
     // than that the extra nodes only fall below the threshold found afterwards.
-    const bool spec = bulk && rows_pre >= 2 && L >= 2 && 1 + K + K * K <= p.ncap;
+    const bool spec = bulk && rows_pre >= 2 && L >= 2 && 1 + K + K * K <= ncap;
     if (spec && warp >= 1) {
         mbar_wait_bounded(smem_u32(&rows_bar), 0, &rows_abort);
         const int t1 = tid - 32, nth = TREE_THREADS - 32;
@@ -778,7 +779,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 // (the level's real children overwrite them), which then gives a bound closer to the final one and a
                 // level 2 that appends a third of what it would.
                 int nsel = ntot;
-                if (L > 2 && rows_done > 2 && ntot + K * K <= p.ncap) {  // (uniform)
+                if (L > 2 && rows_done > 2 && ntot + K * K <= ncap) {  // (uniform)
                     for (int j = tid; j < K * K; j += TREE_THREADS) {
                         const int x = 1 + K + j;
                         const uint32_t kx = sm.nkey[x];
@@ -819,7 +820,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                 // no threshold yet (fewer than B nodes so far): every child of every node of the level is appended,
                 // one thread per (node, child), at a position that needs no atomic
                 const int total = (b1 - b0) * K;
-                if (ntot + total > p.ncap) {
+                if (ntot + total > ncap) {
                     over = true;
                 } else {
                     for (int j = tid; j < total; j += TREE_THREADS) {
@@ -912,14 +913,14 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     total = __shfl_sync(0xFFFFFFFFu, wincl, 31);
                     pre[tid] = __shfl_sync(0xFFFFFFFFu, wincl - wt, warp) + incl;
                     __syncthreads();
-                    if (attempt == 0 && total >= budget && (total > flood || cur + total > p.ncap)) {  // (uniform) the search below uses the scan's space: count again
+                    if (attempt == 0 && total >= budget && (total > flood || cur + total > ncap)) {  // (uniform) the search below uses the scan's space: count again
                         const uint32_t tl = cta_kth_largest_of_children(sm, cnt, kx, sx, row, cx, K, budget, theta, tid);
                         theta = tl > theta ? tl : theta;
                         continue;
                     }
                     break;
                   }
-                    if (cur + total > p.ncap) {  // (uniform)
+                    if (cur + total > ncap) {  // (uniform)
                         over = true;
                         break;
                     }
@@ -1305,7 +1306,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     // which are contiguous in the output, with coalesced writes.  Padding rows are zero-filled directly.
     {
         const size_t stage_off = (((size_t)nmax * 2 + 15) & ~(size_t)15) + (((size_t)nmax * 4 + 15) & ~(size_t)15);
-        const size_t region = (size_t)p.ncap * 12 > stage_off + (size_t)8 * 32 * W * 4 ? (size_t)p.ncap * 12
+        const size_t region = (size_t)ncap * 12 > stage_off + (size_t)8 * 32 * W * 4 ? (size_t)ncap * 12
                                                                                          : stage_off + (size_t)8 * 32 * W * 4;
         int mw = (int)((region - stage_off) / ((size_t)32 * W * 4));
         mw = mw > TREE_THREADS / 32 ? TREE_THREADS / 32 : mw;
@@ -1514,7 +1515,7 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     // deeper rows on demand)
     const bool usual = cfg.m == 128 && p.lazy && p.saba_pre != nullptr;
     void (*kern)(const TreeParams) = tree_kernel<0, 0, false>;
-    if (usual && cfg.K == 32) kern = ctx->nmax == 513 ? tree_kernel<32, 128, true, 513> : tree_kernel<32, 128, true>;
+    if (usual && cfg.K == 32) kern = (ctx->nmax == 513 && p.ncap == 6144) ? tree_kernel<32, 128, true, 513> : tree_kernel<32, 128, true>;
     if (usual && cfg.K == 16) kern = tree_kernel<16, 128, true>;
     if (usual && cfg.K == 8) kern = tree_kernel<8, 128, true>;
     const cudaError_t e = launch_pdl(kern, dim3(batch), dim3(TREE_THREADS), tree_smem_bytes(cfg), st, p);
