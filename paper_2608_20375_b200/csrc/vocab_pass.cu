@@ -457,11 +457,11 @@ __device__ __forceinline__ uint32_t vec_max_ord(const uint4& x) {
 // When the buffer fills up, the best K are kept and the filter rises.
 template <bool BF16>
 __device__ int warp_fallback_select(EpiShared* sh, const VpParams& p, const Seg& sg,
-                                    const typename VT<BF16>::cm_t* cmx, int lane) {
+                                    const typename VT<BF16>::cm_t* cmx, int lane, uint64_t thr) {
     using T = VT<BF16>;
     const int K = p.K;
     const char* rowp = p.logits + (size_t)sg.row * p.V * T::ESZ;
-    uint64_t thr = 0;  // keys must beat this one
+    // thr: keys must beat this one (on entry: what the threshold T of the fast path rules out, or 0)
     int n = 0, ovf = 0;
     // ranking n keys against each other costs n^2 / 32 steps per lane: the buffer is cut back to its best K well
     // before it is full (224 more keys at a time)
@@ -977,7 +977,10 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     if (i < ncand && (etid & 1) == 0 && rank < p.K) es->outk[rank] = key;
                 }
             } else if (ew == 0) {
-                nk = warp_fallback_select<BF16>(es, p, sg, cmx, lane);
+                // (T is a lower bound of the K-th largest element: the filter starts there, not at nothing -- a row sorted
+                // in ascending order would otherwise send every element through the buffer; with the threshold moved up
+                // from -inf, elements equal to -inf may be among the K best and nothing is ruled out)
+                nk = warp_fallback_select<BF16>(es, p, sg, cmx, lane, es->fill_ninf ? 0ull : ((uint64_t)Tv << 32) - 1ull);
             }
             epi_bar(grp);
             if (ew != 0) continue;
