@@ -464,8 +464,8 @@ __device__ int warp_fallback_select(EpiShared* sh, const VpParams& p, const Seg&
     // thr: keys must beat this one (on entry: what the threshold T of the fast path rules out, or 0)
     int n = 0, ovf = 0;
     // ranking n keys against each other costs n^2 / 32 steps per lane: the buffer is cut back to its best K well
-    // before it is full (224 more keys at a time)
-    constexpr int kFallbackFill = 256 - 32;
+    // before it is full (96 more keys at a time)
+    constexpr int kFallbackFill = 128 - 32;
     auto shrink = [&]() {  // keep the best K of the buffer
         if (n > K) {
             warp_select_topk(sh, n, K, lane);
@@ -959,7 +959,10 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 epi_bar(grp);
             }
             // (f) exact top-K of the candidates by rank counting (keys are distinct, so ranks are a permutation)
-            const bool overflow = es->ovf != 0 || es->ncand > kVpCandCap;
+            // (ranking n candidates costs n^2 compares shared by 128 threads: beyond 512 -- rows whose large elements sit
+            // side by side, such as sorted rows, fill every chunk that reaches T with candidates -- the exact selection
+            // with its rising filter is the faster way)
+            const bool overflow = es->ovf != 0 || es->ncand > kVpRankCap;
             const int ncand = es->ncand < kVpCandCap ? es->ncand : kVpCandCap;
             int nk = ncand < p.K ? ncand : p.K;
             if (!overflow) {

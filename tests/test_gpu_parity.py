@@ -153,6 +153,28 @@ def test_vocab_pass_bulk_ties_beside_larger_values(V, dtype):
     _vocab_case(zs.to(torch.bfloat16) if dtype == "bf16" else zs, K, dtype)
 
 
+@pytest.mark.parametrize("V,dtype", [(151936, "bf16"), (40003, "bf16"), (40003, "f32")])
+def test_vocab_pass_sorted_rows(V, dtype):
+    """Rows in ascending and descending order (distinct values, values that tie in blocks after rounding to bf16, a
+    sorted half beside an ordinary one): the large elements sit side by side, so every chunk that reaches the filter's
+    threshold is full of candidates and the selection runs through the exact path with its rising filter."""
+    K, L = 32, 8
+    g = torch.Generator().manual_seed(V + 1)
+    srt = torch.sort(2.0 * torch.randn(V, generator=g)).values
+    ar = torch.arange(V, dtype=torch.float32)
+    z = torch.empty((2, L, V))
+    z[0, 0] = srt
+    z[0, 1] = srt.flip(0)
+    z[0, 2] = ar * 1e-3
+    z[0, 3] = -ar * 1e-3
+    z[0, 4] = ar
+    z[0, 5] = -ar * 0.1
+    z[0, 6] = torch.cat([2.0 * torch.randn(V // 2, generator=g), srt[V // 2:] - 1.0])
+    z[0, 7] = torch.roll(srt, V // 3)
+    z[1] = z[0].flip(0)
+    _vocab_case(z.to(torch.bfloat16) if dtype == "bf16" else z, K, dtype)
+
+
 @pytest.mark.parametrize("V,dtype", [(3, "bf16"), (6, "f32"), (14, "bf16"), (4099, "bf16"), (4097, "f32")])
 def test_vocab_pass_dominant_logit_outside_the_bulk_copies(V, dtype):
     """One logit 30 above the rest, placed where the 16-byte bulk copies do not reach (tiny rows, the ragged first
