@@ -23,7 +23,7 @@ constexpr int kVpTileBytes = 32768;                  // one ring stage (2 KiB pe
 constexpr int kVpQuantum = 2048;                     // elements; granularity of the work partition
 constexpr int kVpCandCap = 1024;                     // candidate keys held in shared memory
 constexpr int kVpHitCap = 512;                       // chunk hits held in shared memory
-constexpr int kVpRankCap = 512;                      // candidates ranked against each other at most
+constexpr int kVpRankCap = 256;                      // candidates ranked against each other at most
 
 // What one CTA leaves behind for a row that it shares with other CTAs.
 struct VpRecord {

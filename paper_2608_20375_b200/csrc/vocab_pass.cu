@@ -390,6 +390,7 @@ struct __align__(16) EpiShared {  // private to one epilogue group
     uint32_t hits[kVpHitCap];
     uint16_t hthreads[NT];  // streaming threads whose maximum reaches T
     int nhits, ncand, nht, ovf;
+    int tie_groups;  // groups of threads whose maximum is T (to 16 bits): many of them means bulk ties at T
     int fill_ninf;  // the threshold fell on -inf: the candidates are the finite elements plus the first -inf ones
     int fill_tie;   // too many chunks reach the threshold T (bulk ties at T): the candidates are the elements above T
                     // plus the first elements equal to T
@@ -437,6 +438,120 @@ __device__ void warp_select_topk(EpiShared* sh, int n, int K, int lane) {
         if (rank < K) sh->outk[rank] = key;
     }
     __syncwarp();
+}
+
+// The K-th largest chunk maximum of a segment (every streaming thread leaves one 16-bit maximum per tile), as a 16-bit
+// order-preserving pattern; 0 when the segment has fewer than K chunks.  All 128 threads of an epilogue group; two
+// histogram passes of eight bits each over the idle hit list.  Out of line: rows that need it are rare.
+__device__ __noinline__ uint32_t epi_kth_chunk_max(EpiShared* es, const uint16_t* cmx, int max_tiles, int ntiles, int K,
+                                                   int etid, int grp) {
+    uint32_t* hist = es->hits;  // [0, 256) counts, [256] the bin found, [257] the count above it
+    uint32_t prefix = 0u;
+    int want = K;
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {
+        for (int i = etid; i < 258; i += kVpEpiThreads) hist[i] = 0u;
+        epi_bar(grp);
+#pragma unroll 1
+        for (int t = etid; t < NT; t += kVpEpiThreads) {
+            const uint16_t* row = cmx + (size_t)t * max_tiles;
+#pragma unroll 1
+            for (int tile = 0; tile < ntiles; ++tile) {
+                const uint32_t v = ord_from_bits((uint32_t)row[tile] << 16) >> 16;
+                if (pass == 0)
+                    atomicAdd(&hist[v >> 8], 1u);
+                else if ((v >> 8) == prefix)
+                    atomicAdd(&hist[v & 255u], 1u);
+            }
+        }
+        epi_bar(grp);
+        if (etid < 32) {  // the bin in which the count from the top reaches `want`: eight bins a lane
+            uint32_t own = 0u;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) own += hist[8 * etid + i];
+            uint32_t above = own;  // inclusive sum over the lanes from this one up
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, above, d);
+                if (etid + d < 32) above += o;
+            }
+            if (above >= (uint32_t)want && above - own < (uint32_t)want) {  // (one lane at most)
+                uint32_t acc = above - own;
+                for (int i = 7; i >= 0; --i) {
+                    const uint32_t c = hist[8 * etid + i];
+                    if (acc + c >= (uint32_t)want) {
+                        hist[256] = (uint32_t)(8 * etid + i) | 0x100u;
+                        hist[257] = acc;
+                        break;
+                    }
+                    acc += c;
+                }
+            }
+        }
+        epi_bar(grp);
+        const uint32_t bin = hist[256];
+        if (bin == 0u) {  // fewer than K chunks (uniform)
+            prefix = 0u;
+            pass = 2;
+        } else {
+            prefix = (prefix << 8) | (bin & 255u);
+            want -= (int)hist[257];
+        }
+        epi_bar(grp);  // (read before the next pass clears it)
+    }
+    return prefix;
+}
+
+// Exact top-K of cand[0..n) for hundreds of keys, K < n: ranking them against each other costs n^2 compares; here the
+// K-th largest key is found by a search over its bits, two at a time with three counts each (keys are distinct, so
+// exactly K keys reach it), and the K keys that reach it are ranked into outk.  Whatever the keys' order or values.
+// All 128 threads of an epilogue group; the counts of its warps meet in the idle hit list.  Out of line: rows that
+// need it are rare.
+__device__ __noinline__ void epi_select_many(EpiShared* es, int n, int K, int etid, int grp) {
+    uint32_t* cnt = es->hits;                       // [3 * 32] counts, [96] number of keys kept
+    uint64_t* kept = (uint64_t*)(es->hits + 128);   // [K] the keys that reach the K-th largest
+    for (int i = etid; i < 97; i += kVpEpiThreads) cnt[i] = 0u;
+    epi_bar(grp);
+    uint64_t kth = 0ull;
+#pragma unroll 1
+    for (int step = 0; step < 32; ++step) {
+        const int bit = 62 - 2 * step;
+        const uint64_t t1 = kth | (1ull << bit), t2 = kth | (2ull << bit), t3 = kth | (3ull << bit);
+        int c1 = 0, c2 = 0, c3 = 0;
+#pragma unroll 2
+        for (int i = etid; i < n; i += kVpEpiThreads) {
+            const uint64_t k = es->cand[i];
+            c1 += (k >= t1) ? 1 : 0;
+            c2 += (k >= t2) ? 1 : 0;
+            c3 += (k >= t3) ? 1 : 0;
+        }
+        c1 = __reduce_add_sync(0xFFFFFFFFu, c1);
+        c2 = __reduce_add_sync(0xFFFFFFFFu, c2);
+        c3 = __reduce_add_sync(0xFFFFFFFFu, c3);
+        if ((etid & 31) == 0) {
+            atomicAdd(&cnt[3 * step], (uint32_t)c1);
+            atomicAdd(&cnt[3 * step + 1], (uint32_t)c2);
+            atomicAdd(&cnt[3 * step + 2], (uint32_t)c3);
+        }
+        epi_bar(grp);
+        const int n1 = (int)cnt[3 * step], n2 = (int)cnt[3 * step + 1], n3 = (int)cnt[3 * step + 2];
+        kth = n3 >= K ? t3 : (n2 >= K ? t2 : (n1 >= K ? t1 : kth));
+    }
+    for (int i = etid; i < n; i += kVpEpiThreads) {
+        const uint64_t k = es->cand[i];
+        if (k >= kth) {
+            const uint32_t pos = atomicAdd(&cnt[96], 1u);
+            if (pos < (uint32_t)kMaxK) kept[pos] = k;
+        }
+    }
+    epi_bar(grp);
+    const int m = (int)cnt[96] < K ? (int)cnt[96] : K;
+    if (etid < m) {
+        const uint64_t k = kept[etid];
+        int rank = 0;
+        for (int j2 = 0; j2 < m; ++j2) rank += (kept[j2] > k) ? 1 : 0;
+        es->outk[rank] = k;
+    }
 }
 
 // ord() of the largest element of a 16-byte vector
@@ -768,6 +883,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 // (c) T = the K-th largest group maximum, truncated to its top 16 bits: a lower bound of
                 //     the K-th largest element of the segment's body (0 when fewer than K threads saw data)
                 uint32_t Tv = 0;
+                int tie_groups = 0;
                 {
                     // over 64 group maxima rather than the 512 thread maxima: any partition of the elements into
                     // at least K groups gives a lower bound, and this one costs an eighth of the compares for about
@@ -794,6 +910,9 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                         c3 = __reduce_add_sync(0xFFFFFFFFu, c3);
                         Tv = c3 >= p.K ? t3 : (c2 >= p.K ? t2 : (c1 >= p.K ? t1 : Tv));
                     }
+#pragma unroll
+                    for (int i = 0; i < kVpGroups / 32; ++i) tie_groups += ((mine[i] ^ Tv) >> 16) == 0u ? 1 : 0;
+                    tie_groups = __reduce_add_sync(0xFFFFFFFFu, tie_groups);
                 }
                 // fold (c, s, max) across the warp
 #pragma unroll
@@ -818,10 +937,11 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     es->nht = 0;
                     es->ncand = ncand;
                     es->ovf = overflow;
+                    es->tie_groups = tie_groups;
                 }
             }
             epi_bar(grp);
-            const uint32_t Tv = es->Tv;
+            uint32_t Tv = es->Tv;
             // (d) chunks whose stored maximum reaches T: only threads whose own maximum reaches T can have one.
             //     List positions come from shared-memory atomics (the order does not matter: the final selection
             //     ranks exact keys).  A hit is recorded as the byte offset of the chunk's first vector.
@@ -830,11 +950,15 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 if (x >= Tv && x != 0u) es->hthreads[atomicAdd(&es->nht, 1)] = (uint16_t)t;
             }
             epi_bar(grp);
-            // Te: what a chunk's maximum (and, below, an element) must reach.  T itself at first; if more chunks reach T
-            // than the list holds -- thousands of elements tie with T -- the scan is repeated for what lies above T, and
-            // the elements equal to T are taken in id order from the front of the segment further down.
+            // Te: what a chunk's maximum (and, below, an element) must reach.  T itself at first.  If more chunks reach T
+            // than the list holds, T was a poor bound (the 64 groups of threads are a partition that a pattern in step
+            // with the lanes defeats: a row of ramps as long as a warp's block leaves half the groups' maxima far down
+            // every ramp): T is raised to the K-th largest chunk maximum, the best bound the chunk maxima give, and the
+            // scan is repeated.  If the list overflows again, thousands of elements tie with T: the scan is repeated
+            // once more for what lies above T, and the elements equal to T are taken in id order from the front of the
+            // segment further down.
             uint32_t Te = Tv;
-            for (int mode = 0; mode < 2; ++mode) {  // (uniform)
+            for (int mode = 0; mode < 3; ++mode) {  // (uniform)
                 // (listed thread, tile) pairs, four per thread at a time with their loads in flight together; the pair's
                 // thread comes from a multiplication (idx / ntiles for idx < 2^16 and ntiles < 2^16, exactly)
                 const int npairs = es->nht * sg.ntiles;
@@ -867,8 +991,24 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     }
                 }
                 epi_bar(grp);
-                if (mode == 1 || !BF16 || es->fill_ninf || es->nhits <= kVpHitCap) break;  // (uniform)
+                if (mode == 2 || es->fill_ninf || es->nhits <= kVpHitCap) break;  // (uniform)
                 epi_bar(grp);  // (everybody has read the count)
+                if (mode == 0 && es->tie_groups < 16) {
+                    uint32_t kth = epi_kth_chunk_max(es, cmx, p.max_tiles, sg.ntiles, p.K, etid, grp);
+                    // (fp32 logits: the stored maxima are rounded up to bf16, the pattern below is a bound)
+                    if (!BF16 && kth > 0u) kth -= 1u;
+                    if ((kth << 16) > Tv) {  // (uniform)
+                        Tv = Te = kth << 16;
+                        if (etid == 0) {
+                            es->nhits = 0;
+                            es->Tv = Tv;
+                        }
+                        epi_bar(grp);
+                        continue;
+                    }
+                    mode = 1;  // no better bound: ties
+                }
+                if (!BF16) break;
                 if (etid == 0) {
                     es->nhits = 0;
                     es->fill_tie = 1;
@@ -959,9 +1099,9 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 epi_bar(grp);
             }
             // (f) exact top-K of the candidates by rank counting (keys are distinct, so ranks are a permutation)
-            // (ranking n candidates costs n^2 compares shared by 128 threads: beyond 512 -- rows whose large elements sit
-            // side by side, such as sorted rows, fill every chunk that reaches T with candidates -- the exact selection
-            // with its rising filter is the faster way)
+            // (ranking n candidates costs n^2 compares shared by 128 threads: beyond 256 -- rows whose large elements sit
+            // side by side, such as sorted rows, fill every chunk that reaches T with candidates -- one warp finds the
+            // K-th largest key by its bits instead)
             const bool overflow = es->ovf != 0 || es->ncand > kVpRankCap;
             const int ncand = es->ncand < kVpCandCap ? es->ncand : kVpCandCap;
             int nk = ncand < p.K ? ncand : p.K;
@@ -979,6 +1119,8 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     rank += __shfl_xor_sync(0xFFFFFFFFu, rank, 1);
                     if (i < ncand && (etid & 1) == 0 && rank < p.K) es->outk[rank] = key;
                 }
+            } else if (es->ovf == 0 && es->ncand <= kVpCandCap) {  // (uniform; every candidate is in the buffer)
+                epi_select_many(es, ncand, p.K, etid, grp);
             } else if (ew == 0) {
                 // (T is a lower bound of the K-th largest element: the filter starts there, not at nothing -- a row sorted
                 // in ascending order would otherwise send every element through the buffer; with the threshold moved up

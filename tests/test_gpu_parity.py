@@ -175,6 +175,22 @@ def test_vocab_pass_sorted_rows(V, dtype):
     _vocab_case(z.to(torch.bfloat16) if dtype == "bf16" else z, K, dtype)
 
 
+@pytest.mark.parametrize("V,dtype", [(151936, "bf16"), (40003, "bf16"), (151936, "f32")])
+def test_vocab_pass_rows_of_ramps(V, dtype):
+    """Rows made of ramps as long as a chunk, a streaming warp's block, a tile, or three quanta of the partition, rising
+    or falling: patterns in step with the kernel's lanes, for which the maxima of its 64 groups of threads bound the
+    K-th largest element poorly (more chunks reach that bound than the hit list holds) and the bound is taken from the
+    chunk maxima instead."""
+    K, L = 32, 8
+    ar = torch.arange(V, dtype=torch.float32)
+    z = torch.empty((2, L, V))
+    for j, per in enumerate((32, 1024, 16384, 6144)):
+        z[0, 2 * j] = (ar % per) / per * 8 + ar * 1e-6
+        z[0, 2 * j + 1] = -(ar % per) / per * 8
+    z[1] = z[0].flip(0).roll(515, 1)
+    _vocab_case(z.to(torch.bfloat16) if dtype == "bf16" else z, K, dtype)
+
+
 @pytest.mark.parametrize("V,dtype", [(3, "bf16"), (6, "f32"), (14, "bf16"), (4099, "bf16"), (4097, "f32")])
 def test_vocab_pass_dominant_logit_outside_the_bulk_copies(V, dtype):
     """One logit 30 above the rest, placed where the 16-byte bulk copies do not reach (tiny rows, the ragged first
