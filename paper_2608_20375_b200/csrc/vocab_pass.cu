@@ -14,8 +14,11 @@
 //   * top-K needs no per-element work in the stream: after the segment, the K-th largest of 64 group maxima
 //     is a lower bound T for the K-th largest element; only chunks whose stored max reaches T
 //     (about K of them) are re-read, their elements >= T become 64-bit keys (value desc, id asc) and the
-//     exact top-K is found by rank counting.  An overflow of the small key buffer (adversarial rows)
-//     falls back to an exact sliced selection;
+//     exact top-K is found by rank counting.  Rows that defeat the bound: when more chunks reach T than the
+//     hit list holds, T is raised to the K-th largest chunk maximum (or, where the group maxima tie, the
+//     elements above T and the first ones equal to T are taken); hundreds of keys are selected by a search
+//     over the key's bits instead of ranked; an overflow of the key buffer falls back to an exact selection
+//     over the segment whose filter starts at T;
 //   * rows shared by several CTAs are merged by the last CTA to arrive (a counter, no waiting);
 //   * vocabulary-parallel use: the row's pieces are left for a merge over shards instead (vocab_merge_kernel).
 // Every wait on an mbarrier is bounded; when one runs out the kernel raises an error flag and drains.
