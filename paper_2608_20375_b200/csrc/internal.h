@@ -21,7 +21,7 @@ constexpr int kVpGroups = 64;   // groups of streaming threads whose maxima boun
 constexpr int kVpThreads = kVpConsumers + kVpEpiGroups * kVpEpiThreads + 64;  // + one producer warp + one cosine warp
 constexpr int kVpTileBytes = 32768;                  // one ring stage (2 KiB per streaming warp)
 constexpr int kVpQuantum = 2048;                     // elements; granularity of the work partition
-constexpr int kVpCandCap = 1024;                     // candidate keys held in shared memory
+constexpr int kVpCandCap = 1280;                     // candidate keys held in shared memory (K chunks of 32 elements and their ties)
 constexpr int kVpHitCap = 512;                       // chunk hits held in shared memory
 constexpr int kVpRankCap = 256;                      // candidates ranked against each other at most
 

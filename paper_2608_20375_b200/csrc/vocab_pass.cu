@@ -958,8 +958,8 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             // with the lanes defeats: a row of ramps as long as a warp's block leaves half the groups' maxima far down
             // every ramp): T is raised to the K-th largest chunk maximum, the best bound the chunk maxima give, and the
             // scan is repeated.  If the list overflows again, thousands of elements tie with T: the scan is repeated
-            // once more for what lies above T, and the elements equal to T are taken in id order from the front of the
-            // segment further down.
+            // once more for what lies above T, and the first elements equal to T in id order are taken by a walk over
+            // the chunks further down.
             uint32_t Te = Tv;
             for (int mode = 0; mode < 3; ++mode) {  // (uniform)
                 // (listed thread, tile) pairs, four per thread at a time with their loads in flight together; the pair's
@@ -1016,7 +1016,7 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     es->nhits = 0;
                     es->fill_tie = 1;
                 }
-                Te = Tv + 1u;
+                Te = Tv + 0x10000u;  // (the next bf16 value up, whatever the sign: T holds the value's upper 16 bits)
                 epi_bar(grp);
             }
             // (e) the 16-byte vectors of the hit chunks, re-read from global memory; elements >= T become keys.
@@ -1074,30 +1074,44 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             epi_bar(grp);
             if (es->fill_ninf || es->fill_tie) {  // (uniform)
                 if (ew == 0) {
-                    // (the same walk serves bulk ties at T: the first K elements equal to T, looked for in the segment's
-                    // first 2048 elements only -- where ties are that many they are found at once)
+                    // The first K elements equal to -inf (or, for bulk ties, to T) of the segment's body in id order (the
+                    // few elements before and after the body are candidates already): a walk over the chunks in id
+                    // order -- tile, streaming warp, lane -- that reads only chunks whose stored maximum reaches T (any
+                    // chunk when the value looked for is -inf), 32 elements at a time.  Every chunk read for ties holds
+                    // one at least unless a larger element put it on the list, so the walk is short wherever the ties
+                    // are; after 256 chunks it gives up and the exact selection takes over.
                     const bool tie = es->fill_tie != 0;
-                    // the first K elements equal to -inf of the segment's body, in id order (the few elements before
-                    // and after the body are candidates already); a segment that does not show K of them within
-                    // its first 8192 elements goes to the exact selection instead
-                    const int kScan = tie ? 2048 : 8192;
-                    int found = 0, e0 = sg.e_body0;
-                    for (; e0 < sg.e_tail0 && e0 - sg.e_body0 < kScan && found < p.K; e0 += 32) {
-                        const int e = e0 + lane;
-                        uint32_t xb = 0u;
-                        bool is = false;
-                        if (e < sg.e_tail0) {
-                            xb = __float_as_uint(load_elem_f32(rowp + (size_t)e * T::ESZ, BF16));
-                            is = tie ? ord_from_bits(xb) == Tv : xb == 0xFF800000u;  // (-0 and +0 are one value)
+                    const uint32_t T16 = Tv >> 16;
+                    int need = p.K, visits = 0;
+                    bool gave_up = false;
+                    for (int blk = 0; blk < sg.ntiles * NW && need > 0; ++blk) {
+                        const int tile = blk / NW, w = blk % NW;
+                        const uint32_t cm = ord_from_bits((uint32_t)cmx[(size_t)(w * 32 + lane) * p.max_tiles + tile] << 16) >> 16;
+                        uint32_t todo = __ballot_sync(0xFFFFFFFFu, !tie || cm >= T16);
+                        while (todo != 0u && need > 0) {  // (uniform)
+                            if (++visits > 256) {
+                                gave_up = true;
+                                need = 0;
+                                break;
+                            }
+                            const uint32_t off = (uint32_t)tile * TILE + (uint32_t)w * WBLK + (uint32_t)(__ffs(todo) - 1) * 64u +
+                                                 (uint32_t)lane * T::ESZ;
+                            todo &= todo - 1u;
+                            uint32_t xb = 0u;
+                            bool is = false;
+                            if (lane < 64 / T::ESZ && off < sg.body_bytes) {
+                                xb = __float_as_uint(load_elem_f32(sg.body + off, BF16));
+                                is = tie ? (ord_from_bits(xb) >> 16) == T16 : xb == 0xFF800000u;  // (-0 and +0 are one value)
+                            }
+                            const uint32_t mk = __ballot_sync(0xFFFFFFFFu, is);
+                            if (is && __popc(mk & ((1u << lane) - 1u)) < need) {
+                                const int pos = atomicAdd(&es->ncand, 1);
+                                if (pos < kVpCandCap) es->cand[pos] = make_key(xb, (uint32_t)sg.e_body0 + off / T::ESZ);
+                            }
+                            need -= __popc(mk);
                         }
-                        const uint32_t mk = __ballot_sync(0xFFFFFFFFu, is);
-                        if (is && found + __popc(mk & ((1u << lane) - 1u)) < p.K) {
-                            const int pos = atomicAdd(&es->ncand, 1);
-                            if (pos < kVpCandCap) es->cand[pos] = make_key(xb, (uint32_t)e);
-                        }
-                        found += __popc(mk);
                     }
-                    if (found < p.K && e0 < sg.e_tail0 && lane == 0) es->ovf = 1;
+                    if (gave_up && lane == 0) es->ovf = 1;
                 }
                 epi_bar(grp);
             }

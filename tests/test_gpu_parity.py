@@ -191,6 +191,73 @@ def test_vocab_pass_rows_of_ramps(V, dtype):
     _vocab_case(z.to(torch.bfloat16) if dtype == "bf16" else z, K, dtype)
 
 
+@pytest.mark.parametrize("V,dtype", [(151936, "bf16"), (40003, "bf16"), (151936, "f32")])
+def test_vocab_pass_sparse_ties(V, dtype):
+    """Hundreds of elements tie with the K-th largest value, one in every 256 or 4096 elements, over a lower random
+    rest: the tied elements of smallest id are wanted, and they are chunks apart -- at a positive and at a negative
+    value, alone, under a few larger elements, and starting far into the row."""
+    K, L = 32, 8
+    g = torch.Generator().manual_seed(V + 7)
+    z = -2.0 - 6.0 * torch.rand((2, L, V), generator=g)
+    z[0, 0, ::256] = 1.5
+    z[0, 1, ::256] = -1.5
+    z[0, 2, 5::4096] = 0.25
+    z[0, 2, torch.randint(0, V, (7,), generator=g)] = 3.0
+    z[0, 3, 5::4096] = -0.75
+    z[0, 3, torch.randint(0, V, (40,), generator=g)] = 3.0   # more winners than K: no tied element is wanted
+    z[0, 4, V // 2::256] = 1.0                                # the ties start half-way into the row
+    z[0, 5, 3::256] = -1.0
+    z[0, 5, 3 + 256 * 9] = -0.5                               # a winner in the place of a tied element
+    z[0, 6, ::33] = 0.0                                       # a tie in every chunk but not at a fixed lane
+    z[0, 7, 31::32] = -1.25                                   # the last element of every chunk
+    z[1] = z[0].flip(0).roll(771, 1)
+    _vocab_case(z.to(torch.bfloat16) if dtype == "bf16" else z, K, dtype)
+
+
+def test_vocab_pass_whole_row_segments_of_rows_that_defeat_the_filter():
+    """At the benchmark's width and batch (64 x 16 rows of 151,936 bf16 logits) a CTA's segments are whole rows of ten
+    tiles: there the hit list overflows on rows of ramps and on sparse ties (hundreds of chunks reach the bound), the
+    bound is taken from the chunk maxima, the tie walk follows the chunk maxima, and sorted rows fill the key buffer.
+    Sixteen such shapes, rolled differently for every sequence; sampled rows against the oracle."""
+    from paper_2608_20375_b200 import Graft
+    V, K, L, Bt = 151936, 32, 16, 64
+    g = torch.Generator().manual_seed(77)
+    ar = torch.arange(V, dtype=torch.float32)
+    low = lambda: -2.0 - 6.0 * torch.rand(V, generator=g)
+    srt = torch.sort(2.0 * torch.randn(V, generator=g)).values
+    pats = []
+    for per in (256, 1024, 6144, 16384):
+        pats.append((ar % per) / per * 8)
+        pats.append(-(ar % per) / per * 8)
+    x = low(); x[::256] = 1.5; pats.append(x)                         # sparse ties, positive
+    x = low(); x[::256] = -1.5; pats.append(x)                        # ... negative
+    x = low(); x[5::4096] = 0.25; x[torch.randint(0, V, (7,), generator=g)] = 3.0; pats.append(x)
+    x = low(); x[V // 2::256] = 1.0; pats.append(x)                   # the ties start half-way into the row
+    pats.append(srt)
+    pats.append(srt.flip(0))
+    pats.append(ar * 1e-3)
+    x = 2.0 * torch.randn(V, generator=g); x[20000:25000] = 20.0 + torch.sort(torch.randn(5000, generator=g)).values
+    pats.append(x)
+    assert len(pats) == L
+    row = torch.stack(pats).to(torch.bfloat16)
+    z = torch.stack([torch.roll(row, 37 * b * (b % 3), 1) for b in range(Bt)])      # [Bt, L, V]
+    gr = Graft(V, L, K, 16, 8, Bt, 8, 8, 8, 0.0, 1, DT["bf16"], 0)
+    ids = torch.empty((Bt, L, K), dtype=torch.int32, device="cuda")
+    lp = torch.empty((Bt, L, K), dtype=torch.float32, device="cuda")
+    lse = torch.empty((Bt, L), dtype=torch.float32, device="cuda")
+    rs = torch.empty((Bt, L), dtype=torch.int32, device="cuda")
+    gr.vocab_pass(z.cuda(), ids, lp, lse, rs)
+    torch.cuda.synchronize()
+    gr.destroy()
+    sample = [b * L + d for b in (0, 1, 2, 7, 30, 63) for d in range(L)]
+    o_ids, o_lp, o_lse, o_st = oracle.vocab_pass(z.reshape(Bt * L, V)[sample], K)
+    ids, lp, lse, rs = (t.cpu().numpy().reshape(Bt * L, -1)[sample] for t in (ids, lp, lse, rs))
+    assert np.array_equal(rs[:, 0], o_st) and not o_st.any()
+    assert np.array_equal(ids, o_ids)
+    assert np.all(np.abs(lp.astype(np.float64) - o_lp) <= tolerance(o_lp))
+    assert np.all(np.abs(lse[:, 0] - o_lse) <= tolerance(o_lse))
+
+
 @pytest.mark.parametrize("V,dtype", [(3, "bf16"), (6, "f32"), (14, "bf16"), (4099, "bf16"), (4097, "f32")])
 def test_vocab_pass_dominant_logit_outside_the_bulk_copies(V, dtype):
     """One logit 30 above the rest, placed where the 16-byte bulk copies do not reach (tiny rows, the ragged first
