@@ -994,14 +994,18 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     }
                 }
                 epi_bar(grp);
-                if (mode == 2 || es->fill_ninf || es->nhits <= kVpHitCap) break;  // (uniform)
+                // (a list several times as long as a good bound leaves it -- about K chunks -- also says that T is poor:
+                // its chunks would overflow the key buffer)
+                const bool over = es->nhits > kVpHitCap;
+                if (mode == 2 || es->fill_ninf) break;  // (uniform)
+                if (!over && !(mode == 0 && es->nhits > 5 * p.K && es->tie_groups < 16)) break;  // (uniform)
                 epi_bar(grp);  // (everybody has read the count)
                 if (mode == 0 && es->tie_groups < 16) {
                     uint32_t kth = epi_kth_chunk_max(es, cmx, p.max_tiles, sg.ntiles, p.K, etid, grp);
                     // (fp32 logits: the stored maxima are rounded up to bf16, the pattern below is a bound)
                     if (!BF16 && kth > 0u) kth -= 1u;
-                    if ((kth << 16) > Tv) {  // (uniform)
-                        Tv = Te = kth << 16;
+                    if ((kth << 16) > Tv || !over) {  // (uniform; the search used the hit list: scan again in any case)
+                        if ((kth << 16) > Tv) Tv = Te = kth << 16;
                         if (etid == 0) {
                             es->nhits = 0;
                             es->Tv = Tv;
