@@ -506,49 +506,79 @@ __device__ __noinline__ uint32_t epi_kth_chunk_max(EpiShared* es, const uint16_t
 }
 
 // Exact top-K of cand[0..n) for hundreds of keys, K < n: ranking them against each other costs n^2 compares; here the
-// K-th largest key is found by a search over its bits, two at a time with three counts each (keys are distinct, so
-// exactly K keys reach it), and the K keys that reach it are ranked into outk.  Whatever the keys' order or values.
-// All 128 threads of an epilogue group; the counts of its warps meet in the idle hit list.  Out of line: rows that
-// need it are rare.
+// K-th largest key is found by a search over its bits, two at a time with three counts each -- over the value word
+// first; over the id word, among the keys of that value, only if more keys share the K-th largest value than are
+// wanted -- and the K keys that reach it (keys are distinct: exactly K) are ranked into outk.  Whatever the keys'
+// order or values.  All 128 threads of an epilogue group; the counts of its warps meet in the idle hit list.  Out of
+// line: rows that need it are rare.
 __device__ __noinline__ void epi_select_many(EpiShared* es, int n, int K, int etid, int grp) {
-    uint32_t* cnt = es->hits;                       // [3 * 32] counts, [96] number of keys kept
+    uint32_t* cnt = es->hits;                       // [2 * 16 * 3] counts of the steps, [96], [97] above / at the value, [98] kept
     uint64_t* kept = (uint64_t*)(es->hits + 128);   // [K] the keys that reach the K-th largest
-    for (int i = etid; i < 97; i += kVpEpiThreads) cnt[i] = 0u;
+    const uint32_t* word = (const uint32_t*)es->cand;  // key i: id word at 2 i, value word at 2 i + 1
+    for (int i = etid; i < 99; i += kVpEpiThreads) cnt[i] = 0u;
     epi_bar(grp);
-    uint64_t kth = 0ull;
+    uint32_t vk = 0u, ik = 0u;  // the K-th largest key's value word and id word
+    int want = K;
 #pragma unroll 1
-    for (int step = 0; step < 32; ++step) {
-        const int bit = 62 - 2 * step;
-        const uint64_t t1 = kth | (1ull << bit), t2 = kth | (2ull << bit), t3 = kth | (3ull << bit);
-        int c1 = 0, c2 = 0, c3 = 0;
+    for (int phase = 0; phase < 2; ++phase) {
+        uint32_t kth = 0u;
+#pragma unroll 1
+        for (int step = 0; step < 16; ++step) {
+            const int bit = 30 - 2 * step;
+            const uint32_t t1 = kth | (1u << bit), t2 = kth | (2u << bit), t3 = kth | (3u << bit);
+            int c1 = 0, c2 = 0, c3 = 0;
 #pragma unroll 2
-        for (int i = etid; i < n; i += kVpEpiThreads) {
-            const uint64_t k = es->cand[i];
-            c1 += (k >= t1) ? 1 : 0;
-            c2 += (k >= t2) ? 1 : 0;
-            c3 += (k >= t3) ? 1 : 0;
+            for (int i = etid; i < n; i += kVpEpiThreads) {
+                const uint32_t hi = word[2 * i + 1];
+                const uint32_t x = phase == 0 ? hi : (hi == vk ? word[2 * i] : 0u);  // (an id word is never 0)
+                c1 += (x >= t1) ? 1 : 0;
+                c2 += (x >= t2) ? 1 : 0;
+                c3 += (x >= t3) ? 1 : 0;
+            }
+            c1 = __reduce_add_sync(0xFFFFFFFFu, c1);
+            c2 = __reduce_add_sync(0xFFFFFFFFu, c2);
+            c3 = __reduce_add_sync(0xFFFFFFFFu, c3);
+            uint32_t* slot = cnt + (phase * 16 + step) * 3;
+            if ((etid & 31) == 0) {
+                atomicAdd(&slot[0], (uint32_t)c1);
+                atomicAdd(&slot[1], (uint32_t)c2);
+                atomicAdd(&slot[2], (uint32_t)c3);
+            }
+            epi_bar(grp);
+            const int n1 = (int)slot[0], n2 = (int)slot[1], n3 = (int)slot[2];
+            kth = n3 >= want ? t3 : (n2 >= want ? t2 : (n1 >= want ? t1 : kth));
         }
-        c1 = __reduce_add_sync(0xFFFFFFFFu, c1);
-        c2 = __reduce_add_sync(0xFFFFFFFFu, c2);
-        c3 = __reduce_add_sync(0xFFFFFFFFu, c3);
+        if (phase == 1) {
+            ik = kth;
+            break;
+        }
+        vk = kth;
+        int above = 0, at = 0;
+        for (int i = etid; i < n; i += kVpEpiThreads) {
+            const uint32_t hi = word[2 * i + 1];
+            above += (hi > vk) ? 1 : 0;
+            at += (hi == vk) ? 1 : 0;
+        }
+        above = __reduce_add_sync(0xFFFFFFFFu, above);
+        at = __reduce_add_sync(0xFFFFFFFFu, at);
         if ((etid & 31) == 0) {
-            atomicAdd(&cnt[3 * step], (uint32_t)c1);
-            atomicAdd(&cnt[3 * step + 1], (uint32_t)c2);
-            atomicAdd(&cnt[3 * step + 2], (uint32_t)c3);
+            atomicAdd(&cnt[96], (uint32_t)above);
+            atomicAdd(&cnt[97], (uint32_t)at);
         }
         epi_bar(grp);
-        const int n1 = (int)cnt[3 * step], n2 = (int)cnt[3 * step + 1], n3 = (int)cnt[3 * step + 2];
-        kth = n3 >= K ? t3 : (n2 >= K ? t2 : (n1 >= K ? t1 : kth));
+        want = K - (int)cnt[96];
+        if ((int)cnt[97] == want) break;  // (uniform) every key of that value is wanted: ik = 0 lets them all through
     }
+    const uint64_t kth_key = ((uint64_t)vk << 32) | ik;
     for (int i = etid; i < n; i += kVpEpiThreads) {
         const uint64_t k = es->cand[i];
-        if (k >= kth) {
-            const uint32_t pos = atomicAdd(&cnt[96], 1u);
+        if (k >= kth_key) {
+            const uint32_t pos = atomicAdd(&cnt[98], 1u);
             if (pos < (uint32_t)kMaxK) kept[pos] = k;
         }
     }
     epi_bar(grp);
-    const int m = (int)cnt[96] < K ? (int)cnt[96] : K;
+    const int m = (int)cnt[98] < K ? (int)cnt[98] : K;
     if (etid < m) {
         const uint64_t k = kept[etid];
         int rank = 0;
