@@ -800,6 +800,48 @@ def run_styles(args):
                       "rounds_timed": args.steps, "rows": rows}))
 
 
+def run_rows(args):
+    """`--rows`: the vocab pass alone, launched back to back, on rows that defeat its top-K filter
+    (graft_inputs.adversarial_rows): every row of the batch is the same shape, rolled differently per sequence so
+    that the CTAs' segments cut it in different places.  One JSON line."""
+    from paper_2608_20375_b200 import Graft
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w = gi.WORKLOADS[args.workload]
+    bf16 = w.logits_dtype == "bf16"
+    g = Graft(w.V, w.L, w.K, w.m, 8, w.batch, w.budget_min, w.budget_max, w.budget_step, 0.0, 1, 1 if bf16 else 0, 0)
+    ids = torch.empty((w.batch, w.L, w.K), dtype=torch.int32, device=dev)
+    lp = torch.empty((w.batch, w.L, w.K), dtype=torch.float32, device=dev)
+    lse = torch.empty((w.batch, w.L), dtype=torch.float32, device=dev)
+    rs = torch.empty((w.batch, w.L), dtype=torch.int32, device=dev)
+    gen = torch.Generator().manual_seed(11)
+    out = []
+    for name, row in gi.adversarial_rows(w.V, gen):
+        r = row.to(torch.bfloat16 if bf16 else torch.float32).to(dev)
+        # two input sets (each larger than L2 at the benchmark's shapes), every row rolled by its own offset
+        sets = []
+        for k in range(2):
+            z = torch.stack([torch.roll(r, (131 * i + 7919 * k) % w.V) for i in range(w.batch * w.L)])
+            sets.append(z.reshape(w.batch, w.L, w.V).contiguous())
+        for _ in range(3):
+            for z in sets:
+                g.vocab_pass(z, ids, lp, lse, rs)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        torch.cuda.synchronize()
+        ev[0].record()
+        for _ in range(args.steps):
+            for z in sets:
+                g.vocab_pass(z, ids, lp, lse, rs)
+        ev[1].record()
+        torch.cuda.synchronize()
+        out.append(dict(row=name, vocab_pass_us=round(ev[0].elapsed_time(ev[1]) * 1e3 / (2 * args.steps), 1),
+                        status_or=int(rs.max())))
+        del sets
+    g.destroy()
+    print(json.dumps({"rows": "the vocab pass alone, back to back, on rows that defeat its filter", "shape": w.name,
+                      "launches_timed": 2 * args.steps, "times": out}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -822,6 +864,8 @@ def main():
                     help="instead of the benchmark: time the least-squares fit of the SABA models")
     ap.add_argument("--styles", action="store_true",
                     help="instead of the benchmark: the round's kernels timed on degenerate inputs (own JSON line)")
+    ap.add_argument("--rows", action="store_true",
+                    help="instead of the benchmark: the vocab pass timed on rows that defeat its filter (own JSON line)")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the benchmark: fixed-budget / beta sweeps on synthetic acceptance (own JSON line)")
     ap.add_argument("--sweep-fixed-budget", type=int, default=256, help="the fixed budget of the DDTree-style arms")
@@ -829,6 +873,10 @@ def main():
     if args.styles and args.impl == "graft":
         args.steps = 20 if args.steps is None else args.steps
         run_styles(args)
+        return
+    if args.rows and args.impl == "graft":
+        args.steps = 10 if args.steps is None else args.steps
+        run_rows(args)
         return
     if args.sweep and args.impl == "graft":
         if "--workload" not in sys.argv:

@@ -300,6 +300,53 @@ def styled_logits(z, style, rng, gen, K):
     return z
 
 
+def adversarial_rows(V, gen):
+    """Named single rows (fp32 [V]) that defeat a top-K filter built on partitions of a row: sorted rows, blocks of
+    large elements, rows of ramps of several periods, bulk and sparse ties, masked halves.  For timing the vocab pass
+    on its worst cases; `gen` is a seeded torch.Generator."""
+    ar = torch.arange(V, dtype=torch.float32)
+    base = 2.0 * torch.randn(V, generator=gen)
+    srt = torch.sort(2.0 * torch.randn(V, generator=gen)).values
+    low = -1.0 - 7.0 * torch.rand(V, generator=gen)
+    rows = [("ordinary", base), ("sorted ascending", srt), ("sorted descending", srt.flip(0))]
+    for s in (1e-3, 0.1, 1.0):
+        rows.append((f"ramp up, step {s:g} (ties in bf16)", ar * s))
+        rows.append((f"ramp down, step {s:g} (ties in bf16)", -ar * s))
+    for n in (1000, 5000, 50000):
+        n = min(n, V // 2)
+        at = V // 8
+        z = base.clone()
+        z[at:at + n] += 20.0
+        rows.append((f"block of {n} large elements", z))
+        z = base.clone()
+        z[at:at + n] = 20.0 + torch.sort(torch.randn(n, generator=gen)).values
+        rows.append((f"sorted block of {n} large elements", z))
+    for per in (32, 256, 512, 1024, 2048, 4096, 6144, 16384):
+        rows.append((f"ramps of period {per}, rising", (ar % per) / per * 8))
+        rows.append((f"ramps of period {per}, falling", -(ar % per) / per * 8))
+    rows.append(("ramps of period 1024, falling, distinct tops", -(ar % 1024) / 1024 * 8 + (ar // 1024) * 1e-2))
+    rows.append(("all equal", torch.zeros(V)))
+    rows.append(("alternating +1 / -1", torch.where(ar % 2 == 0, 1.0, -1.0)))
+    rows.append(("two values at random", torch.where(torch.rand(V, generator=gen) < 0.5, 1.0, 0.0)))
+    rows.append(("coarse grid of 1/8", torch.round(base * 8) / 8))
+    z = low.clone()
+    z[::1024] = 0.0
+    rows.append(("one tied winner in 1024 over a lower rest", z))
+    z = low.clone()
+    z[::256] = 0.0
+    rows.append(("one tied winner in 256 over a lower rest", z))
+    rows.append(("forty winners at the end of a flat row", torch.cat([torch.zeros(V - 40), torch.arange(40).float()])))
+    rows.append(("2000 rising elements at the end", torch.cat([base[: V - min(2000, V // 2)], 10 + torch.arange(min(2000, V // 2)).float() * 0.01])))
+    z = base.clone()
+    z[::2] = float("-inf")
+    rows.append(("every second element -inf", z))
+    z = base.clone()
+    z[: V // 2] = float("-inf")
+    rows.append(("front half -inf", z))
+    rows.append(("heavy tail (cubed)", base ** 3))
+    return rows
+
+
 def small(name: str = "T", **kw) -> Workload:
     """A small workload for tests; override any field."""
     base = dict(name=name, batch=2, L=4, V=1000, K=4, hidden_dim=32, logits_dtype="f32", hidden_dtype="f32",

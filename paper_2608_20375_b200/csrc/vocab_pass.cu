@@ -984,14 +984,16 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
             }
             epi_bar(grp);
             // Te: what a chunk's maximum (and, below, an element) must reach.  T itself at first.  If more chunks reach T
-            // than the list holds, T was a poor bound (the 64 groups of threads are a partition that a pattern in step
-            // with the lanes defeats: a row of ramps as long as a warp's block leaves half the groups' maxima far down
-            // every ramp): T is raised to the K-th largest chunk maximum, the best bound the chunk maxima give, and the
-            // scan is repeated.  If the list overflows again, thousands of elements tie with T: the scan is repeated
-            // once more for what lies above T, and the first elements equal to T in id order are taken by a walk over
-            // the chunks further down.
+            // than the list holds, either thousands of elements tie with T (a flat rest under a few winners: most of the
+            // 64 group maxima are T itself) or T is a poor bound (the groups of threads are a partition that a pattern in
+            // step with the lanes defeats: a row of ramps as long as a warp's block leaves half the groups' maxima far down
+            // every ramp).  Ties: the scan is repeated for what lies above T, and the first elements equal to T in id
+            // order are taken by a walk over the chunks further down.  A poor bound: T is raised to the K-th largest chunk
+            // maximum, the best bound the chunk maxima give, and the scan is repeated.  Whichever comes first, the other
+            // follows if the list overflows again: four scans at most, then the exact selection.
             uint32_t Te = Tv;
-            for (int mode = 0; mode < 3; ++mode) {  // (uniform)
+            bool refined = false, tied = false;
+            for (int pass = 0;; ++pass) {  // (uniform)
                 // (listed thread, tile) pairs, four per thread at a time with their loads in flight together; the pair's
                 // thread comes from a multiplication (idx / ntiles for idx < 2^16 and ntiles < 2^16, exactly)
                 const int npairs = es->nht * sg.ntiles;
@@ -1027,25 +1029,30 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                 // (a list several times as long as a good bound leaves it -- about K chunks -- also says that T is poor:
                 // its chunks would overflow the key buffer)
                 const bool over = es->nhits > kVpHitCap;
-                if (mode == 2 || es->fill_ninf) break;  // (uniform)
-                if (!over && !(mode == 0 && es->nhits > 5 * p.K && es->tie_groups < 16)) break;  // (uniform)
+                if (es->fill_ninf || (refined && tied)) break;  // (uniform)
+                if (!over && !(pass == 0 && es->nhits > 5 * p.K && es->tie_groups < 16)) break;  // (uniform)
                 epi_bar(grp);  // (everybody has read the count)
-                if (mode == 0 && es->tie_groups < 16) {
+                if (!refined && (tied || !BF16 || es->tie_groups < 16)) {
                     uint32_t kth = epi_kth_chunk_max(es, cmx, p.max_tiles, sg.ntiles, p.K, etid, grp);
                     // (fp32 logits: the stored maxima are rounded up to bf16, the pattern below is a bound)
                     if (!BF16 && kth > 0u) kth -= 1u;
+                    refined = true;
                     if ((kth << 16) > Tv || !over) {  // (uniform; the search used the hit list: scan again in any case)
-                        if ((kth << 16) > Tv) Tv = Te = kth << 16;
+                        if ((kth << 16) > Tv) Tv = kth << 16;
+                        Te = Tv;
+                        tied = false;
                         if (etid == 0) {
                             es->nhits = 0;
+                            es->fill_tie = 0;
                             es->Tv = Tv;
                         }
                         epi_bar(grp);
                         continue;
                     }
-                    mode = 1;  // no better bound: ties
+                    if (tied) break;  // (no better bound and what lies above T overflows the list: the exact selection)
                 }
-                if (!BF16) break;
+                if (!BF16 || tied) break;
+                tied = true;
                 if (etid == 0) {
                     es->nhits = 0;
                     es->fill_tie = 1;
@@ -1113,17 +1120,20 @@ __global__ void __launch_bounds__(kVpThreads, 1) vocab_pass_kernel(const VpParam
                     // order -- tile, streaming warp, lane -- that reads only chunks whose stored maximum reaches T (any
                     // chunk when the value looked for is -inf), 32 elements at a time.  Every chunk read for ties holds
                     // one at least unless a larger element put it on the list, so the walk is short wherever the ties
-                    // are; after 256 chunks it gives up and the exact selection takes over.
+                    // are; the walk for -inf gives up after 256 chunks and the exact selection takes over.
                     const bool tie = es->fill_tie != 0;
                     const uint32_t T16 = Tv >> 16;
-                    int need = p.K, visits = 0;
+                    // (K chunks or more with an element above T: no tied element is wanted.  Otherwise fewer than 2 K
+                    // visits find K tied elements or the end of the segment.)
+                    int need = tie && es->nhits >= p.K ? 0 : p.K, visits = 0;
+                    const int max_visits = tie ? 2 * p.K : 256;
                     bool gave_up = false;
                     for (int blk = 0; blk < sg.ntiles * NW && need > 0; ++blk) {
                         const int tile = blk / NW, w = blk % NW;
                         const uint32_t cm = ord_from_bits((uint32_t)cmx[(size_t)(w * 32 + lane) * p.max_tiles + tile] << 16) >> 16;
                         uint32_t todo = __ballot_sync(0xFFFFFFFFu, !tie || cm >= T16);
                         while (todo != 0u && need > 0) {  // (uniform)
-                            if (++visits > 256) {
+                            if (++visits > max_visits) {
                                 gave_up = true;
                                 need = 0;
                                 break;
