@@ -312,8 +312,7 @@ def adversarial_rows(V, gen):
     for s in (1e-3, 0.1, 1.0):
         rows.append((f"ramp up, step {s:g} (ties in bf16)", ar * s))
         rows.append((f"ramp down, step {s:g} (ties in bf16)", -ar * s))
-    for n in (1000, 5000, 50000):
-        n = min(n, V // 2)
+    for n in sorted({min(n, V // 2) for n in (1000, 5000, 50000)}):
         at = V // 8
         z = base.clone()
         z[at:at + n] += 20.0

@@ -40,3 +40,25 @@ def test_gpu_arm_line():
     assert d["e2e"]["h2d_bytes_per_step"] > 0 and d["e2e"]["d2h_bytes_per_step"] > 0
     assert abs(d["value"] - 16 / (d["ms_per_step"] * 1e-3)) / d["value"] < 1e-6
     assert d["status_or"] == 0
+
+
+def test_adversarial_rows_are_seeded_and_whole():
+    """The rows of `bench.py --rows`: named, of the asked width at small and full widths, the same for the same seed."""
+    import torch
+    sys.path.insert(0, ROOT)
+    import graft_inputs as gi
+    for V in (4099, 40003):
+        a = gi.adversarial_rows(V, torch.Generator().manual_seed(11))
+        b = gi.adversarial_rows(V, torch.Generator().manual_seed(11))
+        assert len(a) >= 40 and len({n for n, _ in a}) == len(a), [n for n, _ in a]
+        for (na, ra), (nb_, rb) in zip(a, b):
+            assert na == nb_ and ra.shape == (V,) and ra.dtype == torch.float32
+            assert torch.equal(torch.nan_to_num(ra, neginf=-1e30), torch.nan_to_num(rb, neginf=-1e30))
+            assert not torch.isnan(ra).any() and not torch.isposinf(ra).any()
+
+
+@pytest.mark.gpu
+def test_gpu_rows_line():
+    d = _run(["--rows", "--workload", "C2", "--steps", "1"])
+    assert d["shape"] == "C2" and len(d["times"]) >= 40
+    assert all(t["vocab_pass_us"] > 0 and t["status_or"] == 0 for t in d["times"])
