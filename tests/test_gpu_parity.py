@@ -259,6 +259,55 @@ def test_vocab_pass_whole_row_segments_of_rows_that_defeat_the_filter():
     assert np.all(np.abs(lse[:, 0] - o_lse) <= tolerance(o_lse))
 
 
+@pytest.mark.parametrize("seed,dtype", [(0, "bf16"), (1, "f32"), (2, "bf16"), (3, "bf16")])
+def test_vocab_pass_compositions_of_rows_that_defeat_the_filter(seed, dtype):
+    """Random compositions of `graft_inputs.adversarial_rows` at the benchmark's batch and width (whole-row segments):
+    a row as it is, reversed, negated, scaled, spliced with another, or with a few winners planted on top; every
+    sequence rolled by its own offset; 96 sampled rows against the oracle."""
+    from paper_2608_20375_b200 import Graft
+    V, K, L, Bt = 151936, 32, 16, 64
+    g0 = torch.Generator().manual_seed(1000 + seed)
+    rng = np.random.default_rng(seed)
+    pool = gi.adversarial_rows(V, g0)
+    pats = []
+    for d in range(L):
+        r = pool[int(rng.integers(len(pool)))][1].clone()
+        op = int(rng.integers(6))
+        if op == 1:
+            r = r.flip(0)
+        elif op == 2:
+            r = -r
+        elif op == 3:
+            cut = int(rng.integers(1, V - 1))
+            r[cut:] = pool[int(rng.integers(len(pool)))][1][cut:]
+        elif op == 4:
+            r = r * float(rng.choice([0.1, 3.0, 17.0]))
+        elif op == 5:
+            r[torch.randint(0, V, (int(rng.integers(1, 60)),), generator=g0)] = r[torch.isfinite(r)].max() + 1.0
+        pats.append(torch.nan_to_num(r, nan=0.0, posinf=1e4))
+    row = torch.stack(pats).to(torch.bfloat16 if dtype == "bf16" else torch.float32)
+    z = torch.stack([torch.roll(row, int(rng.integers(V)), 1) for b in range(Bt)])
+    gr = Graft(V, L, K, 16, 8, Bt, 8, 8, 8, 0.0, 1, DT[dtype], 0)
+    ids = torch.empty((Bt, L, K), dtype=torch.int32, device="cuda")
+    lp = torch.empty((Bt, L, K), dtype=torch.float32, device="cuda")
+    lse = torch.empty((Bt, L), dtype=torch.float32, device="cuda")
+    rs = torch.empty((Bt, L), dtype=torch.int32, device="cuda")
+    gr.vocab_pass(z.cuda(), ids, lp, lse, rs)
+    torch.cuda.synchronize()
+    gr.destroy()
+    sample = sorted(set(int(x) for x in rng.integers(0, Bt * L, 96)))
+    o_ids, o_lp, o_lse, o_st = oracle.vocab_pass(z.reshape(Bt * L, V)[sample], K)
+    ids, lp, lse, rs = (t.cpu().numpy().reshape(Bt * L, -1)[sample] for t in (ids, lp, lse, rs))
+    assert np.array_equal(rs[:, 0], o_st)
+    good = o_st == 0
+    assert good.any() and np.array_equal(ids[good], o_ids[good])
+    a, b = lp[good].astype(np.float64), o_lp[good]
+    fin = np.isfinite(b)
+    assert np.array_equal(np.isneginf(a), np.isneginf(b))
+    assert np.all(np.abs(a[fin] - b[fin]) <= tolerance(b[fin]))
+    assert np.all(np.abs(lse[good, 0] - o_lse[good]) <= tolerance(o_lse[good]))
+
+
 @pytest.mark.parametrize("V,dtype", [(3, "bf16"), (6, "f32"), (14, "bf16"), (4099, "bf16"), (4097, "f32")])
 def test_vocab_pass_dominant_logit_outside_the_bulk_copies(V, dtype):
     """One logit 30 above the rest, placed where the 16-byte bulk copies do not reach (tiny rows, the ragged first
