@@ -770,7 +770,8 @@ def run_styles(args):
     for style in gi.STYLES:
         w = gi.small(batch=w0.batch, L=w0.L, V=w0.V, K=w0.K, budget_min=w0.budget_min, budget_max=w0.budget_max,
                      budget_step=w0.budget_step, m=w0.m, hidden_dim=256, logits_dtype=w0.logits_dtype,
-                     hidden_dtype=w0.hidden_dtype, beta=w0.beta, seed=123)
+                     hidden_dtype=w0.hidden_dtype, beta=w0.beta if args.styles_beta is None else args.styles_beta,
+                     seed=123)
         g = Graft(w.V, w.L, w.K, w.m, w.hidden_dim, w.batch, w.budget_min, w.budget_max, w.budget_step, w.beta, 1,
                   1 if w.logits_dtype == "bf16" else 0, 1 if w.hidden_dtype == "bf16" else 0)
         tb = gi.tdes_tables(w)
@@ -797,7 +798,7 @@ def run_styles(args):
                          status_or=int(out.status.max())))
         g.destroy()
     print(json.dumps({"styles": "per-kernel times of the round on degenerate inputs", "shape": w0.name,
-                      "rounds_timed": args.steps, "rows": rows}))
+                      "beta": w.beta, "rounds_timed": args.steps, "rows": rows}))
 
 
 def run_rows(args):
@@ -864,6 +865,8 @@ def main():
                     help="instead of the benchmark: time the least-squares fit of the SABA models")
     ap.add_argument("--styles", action="store_true",
                     help="instead of the benchmark: the round's kernels timed on degenerate inputs (own JSON line)")
+    ap.add_argument("--styles-beta", type=float, default=None,
+                    help="with --styles: the weight of the edge scores instead of the workload's (0: none, as in DDTree)")
     ap.add_argument("--rows", action="store_true",
                     help="instead of the benchmark: the vocab pass timed on rows that defeat its filter (own JSON line)")
     ap.add_argument("--sweep", action="store_true",

@@ -513,6 +513,13 @@ __device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, 
     return v;
 }
 
+// The order in which best-first takes prefixes of equal key, as one number (larger = earlier): path score, then
+// shallower, then the parent's place in the table, then the place in the parent's sorted row.
+__device__ __forceinline__ uint64_t tie_order(float S, uint32_t info) {
+    return ((uint64_t)ord_from_float(S) << 24) |
+           (uint64_t)(((63u - ((info >> 18) & 63u)) << 18) | ((8191u - (info & 8191u)) << 5) | (31u - ((info >> 24) & 31u)));
+}
+
 // ---- edge scores on demand --------------------------------------------------------------------------------------
 // Row j of the edge scores (children at depth j+1), Eq. 4-6: the table rows P[parent token], C[child token] and
 // u_j are copied into shared memory asynchronously (16-byte cp.async chunks spread over the CTA, issued while the
@@ -597,7 +604,11 @@ __device__ __forceinline__ void lazy_score_row(const TreeParams& p, const TreeSm
 // configured workloads' K = 32, m = 128: every index computation with K becomes a shift), or 0: taken from the parameters
 // FAST: the usual round is known at compile time as well -- the budget comes from the edge-score kernel (no SABA
 // arithmetic in this instance) and deeper rows are scored on demand
-template <int KC, int MC, bool FAST, int NMAXC = 0>
+// TIES: the instance for rounds without edge scores (beta = 0), where exactly equal probabilities make hundreds of
+// prefixes tie with the B-th largest key: it resolves them in parallel (the other instances leave more than 32 tied
+// keys to the sequential expansion; with edge scores in the keys such ties do not occur in tens, and the code's mere
+// presence costs this register-bound kernel 0.4 us a round)
+template <int KC, int MC, bool FAST, int NMAXC = 0, bool TIES = false>
 __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int K = KC ? KC : p.K, p_m = MC ? MC : p.m;
@@ -1051,6 +1062,59 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                         }
                         __syncthreads();
                         ordered = true;
+                    } else if (TIES) {
+                        // Many keys tie with the B-th largest: exactly equal probabilities (flat or one-hot rows) and no
+                        // edge scores to tell them apart.  Where every tied node whose parent is tied too stands behind
+                        // that parent in the order of equal keys -- path scores that do not rise along a path: always so
+                        // without edge scores -- the best available tied node is always the best remaining one, so
+                        // best-first takes the tied nodes in that order outright: the `want` first of them are found by
+                        // a search over the bits of the order (path score, then shallower, parent's place, place in the
+                        // parent's row: 56 bits, two a step with three counts each).  Otherwise: the sequential
+                        // expansion below.
+                        const int want = budget - (n_reach - nt);
+                        int mono = 1, same = 1;  // same: every tied node's own path score is theta (the usual tie)
+                        for (int i = i0 > 1 ? i0 : 1; i < i1; ++i) {
+                            if (sm.nkey[i] != theta) continue;
+                            same &= ord_from_float(sm.nS[i]) == theta ? 1 : 0;
+                            const int par = (int)(sm.ninfo[i] & 8191u);
+                            if (sm.nkey[par] == theta && !(tie_order(sm.nS[par], sm.ninfo[par]) > tie_order(sm.nS[i], sm.ninfo[i])))
+                                mono = 0;
+                        }
+                        uint32_t* cnt = sm.hist + 64;  // [3 * 28] the counts of the steps
+                        if (tid < 84) cnt[tid] = 0u;
+                        same = __syncthreads_and(same);
+                        if (__syncthreads_and(mono)) {  // (uniform)
+                            // (equal path scores: the upper 32 bits of the order are known, twelve steps remain)
+                            uint64_t kth = same ? (uint64_t)theta << 24 : 0ull;
+#pragma unroll 1
+                            for (int step = same ? 16 : 0; step < 28; ++step) {
+                                const int bit = 54 - 2 * step;
+                                const uint64_t t1 = kth | (1ull << bit), t2 = kth | (2ull << bit), t3 = kth | (3ull << bit);
+                                int c1 = 0, c2 = 0, c3 = 0;
+                                for (int i = i0 > 1 ? i0 : 1; i < i1; ++i) {
+                                    if (sm.nkey[i] != theta) continue;
+                                    const uint64_t o = tie_order(sm.nS[i], sm.ninfo[i]);
+                                    c1 += (o >= t1) ? 1 : 0;
+                                    c2 += (o >= t2) ? 1 : 0;
+                                    c3 += (o >= t3) ? 1 : 0;
+                                }
+                                c1 = __reduce_add_sync(0xFFFFFFFFu, c1);
+                                c2 = __reduce_add_sync(0xFFFFFFFFu, c2);
+                                c3 = __reduce_add_sync(0xFFFFFFFFu, c3);
+                                if (lane == 0 && c1) {
+                                    atomicAdd(&cnt[3 * step], (uint32_t)c1);
+                                    atomicAdd(&cnt[3 * step + 1], (uint32_t)c2);
+                                    atomicAdd(&cnt[3 * step + 2], (uint32_t)c3);
+                                }
+                                __syncthreads();
+                                const int n1 = (int)cnt[3 * step], n2 = (int)cnt[3 * step + 1], n3 = (int)cnt[3 * step + 2];
+                                kth = n3 >= want ? t3 : (n2 >= want ? t2 : (n1 >= want ? t1 : kth));
+                            }
+                            for (int i = i0 > 1 ? i0 : 1; i < i1; ++i)
+                                if (sm.nkey[i] == theta && tie_order(sm.nS[i], sm.ninfo[i]) >= kth) sm.nkey[i] = theta + 1u;
+                            __syncthreads();
+                            ordered = true;
+                        }
                     }
                 }
             } else if (ntot - 1 < budget) {
@@ -1465,6 +1529,8 @@ cudaError_t tree_configure(const graft_config& cfg) {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<32, 128, true, 513>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<16, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<8, 128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<0, 0, false, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tree_kernel<32, 128, true, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     return e;
 }
 
@@ -1518,6 +1584,7 @@ cudaError_t tree_launch(graft_ctx* ctx, int batch, const int32_t* d_topk_id, con
     if (usual && cfg.K == 32) kern = (ctx->nmax == 513 && p.ncap == 6144) ? tree_kernel<32, 128, true, 513> : tree_kernel<32, 128, true>;
     if (usual && cfg.K == 16) kern = tree_kernel<16, 128, true>;
     if (usual && cfg.K == 8) kern = tree_kernel<8, 128, true>;
+    if (p.beta == 0.0f) kern = (usual && cfg.K == 32) ? tree_kernel<32, 128, true, 0, true> : tree_kernel<0, 0, false, 0, true>;
     const cudaError_t e = launch_pdl(kern, dim3(batch), dim3(TREE_THREADS), tree_smem_bytes(cfg), st, p);
     ctx->launches += 1;
     return e != cudaSuccess ? e : cudaGetLastError();

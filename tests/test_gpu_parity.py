@@ -645,6 +645,51 @@ def test_round_every_cut_through_small_groups_of_tied_prefixes(beta):
     compare_accept(oracle, gi, g, w, out, gpu)
 
 
+@pytest.mark.parametrize("beta", [0.0, 0.2])
+@pytest.mark.parametrize("shape", ["all equal", "16 equal winners", "32 equal winners", "one-hot", "two-hot", "mixed"])
+def test_round_every_cut_through_large_groups_of_tied_prefixes(shape, beta):
+    """Rows of exactly equal probabilities at the benchmark's K and L: all K candidates of every position equal, 16
+    equal winners over 16 equal others, one token of probability 1 (its chain ties with nothing, everything else ties
+    in hundreds), two tokens of probability 1/2, and a mix of these along the depth.  Without edge scores (beta = 0)
+    hundreds to thousands of prefixes tie with the B-th largest key; 64 fixed budgets from 1 to 512 cut those groups
+    everywhere.  The tree must be the oracle's, node for node."""
+    nb, K, L, V = 64, 32, 16, 1000
+    w = gi.small(batch=nb, L=L, V=V, K=K, budget_min=1, budget_max=512, budget_step=1, fixed_budget=1, beta=beta, m=16,
+                 seed=9)
+    g = _graft(w)
+    tb, saba_kw, keep = _setup(w, g)
+    x = gi.batch_inputs(w)
+    row = torch.full((L, V), -30.0)
+    for d in range(L):
+        kind = shape if shape != "mixed" else ("all equal", "one-hot", "16 equal winners", "two-hot")[d % 4]
+        at = 3 * d
+        if kind == "all equal":
+            row[d] = 0.0
+        elif kind == "16 equal winners":
+            row[d, at:at + 32] = 0.0
+            row[d, at:at + 16] = 1.0
+        elif kind == "32 equal winners":
+            row[d, at:at + 32] = 3.0
+        elif kind == "one-hot":
+            row[d] = -60.0
+            row[d, at] = 0.0
+        elif kind == "two-hot":
+            row[d] = -60.0
+            row[d, at] = 0.0
+            row[d, at + 5] = 0.0
+    x["logits"][:] = row.to(x["logits"].dtype)
+    for k in ("root_token", "hist", "prefix_len", "hidden"):
+        x[k][:] = x[k][0]
+    x["fixed_budget"] = torch.tensor([1 + (511 * i) // (nb - 1) for i in range(nb)], dtype=torch.int32)
+    out, gpu = gpu_round(g, w, x)
+    orc = oracle_round(oracle, w, x, tb, saba_kw)
+    stats = compare_round(oracle, w, x, tb, saba_kw, gpu, orc)
+    assert stats["excused_budget"] == 0 and stats["excused_tree"] == 0, stats
+    for k in ("n_nodes", "token", "parent", "depth", "mask", "status"):
+        assert np.array_equal(gpu[k], orc[k]), k
+    compare_accept(oracle, gi, g, w, out, gpu)
+
+
 @pytest.mark.parametrize("budget", [20, 50, 150])
 def test_round_with_equal_scores_across_depths_and_masked_tokens(budget):
     """Sequence 0: below a uniform first position every later position has one token of probability 1 to fp32
