@@ -513,6 +513,26 @@ __device__ uint32_t cta_finish_select(const TreeSmem& sm, const uint32_t* keys, 
     return v;
 }
 
+// The smallest of keys[lo_i..hi_i) that reaches the bound `theta` of the B-th largest key: a bound of it as well (the
+// B-th largest is one of those keys), reached by the same keys, and an actual key -- where hundreds of keys tie just
+// above a bucket's edge, their value.  The whole CTA; word: one word of scratch.
+__device__ __forceinline__ uint32_t cta_snap_to_key(const uint32_t* keys, int lo_i, int hi_i, uint32_t theta, uint32_t* word,
+                                                    int tid) {
+    if (tid == 0) *word = 0xFFFFFFFFu;
+    __syncthreads();
+    uint32_t mn = 0xFFFFFFFFu;
+    for (int i = lo_i + tid; i < hi_i; i += TREE_THREADS) {
+        const uint32_t k = keys[i];
+        mn = (k >= theta && k < mn) ? k : mn;
+    }
+    mn = __reduce_min_sync(0xFFFFFFFFu, mn);
+    if ((tid & 31) == 0 && mn != 0xFFFFFFFFu) atomicMin(word, mn);
+    __syncthreads();
+    const uint32_t v = *word;
+    __syncthreads();
+    return v == 0xFFFFFFFFu ? theta : v;
+}
+
 // The order in which best-first takes prefixes of equal key, as one number (larger = earlier): path score, then
 // shallower, then the parent's place in the table, then the place in the parent's sorted row.
 __device__ __forceinline__ uint64_t tie_order(float S, uint32_t info) {
@@ -776,6 +796,14 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
     bool ordered = false;
     int n_reach = -1;  // keys that reach the final theta, if the search that found it counted them
     uint32_t theta = 0u;
+    // (TIES instances) th_depth: the depth of the deepest node whose key theta counts -- at least B keys of nodes that
+    // deep or shallower reach theta.  A child deeper than that whose own path score equals theta exactly stands behind
+    // all of them in best-first's order of equal keys (its score is no higher than any of theirs and it is deeper; each
+    // of them becomes available before it could be taken, since their ancestors stand before it too): it can never be
+    // selected and is not appended.  theta is moved up to an actual key after every search so that the equality is met
+    // where it matters: when hundreds of prefixes tie at theta and their best children (probability 1) tie there as
+    // well, level after level, until the table overflows.
+    int th_depth = 99;
     if (budget > 0) {
         int ntot = 1, n_at_select = 1;
         SelBucket sel;
@@ -802,6 +830,11 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     __syncthreads();
                 }
                 theta = cta_select_bucket(sm, sm.nkey, 1, nsel, budget, sel_top, sel, tid);
+                if (TIES) {
+                    __syncthreads();
+                    theta = cta_snap_to_key(sm.nkey, 1, nsel, theta, sm.hist + 1100, tid);
+                    th_depth = nsel != ntot ? 3 : 2;
+                }
                 if (nsel != ntot) sel.valid = false;  // (the bucket counts keys that are not in the table)
                 n_at_select = ntot;
             }
@@ -866,6 +899,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                   const int x = c0 + tid;
                   int total = 0;
                   for (int attempt = 0;; ++attempt) {  // (uniform: at most two rounds)
+                    const uint32_t th_in = theta + ((TIES && d + 1 > th_depth) ? 1u : 0u);  // what a child's score must reach
                     int cnt = 0;
                     uint32_t mask = 0u, kx = 0u;
                     float sx = 0.0f;
@@ -880,7 +914,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                             while (lo_r < hi_r) {
                                 const int mid = (lo_r + hi_r) >> 1;
                                 const uint32_t oc = ord_from_float(sx + sm.es[row + es_col(mid, cx, K)]);
-                                if (oc >= theta)  // (kx >= theta already: the child's key min(kx, oc) reaches theta iff oc does)
+                                if (oc >= th_in)  // (kx >= theta already: the child's key min(kx, oc) reaches theta iff oc does)
                                     lo_r = mid + 1;
                                 else
                                     hi_r = mid;
@@ -927,6 +961,7 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
                     if (attempt == 0 && total >= budget && (total > flood || cur + total > ncap)) {  // (uniform) the search below uses the scan's space: count again
                         const uint32_t tl = cta_kth_largest_of_children(sm, cnt, kx, sx, row, cx, K, budget, theta, tid);
                         theta = tl > theta ? tl : theta;
+                        if (TIES) th_depth = d + 1;
                         continue;
                     }
                     break;
@@ -985,6 +1020,11 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_kernel(const TreeParams p) 
             if (ntot - 1 >= budget && (theta == 0u || ntot - n_at_select >= ntot / 8)) {
                 sel_top = 0.0f + sm.es[0];  // the root's best child
                 theta = cta_select_bucket(sm, sm.nkey, 1, ntot, budget, sel_top, sel, tid);  // a lower bound
+                if (TIES) {
+                    __syncthreads();
+                    theta = cta_snap_to_key(sm.nkey, 1, ntot, theta, sm.hist + 1100, tid);
+                    th_depth = d + 1;
+                }
                 n_at_select = ntot;
                 __syncthreads();  // (its bins share the space of the next level's scan)
             }
